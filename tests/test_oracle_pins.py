@@ -1,0 +1,359 @@
+"""Pins for the fp64 oracle: each function is checked against something other than itself --
+brute force on explicitly padded tiny inputs, closed forms, exact identities of the formulas,
+finite differences, and hand-computed values (tests/golden/)."""
+import itertools
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from oracle import net as onet
+from paper_2503_23186_b200 import workloads as wl
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+rng = np.random.default_rng(1234)
+
+
+# ------------------------------------------------------------------ bf16 rounding helper
+def test_bf16_rne_ties_and_edges():
+    r = oracle.lib().orc_bf16_rne
+    u = 2.0 ** -7  # bf16 spacing in [1,2)
+    assert r(1.0 + u / 2) == 1.0                 # tie -> even mantissa (…0)
+    assert r(1.0 + 3 * u / 2) == 1.0 + 2 * u     # tie -> even mantissa
+    assert r(1.0 + u / 2 + 2.0 ** -30) == 1.0 + u
+    assert r(1.0 + u / 2 - 2.0 ** -30) == 1.0
+    assert r(-(1.0 + 3 * u / 2)) == -(1.0 + 2 * u)
+    assert r(0.0) == 0.0 and np.signbit(r(-0.0))
+    big = (2.0 - 2.0 ** -7) * 2.0 ** 127         # largest finite bf16
+    assert r(big) == big
+    assert np.isinf(r(big * (1 + 2.0 ** -8)))    # rounds up past the largest finite value
+    sub = 2.0 ** -133                            # smallest bf16 subnormal
+    assert r(sub) == sub and r(sub * 0.5) == 0.0 and r(sub * 1.5) == 2 * sub and r(sub * 0.75) == sub
+
+
+def test_bf16_rne_matches_library_cast_from_fp32():
+    import torch
+    x = rng.standard_normal(20000).astype(np.float32) * np.float32(10.0) ** rng.integers(-6, 6, 20000).astype(np.float32)
+    ref = torch.from_numpy(x).to(torch.bfloat16).to(torch.float64).numpy()
+    assert np.array_equal(oracle.round_bf16(x.astype(np.float64)), ref)
+
+
+# ------------------------------------------------------------------ convolution forward
+def brute_conv(x, w, stride, pad):
+    """Seven plain loops over an explicitly zero-padded copy."""
+    N, H, W, C = x.shape
+    K, R, S, _ = w.shape
+    xp = np.zeros((N, H + 2 * pad, W + 2 * pad, C))
+    xp[:, pad:pad + H, pad:pad + W, :] = x
+    P, Q = (H + 2 * pad - R) // stride + 1, (W + 2 * pad - S) // stride + 1
+    y = np.zeros((N, P, Q, K))
+    for n, p, q, k, r, s, c in itertools.product(range(N), range(P), range(Q), range(K), range(R), range(S), range(C)):
+        y[n, p, q, k] += xp[n, p * stride + r, q * stride + s, c] * w[k, r, s, c]
+    return y
+
+
+@pytest.mark.parametrize("R,stride", [(3, 1), (3, 2), (1, 1), (1, 2)])
+@pytest.mark.parametrize("H,W", [(5, 6), (4, 4)])
+def test_conv_fwd_brute_force(R, stride, H, W):
+    x = rng.standard_normal((2, H, W, 3))
+    w = rng.standard_normal((4, R, R, 3))
+    pad = (R - 1) // 2
+    np.testing.assert_allclose(oracle.conv2d_fwd(x, w, stride, pad), brute_conv(x, w, stride, pad), rtol=1e-13, atol=1e-13)
+
+
+def test_conv_delta_and_shift_kernels():
+    x = rng.standard_normal((2, 6, 7, 4))
+    w = np.zeros((4, 3, 3, 4))
+    w[np.arange(4), 1, 1, np.arange(4)] = 1.0            # centre tap identity
+    assert np.array_equal(oracle.conv2d_fwd(x, w, 1, 1), x)
+    w = np.zeros((4, 3, 3, 4))
+    w[np.arange(4), 0, 0, np.arange(4)] = 1.0            # tap (0,0): y[p,q] = x[p-1,q-1]
+    y = oracle.conv2d_fwd(x, w, 1, 1)
+    assert np.array_equal(y[:, 1:, 1:, :], x[:, :-1, :-1, :])
+    assert np.all(y[:, 0, :, :] == 0) and np.all(y[:, :, 0, :] == 0)
+    w = np.zeros((4, 3, 3, 4))
+    w[np.arange(4), 2, 1, np.arange(4)] = 1.0            # tap (2,1): y[p,q] = x[p+1,q]
+    y = oracle.conv2d_fwd(x, w, 1, 1)
+    assert np.array_equal(y[:, :-1, :, :], x[:, 1:, :, :]) and np.all(y[:, -1, :, :] == 0)
+
+
+def test_conv_all_ones_counts_taps():
+    C = 5
+    y = oracle.conv2d_fwd(np.ones((1, 6, 6, C)), np.ones((2, 3, 3, C)), 1, 1)
+    assert np.all(y[0, 1:-1, 1:-1] == 9 * C)
+    assert np.all(y[0, 0, 1:-1] == 6 * C) and np.all(y[0, 1:-1, -1] == 6 * C)
+    assert y[0, 0, 0, 0] == 4 * C and y[0, -1, -1, 1] == 4 * C
+
+
+def test_conv_stride2_geometry():
+    # H=8, stride 2, pad 1: P=4; p=3 reads rows 5..7, so the bottom pad row is never read but the top one is.
+    x = np.zeros((1, 8, 8, 1))
+    x[0, 7, 7, 0] = 1.0
+    w = rng.standard_normal((1, 3, 3, 1))
+    y = oracle.conv2d_fwd(x, w, 2, 1)
+    assert y.shape == (1, 4, 4, 1)
+    expect = np.zeros((4, 4))
+    expect[3, 3] = w[0, 2, 2, 0]   # 7 = 3*2 + r - 1 -> r = 2
+    assert np.array_equal(y[0, :, :, 0], expect)
+
+
+def test_conv_linearity():
+    x1, x2 = rng.standard_normal((2, 1, 5, 5, 3))
+    w1, w2 = rng.standard_normal((2, 2, 3, 3, 3))
+    f = lambda x, w: oracle.conv2d_fwd(x, w, 2, 1)
+    np.testing.assert_allclose(f(2 * x1 - x2, w1), 2 * f(x1, w1) - f(x2, w1), atol=1e-12)
+    np.testing.assert_allclose(f(x1, w1 + 3 * w2), f(x1, w1) + 3 * f(x1, w2), atol=1e-12)
+
+
+# ------------------------------------------------------------------ dgrad / wgrad
+@pytest.mark.parametrize("R,stride,H,W", [(3, 1, 6, 5), (3, 2, 8, 8), (3, 2, 7, 6), (1, 2, 8, 8), (1, 1, 4, 4)])
+def test_adjoint_identities(R, stride, H, W):
+    pad = (R - 1) // 2
+    x = rng.standard_normal((2, H, W, 3))
+    w = rng.standard_normal((4, R, R, 3))
+    y = oracle.conv2d_fwd(x, w, stride, pad)
+    g = rng.standard_normal(y.shape)
+    lhs = np.vdot(y, g)
+    dx = oracle.conv2d_dgrad(g, w, x.shape, stride, pad)
+    dw = oracle.conv2d_wgrad(g, x, R, R, stride, pad)
+    assert abs(lhs - np.vdot(x, dx)) <= 1e-12 * abs(lhs)      # <conv(x;w),g> = <x,dgrad(g;w)>
+    assert abs(lhs - np.vdot(w, dw)) <= 1e-12 * abs(lhs)      # conv is linear in w
+
+
+def test_dgrad_wgrad_finite_differences():
+    x = rng.standard_normal((1, 5, 5, 2))
+    w = rng.standard_normal((3, 3, 3, 2))
+    g = rng.standard_normal((1, 3, 3, 3))
+    L = lambda x_, w_: np.vdot(oracle.conv2d_fwd(x_, w_, 2, 1), g)
+    dx = oracle.conv2d_dgrad(g, w, x.shape, 2, 1)
+    dw = oracle.conv2d_wgrad(g, x, 3, 3, 2, 1)
+    h = 1e-6
+    for idx in [(0, 0, 0, 0), (0, 2, 3, 1), (0, 4, 4, 0), (0, 1, 4, 1)]:
+        e = np.zeros_like(x); e[idx] = h
+        assert abs((L(x + e, w) - L(x - e, w)) / (2 * h) - dx[idx]) < 1e-7
+    for idx in [(0, 0, 0, 0), (2, 1, 2, 1), (1, 2, 2, 0)]:
+        e = np.zeros_like(w); e[idx] = h
+        assert abs((L(x, w + e) - L(x, w - e)) / (2 * h) - dw[idx]) < 1e-7
+
+
+def test_dgrad_brute_force_gather():
+    # independent gather form: dx[h,w] sums dy[p,q] over taps with p*st+r-pad = h
+    x_shape = (1, 6, 6, 2); st, pad, R = 2, 1, 3
+    w = rng.standard_normal((3, R, R, 2))
+    g = rng.standard_normal((1, 3, 3, 3))
+    dx = oracle.conv2d_dgrad(g, w, x_shape, st, pad)
+    ref = np.zeros(x_shape)
+    for h, ww, c, k, r, s in itertools.product(range(6), range(6), range(2), range(3), range(R), range(R)):
+        ph, qw = h + pad - r, ww + pad - s
+        if ph % st or qw % st:
+            continue
+        p, q = ph // st, qw // st
+        if 0 <= p < 3 and 0 <= q < 3:
+            ref[0, h, ww, c] += g[0, p, q, k] * w[k, r, s, c]
+    np.testing.assert_allclose(dx, ref, atol=1e-13)
+
+
+# ------------------------------------------------------------------ batch norm
+def test_bn_forward_closed_forms():
+    eps = 1e-5
+    y = rng.standard_normal((64, 3)) * np.array([1.0, 4.0, 0.3]) + np.array([0.0, 5.0, -2.0])
+    gamma, beta = np.array([1.5, 0.5, 2.0]), np.array([0.1, -0.2, 0.3])
+    mean, var, invstd = oracle.bn_stats(y, eps)
+    np.testing.assert_allclose(mean, y.mean(0), atol=1e-14)
+    np.testing.assert_allclose(var, y.var(0), rtol=1e-13)
+    z = oracle.bn_relu_apply(y, mean, invstd, gamma, beta, None, False)
+    np.testing.assert_allclose(z.mean(0), beta, atol=1e-13)
+    np.testing.assert_allclose(z.var(0), gamma ** 2 * var / (var + eps), rtol=1e-12)
+    # two-element channel (-t, t): xhat = -+ t/sqrt(t^2+eps)
+    t = 0.7
+    y2 = np.array([[-t], [t]])
+    m2, v2, i2 = oracle.bn_stats(y2, eps)
+    z2 = oracle.bn_relu_apply(y2, m2, i2, np.ones(1), np.zeros(1), None, False)
+    np.testing.assert_allclose(z2[:, 0], np.array([-t, t]) / np.sqrt(t * t + eps), rtol=1e-14)
+    # constant channel -> z = beta ; relu and residual
+    yc = np.full((8, 1), 3.25)
+    mc, vc, ic = oracle.bn_stats(yc, eps)
+    assert vc[0] == 0 and np.allclose(oracle.bn_relu_apply(yc, mc, ic, np.array([2.0]), np.array([0.5]), None, False), 0.5)
+    res = rng.standard_normal(y.shape)
+    a = oracle.bn_relu_apply(y, mean, invstd, gamma, beta, res, True)
+    np.testing.assert_allclose(a, np.maximum(z + res, 0.0), atol=1e-14)
+
+
+def _bn_loss(y, gamma, beta, res, G, relu):
+    mean, var, invstd = oracle.bn_stats(y, 1e-5)
+    return np.vdot(oracle.bn_relu_apply(y, mean, invstd, gamma, beta, res, relu), G)
+
+
+@pytest.mark.parametrize("relu,use_res,two", [(True, True, True), (False, False, False), (True, False, True)])
+def test_bn_backward_identities_and_finite_differences(relu, use_res, two):
+    M, C = 12, 3
+    y = rng.standard_normal((M, C)) * 2 + 1
+    gamma, beta = rng.standard_normal(C) + 2, rng.standard_normal(C)
+    res = rng.standard_normal((M, C)) if use_res else None
+    da1 = rng.standard_normal((M, C))
+    da2 = rng.standard_normal((M, C)) if two else None
+    G = da1 + (da2 if two else 0)
+    mean, var, invstd = oracle.bn_stats(y, 1e-5)
+    a = oracle.bn_relu_apply(y, mean, invstd, gamma, beta, res, relu)
+    dy, dres, dgamma, dbeta = oracle.bn_relu_bwd(da1, da2, y, a, gamma, mean, invstd, relu, use_res)
+    xhat = (y - mean) * invstd
+    assert np.all(np.abs(dy.sum(0)) < 1e-12)
+    # sum(dy*xhat) = gamma*invstd*dgamma*(1 - sum(xhat^2)/M) = gamma*invstd*dgamma*eps/(var+eps): zero only for eps = 0
+    np.testing.assert_allclose((dy * xhat).sum(0), gamma * invstd * dgamma * 1e-5 / (var + 1e-5), atol=1e-12)
+    dz = G * (a > 0) if relu else G
+    np.testing.assert_allclose(dbeta, dz.sum(0), atol=1e-13)
+    np.testing.assert_allclose(dgamma, (dz * xhat).sum(0), atol=1e-13)
+    if use_res:
+        np.testing.assert_allclose(dres, dz, atol=0)
+    h = 1e-6
+    for idx in [(0, 0), (5, 1), (11, 2)]:
+        e = np.zeros_like(y); e[idx] = h
+        fd = (_bn_loss(y + e, gamma, beta, res, G, relu) - _bn_loss(y - e, gamma, beta, res, G, relu)) / (2 * h)
+        assert abs(fd - dy[idx]) < 2e-7
+    for c in range(C):
+        e = np.zeros(C); e[c] = h
+        fd = (_bn_loss(y, gamma + e, beta, res, G, relu) - _bn_loss(y, gamma - e, beta, res, G, relu)) / (2 * h)
+        assert abs(fd - dgamma[c]) < 2e-7
+        fd = (_bn_loss(y, gamma, beta + e, res, G, relu) - _bn_loss(y, gamma, beta - e, res, G, relu)) / (2 * h)
+        assert abs(fd - dbeta[c]) < 2e-7
+
+
+# ------------------------------------------------------------------ pooling
+def test_avgpool_pair():
+    a = rng.standard_normal((3, 4, 4, 5))
+    np.testing.assert_allclose(oracle.avgpool_fwd(a), a.mean(axis=(1, 2)), atol=1e-14)
+    g = rng.standard_normal((3, 5))
+    da = oracle.avgpool_bwd(g, 4, 4)
+    assert abs(np.vdot(oracle.avgpool_fwd(a), g) - np.vdot(a, da)) < 1e-12
+
+
+# ------------------------------------------------------------------ softmax cross-entropy
+def _golden(name):
+    rows = {}
+    with open(os.path.join(GOLD, name)) as f:
+        for line in f:
+            line = line.split("#")[0].strip()
+            if line:
+                k, v = line.split("=")
+                rows[k.strip()] = float(v)
+    return rows
+
+
+def test_softmax_xent_hand_values():
+    gold = _golden("softmax_xent_hand_values.txt")
+    loss, dz = oracle.softmax_xent(np.zeros((4, 100)), np.array([0, 7, 50, 99]), 0.25)
+    assert abs(loss - gold["uniform100_loss"]) < 1e-9          # ln 100
+    assert np.allclose(dz[1, 7], gold["uniform100_on_label"] * 0.25) and np.allclose(dz[1, 8], gold["uniform100_off_label"] * 0.25)
+    loss, dz = oracle.softmax_xent(np.array([[0.0, np.log(3.0)]]), np.array([1]), 1.0)
+    assert abs(loss - gold["two_class_loss"]) < 1e-9           # ln(4/3)
+    np.testing.assert_allclose(dz[0], [gold["two_class_p0"], gold["two_class_p1"] - 1.0], atol=1e-12)
+
+
+def test_softmax_xent_invariants():
+    z = rng.standard_normal((6, 10)) * 3
+    lab = rng.integers(0, 10, 6)
+    loss, dz = oracle.softmax_xent(z, lab, 1.0 / 6)
+    assert np.all(np.abs(dz.sum(1)) < 1e-15)
+    loss2, dz2 = oracle.softmax_xent(z + 123.0, lab, 1.0 / 6)
+    assert abs(loss - loss2) < 1e-10 and np.allclose(dz, dz2, atol=1e-12)
+    big = np.array([[80.0, -80.0, 0.0]])
+    l3, d3 = oracle.softmax_xent(big, np.array([1]), 1.0)
+    assert np.isfinite(l3) and abs(l3 - 160.0) < 1e-9 and np.all(np.isfinite(d3))
+    # gradient is the derivative of the mean loss times N*grad_scale
+    h = 1e-6
+    e = np.zeros_like(z); e[2, 3] = h
+    fd = (oracle.softmax_xent(z + e, lab, 1)[0] - oracle.softmax_xent(z - e, lab, 1)[0]) / (2 * h)
+    assert abs(fd - dz[2, 3]) < 1e-8
+    with pytest.raises(ValueError):
+        oracle.softmax_xent(z, np.full(6, 10), 1.0)
+
+
+# ------------------------------------------------------------------ SGD
+def test_sgd_hand_value_and_micro_batch_average():
+    gold = _golden("sgd_hand_values.txt")
+    w, v = oracle.sgd_momentum(np.array([1.0]), np.array([0.5]), np.array([0.2]), 1.0, 0.1, 0.9, 5e-4)
+    assert abs(v[0] - gold["v_new"]) < 1e-15 and abs(w[0] - gold["w_new"]) < 1e-15
+    w8, v8 = oracle.sgd_momentum(np.array([1.0]), np.array([0.5]), np.array([8 * 0.2]), 1.0 / 8, 0.1, 0.9, 5e-4)
+    assert abs(w8[0] - w[0]) < 1e-15 and abs(v8[0] - v[0]) < 1e-15
+
+
+# ------------------------------------------------------------------ whole network
+def _tiny():
+    spec = wl.tiny_net_spec(classes=10, hw=8, c=4, width=4, width2=8)
+    params = wl.perturb_bn_params(wl.init_params(spec, 3), 3)
+    params = {k: v.astype(np.float64) for k, v in params.items()}
+    images = rng.standard_normal((4, 8, 8, 4))
+    labels = rng.integers(0, 10, 4).astype(np.int32)
+    return spec, params, images, labels
+
+
+def test_net_gradients_finite_differences():
+    spec, params, images, labels = _tiny()
+    fw = onet.forward(spec, params, images, labels, rounding=False)
+    grads, _ = onet.backward(spec, params, fw, rounding=False)
+    assert set(grads) == set(params)
+    h = 1e-6
+    for name in params:
+        flat = params[name].reshape(-1)
+        for j in sorted(set([0, flat.size // 2, flat.size - 1])):
+            old = flat[j]
+            flat[j] = old + h; lp = onet.forward(spec, params, images, labels, rounding=False)["loss"]
+            flat[j] = old - h; lm = onet.forward(spec, params, images, labels, rounding=False)["loss"]
+            flat[j] = old
+            fd = (lp - lm) / (2 * h)
+            g = grads[name].reshape(-1)[j]
+            assert abs(fd - g) < 1e-6 * max(1.0, abs(g)), (name, j, fd, g)
+
+
+def test_net_scale_invariance_of_conv_before_bn():
+    # a conv followed by BN is scale invariant: <w, dL/dw> ~ 0 (exactly 0 for eps = 0)
+    spec, params, images, labels = _tiny()
+    fw = onet.forward(spec, params, images, labels, rounding=False)
+    grads, _ = onet.backward(spec, params, fw, rounding=False)
+    for i, L in enumerate(spec):
+        if L["kind"] == "conv":
+            g, w = grads[f"w{i}"], params[f"w{i}"]
+            assert abs(np.vdot(g, w)) < 1e-3 * np.linalg.norm(g) * np.linalg.norm(w)
+
+
+def test_train_step_micro_batches():
+    spec, params, images, labels = _tiny()
+    vel = {k: rng.standard_normal(v.shape) * 0.01 for k, v in params.items()}
+    one = onet.train_step(spec, params, vel, images, labels, 1, 0.1, 0.9, 5e-4, rounding=False)
+    # identical micro-batches: the average equals a single micro-batch
+    rep = onet.train_step(spec, params, vel, np.concatenate([images] * 3), np.concatenate([labels] * 3), 3,
+                          0.1, 0.9, 5e-4, rounding=False)
+    for k in params:
+        np.testing.assert_allclose(rep["params"][k], one["params"][k], rtol=1e-12, atol=1e-14)
+    # order of micro-batches does not matter
+    im2, lb2 = rng.standard_normal(images.shape), rng.integers(0, 10, 4).astype(np.int32)
+    ab = onet.train_step(spec, params, vel, np.concatenate([images, im2]), np.concatenate([labels, lb2]), 2, 0.1, 0.9, 5e-4, False)
+    ba = onet.train_step(spec, params, vel, np.concatenate([im2, images]), np.concatenate([lb2, labels]), 2, 0.1, 0.9, 5e-4, False)
+    for k in params:
+        np.testing.assert_allclose(ab["params"][k], ba["params"][k], rtol=1e-12, atol=1e-14)
+    assert abs(ab["loss"] - ba["loss"]) < 1e-13
+    # the update is w - lr*(mu*v + mean-gradient + wd*w)
+    k = "w0"
+    g = ab["grads"][k] / 2 + 5e-4 * params[k]
+    np.testing.assert_allclose(ab["params"][k], params[k] - 0.1 * (0.9 * vel[k] + g), rtol=1e-12, atol=1e-14)
+
+
+def test_rounding_points_are_small_perturbations():
+    spec, params, images, labels = _tiny()
+    images = wl.to_bf16_grid(images).astype(np.float64)
+    a = onet.train_step(spec, params, {k: np.zeros_like(v) for k, v in params.items()}, images, labels, 1, 0.1, 0.9, 5e-4, True)
+    b = onet.train_step(spec, params, {k: np.zeros_like(v) for k, v in params.items()}, images, labels, 1, 0.1, 0.9, 5e-4, False)
+    assert abs(a["loss"] - b["loss"]) < 0.05 * abs(b["loss"])
+    for k in ("w0", f"w{len(spec) - 2}"):
+        assert np.linalg.norm(a["grads"][k] - b["grads"][k]) < 0.1 * np.linalg.norm(b["grads"][k])
+
+
+def test_network_shapes_match_published_parameter_counts():
+    def count(spec):
+        p = wl.init_params(spec, 0)
+        conv_fc = sum(v.size for k, v in p.items() if k.startswith("w"))
+        bn = sum(v.size for k, v in p.items() if k.startswith(("gamma", "beta")))
+        return conv_fc, bn
+    assert count(wl.resnet18_spec()) == (11210432, 9600)
+    assert count(wl.wrn28_10_spec()) == (36518832, 20192)
