@@ -1,0 +1,530 @@
+// C ABI: context, convolution entry points, and the training step over a layer list.
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "common.h"
+
+using namespace b2c;
+
+extern "C" {
+
+b2c_status b2c_create(b2c_ctx** out, int device)
+{
+    if (!out) return B2C_ERR_INVALID_ARG;
+    *out = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) return B2C_ERR_CUDA;
+    cudaDeviceProp prop;
+    B2C_CUDA(cudaGetDeviceProperties(&prop, device));
+    if (prop.major != 10) return B2C_ERR_ARCH;
+    B2C_CUDA(cudaSetDevice(device));
+    b2c_ctx* ctx = new (std::nothrow) b2c_ctx();
+    if (!ctx) return B2C_ERR_CUDA;
+    ctx->device = device;
+    ctx->sm_count = prop.multiProcessorCount;
+    ctx->spin_limit = 1u << 22;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || fn == nullptr ||
+        qres != cudaDriverEntryPointSuccess) {
+        delete ctx;
+        return B2C_ERR_CUDA;
+    }
+    ctx->encode_tiled = reinterpret_cast<b2c_encode_tiled_fn>(fn);
+    if (cudaMalloc(&ctx->d_status, sizeof(unsigned)) != cudaSuccess || cudaMemset(ctx->d_status, 0, sizeof(unsigned)) != cudaSuccess) {
+        delete ctx;
+        return B2C_ERR_CUDA;
+    }
+    *out = ctx;
+    return B2C_OK;
+}
+
+void b2c_destroy(b2c_ctx* ctx)
+{
+    if (!ctx) return;
+    cudaFree(ctx->d_status);
+    delete ctx;
+}
+
+const char* b2c_status_string(b2c_status s)
+{
+    switch (s) {
+        case B2C_OK: return "ok";
+        case B2C_ERR_INVALID_ARG: return "invalid argument";
+        case B2C_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+        case B2C_ERR_MISALIGNED: return "misaligned pointer";
+        case B2C_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case B2C_ERR_CUDA: return "CUDA runtime or driver error";
+        case B2C_ERR_ARCH: return "device is not compute capability 10.x";
+        case B2C_ERR_DEVICE_TIMEOUT: return "a device-side wait exhausted its spin budget";
+        case B2C_ERR_BAD_LABEL: return "label outside [0, classes)";
+    }
+    return "unknown status";
+}
+
+b2c_status b2c_get_device_status(b2c_ctx* ctx, void* stream)
+{
+    if (!ctx) return B2C_ERR_INVALID_ARG;
+    unsigned word = 0;
+    B2C_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+    B2C_CUDA(cudaMemcpy(&word, ctx->d_status, sizeof(word), cudaMemcpyDeviceToHost));
+    if (word) B2C_CUDA(cudaMemset(ctx->d_status, 0, sizeof(word)));
+    if (word & B2C_DEV_TIMEOUT) return B2C_ERR_DEVICE_TIMEOUT;
+    if (word & B2C_DEV_BAD_LABEL) return B2C_ERR_BAD_LABEL;
+    return B2C_OK;
+}
+
+void b2c_set_spin_limit(b2c_ctx* ctx, unsigned limit)
+{
+    if (ctx && limit > 0) ctx->spin_limit = limit;
+}
+
+// ------------------------------------------------------------------------------ convolution
+static b2c_status check_desc(const b2c_conv_desc* d, int* p, int* q)
+{
+    if (!d) return B2C_ERR_INVALID_ARG;
+    if (d->n < 1 || d->h < 1 || d->w < 1 || d->c < 1 || d->k < 1) return B2C_ERR_INVALID_ARG;
+    if (d->r != d->s || !(d->r == 1 || d->r == 3) || !(d->stride == 1 || d->stride == 2) || d->pad != (d->r - 1) / 2)
+        return B2C_ERR_UNSUPPORTED_SHAPE;
+    *p = (d->h + 2 * d->pad - d->r) / d->stride + 1;
+    *q = (d->w + 2 * d->pad - d->s) / d->stride + 1;
+    if (*p * d->stride != d->h || *q * d->stride != d->w) return B2C_ERR_UNSUPPORTED_SHAPE;
+    return B2C_OK;
+}
+
+b2c_status b2c_conv2d_fwd(b2c_ctx* ctx, const b2c_conv_desc* d, const void* x, const void* w_krsc, void* y, int y_is_f32, const float* bias,
+                          double* ch_stats, void* stream)
+{
+    if (!ctx || !x || !w_krsc || !y) return B2C_ERR_INVALID_ARG;
+    int p, q;
+    b2c_status st = check_desc(d, &p, &q);
+    if (st != B2C_OK) return st;
+    if (ch_stats && y_is_f32) return B2C_ERR_INVALID_ARG;
+    KMajorProblem pb{};
+    pb.n = d->n; pb.ih = d->h; pb.iw = d->w; pb.ic = d->c;
+    pb.oh = p; pb.ow = q; pb.oc = d->k;
+    pb.r = d->r; pb.stride = d->stride; pb.pad = d->pad;
+    pb.dgrad = false;
+    pb.in = x; pb.wt = w_krsc; pb.out = y;
+    pb.out_f32 = y_is_f32 != 0; pb.bias = bias; pb.stats = ch_stats;
+    return launch_conv_kmajor(ctx, pb, (cudaStream_t)stream);
+}
+
+b2c_status b2c_conv2d_dgrad(b2c_ctx* ctx, const b2c_conv_desc* d, const void* dy, const void* w_crsk_flipped, void* dx, void* stream)
+{
+    if (!ctx || !dy || !w_crsk_flipped || !dx) return B2C_ERR_INVALID_ARG;
+    int p, q;
+    b2c_status st = check_desc(d, &p, &q);
+    if (st != B2C_OK) return st;
+    KMajorProblem pb{};
+    pb.n = d->n; pb.ih = p; pb.iw = q; pb.ic = d->k;
+    pb.oh = d->h; pb.ow = d->w; pb.oc = d->c;
+    pb.r = d->r; pb.stride = d->stride; pb.pad = d->pad;
+    pb.dgrad = true;
+    pb.in = dy; pb.wt = w_crsk_flipped; pb.out = dx;
+    pb.out_f32 = false; pb.bias = nullptr; pb.stats = nullptr;
+    return launch_conv_kmajor(ctx, pb, (cudaStream_t)stream);
+}
+
+b2c_status b2c_conv2d_wgrad(b2c_ctx* ctx, const b2c_conv_desc* d, const void* dy, const void* x, float* dw_krsc, int accumulate, void* stream)
+{
+    if (!ctx || !dy || !x || !dw_krsc) return B2C_ERR_INVALID_ARG;
+    int p, q;
+    b2c_status st = check_desc(d, &p, &q);
+    if (st != B2C_OK) return st;
+    WgradProblem pb{};
+    pb.n = d->n; pb.h = d->h; pb.w = d->w; pb.c = d->c;
+    pb.p = p; pb.q = q; pb.k = d->k;
+    pb.r = d->r; pb.stride = d->stride; pb.pad = d->pad;
+    pb.dy = dy; pb.x = x; pb.dw = dw_krsc;
+    if (d->c % 16 || d->k % 16) return B2C_ERR_UNSUPPORTED_SHAPE;
+    if (!accumulate) B2C_CUDA(cudaMemsetAsync(dw_krsc, 0, sizeof(float) * (size_t)d->k * d->r * d->s * d->c, (cudaStream_t)stream));
+    return launch_conv_wgrad(ctx, pb, (cudaStream_t)stream);
+}
+
+}  // extern "C"
+
+// ------------------------------------------------------------------------------ layer list
+namespace {
+
+struct TensorPlan {
+    int n = 0, h = 1, w = 1, c = 0;  // c = stored (padded) channels
+    bool f32 = false;
+    bool exists = false;
+    long long act_off = -1;        // bytes into the workspace (-1 for tensor 0 when it is read in place)
+    long long stats_off = -1;      // fp64 [2c] sum / sum of squares, for convolution outputs
+    long long grad_off[2] = {-1, -1};
+    int n_contrib = 0;             // gradient contributions expected
+    int producer = -1;             // layer index
+    size_t elems() const { return (size_t)n * h * w * c; }
+};
+
+struct LayerPlan {
+    b2c_layer_desc d;
+    int c_pad = 0, k_pad = 0;      // stored input / output channels of conv and fc layers
+    int p = 0, q = 0;
+    long long w_off = -1, gamma_off = -1, beta_off = -1, bias_off = -1;   // elements into the flat parameter arrays
+    long long mean_off = -1, invstd_off = -1, bwd_ws_off = -1;            // bytes into the workspace
+    int src_slot = -1, res_slot = -1;                                     // which gradient buffer of src / res this layer writes
+};
+
+inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
+
+}  // namespace
+
+struct b2c_net {
+    b2c_ctx* ctx = nullptr;
+    int micro_batch = 0;
+    int image_h = 0, image_w = 0, image_c = 0, image_c_pad = 0;
+    std::vector<LayerPlan> layers;
+    std::vector<TensorPlan> tensors;
+    std::vector<b2c_weight_seg> segs;
+    size_t param_count = 0;
+    size_t ws_bytes = 0;
+    long long stats_begin = 0, stats_end = 0;   // fp64 region zeroed before every forward pass
+    float *w = nullptr, *v = nullptr, *g = nullptr;
+    char *w_bf16 = nullptr, *w_dgrad = nullptr, *ws = nullptr;
+    bool fuse_stats = true;
+};
+
+extern "C" {
+
+b2c_status b2c_net_create(b2c_ctx* ctx, const b2c_layer_desc* layers, int n_layers, int micro_batch, b2c_net** out)
+{
+    if (!ctx || !layers || !out || n_layers < 1 || micro_batch < 1) return B2C_ERR_INVALID_ARG;
+    *out = nullptr;
+    b2c_net* net = new (std::nothrow) b2c_net();
+    if (!net) return B2C_ERR_CUDA;
+    net->ctx = ctx;
+    net->micro_batch = micro_batch;
+    const char* env = std::getenv("B2C_FUSE_BN_STATS");
+    net->fuse_stats = !(env && env[0] == '0');
+    net->layers.resize(n_layers);
+    net->tensors.resize(n_layers + 1);
+    auto fail = [&](b2c_status s) { delete net; return s; };
+
+    size_t ws = 0;
+    auto alloc = [&](size_t bytes) { long long off = (long long)ws; ws += (bytes + 255) & ~size_t(255); return off; };
+    size_t pc = 0;
+    auto palloc = [&](size_t elems) { long long off = (long long)pc; pc += (elems + 7) & ~size_t(7); return off; };
+
+    // the first layer must be a convolution reading tensor 0: it fixes the image shape
+    if (layers[0].kind != B2C_LAYER_CONV || layers[0].src != 0) return fail(B2C_ERR_INVALID_ARG);
+    net->image_h = layers[0].h; net->image_w = layers[0].w; net->image_c = layers[0].c;
+    net->image_c_pad = round_up(layers[0].c, 16);
+    {
+        TensorPlan& t0 = net->tensors[0];
+        t0.n = micro_batch; t0.h = net->image_h; t0.w = net->image_w; t0.c = net->image_c_pad; t0.exists = true;
+        if (net->image_c_pad != net->image_c) t0.act_off = alloc(t0.elems() * 2);
+    }
+    // forward shapes and parameters
+    for (int i = 0; i < n_layers; ++i) {
+        LayerPlan& L = net->layers[i];
+        L.d = layers[i];
+        const b2c_layer_desc& d = L.d;
+        if (d.src < 0 || d.src > i || !net->tensors[d.src].exists) return fail(B2C_ERR_INVALID_ARG);
+        const TensorPlan& in = net->tensors[d.src];
+        TensorPlan& o = net->tensors[i + 1];
+        o.producer = i;
+        switch (d.kind) {
+            case B2C_LAYER_CONV: {
+                if (in.f32 || d.h != in.h || d.w != in.w || round_up(d.c, 16) != in.c) return fail(B2C_ERR_INVALID_ARG);
+                if (d.k % 16 || !(d.r == 1 || d.r == 3) || !(d.stride == 1 || d.stride == 2)) return fail(B2C_ERR_UNSUPPORTED_SHAPE);
+                if (d.src != 0 && d.c % 16) return fail(B2C_ERR_UNSUPPORTED_SHAPE);
+                const int pad = (d.r - 1) / 2;
+                L.c_pad = in.c; L.k_pad = d.k;
+                L.p = (d.h + 2 * pad - d.r) / d.stride + 1; L.q = (d.w + 2 * pad - d.r) / d.stride + 1;
+                if (L.p * d.stride != d.h || L.q * d.stride != d.w || !b2c_is_pow2(L.p) || !b2c_is_pow2(L.q)) return fail(B2C_ERR_UNSUPPORTED_SHAPE);
+                o.n = micro_batch; o.h = L.p; o.w = L.q; o.c = d.k; o.exists = true;
+                o.act_off = alloc(o.elems() * 2);
+                L.w_off = palloc((size_t)d.k * d.r * d.r * L.c_pad);
+                net->segs.push_back(b2c_weight_seg{L.w_off, d.k, d.r * d.r, L.c_pad});
+                break;
+            }
+            case B2C_LAYER_BN: {
+                if (in.f32 || d.c != in.c || d.c % 8) return fail(B2C_ERR_INVALID_ARG);
+                if (d.res >= 0) {
+                    if (d.res > i || !net->tensors[d.res].exists) return fail(B2C_ERR_INVALID_ARG);
+                    const TensorPlan& r = net->tensors[d.res];
+                    if (r.n != in.n || r.h != in.h || r.w != in.w || r.c != in.c || d.res == 0) return fail(B2C_ERR_INVALID_ARG);
+                }
+                o = in; o.producer = i; o.n_contrib = 0; o.grad_off[0] = o.grad_off[1] = -1; o.stats_off = -1;
+                o.act_off = alloc(o.elems() * 2);
+                break;
+            }
+            case B2C_LAYER_AVGPOOL: {
+                if (in.f32 || d.c != in.c) return fail(B2C_ERR_INVALID_ARG);
+                o.n = micro_batch; o.h = 1; o.w = 1; o.c = in.c; o.exists = true;
+                o.act_off = alloc(o.elems() * 2);
+                break;
+            }
+            case B2C_LAYER_FC: {
+                if (in.f32 || in.h != 1 || in.w != 1 || d.c != in.c || d.c % 16 || d.k < 1) return fail(B2C_ERR_INVALID_ARG);
+                L.c_pad = in.c; L.k_pad = round_up(d.k, 64);
+                L.p = L.q = 1;
+                o.n = micro_batch; o.h = 1; o.w = 1; o.c = L.k_pad; o.f32 = true; o.exists = true;
+                o.act_off = alloc(o.elems() * 4);
+                L.w_off = palloc((size_t)L.k_pad * L.c_pad);
+                net->segs.push_back(b2c_weight_seg{L.w_off, L.k_pad, 1, L.c_pad});
+                break;
+            }
+            case B2C_LAYER_XENT: {
+                if (!in.f32 || i != n_layers - 1 || net->layers[in.producer].d.kind != B2C_LAYER_FC || d.k != net->layers[in.producer].d.k)
+                    return fail(B2C_ERR_INVALID_ARG);
+                break;
+            }
+            default: return fail(B2C_ERR_INVALID_ARG);
+        }
+    }
+    if (layers[n_layers - 1].kind != B2C_LAYER_XENT) return fail(B2C_ERR_INVALID_ARG);
+    if (net->segs.size() > 128) return fail(B2C_ERR_UNSUPPORTED_SHAPE);
+    // BatchNorm / bias parameters after all filter banks
+    for (int i = 0; i < n_layers; ++i) {
+        LayerPlan& L = net->layers[i];
+        if (L.d.kind == B2C_LAYER_BN) { L.gamma_off = palloc(L.d.c); L.beta_off = palloc(L.d.c); }
+        if (L.d.kind == B2C_LAYER_FC) L.bias_off = palloc(L.k_pad);
+    }
+    net->param_count = (pc + 3) & ~size_t(3);
+
+    // backward plan: gradient buffers, in the order the backward pass produces them
+    auto add_contrib = [&](int t) -> int {
+        TensorPlan& T = net->tensors[t];
+        if (T.n_contrib >= 2) return -1;
+        const int slot = T.n_contrib++;
+        T.grad_off[slot] = alloc(T.elems() * 2);
+        return slot;
+    };
+    for (int i = n_layers - 1; i >= 0; --i) {
+        LayerPlan& L = net->layers[i];
+        const int kind = L.d.kind;
+        if (kind == B2C_LAYER_XENT || kind == B2C_LAYER_FC || kind == B2C_LAYER_AVGPOOL || kind == B2C_LAYER_BN ||
+            (kind == B2C_LAYER_CONV && L.d.src != 0)) {
+            if (kind != B2C_LAYER_XENT && net->tensors[i + 1].n_contrib < 1) return fail(B2C_ERR_INVALID_ARG);   // dead output
+            if (kind != B2C_LAYER_BN && kind != B2C_LAYER_XENT && net->tensors[i + 1].n_contrib != 1) return fail(B2C_ERR_UNSUPPORTED_SHAPE);
+            if ((L.src_slot = add_contrib(L.d.src)) < 0) return fail(B2C_ERR_UNSUPPORTED_SHAPE);
+            if (kind == B2C_LAYER_BN && L.d.res >= 0 && (L.res_slot = add_contrib(L.d.res)) < 0) return fail(B2C_ERR_UNSUPPORTED_SHAPE);
+        }
+    }
+    // small per-layer buffers; the fp64 statistics are contiguous so one memset clears them
+    for (int i = 0; i < n_layers; ++i) {
+        LayerPlan& L = net->layers[i];
+        if (L.d.kind == B2C_LAYER_BN) { L.mean_off = alloc(4 * (size_t)L.d.c); L.invstd_off = alloc(4 * (size_t)L.d.c); }
+    }
+    net->stats_begin = (long long)ws;
+    for (int i = 0; i < n_layers; ++i) {
+        LayerPlan& L = net->layers[i];
+        if (L.d.kind == B2C_LAYER_CONV) net->tensors[i + 1].stats_off = alloc(16 * (size_t)L.d.k);
+        if (L.d.kind == B2C_LAYER_BN) L.bwd_ws_off = alloc(b2c_bn_relu_bwd_workspace_bytes(L.d.c));
+    }
+    net->stats_end = (long long)ws;
+    net->ws_bytes = ws;
+    *out = net;
+    return B2C_OK;
+}
+
+void b2c_net_destroy(b2c_net* net) { delete net; }
+size_t b2c_net_param_count(const b2c_net* net) { return net ? net->param_count : 0; }
+size_t b2c_net_workspace_bytes(const b2c_net* net) { return net ? net->ws_bytes : 0; }
+int b2c_net_padded_image_channels(const b2c_net* net) { return net ? net->image_c_pad : 0; }
+
+long long b2c_net_param_offset(const b2c_net* net, int layer, int which)
+{
+    if (!net || layer < 0 || layer >= (int)net->layers.size()) return -1;
+    const LayerPlan& L = net->layers[layer];
+    switch (which) {
+        case 0: return L.w_off;
+        case 1: return L.gamma_off;
+        case 2: return L.beta_off;
+        case 3: return L.bias_off;
+    }
+    return -1;
+}
+
+long long b2c_net_tensor_offset(const b2c_net* net, int tensor, int grad, int which)
+{
+    if (!net || tensor < 0 || tensor >= (int)net->tensors.size()) return -1;
+    const TensorPlan& T = net->tensors[tensor];
+    if (!grad) return T.act_off;
+    if (which < 0 || which > 1) return -1;
+    return T.grad_off[which];
+}
+
+b2c_status b2c_net_bind(b2c_net* net, float* w_master, float* velocity, float* grad_sum, void* w_bf16, void* w_bf16_dgrad, void* workspace,
+                        size_t workspace_bytes)
+{
+    if (!net || !w_master || !velocity || !grad_sum || !w_bf16 || !w_bf16_dgrad || !workspace) return B2C_ERR_INVALID_ARG;
+    if (workspace_bytes < net->ws_bytes) return B2C_ERR_WORKSPACE_TOO_SMALL;
+    if (!b2c_aligned16(w_master) || !b2c_aligned16(velocity) || !b2c_aligned16(grad_sum) || !b2c_aligned16(w_bf16) ||
+        !b2c_aligned16(w_bf16_dgrad) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+        return B2C_ERR_MISALIGNED;
+    net->w = w_master; net->v = velocity; net->g = grad_sum;
+    net->w_bf16 = reinterpret_cast<char*>(w_bf16); net->w_dgrad = reinterpret_cast<char*>(w_bf16_dgrad);
+    net->ws = reinterpret_cast<char*>(workspace);
+    return B2C_OK;
+}
+
+static b2c_status net_pack_dgrad(b2c_net* net, void* stream)
+{
+    return b2c_weight_pack_dgrad(net->ctx, net->segs.data(), (int)net->segs.size(), net->w_bf16, net->w_dgrad, stream);
+}
+
+b2c_status b2c_net_sync_weights(b2c_net* net, void* stream)
+{
+    if (!net || !net->ws) return B2C_ERR_INVALID_ARG;
+    // lr = 0, momentum = 1, wd = 0, zero gradient scale: leaves w and v untouched and writes the bf16 copy
+    b2c_status st = b2c_grad_accum_sgd_momentum(net->ctx, net->param_count, net->w, net->v, net->g, 0.f, 0.f, 1.f, 0.f, net->w_bf16, 0, stream);
+    if (st != B2C_OK) return st;
+    return net_pack_dgrad(net, stream);
+}
+
+#define B2C_TRY(call)                   \
+    do {                                \
+        b2c_status s_ = (call);         \
+        if (s_ != B2C_OK) return s_;    \
+    } while (0)
+
+b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* labels, int n_micro, float lr, float momentum, float wd,
+                          float* loss_dev, int update, void* stream_)
+{
+    if (!net || !net->ws || !images || !labels || !loss_dev || n_micro < 1) return B2C_ERR_INVALID_ARG;
+    if (!b2c_aligned16(images)) return B2C_ERR_MISALIGNED;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    b2c_ctx* ctx = net->ctx;
+    const int N = net->micro_batch;
+    const int n_layers = (int)net->layers.size();
+    const __nv_bfloat16* w_bf16 = reinterpret_cast<const __nv_bfloat16*>(net->w_bf16);
+    const __nv_bfloat16* w_dg = reinterpret_cast<const __nv_bfloat16*>(net->w_dgrad);
+    auto act = [&](int t) -> void* { return net->ws + net->tensors[t].act_off; };
+    auto grad = [&](int t, int slot) -> void* { return slot >= 0 && net->tensors[t].grad_off[slot] >= 0 ? net->ws + net->tensors[t].grad_off[slot] : nullptr; };
+
+    B2C_CUDA(cudaMemsetAsync(loss_dev, 0, sizeof(float), stream));
+    const size_t image_bytes = (size_t)N * net->image_h * net->image_w * net->image_c * 2;
+    if (image_bytes % 16) return B2C_ERR_MISALIGNED;
+
+    for (int mb = 0; mb < n_micro; ++mb) {
+        const char* img = reinterpret_cast<const char*>(images) + (size_t)mb * image_bytes;
+        const int32_t* lab = labels + (size_t)mb * N;
+        const void* t0;
+        if (net->tensors[0].act_off >= 0) {
+            B2C_TRY(b2c_pad_channels(ctx, (long)N * net->image_h * net->image_w, net->image_c, net->image_c_pad, img, act(0), stream));
+            t0 = act(0);
+        } else {
+            t0 = img;
+        }
+        auto act_in = [&](int t) -> const void* { return t == 0 ? t0 : act(t); };
+        B2C_CUDA(cudaMemsetAsync(net->ws + net->stats_begin, 0, (size_t)(net->stats_end - net->stats_begin), stream));
+
+        // ---------------- forward pass and loss
+        for (int i = 0; i < n_layers; ++i) {
+            const LayerPlan& L = net->layers[i];
+            const b2c_layer_desc& d = L.d;
+            const TensorPlan& o = net->tensors[i + 1];
+            switch (d.kind) {
+                case B2C_LAYER_CONV: {
+                    KMajorProblem pb{};
+                    pb.n = N; pb.ih = d.h; pb.iw = d.w; pb.ic = L.c_pad; pb.oh = L.p; pb.ow = L.q; pb.oc = d.k;
+                    pb.r = d.r; pb.stride = d.stride; pb.pad = (d.r - 1) / 2; pb.dgrad = false;
+                    pb.in = act_in(d.src); pb.wt = w_bf16 + L.w_off; pb.out = act(i + 1);
+                    pb.stats = net->fuse_stats ? reinterpret_cast<double*>(net->ws + o.stats_off) : nullptr;
+                    B2C_TRY(launch_conv_kmajor(ctx, pb, stream));
+                    break;
+                }
+                case B2C_LAYER_BN: {
+                    const TensorPlan& in = net->tensors[d.src];
+                    const bool ready = net->fuse_stats && in.stats_off >= 0;
+                    double* stats = reinterpret_cast<double*>(net->ws + (in.stats_off >= 0 ? in.stats_off : L.bwd_ws_off));
+                    B2C_TRY(b2c_bn_relu_fwd(ctx, N, in.h, in.w, in.c, act(d.src), stats, ready ? 1 : 0, net->w + L.gamma_off, net->w + L.beta_off,
+                                            d.res >= 0 ? act(d.res) : nullptr, d.relu, 1e-5f, act(i + 1),
+                                            reinterpret_cast<float*>(net->ws + L.mean_off), reinterpret_cast<float*>(net->ws + L.invstd_off),
+                                            nullptr, nullptr, 0.f, stream));
+                    break;
+                }
+                case B2C_LAYER_AVGPOOL: {
+                    const TensorPlan& in = net->tensors[d.src];
+                    B2C_TRY(b2c_avgpool_fwd(ctx, N, in.h * in.w, in.c, act(d.src), act(i + 1), stream));
+                    break;
+                }
+                case B2C_LAYER_FC: {
+                    KMajorProblem pb{};
+                    pb.n = N; pb.ih = 1; pb.iw = 1; pb.ic = L.c_pad; pb.oh = 1; pb.ow = 1; pb.oc = L.k_pad;
+                    pb.r = 1; pb.stride = 1; pb.pad = 0; pb.dgrad = false;
+                    pb.in = act(d.src); pb.wt = w_bf16 + L.w_off; pb.out = act(i + 1);
+                    pb.out_f32 = true; pb.bias = net->w + L.bias_off;
+                    B2C_TRY(launch_conv_kmajor(ctx, pb, stream));
+                    break;
+                }
+                case B2C_LAYER_XENT: {
+                    const TensorPlan& in = net->tensors[d.src];
+                    B2C_TRY(b2c_softmax_xent_fwd_bwd(ctx, N, d.k, reinterpret_cast<const float*>(act(d.src)), in.c, lab,
+                                                     1.f / ((float)N * (float)n_micro), 1.f / (float)N, loss_dev, grad(d.src, L.src_slot), in.c,
+                                                     stream));
+                    break;
+                }
+            }
+        }
+        // ---------------- backward pass, gradients summed into the flat gradient array
+        for (int i = n_layers - 1; i >= 0; --i) {
+            const LayerPlan& L = net->layers[i];
+            const b2c_layer_desc& d = L.d;
+            const TensorPlan& o = net->tensors[i + 1];
+            switch (d.kind) {
+                case B2C_LAYER_XENT: break;
+                case B2C_LAYER_FC: {
+                    const void* dz = grad(i + 1, 0);
+                    WgradProblem wp{};
+                    wp.n = N; wp.h = 1; wp.w = 1; wp.c = L.c_pad; wp.p = 1; wp.q = 1; wp.k = L.k_pad; wp.r = 1; wp.stride = 1; wp.pad = 0;
+                    wp.dy = dz; wp.x = act(d.src); wp.dw = net->g + L.w_off;
+                    B2C_TRY(launch_conv_wgrad(ctx, wp, stream));
+                    B2C_TRY(b2c_bias_grad(ctx, N, L.k_pad, L.k_pad, dz, net->g + L.bias_off, 1, stream));
+                    KMajorProblem pb{};
+                    pb.n = N; pb.ih = 1; pb.iw = 1; pb.ic = L.k_pad; pb.oh = 1; pb.ow = 1; pb.oc = L.c_pad;
+                    pb.r = 1; pb.stride = 1; pb.pad = 0; pb.dgrad = true;
+                    pb.in = dz; pb.wt = w_dg + L.w_off; pb.out = grad(d.src, L.src_slot);
+                    B2C_TRY(launch_conv_kmajor(ctx, pb, stream));
+                    break;
+                }
+                case B2C_LAYER_AVGPOOL: {
+                    const TensorPlan& in = net->tensors[d.src];
+                    B2C_TRY(b2c_avgpool_bwd(ctx, N, in.h * in.w, in.c, grad(i + 1, 0), grad(d.src, L.src_slot), stream));
+                    break;
+                }
+                case B2C_LAYER_BN: {
+                    const TensorPlan& in = net->tensors[d.src];
+                    B2C_TRY(b2c_bn_relu_bwd(ctx, N, in.h, in.w, in.c, grad(i + 1, 0), o.n_contrib > 1 ? grad(i + 1, 1) : nullptr, act(d.src), act(i + 1),
+                                            net->w + L.gamma_off, reinterpret_cast<float*>(net->ws + L.mean_off),
+                                            reinterpret_cast<float*>(net->ws + L.invstd_off), d.relu, grad(d.src, L.src_slot),
+                                            d.res >= 0 ? grad(d.res, L.res_slot) : nullptr, net->g + L.gamma_off, net->g + L.beta_off, 1,
+                                            net->ws + L.bwd_ws_off, b2c_bn_relu_bwd_workspace_bytes(in.c), stream));
+                    break;
+                }
+                case B2C_LAYER_CONV: {
+                    const void* dy = grad(i + 1, 0);
+                    WgradProblem wp{};
+                    wp.n = N; wp.h = d.h; wp.w = d.w; wp.c = L.c_pad; wp.p = L.p; wp.q = L.q; wp.k = d.k;
+                    wp.r = d.r; wp.stride = d.stride; wp.pad = (d.r - 1) / 2;
+                    wp.dy = dy; wp.x = act_in(d.src); wp.dw = net->g + L.w_off;
+                    B2C_TRY(launch_conv_wgrad(ctx, wp, stream));
+                    if (d.src != 0) {
+                        KMajorProblem pb{};
+                        pb.n = N; pb.ih = L.p; pb.iw = L.q; pb.ic = d.k; pb.oh = d.h; pb.ow = d.w; pb.oc = L.c_pad;
+                        pb.r = d.r; pb.stride = d.stride; pb.pad = (d.r - 1) / 2; pb.dgrad = true;
+                        pb.in = dy; pb.wt = w_dg + L.w_off; pb.out = grad(d.src, L.src_slot);
+                        B2C_TRY(launch_conv_kmajor(ctx, pb, stream));
+                    }
+                    break;
+                }
+            }
+        }
+    }
+    // ---------------- gradient average + parameter update, refresh of both bf16 weight copies
+    if (update) {
+        B2C_TRY(b2c_grad_accum_sgd_momentum(ctx, net->param_count, net->w, net->v, net->g, 1.f / (float)n_micro, lr, momentum, wd, net->w_bf16, 1,
+                                            stream));
+        B2C_TRY(net_pack_dgrad(net, stream));
+    }
+    return B2C_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,79 @@
+// Host-side shared declarations of the library: context, status helpers, kernel launchers.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/b2c.h"
+
+// Bits of the sticky device status word.
+#define B2C_DEV_TIMEOUT 1u
+#define B2C_DEV_BAD_LABEL 2u
+
+typedef CUresult (*b2c_encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                        const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                        CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct b2c_ctx {
+    int device;
+    int sm_count;
+    unsigned* d_status;  // one device word
+    unsigned spin_limit;
+    b2c_encode_tiled_fn encode_tiled;
+};
+
+#define B2C_CUDA(call)                               \
+    do {                                             \
+        cudaError_t e_ = (call);                     \
+        if (e_ != cudaSuccess) return B2C_ERR_CUDA;  \
+    } while (0)
+
+static inline bool b2c_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static inline bool b2c_is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
+
+namespace b2c {
+
+// Filter taps of one launch: which tensor map (parity view) a tap gathers from, its pixel
+// offset inside that view, and its index in the weight tensor's tap dimension.
+struct TapList {
+    int count;
+    int8_t map[9], dh[9], dw[9], rs[9];
+};
+
+// bf16 activation tensor [n][h][w][c] as a 4-D tensor map (c, w/step, h/step, n); step 2 selects
+// rows of parity ph and columns of parity pw.  Box = (box_c, box_w, box_h, box_n); swizzle = box_c*2 bytes.
+bool encode_activation_map(b2c_ctx* ctx, CUtensorMap* tm, const void* base, int n, int h, int w, int c, int step, int ph, int pw, int box_c,
+                           int box_w, int box_h, int box_n);
+// Taps of a forward convolution in terms of (parity view, offset): input row = p*stride + r - pad.
+void forward_taps(TapList& tl, int R, int stride, int pad);
+
+// Geometry of one implicit-GEMM launch with K-major operands (forward and data gradient):
+// the "input" is the activation tensor that is gathered (x for fprop, dy for dgrad), the
+// "output" the tensor that is written.  in_pitch / out_pitch are channel strides in elements.
+struct KMajorProblem {
+    int n;                 // images
+    int ih, iw, ic;        // gathered tensor
+    int oh, ow, oc;        // written tensor
+    int r, stride, pad;    // filter taps (r x r), forward stride and padding of the convolution
+    bool dgrad;            // false: forward; true: data gradient (input = dy, weights in [c,r,s,k] flipped layout)
+    const void* in;
+    const void* wt;        // [oc][r*r][ic] bf16
+    void* out;
+    bool out_f32;
+    const float* bias;
+    double* stats;
+};
+b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_t stream);
+
+struct WgradProblem {
+    int n, h, w, c;        // x
+    int p, q, k;           // dy
+    int r, stride, pad;
+    const void* dy;
+    const void* x;
+    float* dw;             // [k][r*r][c] fp32, accumulated into
+};
+b2c_status launch_conv_wgrad(b2c_ctx* ctx, const WgradProblem& pb, cudaStream_t stream);
+
+}  // namespace b2c

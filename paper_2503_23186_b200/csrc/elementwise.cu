@@ -1,0 +1,530 @@
+// HBM-bound kernels of the training step: BatchNorm(+residual)+ReLU forward and backward,
+// global average pool, softmax cross-entropy, bias gradient, the fused gradient-average +
+// SGD-momentum update, channel padding and the dgrad weight re-layout.
+//
+// Access pattern common to the BatchNorm kernels: the tensor is [m rows][c channels] bf16 with
+// channels contiguous; a thread owns 8 consecutive channels (one 16-byte vector) and walks rows
+// with a grid stride, so a warp reads whole 128-byte lines and per-channel reductions stay in
+// registers until the end of the walk.  Row sums are combined in shared memory, then added to
+// global fp64 accumulators (fp32 partials over few rows, fp64 across them: var = E[y^2] - E[y]^2
+// stays accurate for channels whose mean is large against their spread).
+#include "common.h"
+#include "ptx.cuh"
+
+namespace b2c {
+
+static constexpr int kEwThreads = 256;
+
+struct bf16x8 {
+    uint4 raw;
+};
+__device__ __forceinline__ void unpack8(const uint4& u, float (&f)[8])
+{
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        f[2 * i] = __low2float(h[i]);
+        f[2 * i + 1] = __high2float(h[i]);
+    }
+}
+__device__ __forceinline__ uint4 pack8(const float (&f)[8])
+{
+    return make_uint4(pack_bf16x2(f[0], f[1]), pack_bf16x2(f[2], f[3]), pack_bf16x2(f[4], f[5]), pack_bf16x2(f[6], f[7]));
+}
+__device__ __forceinline__ uint4 ld16(const void* base, long long vec_index) { return __ldg(reinterpret_cast<const uint4*>(base) + vec_index); }
+
+// Row/channel-group decomposition shared by the row-walking kernels.
+struct RowWalk {
+    int groups;         // c / 8
+    int rows_per_iter;  // rows a block covers per step
+    __device__ RowWalk(int c) : groups(c >> 3), rows_per_iter(kEwThreads / (c >> 3)) {}
+};
+
+// ------------------------------------------------------------------------------ BN forward
+__global__ void __launch_bounds__(kEwThreads) bn_stats_kernel(const void* __restrict__ y, long long m, int c, double* __restrict__ stats)
+{
+    extern __shared__ float s_acc[];  // [2*c]
+    for (int i = threadIdx.x; i < 2 * c; i += kEwThreads) s_acc[i] = 0.f;
+    __syncthreads();
+    const RowWalk rw(c);
+    const int g = threadIdx.x % rw.groups, rl = threadIdx.x / rw.groups;
+    if (rl < rw.rows_per_iter) {
+        float s[8], ss[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) s[i] = ss[i] = 0.f;
+        const long long step = (long long)gridDim.x * rw.rows_per_iter;
+        for (long long r = (long long)blockIdx.x * rw.rows_per_iter + rl; r < m; r += step) {
+            float f[8];
+            unpack8(ld16(y, r * rw.groups + g), f);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                s[i] += f[i];
+                ss[i] = fmaf(f[i], f[i], ss[i]);
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            atomicAdd(&s_acc[g * 8 + i], s[i]);
+            atomicAdd(&s_acc[c + g * 8 + i], ss[i]);
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < 2 * c; i += kEwThreads) atomicAdd(stats + i, (double)s_acc[i]);
+}
+
+// mean and 1/sqrt(var+eps) from the fp64 sums, identically in every thread that needs them.
+__device__ __forceinline__ void bn_moments(const double* stats, int c, int ch, double inv_m, float eps, float& mean, float& invstd, float& var)
+{
+    const double mu = stats[ch] * inv_m;
+    double v = stats[c + ch] * inv_m - mu * mu;
+    v = v < 0.0 ? 0.0 : v;
+    mean = (float)mu;
+    var = (float)v;
+    invstd = rsqrtf((float)v + eps);
+}
+
+__global__ void __launch_bounds__(kEwThreads) bn_apply_kernel(const void* __restrict__ y, long long m, int c, const double* __restrict__ stats,
+                                                              const float* __restrict__ gamma, const float* __restrict__ beta,
+                                                              const void* __restrict__ residual, int relu, float eps, void* __restrict__ a,
+                                                              float* save_mean, float* save_invstd, float* run_mean, float* run_var,
+                                                              float momentum)
+{
+    const RowWalk rw(c);
+    const int g = threadIdx.x % rw.groups, rl = threadIdx.x / rw.groups;
+    const double inv_m = 1.0 / (double)m;
+    if (blockIdx.x == 0) {
+        for (int ch = threadIdx.x; ch < c; ch += kEwThreads) {
+            float mean, invstd, var;
+            bn_moments(stats, c, ch, inv_m, eps, mean, invstd, var);
+            save_mean[ch] = mean;
+            save_invstd[ch] = invstd;
+            if (run_mean != nullptr) {
+                const float unbiased = m > 1 ? var * (float)((double)m / (double)(m - 1)) : var;
+                run_mean[ch] = (1.f - momentum) * run_mean[ch] + momentum * mean;
+                run_var[ch] = (1.f - momentum) * run_var[ch] + momentum * unbiased;
+            }
+        }
+    }
+    if (rl >= rw.rows_per_iter) return;
+    float scale[8], shift[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        float mean, invstd, var;
+        bn_moments(stats, c, g * 8 + i, inv_m, eps, mean, invstd, var);
+        const float gm = gamma[g * 8 + i];
+        // z = gamma*(y-mean)*invstd + beta, evaluated as (y-mean)*(gamma*invstd) + beta
+        scale[i] = gm * invstd;
+        shift[i] = mean;
+    }
+    float bt[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) bt[i] = beta[g * 8 + i];
+    const long long step = (long long)gridDim.x * rw.rows_per_iter;
+    for (long long r = (long long)blockIdx.x * rw.rows_per_iter + rl; r < m; r += step) {
+        const long long vi = r * rw.groups + g;
+        float f[8], res[8];
+        unpack8(ld16(y, vi), f);
+        if (residual != nullptr) unpack8(ld16(residual, vi), res);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            float z = fmaf(f[i] - shift[i], scale[i], bt[i]);
+            if (residual != nullptr) z += res[i];
+            f[i] = (relu && z < 0.f) ? 0.f : z;
+        }
+        reinterpret_cast<uint4*>(a)[vi] = pack8(f);
+    }
+}
+
+// ------------------------------------------------------------------------------ BN backward
+__global__ void __launch_bounds__(kEwThreads) bn_bwd_reduce_kernel(const void* __restrict__ da1, const void* __restrict__ da2,
+                                                                   const void* __restrict__ y, const void* __restrict__ a, long long m, int c,
+                                                                   const float* __restrict__ mean, const float* __restrict__ invstd, int relu,
+                                                                   double* __restrict__ sums /* [2c]: dbeta, dgamma */)
+{
+    extern __shared__ float s_acc[];
+    for (int i = threadIdx.x; i < 2 * c; i += kEwThreads) s_acc[i] = 0.f;
+    __syncthreads();
+    const RowWalk rw(c);
+    const int g = threadIdx.x % rw.groups, rl = threadIdx.x / rw.groups;
+    if (rl < rw.rows_per_iter) {
+        float mu[8], is[8], sb[8], sg[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            mu[i] = mean[g * 8 + i];
+            is[i] = invstd[g * 8 + i];
+            sb[i] = sg[i] = 0.f;
+        }
+        const long long step = (long long)gridDim.x * rw.rows_per_iter;
+        for (long long r = (long long)blockIdx.x * rw.rows_per_iter + rl; r < m; r += step) {
+            const long long vi = r * rw.groups + g;
+            float d[8], d2[8], fy[8], fa[8];
+            unpack8(ld16(da1, vi), d);
+            if (da2 != nullptr) unpack8(ld16(da2, vi), d2);
+            unpack8(ld16(y, vi), fy);
+            if (relu) unpack8(ld16(a, vi), fa);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                float dz = d[i];
+                if (da2 != nullptr) dz += d2[i];
+                if (relu && !(fa[i] > 0.f)) dz = 0.f;
+                sb[i] += dz;
+                sg[i] = fmaf(dz, (fy[i] - mu[i]) * is[i], sg[i]);
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            atomicAdd(&s_acc[g * 8 + i], sb[i]);
+            atomicAdd(&s_acc[c + g * 8 + i], sg[i]);
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < 2 * c; i += kEwThreads) atomicAdd(sums + i, (double)s_acc[i]);
+}
+
+__global__ void __launch_bounds__(kEwThreads) bn_bwd_apply_kernel(const void* __restrict__ da1, const void* __restrict__ da2,
+                                                                  const void* __restrict__ y, const void* __restrict__ a, long long m, int c,
+                                                                  const float* __restrict__ gamma, const float* __restrict__ mean,
+                                                                  const float* __restrict__ invstd, int relu, const double* __restrict__ sums,
+                                                                  void* __restrict__ dy, void* __restrict__ dres, float* dgamma, float* dbeta,
+                                                                  int acc)
+{
+    const RowWalk rw(c);
+    const int g = threadIdx.x % rw.groups, rl = threadIdx.x / rw.groups;
+    if (blockIdx.x == 0) {
+        for (int ch = threadIdx.x; ch < c; ch += kEwThreads) {
+            const float db = (float)sums[ch], dg = (float)sums[c + ch];
+            dbeta[ch] = acc ? dbeta[ch] + db : db;
+            dgamma[ch] = acc ? dgamma[ch] + dg : dg;
+        }
+    }
+    if (rl >= rw.rows_per_iter) return;
+    const float inv_m = (float)(1.0 / (double)m);
+    float mu[8], is[8], k0[8], kb[8], kg[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int ch = g * 8 + i;
+        mu[i] = mean[ch];
+        is[i] = invstd[ch];
+        k0[i] = gamma[ch] * is[i];                 // gamma*invstd
+        kb[i] = (float)(sums[ch]) * inv_m;         // dbeta/m
+        kg[i] = (float)(sums[c + ch]) * inv_m;     // dgamma/m
+    }
+    const long long step = (long long)gridDim.x * rw.rows_per_iter;
+    for (long long r = (long long)blockIdx.x * rw.rows_per_iter + rl; r < m; r += step) {
+        const long long vi = r * rw.groups + g;
+        float d[8], d2[8], fy[8], fa[8], o[8];
+        unpack8(ld16(da1, vi), d);
+        if (da2 != nullptr) unpack8(ld16(da2, vi), d2);
+        unpack8(ld16(y, vi), fy);
+        if (relu) unpack8(ld16(a, vi), fa);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            float dz = d[i];
+            if (da2 != nullptr) dz += d2[i];
+            if (relu && !(fa[i] > 0.f)) dz = 0.f;
+            d[i] = dz;
+            const float xhat = (fy[i] - mu[i]) * is[i];
+            o[i] = k0[i] * (dz - kb[i] - xhat * kg[i]);
+        }
+        reinterpret_cast<uint4*>(dy)[vi] = pack8(o);
+        if (dres != nullptr) reinterpret_cast<uint4*>(dres)[vi] = pack8(d);
+    }
+}
+
+// ------------------------------------------------------------------------------ pooling, padding
+__global__ void avgpool_fwd_kernel(const void* __restrict__ a, int n, int hw, int c, void* __restrict__ pooled)
+{
+    const int groups = c >> 3;
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (long long)n * groups) return;
+    const int g = (int)(idx % groups);
+    const long long img = idx / groups;
+    float s[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) s[i] = 0.f;
+    for (int j = 0; j < hw; ++j) {
+        float f[8];
+        unpack8(ld16(a, (img * hw + j) * groups + g), f);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) s[i] += f[i];
+    }
+    const float inv = 1.f / (float)hw;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) s[i] *= inv;
+    reinterpret_cast<uint4*>(pooled)[idx] = pack8(s);
+}
+
+__global__ void avgpool_bwd_kernel(const void* __restrict__ dpooled, int n, int hw, int c, void* __restrict__ da)
+{
+    const int groups = c >> 3;
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (long long)n * hw * groups) return;
+    const int g = (int)(idx % groups);
+    const long long img = idx / ((long long)groups * hw);
+    float f[8];
+    unpack8(ld16(dpooled, img * groups + g), f);
+    const float inv = 1.f / (float)hw;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) f[i] *= inv;
+    reinterpret_cast<uint4*>(da)[idx] = pack8(f);
+}
+
+__global__ void pad_channels_kernel(const __nv_bfloat16* __restrict__ x, long long m, int c_in, int c_out, void* __restrict__ y)
+{
+    const int groups = c_out >> 3;
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= m * groups) return;
+    const int g = (int)(idx % groups);
+    const long long row = idx / groups;
+    float f[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int ch = g * 8 + i;
+        f[i] = ch < c_in ? __bfloat162float(x[row * c_in + ch]) : 0.f;
+    }
+    reinterpret_cast<uint4*>(y)[idx] = pack8(f);
+}
+
+// ------------------------------------------------------------------------------ loss
+// One warp per row.
+__global__ void softmax_xent_kernel(const float* __restrict__ logits, int logits_pitch, const int32_t* __restrict__ labels, int n, int classes,
+                                    float loss_scale, float grad_scale, float* loss, __nv_bfloat16* __restrict__ dlogits, int pitch,
+                                    unsigned* status)
+{
+    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (row >= n) return;
+    const float* z = logits + (long long)row * logits_pitch;
+    const int label = labels[row];
+    const bool bad = label < 0 || label >= classes;
+    float mx = -INFINITY;
+    for (int j = lane; j < classes; j += 32) mx = fmaxf(mx, z[j]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    float se = 0.f;
+    for (int j = lane; j < classes; j += 32) se += expf(z[j] - mx);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) se += __shfl_xor_sync(0xffffffffu, se, o);
+    const float lse = mx + logf(se);
+    if (lane == 0) {
+        if (bad)
+            atomicOr(status, B2C_DEV_BAD_LABEL);
+        else
+            atomicAdd(loss, loss_scale * (lse - z[label]));
+    }
+    __nv_bfloat16* d = dlogits + (long long)row * pitch;
+    for (int j = lane; j < pitch; j += 32) {
+        float gval = 0.f;
+        if (j < classes && !bad) gval = (expf(z[j] - lse) - (j == label ? 1.f : 0.f)) * grad_scale;
+        d[j] = __float2bfloat16_rn(gval);
+    }
+}
+
+__global__ void bias_grad_kernel(const __nv_bfloat16* __restrict__ dz, int m, int k, int pitch, float* db, int accumulate)
+{
+    const int ch = blockIdx.x * blockDim.x + threadIdx.x;
+    if (ch >= k) return;
+    float s = 0.f;
+    for (int r = 0; r < m; ++r) s += __bfloat162float(dz[(long long)r * pitch + ch]);
+    db[ch] = accumulate ? db[ch] + s : s;
+}
+
+// ------------------------------------------------------------------------------ update
+__global__ void __launch_bounds__(kEwThreads) sgd_momentum_kernel(float4* __restrict__ w, float4* __restrict__ v, float4* __restrict__ gsum,
+                                                                  long long count4, float inv_n, float lr, float mu, float wd,
+                                                                  uint2* __restrict__ w_bf16, int zero_grad)
+{
+    const long long step = (long long)gridDim.x * blockDim.x;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < count4; i += step) {
+        float4 wi = w[i], vi = v[i];
+        const float4 gi = gsum[i];
+        float* pw = reinterpret_cast<float*>(&wi);
+        float* pv = reinterpret_cast<float*>(&vi);
+        const float* pg = reinterpret_cast<const float*>(&gi);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float g = fmaf(wd, pw[j], pg[j] * inv_n);   // g = g_sum*inv_n + wd*w
+            pv[j] = fmaf(mu, pv[j], g);                      // v = mu*v + g
+            pw[j] = fmaf(-lr, pv[j], pw[j]);                 // w = w - lr*v
+        }
+        w[i] = wi;
+        v[i] = vi;
+        if (zero_grad) gsum[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (w_bf16 != nullptr) w_bf16[i] = make_uint2(pack_bf16x2(pw[0], pw[1]), pack_bf16x2(pw[2], pw[3]));
+    }
+}
+
+struct PackSegs {
+    b2c_weight_seg seg[128];
+};
+__global__ void weight_pack_dgrad_kernel(const __grid_constant__ PackSegs segs, const __nv_bfloat16* __restrict__ src,
+                                         __nv_bfloat16* __restrict__ dst)
+{
+    const b2c_weight_seg sg = segs.seg[blockIdx.y];
+    const long long total = (long long)sg.k * sg.rs * sg.c;
+    const long long j = (long long)blockIdx.x * blockDim.x + threadIdx.x;   // destination index: [c][t][k]
+    if (j >= total) return;
+    const int k = (int)(j % sg.k);
+    const int t = (int)((j / sg.k) % sg.rs);
+    const int c = (int)(j / ((long long)sg.k * sg.rs));
+    dst[sg.offset + j] = src[sg.offset + ((long long)k * sg.rs + (sg.rs - 1 - t)) * sg.c + c];
+}
+
+// ------------------------------------------------------------------------------ launchers
+static int ew_grid(b2c_ctx* ctx, long long m, int rows_per_iter)
+{
+    long long blocks = (m + rows_per_iter - 1) / rows_per_iter;
+    const long long cap = (long long)ctx->sm_count * 8;
+    return (int)(blocks < cap ? (blocks < 1 ? 1 : blocks) : cap);
+}
+
+}  // namespace b2c
+
+using namespace b2c;
+
+extern "C" {
+
+b2c_status b2c_bn_relu_fwd(b2c_ctx* ctx, int n, int h, int w, int c, const void* y, double* ch_stats, int stats_ready, const float* gamma,
+                           const float* beta, const void* residual, int relu, float eps, void* a, float* save_mean, float* save_invstd,
+                           float* run_mean, float* run_var, float momentum, void* stream_)
+{
+    cudaStream_t stream = (cudaStream_t)stream_;
+    if (!ctx || !y || !ch_stats || !gamma || !beta || !a || !save_mean || !save_invstd) return B2C_ERR_INVALID_ARG;
+    if (n < 1 || h < 1 || w < 1 || c < 8 || c % 8 || c > 2048) return B2C_ERR_UNSUPPORTED_SHAPE;
+    if ((run_mean == nullptr) != (run_var == nullptr)) return B2C_ERR_INVALID_ARG;
+    if (!b2c_aligned16(y) || !b2c_aligned16(a) || (residual && !b2c_aligned16(residual)) || (reinterpret_cast<uintptr_t>(ch_stats) & 7u))
+        return B2C_ERR_MISALIGNED;
+    const long long m = (long long)n * h * w;
+    const int rows_per_iter = kEwThreads / (c / 8);
+    const int grid = ew_grid(ctx, m, rows_per_iter);
+    if (!stats_ready) {
+        B2C_CUDA(cudaMemsetAsync(ch_stats, 0, sizeof(double) * 2 * c, stream));
+        bn_stats_kernel<<<grid, kEwThreads, sizeof(float) * 2 * c, stream>>>(y, m, c, ch_stats);
+    }
+    bn_apply_kernel<<<grid, kEwThreads, 0, stream>>>(y, m, c, ch_stats, gamma, beta, residual, relu, eps, a, save_mean, save_invstd, run_mean,
+                                                     run_var, momentum);
+    B2C_CUDA(cudaGetLastError());
+    return B2C_OK;
+}
+
+size_t b2c_bn_relu_bwd_workspace_bytes(int c) { return c > 0 ? sizeof(double) * 2 * (size_t)c : 0; }
+
+b2c_status b2c_bn_relu_bwd(b2c_ctx* ctx, int n, int h, int w, int c, const void* da1, const void* da2, const void* y, const void* a,
+                           const float* gamma, const float* save_mean, const float* save_invstd, int relu, void* dy, void* dres, float* dgamma,
+                           float* dbeta, int acc, void* ws, size_t ws_bytes, void* stream_)
+{
+    cudaStream_t stream = (cudaStream_t)stream_;
+    if (!ctx || !da1 || !y || !gamma || !save_mean || !save_invstd || !dy || !dgamma || !dbeta || !ws) return B2C_ERR_INVALID_ARG;
+    if (relu && !a) return B2C_ERR_INVALID_ARG;
+    if (n < 1 || h < 1 || w < 1 || c < 8 || c % 8 || c > 2048) return B2C_ERR_UNSUPPORTED_SHAPE;
+    if (ws_bytes < b2c_bn_relu_bwd_workspace_bytes(c)) return B2C_ERR_WORKSPACE_TOO_SMALL;
+    if (!b2c_aligned16(da1) || (da2 && !b2c_aligned16(da2)) || !b2c_aligned16(y) || (a && !b2c_aligned16(a)) || !b2c_aligned16(dy) ||
+        (dres && !b2c_aligned16(dres)) || (reinterpret_cast<uintptr_t>(ws) & 7u))
+        return B2C_ERR_MISALIGNED;
+    const long long m = (long long)n * h * w;
+    const int rows_per_iter = kEwThreads / (c / 8);
+    const int grid = ew_grid(ctx, m, rows_per_iter);
+    double* sums = reinterpret_cast<double*>(ws);
+    B2C_CUDA(cudaMemsetAsync(sums, 0, sizeof(double) * 2 * c, stream));
+    bn_bwd_reduce_kernel<<<grid, kEwThreads, sizeof(float) * 2 * c, stream>>>(da1, da2, y, a, m, c, save_mean, save_invstd, relu, sums);
+    bn_bwd_apply_kernel<<<grid, kEwThreads, 0, stream>>>(da1, da2, y, a, m, c, gamma, save_mean, save_invstd, relu, sums, dy, dres, dgamma, dbeta,
+                                                         acc);
+    B2C_CUDA(cudaGetLastError());
+    return B2C_OK;
+}
+
+b2c_status b2c_avgpool_fwd(b2c_ctx* ctx, int n, int hw, int c, const void* a, void* pooled, void* stream_)
+{
+    if (!ctx || !a || !pooled) return B2C_ERR_INVALID_ARG;
+    if (n < 1 || hw < 1 || c < 8 || c % 8) return B2C_ERR_UNSUPPORTED_SHAPE;
+    if (!b2c_aligned16(a) || !b2c_aligned16(pooled)) return B2C_ERR_MISALIGNED;
+    const long long total = (long long)n * (c / 8);
+    avgpool_fwd_kernel<<<(unsigned)((total + 127) / 128), 128, 0, (cudaStream_t)stream_>>>(a, n, hw, c, pooled);
+    B2C_CUDA(cudaGetLastError());
+    return B2C_OK;
+}
+
+b2c_status b2c_avgpool_bwd(b2c_ctx* ctx, int n, int hw, int c, const void* dpooled, void* da, void* stream_)
+{
+    if (!ctx || !dpooled || !da) return B2C_ERR_INVALID_ARG;
+    if (n < 1 || hw < 1 || c < 8 || c % 8) return B2C_ERR_UNSUPPORTED_SHAPE;
+    if (!b2c_aligned16(dpooled) || !b2c_aligned16(da)) return B2C_ERR_MISALIGNED;
+    const long long total = (long long)n * hw * (c / 8);
+    avgpool_bwd_kernel<<<(unsigned)((total + 255) / 256), 256, 0, (cudaStream_t)stream_>>>(dpooled, n, hw, c, da);
+    B2C_CUDA(cudaGetLastError());
+    return B2C_OK;
+}
+
+b2c_status b2c_pad_channels(b2c_ctx* ctx, long m, int c_in, int c_out, const void* x, void* y, void* stream_)
+{
+    if (!ctx || !x || !y) return B2C_ERR_INVALID_ARG;
+    if (m < 1 || c_in < 1 || c_out < c_in || c_out % 8) return B2C_ERR_UNSUPPORTED_SHAPE;
+    if (!b2c_aligned16(y) || (reinterpret_cast<uintptr_t>(x) & 1u)) return B2C_ERR_MISALIGNED;
+    const long long total = (long long)m * (c_out / 8);
+    pad_channels_kernel<<<(unsigned)((total + 255) / 256), 256, 0, (cudaStream_t)stream_>>>(reinterpret_cast<const __nv_bfloat16*>(x), m, c_in,
+                                                                                            c_out, y);
+    B2C_CUDA(cudaGetLastError());
+    return B2C_OK;
+}
+
+b2c_status b2c_softmax_xent_fwd_bwd(b2c_ctx* ctx, int n, int classes, const float* logits, int logits_pitch, const int32_t* labels,
+                                    float loss_scale, float grad_scale, float* loss, void* dlogits, int pitch, void* stream_)
+{
+    if (!ctx || !logits || !labels || !loss || !dlogits) return B2C_ERR_INVALID_ARG;
+    if (n < 1 || classes < 1 || logits_pitch < classes || pitch < classes || pitch % 8) return B2C_ERR_UNSUPPORTED_SHAPE;
+    if (!b2c_aligned16(dlogits)) return B2C_ERR_MISALIGNED;
+    const int warps = 4;
+    softmax_xent_kernel<<<(n + warps - 1) / warps, warps * 32, 0, (cudaStream_t)stream_>>>(logits, logits_pitch, labels, n, classes, loss_scale,
+                                                                                          grad_scale, loss, reinterpret_cast<__nv_bfloat16*>(dlogits),
+                                                                                          pitch, ctx->d_status);
+    B2C_CUDA(cudaGetLastError());
+    return B2C_OK;
+}
+
+b2c_status b2c_bias_grad(b2c_ctx* ctx, int m, int k, int pitch, const void* dz, float* db, int accumulate, void* stream_)
+{
+    if (!ctx || !dz || !db) return B2C_ERR_INVALID_ARG;
+    if (m < 1 || k < 1 || pitch < k) return B2C_ERR_UNSUPPORTED_SHAPE;
+    bias_grad_kernel<<<(k + 127) / 128, 128, 0, (cudaStream_t)stream_>>>(reinterpret_cast<const __nv_bfloat16*>(dz), m, k, pitch, db, accumulate);
+    B2C_CUDA(cudaGetLastError());
+    return B2C_OK;
+}
+
+b2c_status b2c_grad_accum_sgd_momentum(b2c_ctx* ctx, size_t count, float* w, float* v, float* g_accum, float inv_n_micro, float lr,
+                                       float momentum, float wd, void* w_bf16, int zero_grad, void* stream_)
+{
+    if (!ctx || !w || !v || !g_accum) return B2C_ERR_INVALID_ARG;
+    if (count == 0 || count % 4) return B2C_ERR_UNSUPPORTED_SHAPE;
+    if (!b2c_aligned16(w) || !b2c_aligned16(v) || !b2c_aligned16(g_accum) || (w_bf16 && (reinterpret_cast<uintptr_t>(w_bf16) & 7u)))
+        return B2C_ERR_MISALIGNED;
+    const long long count4 = (long long)(count / 4);
+    long long blocks = (count4 + kEwThreads - 1) / kEwThreads;
+    const long long cap = (long long)ctx->sm_count * 8;
+    if (blocks > cap) blocks = cap;
+    sgd_momentum_kernel<<<(unsigned)blocks, kEwThreads, 0, (cudaStream_t)stream_>>>(reinterpret_cast<float4*>(w), reinterpret_cast<float4*>(v),
+                                                                                   reinterpret_cast<float4*>(g_accum), count4, inv_n_micro, lr,
+                                                                                   momentum, wd, reinterpret_cast<uint2*>(w_bf16), zero_grad);
+    B2C_CUDA(cudaGetLastError());
+    return B2C_OK;
+}
+
+b2c_status b2c_weight_pack_dgrad(b2c_ctx* ctx, const b2c_weight_seg* segs, int n_segs, const void* src_bf16, void* dst_bf16, void* stream_)
+{
+    if (!ctx || !segs || !src_bf16 || !dst_bf16) return B2C_ERR_INVALID_ARG;
+    if (n_segs < 1 || n_segs > 128) return B2C_ERR_UNSUPPORTED_SHAPE;
+    PackSegs ps;
+    long long biggest = 0;
+    for (int i = 0; i < n_segs; ++i) {
+        if (segs[i].k < 1 || segs[i].rs < 1 || segs[i].c < 1 || segs[i].offset < 0) return B2C_ERR_INVALID_ARG;
+        ps.seg[i] = segs[i];
+        const long long sz = (long long)segs[i].k * segs[i].rs * segs[i].c;
+        biggest = sz > biggest ? sz : biggest;
+    }
+    dim3 grid((unsigned)((biggest + 255) / 256), (unsigned)n_segs);
+    weight_pack_dgrad_kernel<<<grid, 256, 0, (cudaStream_t)stream_>>>(ps, reinterpret_cast<const __nv_bfloat16*>(src_bf16),
+                                                                      reinterpret_cast<__nv_bfloat16*>(dst_bf16));
+    B2C_CUDA(cudaGetLastError());
+    return B2C_OK;
+}
+
+}  // extern "C"
