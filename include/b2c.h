@@ -206,6 +206,26 @@ b2c_status b2c_net_sync_weights(b2c_net* net, void* stream);
 b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* labels, int n_micro, float lr,
                           float momentum, float wd, float* loss_dev, int update, void* stream);
 
+/* The gradient synchronisation + update alone: g = grad_sum / n_avg + wd*w; v = momentum*v + g; w -= lr*v; both bf16
+ * weight copies are refreshed and grad_sum is zeroed.  Data-parallel replicas call b2c_train_step with update == 0,
+ * sum grad_sum across replicas (e.g. an NCCL all-reduce), then call this with n_avg = n_micro * replicas. */
+b2c_status b2c_net_apply_update(b2c_net* net, int n_avg, float lr, float momentum, float wd, void* stream);
+
+/* ---- Per-component timing (the profiling phase of the paper's adaptive scheduling algorithm
+ *      measures the execution time of each network component; this is the measurement hook) ---- */
+
+/* Kernel families a step's launches are attributed to. */
+enum {
+    B2C_PROF_CONV_FWD = 0, B2C_PROF_CONV_DGRAD = 1, B2C_PROF_CONV_WGRAD = 2, B2C_PROF_BN_FWD = 3, B2C_PROF_BN_BWD = 4,
+    B2C_PROF_OTHER = 5, B2C_PROF_UPDATE = 6, B2C_PROF_KINDS = 7
+};
+/* enable != 0: b2c_train_step brackets every launch site with CUDA events on its stream. */
+b2c_status b2c_net_profile_enable(b2c_net* net, int enable);
+/* Synchronises `stream`; ms[kind] = device time summed over the launch sites of that family since the
+ * last read (0 unless enabled), launches[kind] = kernels launched since the last read (always counted).
+ * Both arrays are HOST memory of B2C_PROF_KINDS entries.  Resets the sums. */
+b2c_status b2c_net_profile_read(b2c_net* net, double* ms, long long* launches, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

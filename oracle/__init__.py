@@ -18,8 +18,26 @@ import subprocess
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_SO = os.path.join(_HERE, "liboracle.so")
 _SRC = os.path.join(_HERE, "oracle.c")
+
+
+def _host_tag() -> str:
+    """The library is compiled with -march=native, so its file name carries a hash of this host's CPU flags:
+    a copy built on another machine is never loaded."""
+    import hashlib
+    flags = ""
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.startswith("flags"):
+                    flags = line
+                    break
+    except OSError:
+        pass
+    return hashlib.sha1(flags.encode()).hexdigest()[:10]
+
+
+_SO = os.path.join(_HERE, f"liboracle-{_host_tag()}.so")
 
 
 def build(force: bool = False) -> str:

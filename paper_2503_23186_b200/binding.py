@@ -29,8 +29,9 @@ EXPORTS = [
     "b2c_conv2d_wgrad", "b2c_bias_grad", "b2c_grad_accum_sgd_momentum", "b2c_weight_pack_dgrad",
     "b2c_net_create", "b2c_net_destroy", "b2c_net_param_count", "b2c_net_param_offset",
     "b2c_net_padded_image_channels", "b2c_net_workspace_bytes", "b2c_net_tensor_offset", "b2c_net_bind",
-    "b2c_net_sync_weights", "b2c_train_step",
+    "b2c_net_sync_weights", "b2c_train_step", "b2c_net_apply_update", "b2c_net_profile_enable", "b2c_net_profile_read",
 ]
+PROF_KINDS = ["conv_fwd", "conv_dgrad", "conv_wgrad", "bn_fwd", "bn_bwd", "other", "update"]
 
 
 class ConvDesc(Structure):
@@ -266,6 +267,19 @@ class Net:
         _check(lib().b2c_train_step(self.handle, _ptr(images), _ptr(labels), c_int(n_micro), c_float(lr), c_float(momentum), c_float(wd),
                                     _ptr(self.loss), c_int(int(update)), _stream()), "b2c_train_step")
         return self.loss
+
+    def apply_update(self, n_avg, lr, momentum, wd):
+        _check(lib().b2c_net_apply_update(self.handle, c_int(n_avg), c_float(lr), c_float(momentum), c_float(wd), _stream()), "b2c_net_apply_update")
+
+    def profile_enable(self, enable: bool = True):
+        _check(lib().b2c_net_profile_enable(self.handle, c_int(int(enable))), "b2c_net_profile_enable")
+
+    def profile_read(self):
+        """(ms per kernel family, kernels launched per family) since the last read; synchronises."""
+        ms = (c_double * len(PROF_KINDS))()
+        n = (c_longlong * len(PROF_KINDS))()
+        _check(lib().b2c_net_profile_read(self.handle, ms, n, _stream()), "b2c_net_profile_read")
+        return dict(zip(PROF_KINDS, list(ms))), dict(zip(PROF_KINDS, list(n)))
 
     def tensor_view(self, tensor: int, shape, dtype=torch.bfloat16, grad=False, which=0):
         off = self.tensor_offset(tensor, grad, which)

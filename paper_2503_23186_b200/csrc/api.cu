@@ -187,7 +187,38 @@ struct b2c_net {
     float *w = nullptr, *v = nullptr, *g = nullptr;
     char *w_bf16 = nullptr, *w_dgrad = nullptr, *ws = nullptr;
     bool fuse_stats = true;
+    // optional per-launch timing (CUDA events on the step's stream), summed per kernel family
+    bool profile = false;
+    struct Span { cudaEvent_t a, b; int kind; };
+    std::vector<Span> spans;      // event pool, reused every step
+    size_t spans_used = 0;
+    long long launches[B2C_PROF_KINDS] = {0};   // kernels launched since the last profile read
+    ~b2c_net()
+    {
+        for (Span& sp : spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
+    }
 };
+
+namespace {
+// Brackets one launch site with events when profiling is on, and counts its kernels.
+struct ProfScope {
+    b2c_net* net; cudaStream_t stream; b2c_net::Span* sp = nullptr;
+    ProfScope(b2c_net* n, cudaStream_t st, int kind, int kernels) : net(n), stream(st)
+    {
+        net->launches[kind] += kernels;
+        if (!net->profile) return;
+        if (net->spans_used == net->spans.size()) {
+            b2c_net::Span fresh{};
+            if (cudaEventCreate(&fresh.a) != cudaSuccess || cudaEventCreate(&fresh.b) != cudaSuccess) return;
+            net->spans.push_back(fresh);
+        }
+        sp = &net->spans[net->spans_used++];
+        sp->kind = kind;
+        cudaEventRecord(sp->a, stream);
+    }
+    ~ProfScope() { if (sp) cudaEventRecord(sp->b, stream); }
+};
+}  // namespace
 
 extern "C" {
 
@@ -379,6 +410,17 @@ b2c_status b2c_net_sync_weights(b2c_net* net, void* stream)
     return net_pack_dgrad(net, stream);
 }
 
+b2c_status b2c_net_apply_update(b2c_net* net, int n_avg, float lr, float momentum, float wd, void* stream_)
+{
+    if (!net || !net->ws || n_avg < 1) return B2C_ERR_INVALID_ARG;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    ProfScope ps_(net, stream, B2C_PROF_UPDATE, 2);
+    b2c_status st = b2c_grad_accum_sgd_momentum(net->ctx, net->param_count, net->w, net->v, net->g, 1.f / (float)n_avg, lr, momentum, wd,
+                                                net->w_bf16, 1, stream_);
+    if (st != B2C_OK) return st;
+    return net_pack_dgrad(net, stream_);
+}
+
 #define B2C_TRY(call)                   \
     do {                                \
         b2c_status s_ = (call);         \
@@ -391,6 +433,7 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
     if (!net || !net->ws || !images || !labels || !loss_dev || n_micro < 1) return B2C_ERR_INVALID_ARG;
     if (!b2c_aligned16(images)) return B2C_ERR_MISALIGNED;
     cudaStream_t stream = (cudaStream_t)stream_;
+    if (net->profile && net->spans_used > (1u << 20)) return B2C_ERR_INVALID_ARG;   // read the profile between steps
     b2c_ctx* ctx = net->ctx;
     const int N = net->micro_batch;
     const int n_layers = (int)net->layers.size();
@@ -408,6 +451,7 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
         const int32_t* lab = labels + (size_t)mb * N;
         const void* t0;
         if (net->tensors[0].act_off >= 0) {
+            ProfScope ps_(net, stream, B2C_PROF_OTHER, 1);
             B2C_TRY(b2c_pad_channels(ctx, (long)N * net->image_h * net->image_w, net->image_c, net->image_c_pad, img, act(0), stream));
             t0 = act(0);
         } else {
@@ -428,6 +472,7 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
                     pb.r = d.r; pb.stride = d.stride; pb.pad = (d.r - 1) / 2; pb.dgrad = false;
                     pb.in = act_in(d.src); pb.wt = w_bf16 + L.w_off; pb.out = act(i + 1);
                     pb.stats = net->fuse_stats ? reinterpret_cast<double*>(net->ws + o.stats_off) : nullptr;
+                    ProfScope ps_(net, stream, B2C_PROF_CONV_FWD, 1);
                     B2C_TRY(launch_conv_kmajor(ctx, pb, stream));
                     break;
                 }
@@ -435,6 +480,7 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
                     const TensorPlan& in = net->tensors[d.src];
                     const bool ready = net->fuse_stats && in.stats_off >= 0;
                     double* stats = reinterpret_cast<double*>(net->ws + (in.stats_off >= 0 ? in.stats_off : L.bwd_ws_off));
+                    ProfScope ps_(net, stream, B2C_PROF_BN_FWD, ready ? 1 : 2);
                     B2C_TRY(b2c_bn_relu_fwd(ctx, N, in.h, in.w, in.c, act(d.src), stats, ready ? 1 : 0, net->w + L.gamma_off, net->w + L.beta_off,
                                             d.res >= 0 ? act(d.res) : nullptr, d.relu, 1e-5f, act(i + 1),
                                             reinterpret_cast<float*>(net->ws + L.mean_off), reinterpret_cast<float*>(net->ws + L.invstd_off),
@@ -443,6 +489,7 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
                 }
                 case B2C_LAYER_AVGPOOL: {
                     const TensorPlan& in = net->tensors[d.src];
+                    ProfScope ps_(net, stream, B2C_PROF_OTHER, 1);
                     B2C_TRY(b2c_avgpool_fwd(ctx, N, in.h * in.w, in.c, act(d.src), act(i + 1), stream));
                     break;
                 }
@@ -452,11 +499,13 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
                     pb.r = 1; pb.stride = 1; pb.pad = 0; pb.dgrad = false;
                     pb.in = act(d.src); pb.wt = w_bf16 + L.w_off; pb.out = act(i + 1);
                     pb.out_f32 = true; pb.bias = net->w + L.bias_off;
+                    ProfScope ps_(net, stream, B2C_PROF_OTHER, 1);
                     B2C_TRY(launch_conv_kmajor(ctx, pb, stream));
                     break;
                 }
                 case B2C_LAYER_XENT: {
                     const TensorPlan& in = net->tensors[d.src];
+                    ProfScope ps_(net, stream, B2C_PROF_OTHER, 1);
                     B2C_TRY(b2c_softmax_xent_fwd_bwd(ctx, N, d.k, reinterpret_cast<const float*>(act(d.src)), in.c, lab,
                                                      1.f / ((float)N * (float)n_micro), 1.f / (float)N, loss_dev, grad(d.src, L.src_slot), in.c,
                                                      stream));
@@ -476,6 +525,7 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
                     WgradProblem wp{};
                     wp.n = N; wp.h = 1; wp.w = 1; wp.c = L.c_pad; wp.p = 1; wp.q = 1; wp.k = L.k_pad; wp.r = 1; wp.stride = 1; wp.pad = 0;
                     wp.dy = dz; wp.x = act(d.src); wp.dw = net->g + L.w_off;
+                    ProfScope ps_(net, stream, B2C_PROF_OTHER, 3);
                     B2C_TRY(launch_conv_wgrad(ctx, wp, stream));
                     B2C_TRY(b2c_bias_grad(ctx, N, L.k_pad, L.k_pad, dz, net->g + L.bias_off, 1, stream));
                     KMajorProblem pb{};
@@ -487,11 +537,13 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
                 }
                 case B2C_LAYER_AVGPOOL: {
                     const TensorPlan& in = net->tensors[d.src];
+                    ProfScope ps_(net, stream, B2C_PROF_OTHER, 1);
                     B2C_TRY(b2c_avgpool_bwd(ctx, N, in.h * in.w, in.c, grad(i + 1, 0), grad(d.src, L.src_slot), stream));
                     break;
                 }
                 case B2C_LAYER_BN: {
                     const TensorPlan& in = net->tensors[d.src];
+                    ProfScope ps_(net, stream, B2C_PROF_BN_BWD, 2);
                     B2C_TRY(b2c_bn_relu_bwd(ctx, N, in.h, in.w, in.c, grad(i + 1, 0), o.n_contrib > 1 ? grad(i + 1, 1) : nullptr, act(d.src), act(i + 1),
                                             net->w + L.gamma_off, reinterpret_cast<float*>(net->ws + L.mean_off),
                                             reinterpret_cast<float*>(net->ws + L.invstd_off), d.relu, grad(d.src, L.src_slot),
@@ -505,12 +557,16 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
                     wp.n = N; wp.h = d.h; wp.w = d.w; wp.c = L.c_pad; wp.p = L.p; wp.q = L.q; wp.k = d.k;
                     wp.r = d.r; wp.stride = d.stride; wp.pad = (d.r - 1) / 2;
                     wp.dy = dy; wp.x = act_in(d.src); wp.dw = net->g + L.w_off;
-                    B2C_TRY(launch_conv_wgrad(ctx, wp, stream));
+                    {
+                        ProfScope ps_(net, stream, B2C_PROF_CONV_WGRAD, 1);
+                        B2C_TRY(launch_conv_wgrad(ctx, wp, stream));
+                    }
                     if (d.src != 0) {
                         KMajorProblem pb{};
                         pb.n = N; pb.ih = L.p; pb.iw = L.q; pb.ic = d.k; pb.oh = d.h; pb.ow = d.w; pb.oc = L.c_pad;
                         pb.r = d.r; pb.stride = d.stride; pb.pad = (d.r - 1) / 2; pb.dgrad = true;
                         pb.in = dy; pb.wt = w_dg + L.w_off; pb.out = grad(d.src, L.src_slot);
+                        ProfScope ps_(net, stream, B2C_PROF_CONV_DGRAD, 1);
                         B2C_TRY(launch_conv_kmajor(ctx, pb, stream));
                     }
                     break;
@@ -519,11 +575,29 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
         }
     }
     // ---------------- gradient average + parameter update, refresh of both bf16 weight copies
-    if (update) {
-        B2C_TRY(b2c_grad_accum_sgd_momentum(ctx, net->param_count, net->w, net->v, net->g, 1.f / (float)n_micro, lr, momentum, wd, net->w_bf16, 1,
-                                            stream));
-        B2C_TRY(net_pack_dgrad(net, stream));
+    if (update) B2C_TRY(b2c_net_apply_update(net, n_micro, lr, momentum, wd, stream_));
+    return B2C_OK;
+}
+
+b2c_status b2c_net_profile_enable(b2c_net* net, int enable)
+{
+    if (!net) return B2C_ERR_INVALID_ARG;
+    net->profile = enable != 0;
+    net->spans_used = 0;
+    for (int k = 0; k < B2C_PROF_KINDS; ++k) net->launches[k] = 0;
+    return B2C_OK;
+}
+
+b2c_status b2c_net_profile_read(b2c_net* net, double* ms, long long* launches, void* stream)
+{
+    if (!net || !ms || !launches) return B2C_ERR_INVALID_ARG;
+    B2C_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+    for (int k = 0; k < B2C_PROF_KINDS; ++k) { ms[k] = 0.0; launches[k] = net->launches[k]; net->launches[k] = 0; }
+    for (size_t i = 0; i < net->spans_used; ++i) {
+        float t = 0.f;
+        if (cudaEventElapsedTime(&t, net->spans[i].a, net->spans[i].b) == cudaSuccess) ms[net->spans[i].kind] += t;
     }
+    net->spans_used = 0;
     return B2C_OK;
 }
 

@@ -1,0 +1,225 @@
+"""End-to-end parity of the layer-list training step (Algorithm 1's inner loop) against the
+rounding-point oracle: loss, every parameter gradient, updated parameters and momentum."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import net as onet
+from paper_2503_23186_b200 import workloads as wl
+from parity import assert_close, dev_bf16, dev_f32, errors, host
+
+pytestmark = pytest.mark.gpu
+
+LR, MU, WD = 0.1, 0.9, 5e-4
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    from paper_2503_23186_b200 import binding
+    c = binding.Context(0)
+    yield c
+    assert c.device_status() == 0
+    c.close()
+
+
+def _compare_step(ctx, spec, params, velocity, images, labels, micro_batch, n_micro, table=None, gate_gradients=True):
+    """Three checks of one optimiser step.
+    (1) Teacher-forced: every layer's device outputs against the oracle applied to that layer's device inputs
+        (per-kernel tolerances; first micro-batch).
+    (2) Free-running: loss, logits, updated parameters and momentum of the library's whole chain against the
+        oracle's whole chain.
+    (3) Free-running parameter gradients: reported per tensor; gated with the conditioning of each sum taken into
+        account (see _gradient_gate)."""
+    from paper_2503_23186_b200 import binding
+    from netcheck import check_step
+    net = binding.Net(ctx, spec, micro_batch)
+    net.load_params(params, velocity)
+    d_img, d_lab = dev_bf16(images), torch.from_numpy(labels).cuda()
+    vel = velocity if velocity is not None else {k: np.zeros_like(v) for k, v in params.items()}
+
+    # (1) first micro-batch alone, state left in the workspace
+    net.train_step(d_img[:micro_batch], d_lab[:micro_batch], 1, LR, MU, WD, update=False)
+    assert ctx.device_status() == 0
+    rep = check_step(net, spec, images[:micro_batch], labels[:micro_batch], micro_batch)
+    if table is not None:
+        table["teacher_forced_worst"] = rep.worst()[:3]
+    rep.assert_ok()
+    net.g.zero_()
+
+    # (2), (3)
+    ref = onet.train_step(spec, params, vel, images.astype(np.float64), labels, n_micro, LR, MU, WD, rounding=True)
+    loss = net.train_step(d_img, d_lab, n_micro, LR, MU, WD, update=False).item()
+    assert ctx.device_status() == 0
+    assert abs(loss - ref["loss"]) <= 2e-3 * abs(ref["loss"]), (loss, ref["loss"])
+    grads = net.unpack(net.g)
+    rows = []
+    for name in sorted(params):
+        rel, mx = errors(grads[name], ref["grads"][name])
+        rows.append((name, rel, mx))
+    if table is not None:
+        table["free_running_gradients"] = rows
+    # zero padding of the flat arrays receives no gradient
+    packed_mask = net.pack({k: np.ones_like(v) for k, v in params.items()})
+    assert torch.count_nonzero(net.g[torch.from_numpy(packed_mask == 0).cuda()]).item() == 0
+    _gradient_gate(rows, grads, ref["grads"], gate_gradients)
+
+    net.g.zero_()
+    loss2 = net.train_step(d_img, d_lab, n_micro, LR, MU, WD, update=True).item()
+    assert ctx.device_status() == 0
+    assert abs(loss2 - loss) <= 1e-3 * abs(loss)   # run-to-run: BatchNorm statistics are combined with atomics
+    w_new = net.unpack(net.w)
+    for name in sorted(params):
+        assert_close(w_new[name], ref["params"][name], f"w_new {name}")
+    assert torch.count_nonzero(net.g).item() == 0
+    assert torch.equal(net.w_bf16, net.w.to(torch.bfloat16))
+    net.close()
+    return rows
+
+
+def _gradient_gate(rows, got, ref, tight):
+    """Free-running gradients differ from the oracle's by the legitimate bf16 rounding flips of every upstream tensor
+    (an fp32 tensor-core sum and an fp64 sum land on opposite sides of a rounding boundary for ~1e-3 of the elements,
+    a relative perturbation of ~1e-4 per stored tensor).  The gradient of a randomly initialised BatchNorm residual
+    network amplifies such perturbations by two to three orders of magnitude (pinned on the oracle alone in
+    tests/test_oracle_pins.py), so the per-tensor budget cannot hold for the free-running chain of a deep net: there
+    the gate is the direction of every gradient (cosine >= 0.9 rules out sign, index and scaling mistakes) and the
+    errors are reported; the per-tensor budget is enforced teacher-forced, layer by layer.  Shallow nets keep a
+    relative gate with slack for the chain length."""
+    for name in got:
+        a, b = np.asarray(got[name], np.float64).reshape(-1), np.asarray(ref[name], np.float64).reshape(-1)
+        cos = float(np.dot(a, b) / max(np.linalg.norm(a) * np.linalg.norm(b), 1e-300))
+        assert cos >= 0.9, (name, cos)
+    if tight:
+        bad = [(n, r, m) for (n, r, m) in rows if r > 2e-2 or m > 5e-2]
+        assert not bad, bad
+
+
+def test_tiny_net_two_micro_batches(ctx):
+    spec = wl.tiny_net_spec(classes=10, hw=8, c=16, width=16, width2=32)
+    params = wl.perturb_bn_params(wl.init_params(spec, 1), 1)
+    vel = {k: (0.01 * wl.rng_for(1, "v" + k).standard_normal(v.shape)).astype(np.float32) for k, v in params.items()}
+    images, labels = wl.image_batch(1, 2 * 12, hw=8, c=16, classes=10)
+    table = {}
+    try:
+        _compare_step(ctx, spec, params, vel, images, labels, 12, 2, table)
+    finally:
+        print("teacher-forced worst:", table.get("teacher_forced_worst"))
+        for row in table.get("free_running_gradients", []):
+            print("free-running grad %-10s relF=%.3e max=%.3e" % row)
+
+
+def test_tiny_net_three_channel_images(ctx):
+    # image channels are zero-extended to 16 inside the library; the oracle convolves the 3 channels directly
+    spec = wl.tiny_net_spec(classes=10, hw=16, c=3, width=16, width2=32)
+    params = wl.perturb_bn_params(wl.init_params(spec, 2), 2)
+    images, labels = wl.image_batch(2, 8, hw=16, c=3, classes=10)
+    _compare_step(ctx, spec, params, None, images, labels, 8, 1)
+
+
+def test_basic_block_config2(ctx):
+    """One ResNet basic block (two 3x3 convs 64->64, BatchNorm, ReLU, identity shortcut), N=128, 32x32,
+    forward + backward from an upstream gradient, through the single-operation entry points."""
+    from paper_2503_23186_b200 import binding
+    N, H, C = 128, 32, 64
+    d = binding.conv_desc(N, H, H, C, C, 3, 1)
+    x = wl.normal_bf16(0, "x", (N, H, H, C))
+    w1 = wl.normal_bf16(0, "w1", (C, 3, 3, C), std=float(np.sqrt(2.0 / (9 * C))))
+    w2 = wl.normal_bf16(0, "w2", (C, 3, 3, C), std=float(np.sqrt(2.0 / (9 * C))))
+    g = wl.normal_bf16(0, "g", (N, H, H, C))
+    gamma, beta = np.ones(C, np.float32), np.zeros(C, np.float32)
+    rb, rf = oracle.round_bf16, oracle.round_f32
+
+    # oracle, with rounding at the storage points
+    y1 = rb(oracle.conv2d_fwd(x, w1, 1, 1))
+    m1, _, i1 = oracle.bn_stats(y1, 1e-5); m1, i1 = rf(m1), rf(i1)
+    a1 = rb(oracle.bn_relu_apply(y1, m1, i1, gamma, beta, None, True))
+    y2 = rb(oracle.conv2d_fwd(a1, w2, 1, 1))
+    m2, _, i2 = oracle.bn_stats(y2, 1e-5); m2, i2 = rf(m2), rf(i2)
+    out = rb(oracle.bn_relu_apply(y2, m2, i2, gamma, beta, x, True))
+    dy2, dres, dg2, db2 = oracle.bn_relu_bwd(g, None, y2, out, gamma, m2, i2, True, True)
+    dy2, dres = rb(dy2), rb(dres)
+    dw2 = oracle.conv2d_wgrad(dy2, a1, 3, 3, 1, 1)
+    da1 = rb(oracle.conv2d_dgrad(dy2, w2, a1.shape, 1, 1))
+    dy1, _, dg1, db1 = oracle.bn_relu_bwd(da1, None, y1, a1, gamma, m1, i1, True, False)
+    dy1 = rb(dy1)
+    dw1 = oracle.conv2d_wgrad(dy1, x, 3, 3, 1, 1)
+    dx = rb(oracle.conv2d_dgrad(dy1, w1, x.shape, 1, 1)) + dres   # two contributions reach the block input
+
+    # library
+    bf = lambda: torch.empty((N, H, H, C), dtype=torch.bfloat16, device="cuda")
+    f32 = lambda n: torch.empty(n, dtype=torch.float32, device="cuda")
+    X, W1, W2, G = dev_bf16(x), dev_bf16(w1), dev_bf16(w2), dev_bf16(g)
+    Gm, Bt = dev_f32(gamma), dev_f32(beta)
+    W1d, W2d = torch.empty_like(W1).reshape(-1), torch.empty_like(W2).reshape(-1)
+    ctx.weight_pack_dgrad([(0, C, 9, C)], W1.reshape(-1), W1d)
+    ctx.weight_pack_dgrad([(0, C, 9, C)], W2.reshape(-1), W2d)
+    Y1, A1, Y2, OUT = bf(), bf(), bf(), bf()
+    st1, st2 = torch.zeros(2 * C, dtype=torch.float64, device="cuda"), torch.zeros(2 * C, dtype=torch.float64, device="cuda")
+    M1, I1, M2, I2 = f32(C), f32(C), f32(C), f32(C)
+    ctx.conv2d_fwd(d, X, W1, Y1, ch_stats=st1)
+    ctx.bn_relu_fwd(N, H, H, C, Y1, st1, True, Gm, Bt, None, True, 1e-5, A1, M1, I1)
+    ctx.conv2d_fwd(d, A1, W2, Y2, ch_stats=st2)
+    ctx.bn_relu_fwd(N, H, H, C, Y2, st2, True, Gm, Bt, X, True, 1e-5, OUT, M2, I2)
+    DY2, DRES, DA1, DY1, DX1 = bf(), bf(), bf(), bf(), bf()
+    DG1, DB1, DG2, DB2 = f32(C), f32(C), f32(C), f32(C)
+    DW1, DW2 = f32(C * 9 * C), f32(C * 9 * C)
+    ws = torch.empty(ctx.bn_relu_bwd_workspace_bytes(C), dtype=torch.uint8, device="cuda")
+    ctx.bn_relu_bwd(N, H, H, C, G, None, Y2, OUT, Gm, M2, I2, True, DY2, DRES, DG2, DB2, False, ws)
+    ctx.conv2d_wgrad(d, DY2, A1, DW2)
+    ctx.conv2d_dgrad(d, DY2, W2d, DA1)
+    ctx.bn_relu_bwd(N, H, H, C, DA1, None, Y1, A1, Gm, M1, I1, True, DY1, None, DG1, DB1, False, ws)
+    ctx.conv2d_wgrad(d, DY1, X, DW1)
+    ctx.conv2d_dgrad(d, DY1, W1d, DX1)
+    assert ctx.device_status() == 0
+
+    assert_close(Y1, y1, "y1"); assert_close(A1, a1, "a1"); assert_close(Y2, y2, "y2"); assert_close(OUT, out, "out")
+    # backward quantities of the free-running chain: per-tensor budget with slack for the chain of rounding flips
+    loose = dict(rel_fro=1e-2, max_rel=3e-2)
+    assert_close(DW2.reshape(C, 3, 3, C), dw2, "dw2", **loose); assert_close(DW1.reshape(C, 3, 3, C), dw1, "dw1", **loose)
+    assert_close(DG2, dg2, "dgamma2", **loose); assert_close(DB2, db2, "dbeta2", **loose)
+    assert_close(DG1, dg1, "dgamma1", **loose); assert_close(DB1, db1, "dbeta1", **loose)
+    # a ReLU mask may legitimately flip where |z| is below fp32 resolution: one element then differs by a whole dz,
+    # so the free-running input gradient is held to the Frobenius budget only
+    assert_close(host(DX1) + host(DRES), dx, "dx", rel_fro=1e-2, max_rel=float("inf"))
+    # the same backward kernels teacher-forced on the device's own tensors: the per-tensor budget proper
+    hy2, hout, ha1, hy1 = host(Y2), host(OUT), host(A1), host(Y1)
+    t_dy2, t_dres, t_dg2, t_db2 = oracle.bn_relu_bwd(g, None, hy2, hout, gamma, host(M2), host(I2), True, True)
+    assert_close(DY2, rb(t_dy2), "dy2 (teacher-forced)"); assert_close(DG2, t_dg2, "dgamma2 (tf)"); assert_close(DB2, t_db2, "dbeta2 (tf)")
+    assert_close(DW2.reshape(C, 3, 3, C), oracle.conv2d_wgrad(host(DY2), ha1, 3, 3, 1, 1), "dw2 (tf)")
+    assert_close(DA1, rb(oracle.conv2d_dgrad(host(DY2), w2, a1.shape, 1, 1)), "da1 (tf)")
+    t_dy1, _, t_dg1, t_db1 = oracle.bn_relu_bwd(host(DA1), None, hy1, ha1, gamma, host(M1), host(I1), True, False)
+    assert_close(DY1, rb(t_dy1), "dy1 (tf)"); assert_close(DG1, t_dg1, "dgamma1 (tf)"); assert_close(DB1, t_db1, "dbeta1 (tf)")
+    assert_close(DW1.reshape(C, 3, 3, C), oracle.conv2d_wgrad(host(DY1), x, 3, 3, 1, 1), "dw1 (tf)")
+    assert_close(DX1, rb(oracle.conv2d_dgrad(host(DY1), w1, x.shape, 1, 1)), "dx1 (tf)")
+
+
+def test_resnet18_batch128_config3(ctx):
+    spec = wl.resnet18_spec()
+    params = wl.init_params(spec, 0)
+    images, labels = wl.image_batch(0, 128)
+    table = {}
+    try:
+        _compare_step(ctx, spec, params, None, images, labels, 128, 1, table, gate_gradients=False)
+    finally:
+        print("teacher-forced worst:", table.get("teacher_forced_worst"))
+        for row in table.get("free_running_gradients", []):
+            print("free-running grad %-10s relF=%.3e max=%.3e" % row)
+
+
+def test_teacher_forced_report_resnet18(ctx, capsys):
+    """Prints the per-layer teacher-forced errors of one ResNet-18-shaped micro-batch (diagnostic table)."""
+    from paper_2503_23186_b200 import binding
+    from netcheck import check_step
+    spec = wl.resnet18_spec()
+    net = binding.Net(ctx, spec, 32)
+    net.load_params(wl.init_params(spec, 0))
+    images, labels = wl.image_batch(0, 32)
+    net.train_step(dev_bf16(images), torch.from_numpy(labels).cuda(), 1, LR, MU, WD, update=False)
+    assert ctx.device_status() == 0
+    rep = check_step(net, spec, images, labels, 32)
+    with capsys.disabled():
+        for name, rel, mx, ok in rep.rows:
+            print("teacher-forced %-22s relF=%.3e max=%.3e %s" % (name, rel, mx, "" if ok else "FAIL"))
+    rep.assert_ok()
+    net.close()
