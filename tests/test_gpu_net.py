@@ -7,7 +7,7 @@ import torch
 import oracle
 from oracle import net as onet
 from paper_2503_23186_b200 import workloads as wl
-from parity import assert_close, dev_bf16, dev_f32, errors, host
+from parity import MAX_REL, REL_FRO, SGD_REL, assert_close, dev_bf16, dev_f32, errors, host
 
 pytestmark = pytest.mark.gpu
 
@@ -64,15 +64,32 @@ def _compare_step(ctx, spec, params, velocity, images, labels, micro_batch, n_mi
     assert torch.count_nonzero(net.g[torch.from_numpy(packed_mask == 0).cuda()]).item() == 0
     _gradient_gate(rows, grads, ref["grads"], gate_gradients)
 
-    net.g.zero_()
+    # the update alone, teacher-forced on the device's own gradient sum: fp32 arithmetic on identical inputs
+    g_dev = net.unpack(net.g)
+    net.apply_update(n_micro, LR, MU, WD)
+    assert ctx.device_status() == 0
+    w_new, v_new = net.unpack(net.w), net.unpack(net.v)
+    for name in sorted(params):
+        rw, rv = oracle.sgd_momentum(params[name], vel[name], g_dev[name], 1.0 / n_micro, LR, MU, WD)
+        assert_close(w_new[name], rw, f"w_new {name} (given the device gradient)", SGD_REL, 1e-5)
+        assert_close(v_new[name], rv, f"v_new {name} (given the device gradient)", SGD_REL, 1e-5)
+    assert torch.count_nonzero(net.g).item() == 0
+    assert torch.equal(net.w_bf16, net.w.to(torch.bfloat16))
+    # free-running: updated parameters against the oracle's whole chain (tensors that start at zero are pure
+    # gradient and fall under the gradient discussion above)
+    for name in sorted(params):
+        if np.any(params[name] != 0):
+            # deep nets: the 20 % free-running gradient error times lr*|g|/|w| ~ 1e-2 shows up here
+            assert_close(w_new[name], ref["params"][name], f"w_new {name}", REL_FRO if gate_gradients else 1e-2, MAX_REL if gate_gradients else 5e-2)
+    # the same step in one call (forward, backward and update fused in b2c_train_step)
+    net.load_params(params, velocity)
     loss2 = net.train_step(d_img, d_lab, n_micro, LR, MU, WD, update=True).item()
     assert ctx.device_status() == 0
     assert abs(loss2 - loss) <= 1e-3 * abs(loss)   # run-to-run: BatchNorm statistics are combined with atomics
-    w_new = net.unpack(net.w)
+    w_again = net.unpack(net.w)
     for name in sorted(params):
-        assert_close(w_new[name], ref["params"][name], f"w_new {name}")
-    assert torch.count_nonzero(net.g).item() == 0
-    assert torch.equal(net.w_bf16, net.w.to(torch.bfloat16))
+        if np.any(params[name] != 0):
+            assert_close(w_again[name], w_new[name], f"w_new {name} (single call)")
     net.close()
     return rows
 
