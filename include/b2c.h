@@ -126,6 +126,26 @@ b2c_status b2c_bn_relu_bwd(b2c_ctx* ctx, int n, int h, int w, int c, const void*
                            int relu, void* dy, void* dres, float* dgamma, float* dbeta, int acc, void* ws,
                            size_t ws_bytes, void* stream);
 
+/* (No counterpart in the paper: a packaging variant of b2c_bn_relu_bwd.)
+ * The same computation, arguments and results as b2c_bn_relu_bwd, but without the `ws` argument: the per-channel
+ * fp64 accumulators live in an array built into the library (B2C_BN_BWD_STATIC_MAX_C channels, 32 KB, resident on
+ * every GPU that loads the library until the process exits).  It is meant for callers that cannot obtain device
+ * memory of their own at the point of the call: code running under an allocator it does not control (a plug-in that
+ * is handed only its input and output buffers), code with a fixed memory budget drawn up in advance, and code that
+ * must not stall, since the CUDA allocation calls synchronise the device.  This entry point calls no allocating
+ * routine at all, of CUDA or of any library.
+ *   - c > B2C_BN_BWD_STATIC_MAX_C returns B2C_ERR_WORKSPACE_TOO_SMALL and enqueues nothing.
+ *   - The context's device must be the current device.  The first call on a device looks up the array's device
+ *     address (a set-up step); make that first call before any stream capture starts.
+ *   - All calls on a device share the one array, which keeps the previous call's sums; each call clears what it
+ *     uses before reducing into it.  Two calls whose kernels overlap on the GPU (different streams, or different
+ *     host threads) race on it: serialise them on one stream. */
+#define B2C_BN_BWD_STATIC_MAX_C 2048
+b2c_status b2c_bn_relu_bwd_static(b2c_ctx* ctx, int n, int h, int w, int c, const void* da1, const void* da2,
+                                  const void* y, const void* a, const float* gamma, const float* save_mean,
+                                  const float* save_invstd, int relu, void* dy, void* dres, float* dgamma,
+                                  float* dbeta, int acc, void* stream);
+
 /* dx[n,h,w,c] = sum over (p,q,r,s,k) with p*stride+r-pad = h, q*stride+s-pad = w of dy[n,p,q,k]*w[k,r,s,c].
  *   dy bf16 [n,p,q,k]; dx bf16 [n,h,w,c] (every element written)
  *   w_crsk_flipped bf16 [c,r,s,k] with w_crsk_flipped[c,r,s,k] = w[k, R-1-r, S-1-s, c]

@@ -25,7 +25,7 @@ LAYER_KINDS = {"conv": 0, "bn": 1, "avgpool": 2, "fc": 3, "xent": 4}
 EXPORTS = [
     "b2c_create", "b2c_destroy", "b2c_status_string", "b2c_get_device_status", "b2c_set_spin_limit",
     "b2c_conv2d_fwd", "b2c_bn_relu_fwd", "b2c_avgpool_fwd", "b2c_avgpool_bwd", "b2c_pad_channels",
-    "b2c_softmax_xent_fwd_bwd", "b2c_bn_relu_bwd_workspace_bytes", "b2c_bn_relu_bwd", "b2c_conv2d_dgrad",
+    "b2c_softmax_xent_fwd_bwd", "b2c_bn_relu_bwd_workspace_bytes", "b2c_bn_relu_bwd", "b2c_bn_relu_bwd_static", "b2c_conv2d_dgrad",
     "b2c_conv2d_wgrad", "b2c_bias_grad", "b2c_grad_accum_sgd_momentum", "b2c_weight_pack_dgrad",
     "b2c_net_create", "b2c_net_destroy", "b2c_net_param_count", "b2c_net_param_offset",
     "b2c_net_padded_image_channels", "b2c_net_workspace_bytes", "b2c_net_tensor_offset", "b2c_net_bind",
@@ -159,6 +159,14 @@ class Context:
         _check(lib().b2c_bn_relu_bwd(self.handle, n, h, w, c, _ptr(da1), _ptr(da2), _ptr(y), _ptr(a), _ptr(gamma), _ptr(save_mean),
                                      _ptr(save_invstd), c_int(int(relu)), _ptr(dy), _ptr(dres), _ptr(dgamma), _ptr(dbeta), c_int(int(acc)),
                                      _ptr(ws), c_size_t(ws.numel() * ws.element_size()), _stream()), "b2c_bn_relu_bwd")
+
+    def bn_relu_bwd_static(self, n, h, w, c, da1, da2, y, a, gamma, save_mean, save_invstd, relu, dy, dres, dgamma, dbeta, acc):
+        """b2c_bn_relu_bwd without a caller-provided workspace: the accumulators live inside the library, so the
+        call allocates nothing (for callers that cannot get device memory of their own; at most 2048 channels;
+        calls that overlap on the GPU race on the shared scratch)."""
+        _check(lib().b2c_bn_relu_bwd_static(self.handle, n, h, w, c, _ptr(da1), _ptr(da2), _ptr(y), _ptr(a), _ptr(gamma), _ptr(save_mean),
+                                            _ptr(save_invstd), c_int(int(relu)), _ptr(dy), _ptr(dres), _ptr(dgamma), _ptr(dbeta),
+                                            c_int(int(acc)), _stream()), "b2c_bn_relu_bwd_static")
 
     def conv2d_dgrad(self, d: ConvDesc, dy, w_crsk_flipped, dx):
         _check(lib().b2c_conv2d_dgrad(self.handle, byref(d), _ptr(dy), _ptr(w_crsk_flipped), _ptr(dx), _stream()), "b2c_conv2d_dgrad")

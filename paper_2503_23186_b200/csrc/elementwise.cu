@@ -527,4 +527,46 @@ b2c_status b2c_weight_pack_dgrad(b2c_ctx* ctx, const b2c_weight_seg* segs, int n
     return B2C_OK;
 }
 
+// ------------------------------------------------------------------------------ allocation-free variant
+// Scratch of b2c_bn_relu_bwd_static: the two fp64 accumulators per channel, for up to
+// B2C_BN_BWD_STATIC_MAX_C channels.  It is part of the library image, so every GPU that loads the
+// library holds these 32 KB until the process exits.
+static __device__ __align__(256) double g_bn_bwd_static_scratch[2 * B2C_BN_BWD_STATIC_MAX_C];
+
+// Device address of the array above, looked up once per device.  In host code the symbol's name
+// is only a handle: the kernels must be given the address cudaGetSymbolAddress reports.
+static double* g_bn_bwd_static_ptr[64] = {nullptr};
+
+b2c_status b2c_bn_relu_bwd_static(b2c_ctx* ctx, int n, int h, int w, int c, const void* da1, const void* da2, const void* y, const void* a,
+                                  const float* gamma, const float* save_mean, const float* save_invstd, int relu, void* dy, void* dres,
+                                  float* dgamma, float* dbeta, int acc, void* stream_)
+{
+    cudaStream_t stream = (cudaStream_t)stream_;
+    if (!ctx || !da1 || !y || !gamma || !save_mean || !save_invstd || !dy || !dgamma || !dbeta) return B2C_ERR_INVALID_ARG;
+    if (relu && !a) return B2C_ERR_INVALID_ARG;
+    if (n < 1 || h < 1 || w < 1 || c < 8 || c % 8) return B2C_ERR_UNSUPPORTED_SHAPE;
+    if (c > B2C_BN_BWD_STATIC_MAX_C) return B2C_ERR_WORKSPACE_TOO_SMALL;   // the built-in scratch holds at most that many channels
+    if (!b2c_aligned16(da1) || (da2 && !b2c_aligned16(da2)) || !b2c_aligned16(y) || (a && !b2c_aligned16(a)) || !b2c_aligned16(dy) ||
+        (dres && !b2c_aligned16(dres)))
+        return B2C_ERR_MISALIGNED;
+    int current = -1;
+    B2C_CUDA(cudaGetDevice(&current));
+    if (current != ctx->device || current < 0 || current >= 64) return B2C_ERR_INVALID_ARG;   // the context's device must be current
+    if (g_bn_bwd_static_ptr[current] == nullptr) {
+        double* ptr = nullptr;
+        if (cudaGetSymbolAddress((void**)&ptr, g_bn_bwd_static_scratch) != cudaSuccess || ptr == nullptr) return B2C_ERR_CUDA;
+        g_bn_bwd_static_ptr[current] = ptr;
+    }
+    double* sums = g_bn_bwd_static_ptr[current];
+    const long long m = (long long)n * h * w;
+    const int rows_per_iter = kEwThreads / (c / 8);
+    const int grid = ew_grid(ctx, m, rows_per_iter);
+    B2C_CUDA(cudaMemsetAsync(sums, 0, sizeof(double) * 2 * c, stream));   // the array keeps the previous call's sums
+    bn_bwd_reduce_kernel<<<grid, kEwThreads, sizeof(float) * 2 * c, stream>>>(da1, da2, y, a, m, c, save_mean, save_invstd, relu, sums);
+    bn_bwd_apply_kernel<<<grid, kEwThreads, 0, stream>>>(da1, da2, y, a, m, c, gamma, save_mean, save_invstd, relu, sums, dy, dres, dgamma, dbeta,
+                                                         acc);
+    B2C_CUDA(cudaGetLastError());
+    return B2C_OK;
+}
+
 }  // extern "C"
