@@ -190,7 +190,7 @@ def run_b2c(args, spec, name, micro_batch, n_micro):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     torch.cuda.set_device(local)
     ctx = binding.Context(local)
-    net = binding.Net(ctx, spec, micro_batch)
+    net = binding.Net(ctx, spec, micro_batch, n_concurrent=args.concurrent if n_micro % args.concurrent == 0 else 1)
     net.load_params(wl.init_params(spec, 0))
     batch = micro_batch * n_micro
     images, labels = wl.image_batch(rank, batch, tag=f"r{rank}")        # each replica gets its own shard
@@ -261,7 +261,7 @@ def run_b2c(args, spec, name, micro_batch, n_micro):
         return
     peaks = measured_peaks()
     work, n_params = algorithmic_work(spec, micro_batch)
-    reps = n_micro * args.steps
+    reps = n_micro * args.steps        # algorithmic work is counted per micro-batch
     kernels = {}
     for fam in ("conv_fwd", "conv_dgrad", "conv_wgrad"):
         ms = fam_ms[fam]
@@ -291,7 +291,7 @@ def run_b2c(args, spec, name, micro_batch, n_micro):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
-        "config": {"workload": name, "global_batch": world * batch, "micro_batch": micro_batch, "n_micro": n_micro, "params": n_params,
+        "config": {"workload": name, "global_batch": world * batch, "micro_batch": micro_batch, "n_micro": n_micro, "micro_batches_per_pass": net.n_concurrent, "params": n_params,
                    "l2": "per-step working set (~0.5 GB of activations) exceeds the 126 MB L2; a 256 MB buffer is rewritten between timed steps (untimed)",
                    "timing": "CUDA events per step on the launching stream, summed; per-launch events enabled (b2c_net_profile_enable)"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(sum(fam_launches.values())),
@@ -309,6 +309,7 @@ def main():
     ap.add_argument("--impl", default="b2c", choices=["b2c", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--concurrent", type=int, default=8, help="micro-batches run side by side per pass")
     args = ap.parse_args()
     builder, micro_batch, n_micro = WORKLOADS[args.workload]
     spec = builder()

@@ -197,6 +197,12 @@ typedef struct {
 
 /* Builds the execution plan for micro-batches of `micro_batch` images of hw x hw x image_c. */
 b2c_status b2c_net_create(b2c_ctx* ctx, const b2c_layer_desc* layers, int n_layers, int micro_batch, b2c_net** out);
+/* As b2c_net_create, but every pass of b2c_train_step runs n_concurrent micro-batches side by side as one
+ * batch of micro_batch*n_concurrent images (larger GEMMs, fewer launches).  BatchNorm statistics stay per
+ * micro-batch, so results equal those of n_concurrent == 1 up to summation order.  The workspace grows by
+ * the same factor and b2c_train_step requires n_micro % n_concurrent == 0. */
+b2c_status b2c_net_create_concurrent(b2c_ctx* ctx, const b2c_layer_desc* layers, int n_layers, int micro_batch,
+                                     int n_concurrent, b2c_net** out);
 void b2c_net_destroy(b2c_net* net);
 /* Elements of the flat parameter arrays (fp32 master, momentum, gradient sum; a bf16 copy and a
  * bf16 dgrad-layout copy of the same length).  Includes zero padding (first conv: input channels

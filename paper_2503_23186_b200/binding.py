@@ -27,7 +27,7 @@ EXPORTS = [
     "b2c_conv2d_fwd", "b2c_bn_relu_fwd", "b2c_avgpool_fwd", "b2c_avgpool_bwd", "b2c_pad_channels",
     "b2c_softmax_xent_fwd_bwd", "b2c_bn_relu_bwd_workspace_bytes", "b2c_bn_relu_bwd", "b2c_bn_relu_bwd_static", "b2c_conv2d_dgrad",
     "b2c_conv2d_wgrad", "b2c_bias_grad", "b2c_grad_accum_sgd_momentum", "b2c_weight_pack_dgrad",
-    "b2c_net_create", "b2c_net_destroy", "b2c_net_param_count", "b2c_net_param_offset",
+    "b2c_net_create", "b2c_net_create_concurrent", "b2c_net_destroy", "b2c_net_param_count", "b2c_net_param_offset",
     "b2c_net_padded_image_channels", "b2c_net_workspace_bytes", "b2c_net_tensor_offset", "b2c_net_bind",
     "b2c_net_sync_weights", "b2c_train_step", "b2c_net_apply_update", "b2c_net_profile_enable", "b2c_net_profile_read",
 ]
@@ -191,14 +191,15 @@ class Context:
 class Net:
     """A layer list bound to device memory; train_step runs the whole optimiser step."""
 
-    def __init__(self, ctx: Context, spec, micro_batch: int):
-        self.ctx, self.spec, self.micro_batch = ctx, spec, micro_batch
+    def __init__(self, ctx: Context, spec, micro_batch: int, n_concurrent: int = 1):
+        self.ctx, self.spec, self.micro_batch, self.n_concurrent = ctx, spec, micro_batch, n_concurrent
         descs = (LayerDesc * len(spec))()
         for i, L in enumerate(spec):
             descs[i] = LayerDesc(LAYER_KINDS[L["kind"]], L["src"], L.get("res", -1), int(L.get("relu", False)), L.get("C", 0), L.get("K", 0),
                                  L.get("R", 0), L.get("stride", 0), L.get("H", 1), L.get("W", 1))
         self.handle = c_void_p()
-        _check(lib().b2c_net_create(ctx.handle, descs, len(spec), micro_batch, byref(self.handle)), "b2c_net_create")
+        _check(lib().b2c_net_create_concurrent(ctx.handle, descs, len(spec), micro_batch, n_concurrent, byref(self.handle)),
+               "b2c_net_create_concurrent")
         self.param_count = lib().b2c_net_param_count(self.handle)
         self.workspace_bytes = lib().b2c_net_workspace_bytes(self.handle)
         self.image_c_pad = lib().b2c_net_padded_image_channels(self.handle)

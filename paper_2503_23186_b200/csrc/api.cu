@@ -154,7 +154,8 @@ struct TensorPlan {
     bool f32 = false;
     bool exists = false;
     long long act_off = -1;        // bytes into the workspace (-1 for tensor 0 when it is read in place)
-    long long stats_off = -1;      // fp64 [2c] sum / sum of squares, for convolution outputs
+    long long stats_off = -1;      // fp64 [groups][2c] sum / sum of squares, for convolution outputs
+    bool fused_stats = false;      // the producing convolution accumulates them in its epilogue
     long long grad_off[2] = {-1, -1};
     int n_contrib = 0;             // gradient contributions expected
     int producer = -1;             // layer index
@@ -177,6 +178,7 @@ inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 struct b2c_net {
     b2c_ctx* ctx = nullptr;
     int micro_batch = 0;
+    int n_conc = 1;            // micro-batches processed side by side in one pass
     int image_h = 0, image_w = 0, image_c = 0, image_c_pad = 0;
     std::vector<LayerPlan> layers;
     std::vector<TensorPlan> tensors;
@@ -224,12 +226,19 @@ extern "C" {
 
 b2c_status b2c_net_create(b2c_ctx* ctx, const b2c_layer_desc* layers, int n_layers, int micro_batch, b2c_net** out)
 {
-    if (!ctx || !layers || !out || n_layers < 1 || micro_batch < 1) return B2C_ERR_INVALID_ARG;
+    return b2c_net_create_concurrent(ctx, layers, n_layers, micro_batch, 1, out);
+}
+
+b2c_status b2c_net_create_concurrent(b2c_ctx* ctx, const b2c_layer_desc* layers, int n_layers, int micro_batch, int n_concurrent, b2c_net** out)
+{
+    if (!ctx || !layers || !out || n_layers < 1 || micro_batch < 1 || n_concurrent < 1) return B2C_ERR_INVALID_ARG;
     *out = nullptr;
     b2c_net* net = new (std::nothrow) b2c_net();
     if (!net) return B2C_ERR_CUDA;
     net->ctx = ctx;
     net->micro_batch = micro_batch;
+    net->n_conc = n_concurrent;
+    const int batch = micro_batch * n_concurrent;   // images per pass
     const char* env = std::getenv("B2C_FUSE_BN_STATS");
     net->fuse_stats = !(env && env[0] == '0');
     net->layers.resize(n_layers);
@@ -247,7 +256,7 @@ b2c_status b2c_net_create(b2c_ctx* ctx, const b2c_layer_desc* layers, int n_laye
     net->image_c_pad = round_up(layers[0].c, 16);
     {
         TensorPlan& t0 = net->tensors[0];
-        t0.n = micro_batch; t0.h = net->image_h; t0.w = net->image_w; t0.c = net->image_c_pad; t0.exists = true;
+        t0.n = batch; t0.h = net->image_h; t0.w = net->image_w; t0.c = net->image_c_pad; t0.exists = true;
         if (net->image_c_pad != net->image_c) t0.act_off = alloc(t0.elems() * 2);
     }
     // forward shapes and parameters
@@ -268,7 +277,7 @@ b2c_status b2c_net_create(b2c_ctx* ctx, const b2c_layer_desc* layers, int n_laye
                 L.c_pad = in.c; L.k_pad = d.k;
                 L.p = (d.h + 2 * pad - d.r) / d.stride + 1; L.q = (d.w + 2 * pad - d.r) / d.stride + 1;
                 if (L.p * d.stride != d.h || L.q * d.stride != d.w || !b2c_is_pow2(L.p) || !b2c_is_pow2(L.q)) return fail(B2C_ERR_UNSUPPORTED_SHAPE);
-                o.n = micro_batch; o.h = L.p; o.w = L.q; o.c = d.k; o.exists = true;
+                o.n = batch; o.h = L.p; o.w = L.q; o.c = d.k; o.exists = true;
                 o.act_off = alloc(o.elems() * 2);
                 L.w_off = palloc((size_t)d.k * d.r * d.r * L.c_pad);
                 net->segs.push_back(b2c_weight_seg{L.w_off, d.k, d.r * d.r, L.c_pad});
@@ -281,13 +290,13 @@ b2c_status b2c_net_create(b2c_ctx* ctx, const b2c_layer_desc* layers, int n_laye
                     const TensorPlan& r = net->tensors[d.res];
                     if (r.n != in.n || r.h != in.h || r.w != in.w || r.c != in.c || d.res == 0) return fail(B2C_ERR_INVALID_ARG);
                 }
-                o = in; o.producer = i; o.n_contrib = 0; o.grad_off[0] = o.grad_off[1] = -1; o.stats_off = -1;
+                o = in; o.producer = i; o.n_contrib = 0; o.grad_off[0] = o.grad_off[1] = -1; o.stats_off = -1; o.fused_stats = false;
                 o.act_off = alloc(o.elems() * 2);
                 break;
             }
             case B2C_LAYER_AVGPOOL: {
                 if (in.f32 || d.c != in.c) return fail(B2C_ERR_INVALID_ARG);
-                o.n = micro_batch; o.h = 1; o.w = 1; o.c = in.c; o.exists = true;
+                o.n = batch; o.h = 1; o.w = 1; o.c = in.c; o.exists = true;
                 o.act_off = alloc(o.elems() * 2);
                 break;
             }
@@ -295,7 +304,7 @@ b2c_status b2c_net_create(b2c_ctx* ctx, const b2c_layer_desc* layers, int n_laye
                 if (in.f32 || in.h != 1 || in.w != 1 || d.c != in.c || d.c % 16 || d.k < 1) return fail(B2C_ERR_INVALID_ARG);
                 L.c_pad = in.c; L.k_pad = round_up(d.k, 64);
                 L.p = L.q = 1;
-                o.n = micro_batch; o.h = 1; o.w = 1; o.c = L.k_pad; o.f32 = true; o.exists = true;
+                o.n = batch; o.h = 1; o.w = 1; o.c = L.k_pad; o.f32 = true; o.exists = true;
                 o.act_off = alloc(o.elems() * 4);
                 L.w_off = palloc((size_t)L.k_pad * L.c_pad);
                 net->segs.push_back(b2c_weight_seg{L.w_off, L.k_pad, 1, L.c_pad});
@@ -341,13 +350,20 @@ b2c_status b2c_net_create(b2c_ctx* ctx, const b2c_layer_desc* layers, int n_laye
     // small per-layer buffers; the fp64 statistics are contiguous so one memset clears them
     for (int i = 0; i < n_layers; ++i) {
         LayerPlan& L = net->layers[i];
-        if (L.d.kind == B2C_LAYER_BN) { L.mean_off = alloc(4 * (size_t)L.d.c); L.invstd_off = alloc(4 * (size_t)L.d.c); }
+        if (L.d.kind == B2C_LAYER_BN) { L.mean_off = alloc(4 * (size_t)L.d.c * n_concurrent); L.invstd_off = alloc(4 * (size_t)L.d.c * n_concurrent); }
     }
     net->stats_begin = (long long)ws;
     for (int i = 0; i < n_layers; ++i) {
         LayerPlan& L = net->layers[i];
-        if (L.d.kind == B2C_LAYER_CONV) net->tensors[i + 1].stats_off = alloc(16 * (size_t)L.d.k);
-        if (L.d.kind == B2C_LAYER_BN) L.bwd_ws_off = alloc(b2c_bn_relu_bwd_workspace_bytes(L.d.c));
+        if (L.d.kind == B2C_LAYER_CONV) {
+            TensorPlan& o = net->tensors[i + 1];
+            o.stats_off = alloc(16 * (size_t)L.d.k * n_concurrent);
+            // the epilogue can own the statistics only if no 128-pixel tile straddles two micro-batches
+            const int pix = L.p * L.q;
+            const int imgs_per_tile = pix >= 128 ? 1 : 128 / pix;
+            o.fused_stats = net->fuse_stats && (micro_batch % imgs_per_tile == 0);
+        }
+        if (L.d.kind == B2C_LAYER_BN) L.bwd_ws_off = alloc(b2c_bn_relu_bwd_workspace_bytes(L.d.c) * n_concurrent);
     }
     net->stats_end = (long long)ws;
     net->ws_bytes = ws;
@@ -431,11 +447,14 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
                           float* loss_dev, int update, void* stream_)
 {
     if (!net || !net->ws || !images || !labels || !loss_dev || n_micro < 1) return B2C_ERR_INVALID_ARG;
+    if (n_micro % net->n_conc) return B2C_ERR_INVALID_ARG;   // whole passes only
     if (!b2c_aligned16(images)) return B2C_ERR_MISALIGNED;
     cudaStream_t stream = (cudaStream_t)stream_;
     if (net->profile && net->spans_used > (1u << 20)) return B2C_ERR_INVALID_ARG;   // read the profile between steps
     b2c_ctx* ctx = net->ctx;
-    const int N = net->micro_batch;
+    const int G = net->n_conc;                 // statistics groups per pass
+    const int N = net->micro_batch * G;        // images per pass
+    const int n_passes = n_micro / G;
     const int n_layers = (int)net->layers.size();
     const __nv_bfloat16* w_bf16 = reinterpret_cast<const __nv_bfloat16*>(net->w_bf16);
     const __nv_bfloat16* w_dg = reinterpret_cast<const __nv_bfloat16*>(net->w_dgrad);
@@ -446,7 +465,7 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
     const size_t image_bytes = (size_t)N * net->image_h * net->image_w * net->image_c * 2;
     if (image_bytes % 16) return B2C_ERR_MISALIGNED;
 
-    for (int mb = 0; mb < n_micro; ++mb) {
+    for (int mb = 0; mb < n_passes; ++mb) {
         const char* img = reinterpret_cast<const char*>(images) + (size_t)mb * image_bytes;
         const int32_t* lab = labels + (size_t)mb * N;
         const void* t0;
@@ -471,20 +490,21 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
                     pb.n = N; pb.ih = d.h; pb.iw = d.w; pb.ic = L.c_pad; pb.oh = L.p; pb.ow = L.q; pb.oc = d.k;
                     pb.r = d.r; pb.stride = d.stride; pb.pad = (d.r - 1) / 2; pb.dgrad = false;
                     pb.in = act_in(d.src); pb.wt = w_bf16 + L.w_off; pb.out = act(i + 1);
-                    pb.stats = net->fuse_stats ? reinterpret_cast<double*>(net->ws + o.stats_off) : nullptr;
+                    pb.stats = o.fused_stats ? reinterpret_cast<double*>(net->ws + o.stats_off) : nullptr;
+                    pb.stats_group_images = net->micro_batch;
                     ProfScope ps_(net, stream, B2C_PROF_CONV_FWD, 1);
                     B2C_TRY(launch_conv_kmajor(ctx, pb, stream));
                     break;
                 }
                 case B2C_LAYER_BN: {
                     const TensorPlan& in = net->tensors[d.src];
-                    const bool ready = net->fuse_stats && in.stats_off >= 0;
+                    const bool ready = in.fused_stats;
                     double* stats = reinterpret_cast<double*>(net->ws + (in.stats_off >= 0 ? in.stats_off : L.bwd_ws_off));
                     ProfScope ps_(net, stream, B2C_PROF_BN_FWD, ready ? 1 : 2);
-                    B2C_TRY(b2c_bn_relu_fwd(ctx, N, in.h, in.w, in.c, act(d.src), stats, ready ? 1 : 0, net->w + L.gamma_off, net->w + L.beta_off,
-                                            d.res >= 0 ? act(d.res) : nullptr, d.relu, 1e-5f, act(i + 1),
-                                            reinterpret_cast<float*>(net->ws + L.mean_off), reinterpret_cast<float*>(net->ws + L.invstd_off),
-                                            nullptr, nullptr, 0.f, stream));
+                    B2C_TRY(launch_bn_fwd(ctx, G, (long long)net->micro_batch * in.h * in.w, in.c, act(d.src), stats, ready, net->w + L.gamma_off,
+                                          net->w + L.beta_off, d.res >= 0 ? act(d.res) : nullptr, d.relu, 1e-5f, act(i + 1),
+                                          reinterpret_cast<float*>(net->ws + L.mean_off), reinterpret_cast<float*>(net->ws + L.invstd_off), nullptr,
+                                          nullptr, 0.f, stream));
                     break;
                 }
                 case B2C_LAYER_AVGPOOL: {
@@ -507,7 +527,8 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
                     const TensorPlan& in = net->tensors[d.src];
                     ProfScope ps_(net, stream, B2C_PROF_OTHER, 1);
                     B2C_TRY(b2c_softmax_xent_fwd_bwd(ctx, N, d.k, reinterpret_cast<const float*>(act(d.src)), in.c, lab,
-                                                     1.f / ((float)N * (float)n_micro), 1.f / (float)N, loss_dev, grad(d.src, L.src_slot), in.c,
+                                                     1.f / ((float)net->micro_batch * (float)n_micro), 1.f / (float)net->micro_batch, loss_dev,
+                                                     grad(d.src, L.src_slot), in.c,
                                                      stream));
                     break;
                 }
@@ -544,11 +565,11 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
                 case B2C_LAYER_BN: {
                     const TensorPlan& in = net->tensors[d.src];
                     ProfScope ps_(net, stream, B2C_PROF_BN_BWD, 2);
-                    B2C_TRY(b2c_bn_relu_bwd(ctx, N, in.h, in.w, in.c, grad(i + 1, 0), o.n_contrib > 1 ? grad(i + 1, 1) : nullptr, act(d.src), act(i + 1),
-                                            net->w + L.gamma_off, reinterpret_cast<float*>(net->ws + L.mean_off),
-                                            reinterpret_cast<float*>(net->ws + L.invstd_off), d.relu, grad(d.src, L.src_slot),
-                                            d.res >= 0 ? grad(d.res, L.res_slot) : nullptr, net->g + L.gamma_off, net->g + L.beta_off, 1,
-                                            net->ws + L.bwd_ws_off, b2c_bn_relu_bwd_workspace_bytes(in.c), stream));
+                    B2C_TRY(launch_bn_bwd(ctx, G, (long long)net->micro_batch * in.h * in.w, in.c, grad(i + 1, 0), o.n_contrib > 1 ? grad(i + 1, 1) : nullptr,
+                                          act(d.src), act(i + 1), net->w + L.gamma_off, reinterpret_cast<float*>(net->ws + L.mean_off),
+                                          reinterpret_cast<float*>(net->ws + L.invstd_off), d.relu, grad(d.src, L.src_slot),
+                                          d.res >= 0 ? grad(d.res, L.res_slot) : nullptr, net->g + L.gamma_off, net->g + L.beta_off, 1,
+                                          reinterpret_cast<double*>(net->ws + L.bwd_ws_off), stream));
                     break;
                 }
                 case B2C_LAYER_CONV: {

@@ -36,6 +36,7 @@ struct alignas(64) ConvKParams {
     int out_is_f32;
     const float* bias;
     double* stats;
+    int stats_group_images;          // images per BatchNorm statistics group (0: one group)
     unsigned* status;
     unsigned spin_limit;
 };
@@ -229,8 +230,9 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
             for (int c = et; c < p.n_tile; c += 128) {
                 const int ch = ktile * p.n_tile + c;
                 if (ch < p.oc_valid) {
-                    atomicAdd(p.stats + ch, (double)s_stats[c]);
-                    atomicAdd(p.stats + p.oc_valid + ch, (double)s_stats[256 + c]);
+                    double* st = p.stats + (size_t)(p.stats_group_images > 0 ? n0 / p.stats_group_images : 0) * 2 * p.oc_valid;
+                    atomicAdd(st + ch, (double)s_stats[c]);
+                    atomicAdd(st + p.oc_valid + ch, (double)s_stats[256 + c]);
                 }
             }
         }
@@ -403,6 +405,8 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
     p.out_is_f32 = pb.out_f32 ? 1 : 0;
     p.bias = pb.bias;
     p.stats = pb.out_f32 ? nullptr : pb.stats;
+    p.stats_group_images = pb.stats_group_images;
+    if (p.stats && p.stats_group_images > 0 && (p.stats_group_images % p.bn) != 0) return B2C_ERR_UNSUPPORTED_SHAPE;  // a tile must not straddle groups
     p.status = ctx->d_status;
     p.spin_limit = ctx->spin_limit;
 

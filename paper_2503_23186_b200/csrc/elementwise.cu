@@ -33,33 +33,48 @@ __device__ __forceinline__ uint4 pack8(const float (&f)[8])
 }
 __device__ __forceinline__ uint4 ld16(const void* base, long long vec_index) { return __ldg(reinterpret_cast<const uint4*>(base) + vec_index); }
 
-// Row/channel-group decomposition shared by the row-walking kernels.
+// Row/channel-group decomposition shared by the row-walking kernels.  blockIdx.y selects the
+// statistics group (a micro-batch): rows [g*m, (g+1)*m) of the tensor, its own accumulators and
+// its own saved mean / invstd.  Each thread keeps kRowsUnroll independent 16-byte loads per tensor
+// in flight (rows beyond the end read as zero and contribute nothing).
+static constexpr int kRowsUnroll = 4;
 struct RowWalk {
     int groups;         // c / 8
     int rows_per_iter;  // rows a block covers per step
     __device__ RowWalk(int c) : groups(c >> 3), rows_per_iter(kEwThreads / (c >> 3)) {}
 };
+__device__ __forceinline__ uint4 ld16_or_zero(const void* base, long long vec_index, bool ok)
+{
+    return ok ? __ldg(reinterpret_cast<const uint4*>(base) + vec_index) : make_uint4(0u, 0u, 0u, 0u);
+}
 
 // ------------------------------------------------------------------------------ BN forward
-__global__ void __launch_bounds__(kEwThreads) bn_stats_kernel(const void* __restrict__ y, long long m, int c, double* __restrict__ stats)
+__global__ void __launch_bounds__(kEwThreads, 2) bn_stats_kernel(const void* __restrict__ y, long long m, int c, double* __restrict__ stats)
 {
     extern __shared__ float s_acc[];  // [2*c]
     for (int i = threadIdx.x; i < 2 * c; i += kEwThreads) s_acc[i] = 0.f;
     __syncthreads();
     const RowWalk rw(c);
     const int g = threadIdx.x % rw.groups, rl = threadIdx.x / rw.groups;
+    const long long base = (long long)blockIdx.y * m * rw.groups;
     if (rl < rw.rows_per_iter) {
         float s[8], ss[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) s[i] = ss[i] = 0.f;
         const long long step = (long long)gridDim.x * rw.rows_per_iter;
-        for (long long r = (long long)blockIdx.x * rw.rows_per_iter + rl; r < m; r += step) {
-            float f[8];
-            unpack8(ld16(y, r * rw.groups + g), f);
+        for (long long r = (long long)blockIdx.x * rw.rows_per_iter + rl; r < m; r += kRowsUnroll * step) {
+            uint4 v[kRowsUnroll];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                s[i] += f[i];
-                ss[i] = fmaf(f[i], f[i], ss[i]);
+            for (int u = 0; u < kRowsUnroll; ++u) v[u] = ld16_or_zero(y, base + (r + u * step) * rw.groups + g, r + u * step < m);
+#pragma unroll
+            for (int u = 0; u < kRowsUnroll; ++u) {
+                float f[8];
+                unpack8(v[u], f);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    s[i] += f[i];
+                    ss[i] = fmaf(f[i], f[i], ss[i]);
+                }
             }
         }
 #pragma unroll
@@ -69,7 +84,8 @@ __global__ void __launch_bounds__(kEwThreads) bn_stats_kernel(const void* __rest
         }
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < 2 * c; i += kEwThreads) atomicAdd(stats + i, (double)s_acc[i]);
+    double* out = stats + (size_t)blockIdx.y * 2 * c;
+    for (int i = threadIdx.x; i < 2 * c; i += kEwThreads) atomicAdd(out + i, (double)s_acc[i]);
 }
 
 // mean and 1/sqrt(var+eps) from the fp64 sums, identically in every thread that needs them.
@@ -83,21 +99,23 @@ __device__ __forceinline__ void bn_moments(const double* stats, int c, int ch, d
     invstd = rsqrtf((float)v + eps);
 }
 
-__global__ void __launch_bounds__(kEwThreads) bn_apply_kernel(const void* __restrict__ y, long long m, int c, const double* __restrict__ stats,
-                                                              const float* __restrict__ gamma, const float* __restrict__ beta,
-                                                              const void* __restrict__ residual, int relu, float eps, void* __restrict__ a,
-                                                              float* save_mean, float* save_invstd, float* run_mean, float* run_var,
-                                                              float momentum)
+__global__ void __launch_bounds__(kEwThreads, 2) bn_apply_kernel(const void* __restrict__ y, long long m, int c, const double* __restrict__ stats_all,
+                                                                 const float* __restrict__ gamma, const float* __restrict__ beta,
+                                                                 const void* __restrict__ residual, int relu, float eps, void* __restrict__ a,
+                                                                 float* save_mean, float* save_invstd, float* run_mean, float* run_var,
+                                                                 float momentum)
 {
     const RowWalk rw(c);
     const int g = threadIdx.x % rw.groups, rl = threadIdx.x / rw.groups;
     const double inv_m = 1.0 / (double)m;
+    const double* stats = stats_all + (size_t)blockIdx.y * 2 * c;
+    const long long base = (long long)blockIdx.y * m * rw.groups;
     if (blockIdx.x == 0) {
         for (int ch = threadIdx.x; ch < c; ch += kEwThreads) {
             float mean, invstd, var;
             bn_moments(stats, c, ch, inv_m, eps, mean, invstd, var);
-            save_mean[ch] = mean;
-            save_invstd[ch] = invstd;
+            save_mean[(size_t)blockIdx.y * c + ch] = mean;
+            save_invstd[(size_t)blockIdx.y * c + ch] = invstd;
             if (run_mean != nullptr) {
                 const float unbiased = m > 1 ? var * (float)((double)m / (double)(m - 1)) : var;
                 run_mean[ch] = (1.f - momentum) * run_mean[ch] + momentum * mean;
@@ -106,69 +124,87 @@ __global__ void __launch_bounds__(kEwThreads) bn_apply_kernel(const void* __rest
         }
     }
     if (rl >= rw.rows_per_iter) return;
-    float scale[8], shift[8];
+    float scale[8], shift[8], bt[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         float mean, invstd, var;
         bn_moments(stats, c, g * 8 + i, inv_m, eps, mean, invstd, var);
-        const float gm = gamma[g * 8 + i];
         // z = gamma*(y-mean)*invstd + beta, evaluated as (y-mean)*(gamma*invstd) + beta
-        scale[i] = gm * invstd;
+        scale[i] = gamma[g * 8 + i] * invstd;
         shift[i] = mean;
+        bt[i] = beta[g * 8 + i];
     }
-    float bt[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) bt[i] = beta[g * 8 + i];
     const long long step = (long long)gridDim.x * rw.rows_per_iter;
-    for (long long r = (long long)blockIdx.x * rw.rows_per_iter + rl; r < m; r += step) {
-        const long long vi = r * rw.groups + g;
-        float f[8], res[8];
-        unpack8(ld16(y, vi), f);
-        if (residual != nullptr) unpack8(ld16(residual, vi), res);
+    for (long long r = (long long)blockIdx.x * rw.rows_per_iter + rl; r < m; r += kRowsUnroll * step) {
+        uint4 vy[kRowsUnroll], vr[kRowsUnroll];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            float z = fmaf(f[i] - shift[i], scale[i], bt[i]);
-            if (residual != nullptr) z += res[i];
-            f[i] = (relu && z < 0.f) ? 0.f : z;
+        for (int u = 0; u < kRowsUnroll; ++u) {
+            const bool ok = r + u * step < m;
+            const long long vi = base + (r + u * step) * rw.groups + g;
+            vy[u] = ld16_or_zero(y, vi, ok);
+            if (residual != nullptr) vr[u] = ld16_or_zero(residual, vi, ok);
         }
-        reinterpret_cast<uint4*>(a)[vi] = pack8(f);
+#pragma unroll
+        for (int u = 0; u < kRowsUnroll; ++u) {
+            if (r + u * step >= m) break;
+            float f[8], res[8];
+            unpack8(vy[u], f);
+            if (residual != nullptr) unpack8(vr[u], res);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                float z = fmaf(f[i] - shift[i], scale[i], bt[i]);
+                if (residual != nullptr) z += res[i];
+                f[i] = (relu && z < 0.f) ? 0.f : z;
+            }
+            reinterpret_cast<uint4*>(a)[base + (r + u * step) * rw.groups + g] = pack8(f);
+        }
     }
 }
 
 // ------------------------------------------------------------------------------ BN backward
-__global__ void __launch_bounds__(kEwThreads) bn_bwd_reduce_kernel(const void* __restrict__ da1, const void* __restrict__ da2,
-                                                                   const void* __restrict__ y, const void* __restrict__ a, long long m, int c,
-                                                                   const float* __restrict__ mean, const float* __restrict__ invstd, int relu,
-                                                                   double* __restrict__ sums /* [2c]: dbeta, dgamma */)
+// Pass 1: S1 = sum dz, S2 = sum dz*y per channel (dgamma = invstd*(S2 - mean*S1) is formed in fp64 by pass 2).
+__global__ void __launch_bounds__(kEwThreads, 2) bn_bwd_reduce_kernel(const void* __restrict__ da1, const void* __restrict__ da2,
+                                                                      const void* __restrict__ y, const void* __restrict__ a, long long m, int c,
+                                                                      int relu, double* __restrict__ sums_all /* [G][2c] */)
 {
     extern __shared__ float s_acc[];
     for (int i = threadIdx.x; i < 2 * c; i += kEwThreads) s_acc[i] = 0.f;
     __syncthreads();
     const RowWalk rw(c);
     const int g = threadIdx.x % rw.groups, rl = threadIdx.x / rw.groups;
+    const long long base = (long long)blockIdx.y * m * rw.groups;
     if (rl < rw.rows_per_iter) {
-        float mu[8], is[8], sb[8], sg[8];
+        float sb[8], sg[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            mu[i] = mean[g * 8 + i];
-            is[i] = invstd[g * 8 + i];
-            sb[i] = sg[i] = 0.f;
-        }
+        for (int i = 0; i < 8; ++i) sb[i] = sg[i] = 0.f;
         const long long step = (long long)gridDim.x * rw.rows_per_iter;
-        for (long long r = (long long)blockIdx.x * rw.rows_per_iter + rl; r < m; r += step) {
-            const long long vi = r * rw.groups + g;
-            float d[8], d2[8], fy[8], fa[8];
-            unpack8(ld16(da1, vi), d);
-            if (da2 != nullptr) unpack8(ld16(da2, vi), d2);
-            unpack8(ld16(y, vi), fy);
-            if (relu) unpack8(ld16(a, vi), fa);
+        constexpr int U = 2;
+        for (long long r = (long long)blockIdx.x * rw.rows_per_iter + rl; r < m; r += U * step) {
+            uint4 v1[U], v2[U], vy[U], va[U];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                float dz = d[i];
-                if (da2 != nullptr) dz += d2[i];
-                if (relu && !(fa[i] > 0.f)) dz = 0.f;
-                sb[i] += dz;
-                sg[i] = fmaf(dz, (fy[i] - mu[i]) * is[i], sg[i]);
+            for (int u = 0; u < U; ++u) {
+                const bool ok = r + u * step < m;
+                const long long vi = base + (r + u * step) * rw.groups + g;
+                v1[u] = ld16_or_zero(da1, vi, ok);
+                if (da2 != nullptr) v2[u] = ld16_or_zero(da2, vi, ok);
+                vy[u] = ld16_or_zero(y, vi, ok);
+                if (relu) va[u] = ld16_or_zero(a, vi, ok);
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                float d[8], d2[8], fy[8], fa[8];
+                unpack8(v1[u], d);
+                if (da2 != nullptr) unpack8(v2[u], d2);
+                unpack8(vy[u], fy);
+                if (relu) unpack8(va[u], fa);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    float dz = d[i];
+                    if (da2 != nullptr) dz += d2[i];
+                    if (relu && !(fa[i] > 0.f)) dz = 0.f;
+                    sb[i] += dz;
+                    sg[i] = fmaf(dz, fy[i], sg[i]);
+                }
             }
         }
 #pragma unroll
@@ -178,56 +214,83 @@ __global__ void __launch_bounds__(kEwThreads) bn_bwd_reduce_kernel(const void* _
         }
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < 2 * c; i += kEwThreads) atomicAdd(sums + i, (double)s_acc[i]);
+    double* out = sums_all + (size_t)blockIdx.y * 2 * c;
+    for (int i = threadIdx.x; i < 2 * c; i += kEwThreads) atomicAdd(out + i, (double)s_acc[i]);
 }
 
-__global__ void __launch_bounds__(kEwThreads) bn_bwd_apply_kernel(const void* __restrict__ da1, const void* __restrict__ da2,
-                                                                  const void* __restrict__ y, const void* __restrict__ a, long long m, int c,
-                                                                  const float* __restrict__ gamma, const float* __restrict__ mean,
-                                                                  const float* __restrict__ invstd, int relu, const double* __restrict__ sums,
-                                                                  void* __restrict__ dy, void* __restrict__ dres, float* dgamma, float* dbeta,
-                                                                  int acc)
+// Pass 2: dy = gamma*invstd*(dz - dbeta/m - xhat*dgamma/m), dres = dz; block 0 of each group emits dgamma, dbeta.
+__global__ void __launch_bounds__(kEwThreads, 2) bn_bwd_apply_kernel(const void* __restrict__ da1, const void* __restrict__ da2,
+                                                                     const void* __restrict__ y, const void* __restrict__ a, long long m, int c,
+                                                                     const float* __restrict__ gamma, const float* __restrict__ mean_all,
+                                                                     const float* __restrict__ invstd_all, int relu,
+                                                                     const double* __restrict__ sums_all, void* __restrict__ dy,
+                                                                     void* __restrict__ dres, float* dgamma, float* dbeta, int acc)
 {
     const RowWalk rw(c);
     const int g = threadIdx.x % rw.groups, rl = threadIdx.x / rw.groups;
+    const double* sums = sums_all + (size_t)blockIdx.y * 2 * c;
+    const float* mean = mean_all + (size_t)blockIdx.y * c;
+    const float* invstd = invstd_all + (size_t)blockIdx.y * c;
+    const long long base = (long long)blockIdx.y * m * rw.groups;
     if (blockIdx.x == 0) {
         for (int ch = threadIdx.x; ch < c; ch += kEwThreads) {
-            const float db = (float)sums[ch], dg = (float)sums[c + ch];
-            dbeta[ch] = acc ? dbeta[ch] + db : db;
-            dgamma[ch] = acc ? dgamma[ch] + dg : dg;
+            const double s1 = sums[ch], s2 = sums[c + ch];
+            const float db = (float)s1, dg = (float)((double)invstd[ch] * (s2 - (double)mean[ch] * s1));
+            if (gridDim.y == 1) {
+                dbeta[ch] = acc ? dbeta[ch] + db : db;
+                dgamma[ch] = acc ? dgamma[ch] + dg : dg;
+            } else {   // several groups add into the same gradient (always accumulating)
+                atomicAdd(dbeta + ch, db);
+                atomicAdd(dgamma + ch, dg);
+            }
         }
     }
     if (rl >= rw.rows_per_iter) return;
-    const float inv_m = (float)(1.0 / (double)m);
-    float mu[8], is[8], k0[8], kb[8], kg[8];
+    const double inv_m = 1.0 / (double)m;
+    float mu[8], k0[8], kb[8], kg[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         const int ch = g * 8 + i;
+        const double s1 = sums[ch], s2 = sums[c + ch];
+        const double is = (double)invstd[ch], dgam = is * (s2 - (double)mean[ch] * s1);
         mu[i] = mean[ch];
-        is[i] = invstd[ch];
-        k0[i] = gamma[ch] * is[i];                 // gamma*invstd
-        kb[i] = (float)(sums[ch]) * inv_m;         // dbeta/m
-        kg[i] = (float)(sums[c + ch]) * inv_m;     // dgamma/m
+        k0[i] = gamma[ch] * invstd[ch];                        // gamma*invstd
+        kb[i] = (float)(s1 * inv_m);                           // dbeta/m
+        kg[i] = (float)(dgam * inv_m * is);                    // (dgamma/m)*invstd, multiplies (y-mean)
     }
     const long long step = (long long)gridDim.x * rw.rows_per_iter;
-    for (long long r = (long long)blockIdx.x * rw.rows_per_iter + rl; r < m; r += step) {
-        const long long vi = r * rw.groups + g;
-        float d[8], d2[8], fy[8], fa[8], o[8];
-        unpack8(ld16(da1, vi), d);
-        if (da2 != nullptr) unpack8(ld16(da2, vi), d2);
-        unpack8(ld16(y, vi), fy);
-        if (relu) unpack8(ld16(a, vi), fa);
+    constexpr int U = 2;
+    for (long long r = (long long)blockIdx.x * rw.rows_per_iter + rl; r < m; r += U * step) {
+        uint4 v1[U], v2[U], vy[U], va[U];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            float dz = d[i];
-            if (da2 != nullptr) dz += d2[i];
-            if (relu && !(fa[i] > 0.f)) dz = 0.f;
-            d[i] = dz;
-            const float xhat = (fy[i] - mu[i]) * is[i];
-            o[i] = k0[i] * (dz - kb[i] - xhat * kg[i]);
+        for (int u = 0; u < U; ++u) {
+            const bool ok = r + u * step < m;
+            const long long vi = base + (r + u * step) * rw.groups + g;
+            v1[u] = ld16_or_zero(da1, vi, ok);
+            if (da2 != nullptr) v2[u] = ld16_or_zero(da2, vi, ok);
+            vy[u] = ld16_or_zero(y, vi, ok);
+            if (relu) va[u] = ld16_or_zero(a, vi, ok);
         }
-        reinterpret_cast<uint4*>(dy)[vi] = pack8(o);
-        if (dres != nullptr) reinterpret_cast<uint4*>(dres)[vi] = pack8(d);
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (r + u * step >= m) break;
+            float d[8], d2[8], fy[8], fa[8], o[8];
+            unpack8(v1[u], d);
+            if (da2 != nullptr) unpack8(v2[u], d2);
+            unpack8(vy[u], fy);
+            if (relu) unpack8(va[u], fa);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                float dz = d[i];
+                if (da2 != nullptr) dz += d2[i];
+                if (relu && !(fa[i] > 0.f)) dz = 0.f;
+                d[i] = dz;
+                o[i] = k0[i] * (dz - kb[i] - (fy[i] - mu[i]) * kg[i]);
+            }
+            const long long vi = base + (r + u * step) * rw.groups + g;
+            reinterpret_cast<uint4*>(dy)[vi] = pack8(o);
+            if (dres != nullptr) reinterpret_cast<uint4*>(dres)[vi] = pack8(d);
+        }
     }
 }
 
@@ -371,11 +434,43 @@ __global__ void weight_pack_dgrad_kernel(const __grid_constant__ PackSegs segs, 
 }
 
 // ------------------------------------------------------------------------------ launchers
-static int ew_grid(b2c_ctx* ctx, long long m, int rows_per_iter)
+// Blocks per statistics group: one wave of two resident blocks per SM across all groups.
+static int ew_grid(b2c_ctx* ctx, int n_groups, long long m, int rows_per_iter)
 {
     long long blocks = (m + rows_per_iter - 1) / rows_per_iter;
-    const long long cap = (long long)ctx->sm_count * 8;
+    long long cap = ((long long)ctx->sm_count * 2 + n_groups - 1) / n_groups;
+    if (cap < 1) cap = 1;
     return (int)(blocks < cap ? (blocks < 1 ? 1 : blocks) : cap);
+}
+
+b2c_status launch_bn_fwd(b2c_ctx* ctx, int G, long long m, int c, const void* y, double* stats, bool stats_ready, const float* gamma,
+                         const float* beta, const void* residual, int relu, float eps, void* a, float* save_mean, float* save_invstd,
+                         float* run_mean, float* run_var, float momentum, cudaStream_t stream)
+{
+    const int rows_per_iter = kEwThreads / (c / 8);
+    dim3 grid((unsigned)ew_grid(ctx, G, m, rows_per_iter), (unsigned)G);
+    if (!stats_ready) {
+        B2C_CUDA(cudaMemsetAsync(stats, 0, sizeof(double) * 2 * c * G, stream));
+        bn_stats_kernel<<<grid, kEwThreads, sizeof(float) * 2 * c, stream>>>(y, m, c, stats);
+    }
+    bn_apply_kernel<<<grid, kEwThreads, 0, stream>>>(y, m, c, stats, gamma, beta, residual, relu, eps, a, save_mean, save_invstd, run_mean, run_var,
+                                                     momentum);
+    B2C_CUDA(cudaGetLastError());
+    return B2C_OK;
+}
+
+b2c_status launch_bn_bwd(b2c_ctx* ctx, int G, long long m, int c, const void* da1, const void* da2, const void* y, const void* a,
+                         const float* gamma, const float* save_mean, const float* save_invstd, int relu, void* dy, void* dres, float* dgamma,
+                         float* dbeta, int acc, double* sums, cudaStream_t stream)
+{
+    const int rows_per_iter = kEwThreads / (c / 8);
+    dim3 grid((unsigned)ew_grid(ctx, G, m, rows_per_iter), (unsigned)G);
+    B2C_CUDA(cudaMemsetAsync(sums, 0, sizeof(double) * 2 * c * G, stream));
+    bn_bwd_reduce_kernel<<<grid, kEwThreads, sizeof(float) * 2 * c, stream>>>(da1, da2, y, a, m, c, relu, sums);
+    bn_bwd_apply_kernel<<<grid, kEwThreads, 0, stream>>>(da1, da2, y, a, m, c, gamma, save_mean, save_invstd, relu, sums, dy, dres, dgamma, dbeta,
+                                                         acc);
+    B2C_CUDA(cudaGetLastError());
+    return B2C_OK;
 }
 
 }  // namespace b2c
@@ -394,17 +489,8 @@ b2c_status b2c_bn_relu_fwd(b2c_ctx* ctx, int n, int h, int w, int c, const void*
     if ((run_mean == nullptr) != (run_var == nullptr)) return B2C_ERR_INVALID_ARG;
     if (!b2c_aligned16(y) || !b2c_aligned16(a) || (residual && !b2c_aligned16(residual)) || (reinterpret_cast<uintptr_t>(ch_stats) & 7u))
         return B2C_ERR_MISALIGNED;
-    const long long m = (long long)n * h * w;
-    const int rows_per_iter = kEwThreads / (c / 8);
-    const int grid = ew_grid(ctx, m, rows_per_iter);
-    if (!stats_ready) {
-        B2C_CUDA(cudaMemsetAsync(ch_stats, 0, sizeof(double) * 2 * c, stream));
-        bn_stats_kernel<<<grid, kEwThreads, sizeof(float) * 2 * c, stream>>>(y, m, c, ch_stats);
-    }
-    bn_apply_kernel<<<grid, kEwThreads, 0, stream>>>(y, m, c, ch_stats, gamma, beta, residual, relu, eps, a, save_mean, save_invstd, run_mean,
-                                                     run_var, momentum);
-    B2C_CUDA(cudaGetLastError());
-    return B2C_OK;
+    return launch_bn_fwd(ctx, 1, (long long)n * h * w, c, y, ch_stats, stats_ready != 0, gamma, beta, residual, relu, eps, a, save_mean, save_invstd,
+                         run_mean, run_var, momentum, stream);
 }
 
 size_t b2c_bn_relu_bwd_workspace_bytes(int c) { return c > 0 ? sizeof(double) * 2 * (size_t)c : 0; }
@@ -421,16 +507,8 @@ b2c_status b2c_bn_relu_bwd(b2c_ctx* ctx, int n, int h, int w, int c, const void*
     if (!b2c_aligned16(da1) || (da2 && !b2c_aligned16(da2)) || !b2c_aligned16(y) || (a && !b2c_aligned16(a)) || !b2c_aligned16(dy) ||
         (dres && !b2c_aligned16(dres)) || (reinterpret_cast<uintptr_t>(ws) & 7u))
         return B2C_ERR_MISALIGNED;
-    const long long m = (long long)n * h * w;
-    const int rows_per_iter = kEwThreads / (c / 8);
-    const int grid = ew_grid(ctx, m, rows_per_iter);
-    double* sums = reinterpret_cast<double*>(ws);
-    B2C_CUDA(cudaMemsetAsync(sums, 0, sizeof(double) * 2 * c, stream));
-    bn_bwd_reduce_kernel<<<grid, kEwThreads, sizeof(float) * 2 * c, stream>>>(da1, da2, y, a, m, c, save_mean, save_invstd, relu, sums);
-    bn_bwd_apply_kernel<<<grid, kEwThreads, 0, stream>>>(da1, da2, y, a, m, c, gamma, save_mean, save_invstd, relu, sums, dy, dres, dgamma, dbeta,
-                                                         acc);
-    B2C_CUDA(cudaGetLastError());
-    return B2C_OK;
+    return launch_bn_bwd(ctx, 1, (long long)n * h * w, c, da1, da2, y, a, gamma, save_mean, save_invstd, relu, dy, dres, dgamma, dbeta, acc,
+                         reinterpret_cast<double*>(ws), stream);
 }
 
 b2c_status b2c_avgpool_fwd(b2c_ctx* ctx, int n, int hw, int c, const void* a, void* pooled, void* stream_)
@@ -557,16 +635,9 @@ b2c_status b2c_bn_relu_bwd_static(b2c_ctx* ctx, int n, int h, int w, int c, cons
         if (cudaGetSymbolAddress((void**)&ptr, g_bn_bwd_static_scratch) != cudaSuccess || ptr == nullptr) return B2C_ERR_CUDA;
         g_bn_bwd_static_ptr[current] = ptr;
     }
-    double* sums = g_bn_bwd_static_ptr[current];
-    const long long m = (long long)n * h * w;
-    const int rows_per_iter = kEwThreads / (c / 8);
-    const int grid = ew_grid(ctx, m, rows_per_iter);
-    B2C_CUDA(cudaMemsetAsync(sums, 0, sizeof(double) * 2 * c, stream));   // the array keeps the previous call's sums
-    bn_bwd_reduce_kernel<<<grid, kEwThreads, sizeof(float) * 2 * c, stream>>>(da1, da2, y, a, m, c, save_mean, save_invstd, relu, sums);
-    bn_bwd_apply_kernel<<<grid, kEwThreads, 0, stream>>>(da1, da2, y, a, m, c, gamma, save_mean, save_invstd, relu, sums, dy, dres, dgamma, dbeta,
-                                                         acc);
-    B2C_CUDA(cudaGetLastError());
-    return B2C_OK;
+    // the array keeps the previous call's sums: the launcher clears the part this call uses
+    return launch_bn_bwd(ctx, 1, (long long)n * h * w, c, da1, da2, y, a, gamma, save_mean, save_invstd, relu, dy, dres, dgamma, dbeta, acc,
+                         g_bn_bwd_static_ptr[current], stream);
 }
 
 }  // extern "C"

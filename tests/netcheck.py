@@ -123,9 +123,10 @@ def _wgrad_samples(rng, dy, x, R, stride, pad, count):
     return idx, out
 
 
-def check_step(net, spec, images, labels, n, n_micro_scale=1, sample=None, seed=0):
+def check_step(net, spec, images, labels, n, n_micro_scale=1, sample=None, seed=0, groups=1):
     """Checks the micro-batch whose state is in the workspace (run train_step with n_micro=1, update=False
-    first).  `images` are the logical (unpadded) images of that micro-batch.  Returns a Report."""
+    first).  `images` are the logical (unpadded) images of that pass: `groups` micro-batches side by side, each
+    with its own BatchNorm statistics (n = total images).  Returns a Report."""
     rep = Report()
     rng = np.random.default_rng(seed)
     rb, rf = oracle.round_bf16, oracle.round_f32
@@ -163,11 +164,15 @@ def check_step(net, spec, images, labels, n, n_micro_scale=1, sample=None, seed=
                 rep.add(f"{name} fwd", y, rb(oracle.conv2d_fwd(x, w, L["stride"], L["pad"])))
         elif k == "bn":
             y = A(L["src"])
-            mean, var, invstd = oracle.bn_stats(y, 1e-5)
-            mean, invstd = rf(mean), rf(invstd)
-            saved[i] = (mean, invstd)
             res = A(L["res"]) if L["res"] >= 0 else None
-            rep.add(f"{name} fwd", A(i + 1), rb(oracle.bn_relu_apply(y, mean, invstd, wm[f"gamma{i}"], wm[f"beta{i}"], res, L["relu"])))
+            per, saved[i], outs = n // groups, [], []
+            for gi in range(groups):
+                sl = slice(gi * per, (gi + 1) * per)
+                mean, var, invstd = oracle.bn_stats(y[sl], 1e-5)
+                mean, invstd = rf(mean), rf(invstd)
+                saved[i].append((mean, invstd))
+                outs.append(oracle.bn_relu_apply(y[sl], mean, invstd, wm[f"gamma{i}"], wm[f"beta{i}"], None if res is None else res[sl], L["relu"]))
+            rep.add(f"{name} fwd", A(i + 1), rb(np.concatenate(outs)))
         elif k == "avgpool":
             rep.add(f"{name} fwd", A(i + 1), rb(oracle.avgpool_fwd(A(L["src"]))))
         elif k == "fc":
@@ -175,7 +180,7 @@ def check_step(net, spec, images, labels, n, n_micro_scale=1, sample=None, seed=
             rep.add(f"{name} fwd", A(i + 1)[:, :L["K"]], z)
         elif k == "xent":
             z = A(L["src"])[:, :L["K"]]
-            loss, dz = oracle.softmax_xent(z, labels, 1.0 / n)
+            loss, dz = oracle.softmax_xent(z, labels, float(groups) / n)
             rep.add("loss", np.array([net.loss.item() * n_micro_scale]), np.array([loss]), 1e-5, 1e-5)
             rep.add("dlogits", grad(L["src"], slots[i][0])[:, :L["K"]], rb(dz))
     for i in reversed(range(len(spec))):
@@ -191,9 +196,16 @@ def check_step(net, spec, images, labels, n, n_micro_scale=1, sample=None, seed=
             rep.add(f"{name} bwd", grad(L["src"], s_slot), rb(oracle.avgpool_bwd(grad(i + 1, 0), L["H"], L["W"])))
         elif k == "bn":
             two = n_contrib[i + 1] == 2
-            mean, invstd = saved[i]
-            dy, dres, dg, db = oracle.bn_relu_bwd(grad(i + 1, 0), grad(i + 1, 1) if two else None, A(L["src"]), A(i + 1), wm[f"gamma{i}"], mean,
-                                                  invstd, L["relu"], L["res"] >= 0)
+            per, parts = n // groups, []
+            g1, g2 = grad(i + 1, 0), (grad(i + 1, 1) if two else None)
+            for gi in range(groups):
+                sl = slice(gi * per, (gi + 1) * per)
+                mean, invstd = saved[i][gi]
+                parts.append(oracle.bn_relu_bwd(g1[sl], None if g2 is None else g2[sl], A(L["src"])[sl], A(i + 1)[sl], wm[f"gamma{i}"], mean, invstd,
+                                                L["relu"], L["res"] >= 0))
+            dy = np.concatenate([q[0] for q in parts])
+            dres = np.concatenate([q[1] for q in parts]) if L["res"] >= 0 else None
+            dg, db = sum(q[2] for q in parts), sum(q[3] for q in parts)
             rep.add(f"{name} bwd dy", grad(L["src"], s_slot), rb(dy))
             if L["res"] >= 0:
                 rep.add(f"{name} bwd dres", grad(L["res"], r_slot), rb(dres))

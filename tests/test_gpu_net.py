@@ -240,3 +240,27 @@ def test_teacher_forced_report_resnet18(ctx, capsys):
             print("teacher-forced %-22s relF=%.3e max=%.3e %s" % (name, rel, mx, "" if ok else "FAIL"))
     rep.assert_ok()
     net.close()
+
+
+def test_concurrent_micro_batches_match_sequential(ctx):
+    """Four micro-batches run side by side in one pass (BatchNorm statistics per micro-batch) against the same four run
+    one after the other: teacher-forced against the oracle, and gradient sums against the sequential run."""
+    from paper_2503_23186_b200 import binding
+    from netcheck import check_step
+    spec = wl.tiny_net_spec(classes=10, hw=16, c=3, width=64, width2=128)
+    params = wl.perturb_bn_params(wl.init_params(spec, 4), 4)
+    images, labels = wl.image_batch(4, 4 * 8, hw=16, c=3, classes=10)
+    d_img, d_lab = dev_bf16(images), torch.from_numpy(labels).cuda()
+    seq = binding.Net(ctx, spec, 8)
+    seq.load_params(params)
+    loss_seq = seq.train_step(d_img, d_lab, 4, LR, MU, WD, update=False).item()
+    par = binding.Net(ctx, spec, 8, n_concurrent=4)
+    par.load_params(params)
+    loss_par = par.train_step(d_img, d_lab, 4, LR, MU, WD, update=False).item()
+    assert ctx.device_status() == 0
+    check_step(par, spec, images, labels, 32, groups=4).assert_ok()
+    assert abs(loss_par - loss_seq) <= 1e-4 * abs(loss_seq)
+    gs, gp = seq.unpack(seq.g), par.unpack(par.g)
+    for name in sorted(params):
+        assert_close(gp[name], gs[name], f"grad {name} (concurrent vs sequential)", 1e-2, 3e-2)
+    seq.close(); par.close()
