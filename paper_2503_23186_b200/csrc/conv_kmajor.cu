@@ -8,9 +8,16 @@
 // gather from four "parity views" of the input (even/odd rows x even/odd columns), each a plain
 // strided tensor map; the stride-2 data gradient is four sub-problems, one per output parity.
 // B is a box (kb channels, one tap, n_tile output channels) of the [out][tap][in] weights.
-// Accumulators live in TMEM; four epilogue warps read them back, add the bias, round to bf16,
-// accumulate per-channel sum / sum of squares for BatchNorm, and store.
 //
+// The kernel is persistent: one CTA per SM walks a list of (pixel tile, channel tile) units.
+//   * Two accumulators in TMEM: while the four epilogue warps drain unit i (bias, bf16 rounding,
+//     BatchNorm sums, stores), the MMA thread already accumulates unit i+1 into the other one, and
+//     the TMA producer runs ahead through the shared-memory ring across unit boundaries.
+//   * Vertical tap reuse (3x3, stride 1, tile inside one image): a stage holds the tile plus one
+//     halo row above and below for one horizontal shift; the three vertical taps read it at row
+//     offsets of one image row (a multiple of the swizzle period), so the input is fetched three
+//     times instead of nine.
+//   * Small filter banks stay resident in shared memory for the whole launch.
 // Warp roles: warp 0 = TMA producer (one lane), warp 1 = TMEM owner + MMA issuer (one lane),
 // warps 2..5 = epilogue.  Every mbarrier wait is bounded.
 #include "common.h"
@@ -22,13 +29,21 @@ struct alignas(64) ConvKParams {
     CUtensorMap tmA[4];
     CUtensorMap tmB;
     TapList taps[4];
-    int bw, bh, bn;                  // pixel box; bw*bh*bn == 128
+    int bw, bh, bn;                  // pixel box of an output tile; bw*bh*bn == 128
     int tiles_w, tiles_h, tiles_n;   // tiles of the output grid
     int n_ktiles, n_tile;            // output-channel tiles, UMMA N
+    int n_par;                       // output parities (stride-2 data gradient: 4)
+    int total_units;
     int kb, c_blocks;                // channels per k-block, k-blocks per tap
-    int stages, swz, tmem_cols;
-    int a_bytes, b_bytes;            // per stage (b rounded up to 1 KB so that every stage stays 1 KB aligned)
-    int tx_bytes;                    // bytes the two TMA loads of a stage deliver
+    int stages, swz;
+    int tmem_cols, acc_cols;         // allocation, columns per accumulator
+    int vreuse;                      // a stage serves the three vertical taps of one horizontal shift
+    int nb;                          // B tiles per stage (1, or 3 with vreuse)
+    int a_bytes, b_bytes;            // shared-memory footprint of the A tile / one B tile (multiples of 1 KB)
+    int tx_a, tx_b;                  // bytes one A / B load delivers
+    int a_step;                      // byte offset of one image row inside the A tile (vreuse)
+    int resident;                    // filter bank of this CTA's channel tile stays in shared memory
+    int resident_bytes;
     int n_valid, oc_valid;           // images / output channels that exist
     long long os_n, os_h, os_w;      // output element strides along the tile grid
     long long off[4];                // output element offset per parity
@@ -45,37 +60,72 @@ static constexpr int kMaxStages = 8;
 static constexpr int kThreads = 192;
 static constexpr uint32_t kDrainPolls = 1u << 22;
 
+struct UnitCoord {
+    int par, ktile, ow0, oh0, n0;
+};
+__device__ __forceinline__ UnitCoord decode_unit(const ConvKParams& p, int u)
+{
+    UnitCoord c;
+    c.ktile = u % p.n_ktiles;
+    u /= p.n_ktiles;
+    c.ow0 = (u % p.tiles_w) * p.bw;
+    u /= p.tiles_w;
+    c.oh0 = (u % p.tiles_h) * p.bh;
+    u /= p.tiles_h;
+    c.n0 = (u % p.tiles_n) * p.bn;
+    c.par = u / p.tiles_n;
+    return c;
+}
+__device__ __forceinline__ int unit_iters(const ConvKParams& p, int par)
+{
+    const int taps = p.taps[par].count;
+    return (p.vreuse ? taps / 3 : taps) * p.c_blocks;
+}
+
+// Issues the MMAs of one stage: nb sub-tiles (vertical taps) x KS k-steps of 16 channels.  Descriptor low words
+// advance by 32 bytes per k-step inside the swizzle atom and by a_step / b_step per sub-tile.
+template <int KS>
+__device__ __forceinline__ void issue_stage(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc, int nb,
+                                            uint32_t a_step16, uint32_t b_step16, bool accumulate_first)
+{
+    uint32_t acc = accumulate_first ? 1u : 0u;
+    for (int j = 0; j < nb; ++j) {
+#pragma unroll
+        for (int k = 0; k < KS; ++k) {
+            const uint64_t ad = ((uint64_t)desc_hi << 32) | (uint64_t)(a_lo + 2u * k);
+            const uint64_t bd = ((uint64_t)desc_hi << 32) | (uint64_t)(b_lo + 2u * k);
+            umma_bf16(d_tmem, ad, bd, idesc, acc);
+            acc = 1u;
+        }
+        a_lo += a_step16;
+        b_lo += b_step16;
+    }
+}
+
 __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_constant__ ConvKParams p)
 {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], accum_bar, drain_bar;
+    __shared__ uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], acc_full[2], acc_empty[2], w_bar, drain_bar;
     __shared__ uint32_t tmem_slot;
     __shared__ uint32_t abort_flag;
-    __shared__ float s_stats[512];
+    __shared__ float s_stats[4][512];   // per epilogue warp: [0,256) sums, [256,512) sums of squares
 
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023u) & ~uintptr_t(1023));
+    uint8_t* ring = smem + p.resident_bytes;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int par = blockIdx.z;
-    const TapList& tl = p.taps[par];
-    const int n_iters = tl.count * p.c_blocks;
     const int S = p.stages;
-
-    // tile decode: neighbouring CTAs share the activation tile and differ in the channel tile
-    int t = blockIdx.x;
-    const int ktile = t % p.n_ktiles;
-    t /= p.n_ktiles;
-    const int tw = t % p.tiles_w;
-    t /= p.tiles_w;
-    const int th = t % p.tiles_h;
-    const int tn = t / p.tiles_h;
-    const int ow0 = tw * p.bw, oh0 = th * p.bh, n0 = tn * p.bn;
+    const int stage_bytes = p.a_bytes + (p.resident ? 0 : p.nb * p.b_bytes);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], 1);
         }
-        mbar_init(&accum_bar, 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&acc_full[b], 1);
+            mbar_init(&acc_empty[b], 4);   // one arrival per epilogue warp
+        }
+        mbar_init(&w_bar, 1);
         mbar_init(&drain_bar, 1);
         abort_flag = 0;
         fence_mbar_init();
@@ -88,85 +138,167 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_slot;
-    const int stage_bytes = p.a_bytes + p.b_bytes;
-    int issued = 0;  // producer lane: k-blocks whose loads were issued
+    int issued = 0;  // producer lane: stages whose loads were issued
 
     if (warp == 0) {
         if (lane == 0) {
+            // ------------------------------------------------------------ TMA producer
             prefetch_tensormap(&p.tmB);
-            for (int it = 0; it < n_iters; ++it, ++issued) {
-                const int s = it % S;
-                const uint32_t ph = (uint32_t)(it / S) & 1u;
-                if (!mbar_wait_bounded(&empty_bar[s], ph ^ 1u, p.spin_limit, &abort_flag)) {
-                    atomicOr(p.status, B2C_DEV_TIMEOUT);
-                    break;
+            prefetch_tensormap(&p.tmA[0]);
+            if (p.resident) {
+                const int ktile = (int)blockIdx.x % p.n_ktiles;   // the grid is a multiple of n_ktiles: fixed per CTA
+                const TapList& tl = p.taps[0];
+                mbar_expect_tx(&w_bar, (uint32_t)(tl.count * p.c_blocks * p.tx_b));
+                for (int t = 0; t < tl.count; ++t)
+                    for (int cb = 0; cb < p.c_blocks; ++cb)
+                        tma_load_3d(smem + (size_t)(t * p.c_blocks + cb) * p.b_bytes, &p.tmB, &w_bar, cb * p.kb, tl.rs[t], ktile * p.n_tile);
+            }
+            bool ok = true;
+            for (int u = (int)blockIdx.x; ok && u < p.total_units; u += (int)gridDim.x) {
+                const UnitCoord c = decode_unit(p, u);
+                const TapList& tl = p.taps[c.par];
+                const int n_it = unit_iters(p, c.par);
+                for (int it = 0; it < n_it; ++it, ++issued) {
+                    const int s = issued % S;
+                    const uint32_t ph = (uint32_t)(issued / S) & 1u;
+                    if (!mbar_wait_bounded(&empty_bar[s], ph ^ 1u, p.spin_limit, &abort_flag)) {
+                        atomicOr(p.status, B2C_DEV_TIMEOUT);
+                        ok = false;
+                        break;
+                    }
+                    const int t0 = it / p.c_blocks, cb = it - t0 * p.c_blocks;   // tap (or horizontal shift) and channel block
+                    uint8_t* a_dst = ring + (size_t)s * stage_bytes;
+                    mbar_expect_tx(&full_bar[s], (uint32_t)(p.tx_a + (p.resident ? 0 : p.nb * p.tx_b)));
+                    // with vreuse the table entry of vertical tap 0 carries the shift of the whole haloed tile
+                    tma_load_4d(a_dst, &p.tmA[tl.map[t0]], &full_bar[s], cb * p.kb, c.ow0 + tl.dw[t0], c.oh0 + tl.dh[t0], c.n0);
+                    if (!p.resident) {
+                        for (int j = 0; j < p.nb; ++j)
+                            tma_load_3d(a_dst + p.a_bytes + (size_t)j * p.b_bytes, &p.tmB, &full_bar[s], cb * p.kb, tl.rs[t0 + 3 * j],
+                                        c.ktile * p.n_tile);
+                    }
                 }
-                const int tap = it / p.c_blocks, cb = it - tap * p.c_blocks;
-                uint8_t* a_dst = smem + (size_t)s * stage_bytes;
-                uint8_t* b_dst = a_dst + p.a_bytes;
-                mbar_expect_tx(&full_bar[s], (uint32_t)p.tx_bytes);
-                tma_load_4d(a_dst, &p.tmA[tl.map[tap]], &full_bar[s], cb * p.kb, ow0 + tl.dw[tap], oh0 + tl.dh[tap], n0);
-                tma_load_3d(b_dst, &p.tmB, &full_bar[s], cb * p.kb, tl.rs[tap], ktile * p.n_tile);
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
+            // ------------------------------------------------------------ MMA issuer
             const uint32_t idesc = make_idesc_bf16(128, p.n_tile, false, false);
             const uint32_t sbo = 8u * (uint32_t)p.kb * 2u;  // eight rows of kb bf16
+            const int ksteps = p.kb >> 4;
+            const uint64_t desc_proto = make_smem_desc(0u, 16u, sbo, (uint32_t)p.swz);
+            const uint32_t desc_hi = (uint32_t)(desc_proto >> 32), desc_lo_base = (uint32_t)desc_proto;
+            const uint32_t smem_addr = smem_u32(smem), ring_addr = smem_u32(ring);
+            const uint32_t a_to_b16 = (uint32_t)p.a_bytes >> 4, a_step16 = (uint32_t)p.a_step >> 4;
+            // B tiles of consecutive vertical taps: adjacent in a stage, three table rows apart in the resident bank
+            const uint32_t b_step16 = (uint32_t)(p.resident ? 3 * p.c_blocks * p.b_bytes : p.b_bytes) >> 4;
             bool ok = true;
-            for (int it = 0; it < n_iters; ++it) {
-                const int s = it % S;
-                const uint32_t ph = (uint32_t)(it / S) & 1u;
-                if (!mbar_wait_bounded(&full_bar[s], ph, p.spin_limit, &abort_flag)) {
+            if (p.resident && !mbar_wait_bounded(&w_bar, 0u, p.spin_limit, &abort_flag)) {
+                atomicOr(p.status, B2C_DEV_TIMEOUT);
+                ok = false;
+            }
+            int consumed = 0, jacc = 0;
+            for (int u = (int)blockIdx.x; ok && u < p.total_units; u += (int)gridDim.x) {
+                const UnitCoord c = decode_unit(p, u);
+                const int n_it = unit_iters(p, c.par);
+                if (n_it == 0) continue;
+                const int buf = jacc & 1;
+                if (!mbar_wait_bounded(&acc_empty[buf], ((uint32_t)(jacc >> 1) & 1u) ^ 1u, p.spin_limit, &abort_flag)) {
                     atomicOr(p.status, B2C_DEV_TIMEOUT);
                     ok = false;
                     break;
                 }
                 tc_fence_after();
-                const uint32_t a_addr = smem_u32(smem + (size_t)s * stage_bytes);
-                const uint32_t b_addr = a_addr + (uint32_t)p.a_bytes;
-                const int ksteps = p.kb >> 4;
-                for (int k = 0; k < ksteps; ++k) {
-                    umma_bf16(tmem_base, make_smem_desc(a_addr + k * 32, 16, sbo, (uint32_t)p.swz),
-                              make_smem_desc(b_addr + k * 32, 16, sbo, (uint32_t)p.swz), idesc, (uint32_t)((it | k) != 0));
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * p.acc_cols);
+                int cur_t0 = 0, cur_cb = 0;   // tap (or horizontal shift) and channel block of the stage
+                for (int it = 0; it < n_it; ++it, ++consumed) {
+                    const int s = consumed % S;
+                    const uint32_t ph = (uint32_t)(consumed / S) & 1u;
+                    if (!mbar_wait_bounded(&full_bar[s], ph, p.spin_limit, &abort_flag)) {
+                        atomicOr(p.status, B2C_DEV_TIMEOUT);
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    // descriptors differ from stage to stage only in the 14-bit address field: add offsets to the low word
+                    const uint32_t a_lo = desc_lo_base + ((ring_addr + (uint32_t)(s * stage_bytes)) >> 4);
+                    uint32_t b_lo;
+                    if (p.resident) {
+                        b_lo = desc_lo_base + ((smem_addr + (uint32_t)((cur_t0 * p.c_blocks + cur_cb) * p.b_bytes)) >> 4);
+                    } else {
+                        b_lo = a_lo + a_to_b16;
+                    }
+                    if (ksteps == 4)
+                        issue_stage<4>(d_tmem, a_lo, b_lo, desc_hi, idesc, p.nb, a_step16, b_step16, it != 0);
+                    else if (ksteps == 2)
+                        issue_stage<2>(d_tmem, a_lo, b_lo, desc_hi, idesc, p.nb, a_step16, b_step16, it != 0);
+                    else
+                        issue_stage<1>(d_tmem, a_lo, b_lo, desc_hi, idesc, p.nb, a_step16, b_step16, it != 0);
+                    if (++cur_cb == p.c_blocks) { cur_cb = 0; ++cur_t0; }
+                    umma_commit(&empty_bar[s]);  // frees the stage once these MMAs have read it
                 }
-                umma_commit(&empty_bar[s]);  // frees the stage once these MMAs have read it
+                if (!ok) break;
+                umma_commit(&acc_full[buf]);
+                ++jacc;
             }
-            if (ok && n_iters > 0) umma_commit(&accum_bar);
         }
     } else {
-        // ---------------------------------------------------------------- epilogue (128 threads)
+        // ---------------------------------------------------------------- epilogue (4 warps)
         const int q = warp & 3;          // TMEM lane quarter this warp may read
         const int m = q * 32 + lane;     // accumulator row = pixel of the tile (w fastest, then h, then image)
-        const int et = threadIdx.x - 64; // 0..127
         const int lw = m % p.bw, lh = (m / p.bw) % p.bh, ln = m / (p.bw * p.bh);
-        const bool row_valid = (n0 + ln) < p.n_valid;
-        const long long row_off = (long long)(n0 + ln) * p.os_n + (long long)(oh0 + lh) * p.os_h + (long long)(ow0 + lw) * p.os_w + p.off[par];
         const bool do_stats = p.stats != nullptr;
-
-        if (do_stats) {
-            for (int i = et; i < 512; i += 128) s_stats[i] = 0.f;
-        }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-
+        float* my_stats = s_stats[q];
+        for (int i = lane; i < 512; i += 32) my_stats[i] = 0.f;
+        __syncwarp();
+        const int n_chunks = p.n_tile >> 4;
+        int jacc = 0, cur_group = -1, cur_ktile = 0;
         bool ok = true;
-        if (n_iters > 0) {
-            ok = mbar_wait_bounded(&accum_bar, 0u, p.spin_limit, &abort_flag);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok && lane == 0) atomicOr(p.status, B2C_DEV_TIMEOUT);
-            tc_fence_after();
-        }
-        if (ok) {
-            for (int c0 = 0; c0 < p.n_tile; c0 += 16) {
-                uint32_t r[16];
-                if (n_iters > 0) {
-                    tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
-                    tmem_ld_wait();
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) r[i] = 0u;
+
+        auto flush_stats = [&]() {   // this warp's partial sums of the finished statistics group -> global fp64
+            __syncwarp();
+            double* st = p.stats + (size_t)cur_group * 2 * p.oc_valid;
+            for (int c = lane; c < p.n_tile; c += 32) {
+                const int ch = cur_ktile * p.n_tile + c;
+                if (ch < p.oc_valid) {
+                    atomicAdd(st + ch, (double)my_stats[c]);
+                    atomicAdd(st + p.oc_valid + ch, (double)my_stats[256 + c]);
                 }
-                const int ch0 = ktile * p.n_tile + c0;  // first output channel of this chunk
+                my_stats[c] = 0.f;
+                my_stats[256 + c] = 0.f;
+            }
+            __syncwarp();
+        };
+
+        for (int u = (int)blockIdx.x; u < p.total_units; u += (int)gridDim.x) {
+            const UnitCoord c = decode_unit(p, u);
+            const int n_it = unit_iters(p, c.par);
+            const bool row_valid = (c.n0 + ln) < p.n_valid;
+            const long long row_off = (long long)(c.n0 + ln) * p.os_n + (long long)(c.oh0 + lh) * p.os_h + (long long)(c.ow0 + lw) * p.os_w + p.off[c.par];
+            int buf = 0;
+            if (n_it > 0) {
+                buf = jacc & 1;
+                ok = mbar_wait_bounded(&acc_full[buf], (uint32_t)(jacc >> 1) & 1u, p.spin_limit, &abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) {
+                    if (lane == 0) atomicOr(p.status, B2C_DEV_TIMEOUT);
+                    break;
+                }
+                tc_fence_after();
+                ++jacc;
+            }
+            if (do_stats) {
+                const int grp = p.stats_group_images > 0 ? c.n0 / p.stats_group_images : 0;
+                if (grp != cur_group) {
+                    if (cur_group >= 0) flush_stats();
+                    cur_group = grp;
+                }
+                cur_ktile = c.ktile;
+            }
+            const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * p.acc_cols);
+
+            // one 16-column chunk: bias, rounding, stores, BatchNorm partial sums
+            auto process = [&](const uint32_t (&r)[16], int c0) {
+                const int ch0 = c.ktile * p.n_tile + c0;  // first output channel of this chunk
                 float v[16];
 #pragma unroll
                 for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
@@ -181,61 +313,86 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
                         for (int i = 0; i < 16; i += 4)
                             if (ch0 + i < p.oc_valid) *reinterpret_cast<float4*>(dst + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
                     }
-                } else {
-                    uint32_t pk[8];
+                    return;
+                }
+                uint32_t pk[8];
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) pk[i] = pack_bf16x2(v[2 * i], v[2 * i + 1]);
-                    if (row_valid) {
-                        __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + row_off + ch0;
-                        if (ch0 < p.oc_valid) *reinterpret_cast<uint4*>(dst) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                        if (ch0 + 8 < p.oc_valid) *reinterpret_cast<uint4*>(dst + 8) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                for (int i = 0; i < 8; ++i) pk[i] = pack_bf16x2(v[2 * i], v[2 * i + 1]);
+                if (row_valid) {
+                    __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + row_off + ch0;
+                    if (ch0 < p.oc_valid) *reinterpret_cast<uint4*>(dst) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    if (ch0 + 8 < p.oc_valid) *reinterpret_cast<uint4*>(dst + 8) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                }
+                if (do_stats) {
+                    // Column sums over the warp's 32 rows of the values as stored: a butterfly that
+                    // halves the number of columns each lane carries (16 -> 8 -> 4 -> 2 -> 1).
+                    float a[16], b[16];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        __nv_bfloat162 h = *reinterpret_cast<__nv_bfloat162*>(&pk[i]);
+                        const float lo = row_valid ? __low2float(h) : 0.f, hi = row_valid ? __high2float(h) : 0.f;
+                        a[2 * i] = lo;
+                        a[2 * i + 1] = hi;
+                        b[2 * i] = lo * lo;
+                        b[2 * i + 1] = hi * hi;
                     }
-                    if (do_stats) {
-                        // Column sums over the warp's 32 rows of the values as stored: a butterfly that
-                        // halves the number of columns each lane carries (16 -> 8 -> 4 -> 2 -> 1).
-                        float a[16], b[16];
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            __nv_bfloat162 h = *reinterpret_cast<__nv_bfloat162*>(&pk[i]);
-                            const float lo = row_valid ? __low2float(h) : 0.f, hi = row_valid ? __high2float(h) : 0.f;
-                            a[2 * i] = lo;
-                            a[2 * i + 1] = hi;
-                            b[2 * i] = lo * lo;
-                            b[2 * i + 1] = hi * hi;
-                        }
+                    for (int width = 8, bit = 16; width >= 1; width >>= 1, bit >>= 1) {
+                        const bool upper = (lane & bit) != 0;
 #pragma unroll
-                        for (int width = 8, bit = 16; width >= 1; width >>= 1, bit >>= 1) {
-                            const bool upper = (lane & bit) != 0;
+                        for (int i = 0; i < width; ++i) {
+                            const float sa = upper ? a[i] : a[i + width], ka = upper ? a[i + width] : a[i];
+                            const float sb = upper ? b[i] : b[i + width], kb_ = upper ? b[i + width] : b[i];
+                            a[i] = ka + __shfl_xor_sync(0xffffffffu, sa, bit);
+                            b[i] = kb_ + __shfl_xor_sync(0xffffffffu, sb, bit);
+                        }
+                    }
+                    a[0] += __shfl_xor_sync(0xffffffffu, a[0], 1);
+                    b[0] += __shfl_xor_sync(0xffffffffu, b[0], 1);
+                    if ((lane & 1) == 0) {   // lane bits 4..1 select the column of the chunk; the array is private to this warp
+                        const int col = c0 + (lane >> 1);
+                        my_stats[col] += a[0];
+                        my_stats[256 + col] += b[0];
+                    }
+                }
+            };
+            // the accumulator is handed back to the MMA thread as soon as its last column has been read
+            auto release = [&]() {
+                if (n_it > 0) {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&acc_empty[buf]);
+                }
+            };
+
+            uint32_t ra[16], rb[16];
+            if (n_it > 0) {
+                tmem_ld16(t_row, ra);
+                tmem_ld_wait();
+            } else {
 #pragma unroll
-                            for (int i = 0; i < width; ++i) {
-                                const float sa = upper ? a[i] : a[i + width], ka = upper ? a[i + width] : a[i];
-                                const float sb = upper ? b[i] : b[i + width], kb_ = upper ? b[i + width] : b[i];
-                                a[i] = ka + __shfl_xor_sync(0xffffffffu, sa, bit);
-                                b[i] = kb_ + __shfl_xor_sync(0xffffffffu, sb, bit);
-                            }
-                        }
-                        a[0] += __shfl_xor_sync(0xffffffffu, a[0], 1);
-                        b[0] += __shfl_xor_sync(0xffffffffu, b[0], 1);
-                        if ((lane & 1) == 0) {
-                            const int col = c0 + (lane >> 1);  // lane bits 4..1 select the column of the chunk
-                            atomicAdd(&s_stats[col], a[0]);
-                            atomicAdd(&s_stats[256 + col], b[0]);
-                        }
+                for (int i = 0; i < 16; ++i) ra[i] = rb[i] = 0u;
+            }
+            if (n_chunks == 1) release();
+            for (int ck = 0; ck < n_chunks; ck += 2) {
+                // chunk ck is in ra; fetch ck+1 into rb while ra is processed, then ck+2 into ra while rb is processed
+                if (n_it > 0 && ck + 1 < n_chunks) tmem_ld16(t_row + (uint32_t)((ck + 1) * 16), rb);
+                process(ra, ck * 16);
+                if (ck + 1 < n_chunks) {
+                    if (n_it > 0) {
+                        tmem_ld_wait();
+                        if (ck + 2 == n_chunks) release();
+                        if (ck + 2 < n_chunks) tmem_ld16(t_row + (uint32_t)((ck + 2) * 16), ra);
+                    }
+                    process(rb, (ck + 1) * 16);
+                    if (n_it > 0 && ck + 2 < n_chunks) {
+                        tmem_ld_wait();
+                        if (ck + 3 == n_chunks) release();
                     }
                 }
             }
         }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        if (do_stats && ok) {
-            for (int c = et; c < p.n_tile; c += 128) {
-                const int ch = ktile * p.n_tile + c;
-                if (ch < p.oc_valid) {
-                    double* st = p.stats + (size_t)(p.stats_group_images > 0 ? n0 / p.stats_group_images : 0) * 2 * p.oc_valid;
-                    atomicAdd(st + ch, (double)s_stats[c]);
-                    atomicAdd(st + p.oc_valid + ch, (double)s_stats[256 + c]);
-                }
-            }
-        }
+        if (do_stats && cur_group >= 0 && ok) flush_stats();
     }
     tc_fence_before();
     __syncthreads();
@@ -243,6 +400,8 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
         // A wait gave up.  Before the CTA may exit, let every bulk copy it issued land and every
         // MMA it issued retire (both finish on their own; the polls here only bound the wait).
         if (warp == 0 && lane == 0) {
+            if (p.resident)
+                for (uint32_t i = 0; i < kDrainPolls && !mbar_try_wait(&w_bar, 0u); ++i) {}
             for (int back = 0; back < S && back < issued; ++back) {
                 const int it = issued - 1 - back;
                 for (uint32_t i = 0; i < kDrainPolls && !mbar_try_wait(&full_bar[it % S], (uint32_t)(it / S) & 1u); ++i) {}
@@ -311,7 +470,7 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
     const int R = pb.r;
     if (!(R == 1 || R == 3) || !(pb.stride == 1 || pb.stride == 2) || pb.pad != (R - 1) / 2) return B2C_ERR_UNSUPPORTED_SHAPE;
     if (pb.n < 1 || pb.ic < 16 || pb.ic % 16 || pb.oc < 16 || pb.oc % 16) return B2C_ERR_UNSUPPORTED_SHAPE;
-    // tile grid = spatial grid each CTA's 128 accumulator rows walk over
+    // tile grid = spatial grid each unit's 128 accumulator rows walk over
     int gh, gw, n_par = 1;
     if (!pb.dgrad) {
         gh = pb.oh; gw = pb.ow;
@@ -330,37 +489,69 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
     p.tiles_w = gw / p.bw;
     p.tiles_h = gh / p.bh;
     p.tiles_n = (pb.n + p.bn - 1) / p.bn;
+    p.n_par = n_par;
 
-    p.kb = (pb.ic % 64 == 0) ? 64 : (pb.ic % 32 == 0) ? 32 : 16;
-    p.c_blocks = pb.ic / p.kb;
-    p.swz = p.kb == 64 ? SWZ_128B : p.kb == 32 ? SWZ_64B : SWZ_32B;
     // output-channel tile: the largest multiple of 16 up to 256 that splits oc evenly
     int n_tile = 16;
     for (int cand = 256; cand >= 16; cand -= 16)
         if (pb.oc % cand == 0) { n_tile = cand; break; }
     p.n_tile = n_tile;
     p.n_ktiles = pb.oc / n_tile;
+    p.acc_cols = ((n_tile + 31) / 32) * 32;
     p.tmem_cols = 32;
-    while (p.tmem_cols < n_tile) p.tmem_cols *= 2;
-    p.a_bytes = 128 * p.kb * 2;
-    p.b_bytes = ((n_tile * p.kb * 2) + 1023) & ~1023;
-    p.tx_bytes = p.a_bytes + n_tile * p.kb * 2;
-    const int stage_bytes = p.a_bytes + p.b_bytes;
-    int stages = (96 * 1024) / stage_bytes;            // two CTAs per SM when the ring is small
-    if (stages < 4) stages = (200 * 1024) / stage_bytes;
-    if (stages > kMaxStages) stages = kMaxStages;
-    if (stages < 2) return B2C_ERR_UNSUPPORTED_SHAPE;
-    p.stages = stages;
-    const size_t smem_bytes = (size_t)stages * stage_bytes + 1024;
+    while (p.tmem_cols < 2 * p.acc_cols) p.tmem_cols *= 2;
+    p.total_units = n_par * p.tiles_n * p.tiles_h * p.tiles_w * p.n_ktiles;
+
+    // launch shape: one persistent CTA per SM; a multiple of n_ktiles so that a CTA keeps its channel tile
+    int grid = ctx->sm_count < p.total_units ? ctx->sm_count : p.total_units;
+    grid -= grid % p.n_ktiles;
+    if (grid < p.n_ktiles) grid = p.n_ktiles;
+    const int units_per_cta = (p.total_units + grid - 1) / grid;
+
+    // shared-memory plan.  Preference: haloed stages (vertical tap reuse) with 64-channel k-blocks, then with
+    // 32-channel k-blocks (smaller stages, so that a ring of at least four still fits), else one tap per stage.
+    const int ring_budget = 200 * 1024;
+    const int kb_natural = (pb.ic % 64 == 0) ? 64 : (pb.ic % 32 == 0) ? 32 : 16;
+    const bool can_vreuse = (R == 3 && pb.stride == 1 && p.bn == 1);
+    const int taps_total = R * R;
+    const int attempts[3][2] = {{kb_natural, 1}, {32, 1}, {kb_natural, 0}};   // (kb, vreuse)
+    for (int a = 0; a < 3; ++a) {
+        const int kb = attempts[a][0], vr = attempts[a][1];
+        if (vr && !can_vreuse) continue;
+        if (kb > kb_natural) continue;
+        p.kb = kb;
+        p.c_blocks = pb.ic / kb;
+        p.swz = kb == 64 ? SWZ_128B : kb == 32 ? SWZ_64B : SWZ_32B;
+        p.vreuse = vr;
+        p.b_bytes = ((n_tile * kb * 2) + 1023) & ~1023;
+        p.tx_b = n_tile * kb * 2;
+        const int a_rows = vr ? (p.bh + 2) * p.bw : 128;
+        p.tx_a = a_rows * kb * 2;
+        p.a_bytes = (p.tx_a + 1023) & ~1023;
+        p.nb = vr ? 3 : 1;
+        p.a_step = vr ? p.bw * kb * 2 : 0;
+        const int bank_bytes = taps_total * p.c_blocks * p.b_bytes;
+        p.resident = (n_par == 1 && bank_bytes <= 96 * 1024 && units_per_cta >= 2) ? 1 : 0;
+        p.resident_bytes = p.resident ? bank_bytes : 0;
+        const int stage_bytes = p.a_bytes + (p.resident ? 0 : p.nb * p.b_bytes);
+        int stages = (ring_budget - p.resident_bytes) / stage_bytes;
+        if (stages > kMaxStages) stages = kMaxStages;
+        p.stages = stages;
+        if (stages >= 4 || !vr) break;
+    }
+    if (p.stages < 2) return B2C_ERR_UNSUPPORTED_SHAPE;
+    const int stage_bytes = p.a_bytes + (p.resident ? 0 : p.nb * p.b_bytes);
+    const size_t smem_bytes = (size_t)p.resident_bytes + (size_t)p.stages * stage_bytes + 1024;
 
     // tensor maps
+    const int box_h = p.vreuse ? p.bh + 2 : p.bh;
     if (!pb.dgrad && pb.stride == 2) {
         for (int ph = 0; ph < 2; ++ph)
             for (int pw = 0; pw < 2; ++pw)
-                if (!encode_activation_map(ctx, &p.tmA[ph * 2 + pw], pb.in, pb.n, pb.ih, pb.iw, pb.ic, 2, ph, pw, p.kb, p.bw, p.bh, p.bn))
+                if (!encode_activation_map(ctx, &p.tmA[ph * 2 + pw], pb.in, pb.n, pb.ih, pb.iw, pb.ic, 2, ph, pw, p.kb, p.bw, box_h, p.bn))
                     return B2C_ERR_CUDA;
     } else {
-        if (!encode_activation_map(ctx, &p.tmA[0], pb.in, pb.n, pb.ih, pb.iw, pb.ic, 1, 0, 0, p.kb, p.bw, p.bh, p.bn)) return B2C_ERR_CUDA;
+        if (!encode_activation_map(ctx, &p.tmA[0], pb.in, pb.n, pb.ih, pb.iw, pb.ic, 1, 0, 0, p.kb, p.bw, box_h, p.bn)) return B2C_ERR_CUDA;
     }
     {
         cuuint64_t dims[3] = {(cuuint64_t)pb.ic, (cuuint64_t)(R * R), (cuuint64_t)pb.oc};
@@ -369,7 +560,7 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
         if (!encode_map(ctx, &p.tmB, pb.wt, 3, dims, str, box, p.kb * 2)) return B2C_ERR_CUDA;
     }
 
-    // tap tables
+    // tap tables (row-major over (r, s); with vreuse entry s of row 0 carries the shift of the haloed tile)
     if (!pb.dgrad) {
         forward_taps(p.taps[0], R, pb.stride, pb.pad);
         p.os_n = (long long)pb.oh * pb.ow * pb.oc; p.os_h = (long long)pb.ow * pb.oc; p.os_w = pb.oc;
@@ -411,10 +602,9 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
     p.spin_limit = ctx->spin_limit;
 
     if (!attr_set) {
-        B2C_CUDA(cudaFuncSetAttribute(conv_kmajor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
+        B2C_CUDA(cudaFuncSetAttribute(conv_kmajor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 212 * 1024));
         attr_set = true;
     }
-    dim3 grid((unsigned)(p.tiles_w * p.tiles_h * p.tiles_n * p.n_ktiles), 1, (unsigned)n_par);
     conv_kmajor_kernel<<<grid, kThreads, smem_bytes, stream>>>(p);
     B2C_CUDA(cudaGetLastError());
     return B2C_OK;
