@@ -62,6 +62,12 @@ b2c_status b2c_get_device_status(b2c_ctx* ctx, void* stream);
  * A wait that exhausts it records B2C_ERR_DEVICE_TIMEOUT and the kernel winds down. */
 void b2c_set_spin_limit(b2c_ctx* ctx, unsigned limit);
 
+/* Pipeline diagnostics of the convolution kernels.  `counters` is a DEVICE array of 8 unsigned 64-bit words owned
+ * by the caller (NULL switches the feature off, the default).  Every CTA of the forward / data-gradient kernel adds
+ * the SM clock cycles its roles spent waiting: [0] TMA producer for a free ring stage, [1] MMA thread for a loaded
+ * stage, [2] MMA thread for a free accumulator, [3] first epilogue warp for a finished accumulator, [4] CTA lifetime. */
+void b2c_set_stall_counters(b2c_ctx* ctx, unsigned long long* counters);
+
 /* ---- Forward pass (Algorithm 1, "Perform forward pass") -------------------------------- */
 
 /* y[n,p,q,k] = sum_{r,s,c} x[n, p*stride+r-pad, q*stride+s-pad, c] * w[k,r,s,c]  (+ bias[k]),

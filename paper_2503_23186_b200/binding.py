@@ -23,7 +23,7 @@ LAYER_KINDS = {"conv": 0, "bn": 1, "avgpool": 2, "fc": 3, "xent": 4}
 
 # every symbol include/b2c.h declares
 EXPORTS = [
-    "b2c_create", "b2c_destroy", "b2c_status_string", "b2c_get_device_status", "b2c_set_spin_limit",
+    "b2c_create", "b2c_destroy", "b2c_status_string", "b2c_get_device_status", "b2c_set_spin_limit", "b2c_set_stall_counters",
     "b2c_conv2d_fwd", "b2c_bn_relu_fwd", "b2c_avgpool_fwd", "b2c_avgpool_bwd", "b2c_pad_channels",
     "b2c_softmax_xent_fwd_bwd", "b2c_bn_relu_bwd_workspace_bytes", "b2c_bn_relu_bwd", "b2c_bn_relu_bwd_static", "b2c_conv2d_dgrad",
     "b2c_conv2d_wgrad", "b2c_bias_grad", "b2c_grad_accum_sgd_momentum", "b2c_weight_pack_dgrad",
@@ -71,6 +71,7 @@ def lib() -> ctypes.CDLL:
         L.b2c_destroy.restype = None
         L.b2c_net_destroy.restype = None
         L.b2c_set_spin_limit.restype = None
+        L.b2c_set_stall_counters.restype = None
         _lib = L
     return _lib
 
@@ -124,6 +125,10 @@ class Context:
 
     def set_spin_limit(self, limit: int):
         lib().b2c_set_spin_limit(self.handle, c_uint(limit))
+
+    def set_stall_counters(self, counters):
+        """counters: int64 device tensor of 8 words (or None to switch the diagnostics off)."""
+        lib().b2c_set_stall_counters(self.handle, _ptr(counters))
 
     # ---- forward
     def conv2d_fwd(self, d: ConvDesc, x, w_krsc, y, bias=None, ch_stats=None):

@@ -25,6 +25,7 @@ b2c_status b2c_create(b2c_ctx** out, int device)
     ctx->device = device;
     ctx->sm_count = prop.multiProcessorCount;
     ctx->spin_limit = 1u << 22;
+    ctx->stall_counters = nullptr;
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || fn == nullptr ||
@@ -75,6 +76,8 @@ b2c_status b2c_get_device_status(b2c_ctx* ctx, void* stream)
     if (word & B2C_DEV_BAD_LABEL) return B2C_ERR_BAD_LABEL;
     return B2C_OK;
 }
+
+void b2c_set_stall_counters(b2c_ctx* ctx, unsigned long long* counters) { if (ctx) ctx->stall_counters = counters; }
 
 void b2c_set_spin_limit(b2c_ctx* ctx, unsigned limit)
 {

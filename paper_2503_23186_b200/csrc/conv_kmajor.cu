@@ -19,7 +19,7 @@
 //     times instead of nine.
 //   * Small filter banks stay resident in shared memory for the whole launch.
 // Warp roles: warp 0 = TMA producer (one lane), warp 1 = TMEM owner + MMA issuer (one lane),
-// warps 2..5 = epilogue.  Every mbarrier wait is bounded.
+// warps 2..9 = epilogue (two per TMEM lane quarter, splitting the columns).  Every mbarrier wait is bounded.
 #include "common.h"
 #include "ptx.cuh"
 
@@ -54,10 +54,12 @@ struct alignas(64) ConvKParams {
     int stats_group_images;          // images per BatchNorm statistics group (0: one group)
     unsigned* status;
     unsigned spin_limit;
+    unsigned long long* stall;       // optional [5]: cycles waited by producer / MMA (ring) / MMA (accumulator) / epilogue, CTA lifetime
 };
 
 static constexpr int kMaxStages = 8;
-static constexpr int kThreads = 192;
+static constexpr int kEpiWarps = 8;
+static constexpr int kThreads = 64 + 32 * kEpiWarps;
 static constexpr uint32_t kDrainPolls = 1u << 22;
 
 struct UnitCoord {
@@ -82,23 +84,255 @@ __device__ __forceinline__ int unit_iters(const ConvKParams& p, int par)
     return (p.vreuse ? taps / 3 : taps) * p.c_blocks;
 }
 
-// Issues the MMAs of one stage: nb sub-tiles (vertical taps) x KS k-steps of 16 channels.  Descriptor low words
-// advance by 32 bytes per k-step inside the swizzle atom and by a_step / b_step per sub-tile.
-template <int KS>
-__device__ __forceinline__ void issue_stage(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc, int nb,
-                                            uint32_t a_step16, uint32_t b_step16, bool accumulate_first)
+// Column sums over the 32 rows a warp holds (one row per lane, 16 columns each): a butterfly that halves the
+// number of columns each lane carries (16 -> 8 -> 4 -> 2 -> 1).  On return lane l holds in a[0], b[0] the totals of
+// column (l >> 1) of the chunk.
+__device__ __forceinline__ void butterfly16(float (&a)[16], float (&b)[16], int lane)
 {
-    uint32_t acc = accumulate_first ? 1u : 0u;
-    for (int j = 0; j < nb; ++j) {
+#pragma unroll
+    for (int width = 8, bit = 16; width >= 1; width >>= 1, bit >>= 1) {
+        const bool upper = (lane & bit) != 0;
+#pragma unroll
+        for (int i = 0; i < width; ++i) {
+            const float sa = upper ? a[i] : a[i + width], ka = upper ? a[i + width] : a[i];
+            const float sb = upper ? b[i] : b[i + width], kb_ = upper ? b[i + width] : b[i];
+            a[i] = ka + __shfl_xor_sync(0xffffffffu, sa, bit);
+            b[i] = kb_ + __shfl_xor_sync(0xffffffffu, sb, bit);
+        }
+    }
+    a[0] += __shfl_xor_sync(0xffffffffu, a[0], 1);
+    b[0] += __shfl_xor_sync(0xffffffffu, b[0], 1);
+}
+
+// Epilogue of one warp over all units of the CTA.  Epilogue warp e reads the TMEM lane quarter its warp index selects and the column half e >> 2
+// of every accumulator.  NCH > 0: the warp owns exactly NCH 16-column chunks per unit and keeps the BatchNorm sums of
+// its rows in registers across units, reducing them over rows once per statistics group.  NCH == 0: any width; sums
+// are reduced over rows per unit into a per-warp shared-memory array.
+template <int NCH>
+__device__ __forceinline__ void epilogue_loop(const ConvKParams& p, uint32_t tmem_base, uint64_t* acc_full, uint64_t* acc_empty,
+                                              uint32_t* abort_flag, float* my_stats, int e, int lane)
+{
+    const int q = (e + 2) & 3;       // TMEM lane quarter this warp may read: (warp index in the CTA) % 4, epilogue warps start at 2
+    const int m = q * 32 + lane;     // accumulator row = pixel of the tile (w fastest, then h, then image)
+    const int lw = m % p.bw, lh = (m / p.bw) % p.bh, ln = m / (p.bw * p.bh);
+    const bool do_stats = p.stats != nullptr;
+    const int n_chunks_all = p.n_tile >> 4;
+    const int first_half = (n_chunks_all + 1) >> 1;
+    const int ck_begin = (e >> 2) ? first_half : 0;
+    const int n_chunks = (e >> 2) ? n_chunks_all - first_half : first_half;   // chunks this warp handles
+    const int col_begin = ck_begin * 16;
+    constexpr int NA = NCH > 0 ? NCH * 16 : 1;
+    float acc_s[NA], acc_q[NA];
+#pragma unroll
+    for (int i = 0; i < NA; ++i) acc_s[i] = acc_q[i] = 0.f;
+    for (int i = lane; i < 256; i += 32) my_stats[i] = 0.f;
+    __syncwarp();
+    int jacc = 0, cur_group = -1, cur_ktile = 0;
+    bool ok = true;
+    long long epi_wait = 0;
+
+    auto flush_stats = [&]() {   // this warp's partial sums of the finished statistics group -> global fp64
+        double* st = p.stats + (size_t)cur_group * 2 * p.oc_valid;
+        if constexpr (NCH > 0) {
+#pragma unroll
+            for (int ck = 0; ck < NCH; ++ck) {
+                float a[16], b[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    a[i] = acc_s[ck * 16 + i];
+                    b[i] = acc_q[ck * 16 + i];
+                    acc_s[ck * 16 + i] = 0.f;
+                    acc_q[ck * 16 + i] = 0.f;
+                }
+                butterfly16(a, b, lane);
+                const int ch = cur_ktile * p.n_tile + col_begin + ck * 16 + (lane >> 1);
+                if ((lane & 1) == 0 && ck < n_chunks && ch < p.oc_valid) {
+                    atomicAdd(st + ch, (double)a[0]);
+                    atomicAdd(st + p.oc_valid + ch, (double)b[0]);
+                }
+            }
+        } else {
+            __syncwarp();
+            for (int c = lane; c < n_chunks * 16; c += 32) {
+                const int ch = cur_ktile * p.n_tile + col_begin + c;
+                if (ch < p.oc_valid) {
+                    atomicAdd(st + ch, (double)my_stats[c]);
+                    atomicAdd(st + p.oc_valid + ch, (double)my_stats[128 + c]);
+                }
+                my_stats[c] = 0.f;
+                my_stats[128 + c] = 0.f;
+            }
+            __syncwarp();
+        }
+    };
+
+    for (int u = (int)blockIdx.x; u < p.total_units; u += (int)gridDim.x) {
+        const UnitCoord c = decode_unit(p, u);
+        const int n_it = unit_iters(p, c.par);
+        const bool row_valid = (c.n0 + ln) < p.n_valid;
+        const long long row_off = (long long)(c.n0 + ln) * p.os_n + (long long)(c.oh0 + lh) * p.os_h + (long long)(c.ow0 + lw) * p.os_w + p.off[c.par];
+        int buf = 0;
+        if (n_it > 0) {
+            buf = jacc & 1;
+            const long long w3 = clock64();
+            ok = mbar_wait_bounded(&acc_full[buf], (uint32_t)(jacc >> 1) & 1u, p.spin_limit, abort_flag);
+            epi_wait += clock64() - w3;
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) {
+                if (lane == 0) atomicOr(p.status, B2C_DEV_TIMEOUT);
+                break;
+            }
+            tc_fence_after();
+            ++jacc;
+        }
+        if (do_stats) {
+            const int grp = p.stats_group_images > 0 ? c.n0 / p.stats_group_images : 0;
+            if (grp != cur_group) {
+                if (cur_group >= 0) flush_stats();
+                cur_group = grp;
+            }
+            cur_ktile = c.ktile;
+        }
+        const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * p.acc_cols + col_begin);
+        // the accumulator is handed back to the MMA thread as soon as this warp has read its last column
+        auto release = [&]() {
+            if (n_it > 0) {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&acc_empty[buf]);
+            }
+        };
+        // bias, rounding and stores of one 16-column chunk; returns the values as stored in pk
+        auto store_chunk = [&](const uint32_t (&r)[16], int c0, uint32_t (&pk)[8]) {
+            const int ch0 = c.ktile * p.n_tile + col_begin + c0;  // first output channel of this chunk
+            float v[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+            if (p.bias != nullptr) {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) v[i] += (ch0 + i < p.oc_valid) ? __ldg(p.bias + ch0 + i) : 0.f;
+            }
+            if (p.out_is_f32) {
+                if (row_valid) {
+                    float* dst = reinterpret_cast<float*>(p.out) + row_off + ch0;
+#pragma unroll
+                    for (int i = 0; i < 16; i += 4)
+                        if (ch0 + i < p.oc_valid) *reinterpret_cast<float4*>(dst + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                }
+                return;
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) pk[i] = pack_bf16x2(v[2 * i], v[2 * i + 1]);
+            if (row_valid) {
+                __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + row_off + ch0;
+                if (ch0 < p.oc_valid) *reinterpret_cast<uint4*>(dst) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                if (ch0 + 8 < p.oc_valid) *reinterpret_cast<uint4*>(dst + 8) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+            }
+        };
+
+        if constexpr (NCH > 0) {
+            // narrow tiles: read all of this warp's columns at once, free the accumulator, then work from registers
+            uint32_t r[NCH][16];
+#pragma unroll
+            for (int ck = 0; ck < NCH; ++ck) {
+                if (n_it > 0 && ck < n_chunks) {
+                    tmem_ld16(t_row + (uint32_t)(ck * 16), r[ck]);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) r[ck][i] = 0u;
+                }
+            }
+            if (n_it > 0) tmem_ld_wait();
+            release();
+#pragma unroll
+            for (int ck = 0; ck < NCH; ++ck) {
+                if (ck < n_chunks) {
+                    uint32_t pk[8];
+                    store_chunk(r[ck], ck * 16, pk);
+                    if (row_valid) {   // sums of the values as stored, kept per row in registers
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            __nv_bfloat162 h = *reinterpret_cast<__nv_bfloat162*>(&pk[i]);
+                            const float lo = __low2float(h), hi = __high2float(h);
+                            acc_s[ck * 16 + 2 * i] += lo;
+                            acc_s[ck * 16 + 2 * i + 1] += hi;
+                            acc_q[ck * 16 + 2 * i] = fmaf(lo, lo, acc_q[ck * 16 + 2 * i]);
+                            acc_q[ck * 16 + 2 * i + 1] = fmaf(hi, hi, acc_q[ck * 16 + 2 * i + 1]);
+                        }
+                    }
+                }
+            }
+        } else {
+            auto process = [&](const uint32_t (&r)[16], int c0) {
+                uint32_t pk[8];
+                store_chunk(r, c0, pk);
+                if (do_stats && !p.out_is_f32) {
+                    float a[16], b[16];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        __nv_bfloat162 h = *reinterpret_cast<__nv_bfloat162*>(&pk[i]);
+                        const float lo = row_valid ? __low2float(h) : 0.f, hi = row_valid ? __high2float(h) : 0.f;
+                        a[2 * i] = lo;
+                        a[2 * i + 1] = hi;
+                        b[2 * i] = lo * lo;
+                        b[2 * i + 1] = hi * hi;
+                    }
+                    butterfly16(a, b, lane);
+                    if ((lane & 1) == 0) {   // the array is private to this warp
+                        const int col = c0 + (lane >> 1);
+                        my_stats[col] += a[0];
+                        my_stats[128 + col] += b[0];
+                    }
+                }
+            };
+            uint32_t ra[16], rb[16];
+            if (n_it > 0 && n_chunks > 0) {
+                tmem_ld16(t_row, ra);
+                tmem_ld_wait();
+            } else {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) ra[i] = rb[i] = 0u;
+            }
+            if (n_chunks <= 1) release();
+            for (int ck = 0; ck < n_chunks; ck += 2) {
+                // chunk ck is in ra; fetch ck+1 into rb while ra is processed, then ck+2 into ra while rb is processed
+                if (n_it > 0 && ck + 1 < n_chunks) tmem_ld16(t_row + (uint32_t)((ck + 1) * 16), rb);
+                process(ra, ck * 16);
+                if (ck + 1 < n_chunks) {
+                    if (n_it > 0) {
+                        tmem_ld_wait();
+                        if (ck + 2 == n_chunks) release();
+                        if (ck + 2 < n_chunks) tmem_ld16(t_row + (uint32_t)((ck + 2) * 16), ra);
+                    }
+                    process(rb, (ck + 1) * 16);
+                    if (n_it > 0 && ck + 2 < n_chunks) {
+                        tmem_ld_wait();
+                        if (ck + 3 == n_chunks) release();
+                    }
+                }
+            }
+        }
+    }
+    if (do_stats && cur_group >= 0 && ok) flush_stats();
+    if (p.stall != nullptr && e == 0 && lane == 0) atomicAdd(p.stall + 3, (unsigned long long)epi_wait);
+}
+
+// Issues the MMAs of one stage: NB sub-tiles (vertical taps) x KS k-steps of 16 channels, fully unrolled so that
+// the issuing thread spends a handful of independent instructions per MMA (its own dependent-issue latency, not the
+// tensor pipe, bounds small-N tiles otherwise).  Descriptor low words advance by 32 bytes per k-step inside the
+// swizzle atom and by a_step / b_step per sub-tile.
+template <int KS, int NB>
+__device__ __forceinline__ void issue_stage(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc,
+                                            uint32_t a_step16, uint32_t b_step16, uint32_t accumulate_first)
+{
+#pragma unroll
+    for (int j = 0; j < NB; ++j) {
 #pragma unroll
         for (int k = 0; k < KS; ++k) {
-            const uint64_t ad = ((uint64_t)desc_hi << 32) | (uint64_t)(a_lo + 2u * k);
-            const uint64_t bd = ((uint64_t)desc_hi << 32) | (uint64_t)(b_lo + 2u * k);
-            umma_bf16(d_tmem, ad, bd, idesc, acc);
-            acc = 1u;
+            const uint64_t ad = ((uint64_t)desc_hi << 32) | (uint64_t)(a_lo + (uint32_t)j * a_step16 + 2u * k);
+            const uint64_t bd = ((uint64_t)desc_hi << 32) | (uint64_t)(b_lo + (uint32_t)j * b_step16 + 2u * k);
+            umma_bf16(d_tmem, ad, bd, idesc, (j == 0 && k == 0) ? accumulate_first : 1u);
         }
-        a_lo += a_step16;
-        b_lo += b_step16;
     }
 }
 
@@ -108,7 +342,7 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
     __shared__ uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], acc_full[2], acc_empty[2], w_bar, drain_bar;
     __shared__ uint32_t tmem_slot;
     __shared__ uint32_t abort_flag;
-    __shared__ float s_stats[4][512];   // per epilogue warp: [0,256) sums, [256,512) sums of squares
+    __shared__ float s_stats[kEpiWarps][256];   // per epilogue warp (128 columns at most): [0,128) sums, [128,256) sums of squares
 
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023u) & ~uintptr_t(1023));
     uint8_t* ring = smem + p.resident_bytes;
@@ -123,7 +357,7 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(&acc_full[b], 1);
-            mbar_init(&acc_empty[b], 4);   // one arrival per epilogue warp
+            mbar_init(&acc_empty[b], kEpiWarps);   // one arrival per epilogue warp
         }
         mbar_init(&w_bar, 1);
         mbar_init(&drain_bar, 1);
@@ -138,6 +372,7 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_slot;
+    const long long t_start = clock64();
     int issued = 0;  // producer lane: stages whose loads were issued
 
     if (warp == 0) {
@@ -154,6 +389,7 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
                         tma_load_3d(smem + (size_t)(t * p.c_blocks + cb) * p.b_bytes, &p.tmB, &w_bar, cb * p.kb, tl.rs[t], ktile * p.n_tile);
             }
             bool ok = true;
+            long long waited = 0;
             for (int u = (int)blockIdx.x; ok && u < p.total_units; u += (int)gridDim.x) {
                 const UnitCoord c = decode_unit(p, u);
                 const TapList& tl = p.taps[c.par];
@@ -161,11 +397,13 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
                 for (int it = 0; it < n_it; ++it, ++issued) {
                     const int s = issued % S;
                     const uint32_t ph = (uint32_t)(issued / S) & 1u;
+                    const long long w0 = clock64();
                     if (!mbar_wait_bounded(&empty_bar[s], ph ^ 1u, p.spin_limit, &abort_flag)) {
                         atomicOr(p.status, B2C_DEV_TIMEOUT);
                         ok = false;
                         break;
                     }
+                    waited += clock64() - w0;
                     const int t0 = it / p.c_blocks, cb = it - t0 * p.c_blocks;   // tap (or horizontal shift) and channel block
                     uint8_t* a_dst = ring + (size_t)s * stage_bytes;
                     mbar_expect_tx(&full_bar[s], (uint32_t)(p.tx_a + (p.resident ? 0 : p.nb * p.tx_b)));
@@ -177,6 +415,10 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
                                         c.ktile * p.n_tile);
                     }
                 }
+            }
+            if (p.stall != nullptr) {
+                atomicAdd(p.stall + 0, (unsigned long long)waited);
+                atomicAdd(p.stall + 4, (unsigned long long)(clock64() - t_start));
             }
         }
     } else if (warp == 1) {
@@ -197,27 +439,32 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
                 ok = false;
             }
             int consumed = 0, jacc = 0;
+            long long wait_ring = 0, wait_acc = 0;
             for (int u = (int)blockIdx.x; ok && u < p.total_units; u += (int)gridDim.x) {
                 const UnitCoord c = decode_unit(p, u);
                 const int n_it = unit_iters(p, c.par);
                 if (n_it == 0) continue;
                 const int buf = jacc & 1;
+                const long long w1 = clock64();
                 if (!mbar_wait_bounded(&acc_empty[buf], ((uint32_t)(jacc >> 1) & 1u) ^ 1u, p.spin_limit, &abort_flag)) {
                     atomicOr(p.status, B2C_DEV_TIMEOUT);
                     ok = false;
                     break;
                 }
+                wait_acc += clock64() - w1;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * p.acc_cols);
                 int cur_t0 = 0, cur_cb = 0;   // tap (or horizontal shift) and channel block of the stage
                 for (int it = 0; it < n_it; ++it, ++consumed) {
                     const int s = consumed % S;
                     const uint32_t ph = (uint32_t)(consumed / S) & 1u;
+                    const long long w2 = clock64();
                     if (!mbar_wait_bounded(&full_bar[s], ph, p.spin_limit, &abort_flag)) {
                         atomicOr(p.status, B2C_DEV_TIMEOUT);
                         ok = false;
                         break;
                     }
+                    wait_ring += clock64() - w2;
                     tc_fence_after();
                     // descriptors differ from stage to stage only in the 14-bit address field: add offsets to the low word
                     const uint32_t a_lo = desc_lo_base + ((ring_addr + (uint32_t)(s * stage_bytes)) >> 4);
@@ -227,12 +474,16 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
                     } else {
                         b_lo = a_lo + a_to_b16;
                     }
-                    if (ksteps == 4)
-                        issue_stage<4>(d_tmem, a_lo, b_lo, desc_hi, idesc, p.nb, a_step16, b_step16, it != 0);
-                    else if (ksteps == 2)
-                        issue_stage<2>(d_tmem, a_lo, b_lo, desc_hi, idesc, p.nb, a_step16, b_step16, it != 0);
-                    else
-                        issue_stage<1>(d_tmem, a_lo, b_lo, desc_hi, idesc, p.nb, a_step16, b_step16, it != 0);
+                    const uint32_t acc0 = it != 0 ? 1u : 0u;
+                    if (p.nb == 3) {
+                        if (ksteps == 4) issue_stage<4, 3>(d_tmem, a_lo, b_lo, desc_hi, idesc, a_step16, b_step16, acc0);
+                        else if (ksteps == 2) issue_stage<2, 3>(d_tmem, a_lo, b_lo, desc_hi, idesc, a_step16, b_step16, acc0);
+                        else issue_stage<1, 3>(d_tmem, a_lo, b_lo, desc_hi, idesc, a_step16, b_step16, acc0);
+                    } else {
+                        if (ksteps == 4) issue_stage<4, 1>(d_tmem, a_lo, b_lo, desc_hi, idesc, a_step16, b_step16, acc0);
+                        else if (ksteps == 2) issue_stage<2, 1>(d_tmem, a_lo, b_lo, desc_hi, idesc, a_step16, b_step16, acc0);
+                        else issue_stage<1, 1>(d_tmem, a_lo, b_lo, desc_hi, idesc, a_step16, b_step16, acc0);
+                    }
                     if (++cur_cb == p.c_blocks) { cur_cb = 0; ++cur_t0; }
                     umma_commit(&empty_bar[s]);  // frees the stage once these MMAs have read it
                 }
@@ -240,159 +491,20 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
                 umma_commit(&acc_full[buf]);
                 ++jacc;
             }
+            if (p.stall != nullptr) {
+                atomicAdd(p.stall + 1, (unsigned long long)wait_ring);
+                atomicAdd(p.stall + 2, (unsigned long long)wait_acc);
+            }
         }
     } else {
-        // ---------------------------------------------------------------- epilogue (4 warps)
-        const int q = warp & 3;          // TMEM lane quarter this warp may read
-        const int m = q * 32 + lane;     // accumulator row = pixel of the tile (w fastest, then h, then image)
-        const int lw = m % p.bw, lh = (m / p.bw) % p.bh, ln = m / (p.bw * p.bh);
-        const bool do_stats = p.stats != nullptr;
-        float* my_stats = s_stats[q];
-        for (int i = lane; i < 512; i += 32) my_stats[i] = 0.f;
-        __syncwarp();
-        const int n_chunks = p.n_tile >> 4;
-        int jacc = 0, cur_group = -1, cur_ktile = 0;
-        bool ok = true;
-
-        auto flush_stats = [&]() {   // this warp's partial sums of the finished statistics group -> global fp64
-            __syncwarp();
-            double* st = p.stats + (size_t)cur_group * 2 * p.oc_valid;
-            for (int c = lane; c < p.n_tile; c += 32) {
-                const int ch = cur_ktile * p.n_tile + c;
-                if (ch < p.oc_valid) {
-                    atomicAdd(st + ch, (double)my_stats[c]);
-                    atomicAdd(st + p.oc_valid + ch, (double)my_stats[256 + c]);
-                }
-                my_stats[c] = 0.f;
-                my_stats[256 + c] = 0.f;
-            }
-            __syncwarp();
-        };
-
-        for (int u = (int)blockIdx.x; u < p.total_units; u += (int)gridDim.x) {
-            const UnitCoord c = decode_unit(p, u);
-            const int n_it = unit_iters(p, c.par);
-            const bool row_valid = (c.n0 + ln) < p.n_valid;
-            const long long row_off = (long long)(c.n0 + ln) * p.os_n + (long long)(c.oh0 + lh) * p.os_h + (long long)(c.ow0 + lw) * p.os_w + p.off[c.par];
-            int buf = 0;
-            if (n_it > 0) {
-                buf = jacc & 1;
-                ok = mbar_wait_bounded(&acc_full[buf], (uint32_t)(jacc >> 1) & 1u, p.spin_limit, &abort_flag);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) {
-                    if (lane == 0) atomicOr(p.status, B2C_DEV_TIMEOUT);
-                    break;
-                }
-                tc_fence_after();
-                ++jacc;
-            }
-            if (do_stats) {
-                const int grp = p.stats_group_images > 0 ? c.n0 / p.stats_group_images : 0;
-                if (grp != cur_group) {
-                    if (cur_group >= 0) flush_stats();
-                    cur_group = grp;
-                }
-                cur_ktile = c.ktile;
-            }
-            const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * p.acc_cols);
-
-            // one 16-column chunk: bias, rounding, stores, BatchNorm partial sums
-            auto process = [&](const uint32_t (&r)[16], int c0) {
-                const int ch0 = c.ktile * p.n_tile + c0;  // first output channel of this chunk
-                float v[16];
-#pragma unroll
-                for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
-                if (p.bias != nullptr) {
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) v[i] += (ch0 + i < p.oc_valid) ? __ldg(p.bias + ch0 + i) : 0.f;
-                }
-                if (p.out_is_f32) {
-                    if (row_valid) {
-                        float* dst = reinterpret_cast<float*>(p.out) + row_off + ch0;
-#pragma unroll
-                        for (int i = 0; i < 16; i += 4)
-                            if (ch0 + i < p.oc_valid) *reinterpret_cast<float4*>(dst + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
-                    }
-                    return;
-                }
-                uint32_t pk[8];
-#pragma unroll
-                for (int i = 0; i < 8; ++i) pk[i] = pack_bf16x2(v[2 * i], v[2 * i + 1]);
-                if (row_valid) {
-                    __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + row_off + ch0;
-                    if (ch0 < p.oc_valid) *reinterpret_cast<uint4*>(dst) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                    if (ch0 + 8 < p.oc_valid) *reinterpret_cast<uint4*>(dst + 8) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
-                }
-                if (do_stats) {
-                    // Column sums over the warp's 32 rows of the values as stored: a butterfly that
-                    // halves the number of columns each lane carries (16 -> 8 -> 4 -> 2 -> 1).
-                    float a[16], b[16];
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        __nv_bfloat162 h = *reinterpret_cast<__nv_bfloat162*>(&pk[i]);
-                        const float lo = row_valid ? __low2float(h) : 0.f, hi = row_valid ? __high2float(h) : 0.f;
-                        a[2 * i] = lo;
-                        a[2 * i + 1] = hi;
-                        b[2 * i] = lo * lo;
-                        b[2 * i + 1] = hi * hi;
-                    }
-#pragma unroll
-                    for (int width = 8, bit = 16; width >= 1; width >>= 1, bit >>= 1) {
-                        const bool upper = (lane & bit) != 0;
-#pragma unroll
-                        for (int i = 0; i < width; ++i) {
-                            const float sa = upper ? a[i] : a[i + width], ka = upper ? a[i + width] : a[i];
-                            const float sb = upper ? b[i] : b[i + width], kb_ = upper ? b[i + width] : b[i];
-                            a[i] = ka + __shfl_xor_sync(0xffffffffu, sa, bit);
-                            b[i] = kb_ + __shfl_xor_sync(0xffffffffu, sb, bit);
-                        }
-                    }
-                    a[0] += __shfl_xor_sync(0xffffffffu, a[0], 1);
-                    b[0] += __shfl_xor_sync(0xffffffffu, b[0], 1);
-                    if ((lane & 1) == 0) {   // lane bits 4..1 select the column of the chunk; the array is private to this warp
-                        const int col = c0 + (lane >> 1);
-                        my_stats[col] += a[0];
-                        my_stats[256 + col] += b[0];
-                    }
-                }
-            };
-            // the accumulator is handed back to the MMA thread as soon as its last column has been read
-            auto release = [&]() {
-                if (n_it > 0) {
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&acc_empty[buf]);
-                }
-            };
-
-            uint32_t ra[16], rb[16];
-            if (n_it > 0) {
-                tmem_ld16(t_row, ra);
-                tmem_ld_wait();
-            } else {
-#pragma unroll
-                for (int i = 0; i < 16; ++i) ra[i] = rb[i] = 0u;
-            }
-            if (n_chunks == 1) release();
-            for (int ck = 0; ck < n_chunks; ck += 2) {
-                // chunk ck is in ra; fetch ck+1 into rb while ra is processed, then ck+2 into ra while rb is processed
-                if (n_it > 0 && ck + 1 < n_chunks) tmem_ld16(t_row + (uint32_t)((ck + 1) * 16), rb);
-                process(ra, ck * 16);
-                if (ck + 1 < n_chunks) {
-                    if (n_it > 0) {
-                        tmem_ld_wait();
-                        if (ck + 2 == n_chunks) release();
-                        if (ck + 2 < n_chunks) tmem_ld16(t_row + (uint32_t)((ck + 2) * 16), ra);
-                    }
-                    process(rb, (ck + 1) * 16);
-                    if (n_it > 0 && ck + 2 < n_chunks) {
-                        tmem_ld_wait();
-                        if (ck + 3 == n_chunks) release();
-                    }
-                }
-            }
-        }
-        if (do_stats && cur_group >= 0 && ok) flush_stats();
+        // ---------------------------------------------------------------- epilogue (8 warps)
+        const int e = warp - 2;
+        if (p.stats != nullptr && p.n_tile <= 32)
+            epilogue_loop<1>(p, tmem_base, acc_full, acc_empty, &abort_flag, s_stats[e], e, lane);
+        else if (p.stats != nullptr && p.n_tile <= 64)
+            epilogue_loop<2>(p, tmem_base, acc_full, acc_empty, &abort_flag, s_stats[e], e, lane);
+        else
+            epilogue_loop<0>(p, tmem_base, acc_full, acc_empty, &abort_flag, s_stats[e], e, lane);
     }
     tc_fence_before();
     __syncthreads();
@@ -600,6 +712,7 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
     if (p.stats && p.stats_group_images > 0 && (p.stats_group_images % p.bn) != 0) return B2C_ERR_UNSUPPORTED_SHAPE;  // a tile must not straddle groups
     p.status = ctx->d_status;
     p.spin_limit = ctx->spin_limit;
+    p.stall = ctx->stall_counters;
 
     if (!attr_set) {
         B2C_CUDA(cudaFuncSetAttribute(conv_kmajor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 212 * 1024));
