@@ -2,45 +2,71 @@
 //
 //   dw[k, tap, c] += sum over pixels  dy[pixel, k] * x[pixel shifted by tap, c]
 //
-// GEMM M = 128 output channels (k), N = ct input channels (c), reduction = pixels.  Both dy and
-// x are stored pixel-major with channels contiguous, i.e. the reduction index is the slow one:
-// TMA boxes of (cw channels, pb pixels) land in shared memory exactly in the swizzled MN-major
-// canonical layout (rows = pixels, cw*2 = 32/64/128 bytes per row).  One CTA owns a
+// GEMM M = 128 output channels (k), N = input channels (c) of one or more taps, reduction = pixels.
+// Both dy and x are stored pixel-major with channels contiguous, i.e. the reduction index is the
+// slow one: TMA boxes of (cw channels, pb pixels) land in shared memory exactly in the swizzled
+// MN-major canonical layout (rows = pixels, cw*2 = 32/64/128 bytes per row).  One CTA owns a
 // (k-tile, c-tile, tap group) and a range of pixel chunks; a stage holds one chunk: the dy boxes
-// (shared by all taps of the group) and, per tap, the x boxes shifted by that tap (zero-filled
-// outside the image by TMA).  Each tap accumulates into its own TMEM column range.  Partial sums
-// of the pixel ranges are added to dw with vector fp32 reductions.
+// and, per x shift of the group, the x boxes gathered at that shift (zero-filled outside the image by
+// TMA).  The x boxes of consecutive shifts are adjacent, so one MMA covers several taps (N up to 256).
+//
+// Layers with 64 output channels would leave half of M = 128 empty.  There two copies of dy, the
+// second gathered one row higher, are stacked on M: with x gathered at (r0 - pad, s - pad) the rows of
+// copy a accumulate tap (r0 + a, s), since sum_p dy[p - (a,0)] x[p + t] = sum_p dy[p] x[p + t + (a,0)].
+// Partial sums of the pixel ranges are added to dw with vector fp32 reductions.
 #include "common.h"
 #include "ptx.cuh"
 
 namespace b2c {
 
+struct WgGroup {
+    int nb;                        // x shifts of the group (column blocks of ct channels)
+    int8_t map[3], dh[3], dw[3];   // tensor map (parity view) and pixel offset of each shift
+    int8_t rs[2][3];               // filter tap accumulated by (dy copy, shift); -1: not used
+};
+
 struct alignas(64) WgradParams {
     CUtensorMap tmDy;
     CUtensorMap tmX[4];
-    TapList taps;
-    int bw, bh, bn, tiles_w, tiles_h;  // pixel chunk box and chunk grid
+    WgGroup groups[3];
+    int n_groups;
+    int stack;                         // two dy copies stacked on M (64 output channels)
+    int bw, bh, bn, tiles_w, tiles_h;  // pixel chunk box and chunk grid (tiles_h covers one extra row when stacked)
     int pb;                            // pixels per chunk
-    int cw, swz;                       // channels per box, descriptor swizzle code
-    int ct;                            // x channels per CTA (UMMA N)
-    int n_ktiles, n_ctiles, n_groups, taps_per_group, n_splits;
+    int cw_a, swz_a, cw_b, swz_b;      // channels per box (= one swizzle row) and descriptor swizzle code: dy, x
+    int ct;                            // x channels per CTA
+    int n_ktiles, n_ctiles, n_splits;
     int chunks_total;
     int stages, tmem_cols;
-    int box_bytes, a_boxes, b_boxes;   // bytes per box; dy boxes per stage; x boxes per tap
+    int box_a, box_b, a_boxes, b_boxes;   // bytes per dy / x box; dy boxes per stage; x boxes per shift
     int stage_bytes;
+    int n_pieces, piece_t0[3], piece_nt[3];   // MMAs per k-step: first shift and number of shifts each covers
     int k_total, c_total, rs_total;
     float* dw;
     unsigned* status;
     unsigned spin_limit;
 };
 
-static constexpr int kWgStages = 4;
+static constexpr int kWgStages = 6;
 static constexpr int kWgThreads = 192;
 static constexpr uint32_t kWgDrainPolls = 1u << 22;
 
 __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d)
 {
     asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+
+// One MMA per k-step of 16 pixels, unrolled: descriptors differ only in their low (address) word.
+template <int KS>
+__device__ __forceinline__ void wg_issue(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t a_hi, uint32_t b_hi, uint32_t idesc,
+                                         uint32_t kstep_a, uint32_t kstep_b, uint32_t accumulate_first)
+{
+#pragma unroll
+    for (int kk = 0; kk < KS; ++kk) {
+        const uint64_t ad = ((uint64_t)a_hi << 32) | (uint64_t)(a_lo + (uint32_t)kk * kstep_a);
+        const uint64_t bd = ((uint64_t)b_hi << 32) | (uint64_t)(b_lo + (uint32_t)kk * kstep_b);
+        umma_bf16(d_tmem, ad, bd, idesc, kk == 0 ? accumulate_first : 1u);
+    }
 }
 
 __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_constant__ WgradParams p)
@@ -59,14 +85,12 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
     t /= p.n_ktiles;
     const int ctile = t % p.n_ctiles;
     t /= p.n_ctiles;
-    const int group = t % p.n_groups;
+    const int gi = t % p.n_groups;
     const int split = t / p.n_groups;
+    const WgGroup& grp = p.groups[gi];
     const int chunk_begin = (int)((long long)p.chunks_total * split / p.n_splits);
     const int chunk_end = (int)((long long)p.chunks_total * (split + 1) / p.n_splits);
     const int n_chunks = chunk_end - chunk_begin;
-    const int tap0 = group * p.taps_per_group;
-    const int n_taps = min(p.taps_per_group, p.taps.count - tap0);
-    const int row_bytes = p.cw * 2;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
@@ -91,7 +115,8 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
     if (warp == 0) {
         if (lane == 0) {
             prefetch_tensormap(&p.tmDy);
-            const uint32_t tx = (uint32_t)((p.a_boxes + n_taps * p.b_boxes) * p.box_bytes);
+            prefetch_tensormap(&p.tmX[0]);
+            const uint32_t tx = (uint32_t)(p.a_boxes * p.box_a + grp.nb * p.b_boxes * p.box_b);
             for (int it = 0; it < n_chunks; ++it, ++issued) {
                 const int s = it % S;
                 const uint32_t ph = (uint32_t)(it / S) & 1u;
@@ -106,23 +131,43 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
                 const int n0 = (ch / p.tiles_h) * p.bn;
                 uint8_t* dst = smem + (size_t)s * p.stage_bytes;
                 mbar_expect_tx(&full_bar[s], tx);
-                for (int j = 0; j < p.a_boxes; ++j)  // boxes past the last channel are zero-filled
-                    tma_load_4d(dst + (size_t)j * p.box_bytes, &p.tmDy, &full_bar[s], ktile * 128 + j * p.cw, ow0, oh0, n0);
-                dst += (size_t)p.a_boxes * p.box_bytes;
-                for (int tl = 0; tl < n_taps; ++tl) {
-                    const int tap = tap0 + tl;
-                    for (int j = 0; j < p.b_boxes; ++j)
-                        tma_load_4d(dst + (size_t)(tl * p.b_boxes + j) * p.box_bytes, &p.tmX[p.taps.map[tap]], &full_bar[s],
-                                    ctile * p.ct + j * p.cw, ow0 + p.taps.dw[tap], oh0 + p.taps.dh[tap], n0);
+                if (p.stack) {
+                    for (int a = 0; a < 2; ++a)   // copy a of dy is gathered a rows higher
+                        tma_load_4d(dst + (size_t)a * p.box_a, &p.tmDy, &full_bar[s], 0, ow0, oh0 - a, n0);
+                } else {
+                    for (int j = 0; j < p.a_boxes; ++j)  // boxes past the last channel are zero-filled
+                        tma_load_4d(dst + (size_t)j * p.box_a, &p.tmDy, &full_bar[s], ktile * 128 + j * p.cw_a, ow0, oh0, n0);
                 }
+                dst += (size_t)p.a_boxes * p.box_a;
+                for (int b = 0; b < grp.nb; ++b)
+                    for (int j = 0; j < p.b_boxes; ++j)
+                        tma_load_4d(dst + (size_t)(b * p.b_boxes + j) * p.box_b, &p.tmX[grp.map[b]], &full_bar[s], ctile * p.ct + j * p.cw_b,
+                                    ow0 + grp.dw[b], oh0 + grp.dh[b], n0);
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            const uint32_t idesc = make_idesc_bf16(128, p.ct, true, true);
-            const uint32_t sbo = 8u * (uint32_t)row_bytes;   // eight pixel rows
-            const uint32_t lbo = (uint32_t)p.box_bytes;      // next block of cw channels
+            // SBO = eight pixel rows, LBO = next block of cw channels (the next box)
+            const uint64_t proto_a = make_smem_desc(0u, (uint32_t)p.box_a, 16u * (uint32_t)p.cw_a, (uint32_t)p.swz_a);
+            const uint64_t proto_b = make_smem_desc(0u, (uint32_t)p.box_b, 16u * (uint32_t)p.cw_b, (uint32_t)p.swz_b);
+            const uint32_t a_hi = (uint32_t)(proto_a >> 32), a_lo_base = (uint32_t)proto_a;
+            const uint32_t b_hi = (uint32_t)(proto_b >> 32), b_lo_base = (uint32_t)proto_b;
+            const uint32_t kstep_a = (uint32_t)(16 * p.cw_a * 2) >> 4, kstep_b = (uint32_t)(16 * p.cw_b * 2) >> 4;   // 16 pixel rows
             const int ksteps = p.pb >> 4;
+            // up to three MMAs per k-step (kept in scalars: the issuing thread must not index local memory)
+            uint32_t idesc0 = 0, idesc1 = 0, idesc2 = 0, boff0 = 0, boff1 = 0, boff2 = 0, dcol0 = 0, dcol1 = 0, dcol2 = 0;
+            int n_pieces = 0;
+            for (int i = 0; i < p.n_pieces; ++i) {
+                if (p.piece_t0[i] >= grp.nb) break;
+                const int nt = min(p.piece_nt[i], grp.nb - p.piece_t0[i]);
+                const uint32_t id = make_idesc_bf16(128, nt * p.ct, true, true);
+                const uint32_t bo = (uint32_t)(p.a_boxes * p.box_a + p.piece_t0[i] * p.b_boxes * p.box_b) >> 4;
+                const uint32_t dc = (uint32_t)(p.piece_t0[i] * p.ct);
+                if (i == 0) { idesc0 = id; boff0 = bo; dcol0 = dc; }
+                else if (i == 1) { idesc1 = id; boff1 = bo; dcol1 = dc; }
+                else { idesc2 = id; boff2 = bo; dcol2 = dc; }
+                ++n_pieces;
+            }
             bool ok = true;
             for (int it = 0; it < n_chunks; ++it) {
                 const int s = it % S;
@@ -133,15 +178,17 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
                     break;
                 }
                 tc_fence_after();
-                const uint32_t a_addr = smem_u32(smem + (size_t)s * p.stage_bytes);
-                const uint32_t b_addr = a_addr + (uint32_t)(p.a_boxes * p.box_bytes);
-                for (int tl = 0; tl < n_taps; ++tl) {
-                    for (int kk = 0; kk < ksteps; ++kk) {
-                        const uint32_t koff = (uint32_t)(kk * 16 * row_bytes);
-                        umma_bf16(tmem_base + (uint32_t)(tl * p.ct), make_smem_desc(a_addr + koff, lbo, sbo, (uint32_t)p.swz),
-                                  make_smem_desc(b_addr + (uint32_t)(tl * p.b_boxes * p.box_bytes) + koff, lbo, sbo, (uint32_t)p.swz), idesc,
-                                  (uint32_t)((it | kk) != 0));
-                    }
+                const uint32_t st16 = smem_u32(smem + (size_t)s * p.stage_bytes) >> 4;
+                const uint32_t a_lo = a_lo_base + st16, b_lo = b_lo_base + st16;
+                const uint32_t acc0 = it != 0 ? 1u : 0u;
+                if (ksteps == 4) {
+                    wg_issue<4>(tmem_base + dcol0, a_lo, b_lo + boff0, a_hi, b_hi, idesc0, kstep_a, kstep_b, acc0);
+                    if (n_pieces > 1) wg_issue<4>(tmem_base + dcol1, a_lo, b_lo + boff1, a_hi, b_hi, idesc1, kstep_a, kstep_b, acc0);
+                    if (n_pieces > 2) wg_issue<4>(tmem_base + dcol2, a_lo, b_lo + boff2, a_hi, b_hi, idesc2, kstep_a, kstep_b, acc0);
+                } else {
+                    wg_issue<2>(tmem_base + dcol0, a_lo, b_lo + boff0, a_hi, b_hi, idesc0, kstep_a, kstep_b, acc0);
+                    if (n_pieces > 1) wg_issue<2>(tmem_base + dcol1, a_lo, b_lo + boff1, a_hi, b_hi, idesc1, kstep_a, kstep_b, acc0);
+                    if (n_pieces > 2) wg_issue<2>(tmem_base + dcol2, a_lo, b_lo + boff2, a_hi, b_hi, idesc2, kstep_a, kstep_b, acc0);
                 }
                 umma_commit(&empty_bar[s]);
             }
@@ -150,7 +197,8 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
     } else {
         const int q = warp & 3;
         const int m = q * 32 + lane;
-        const int k = ktile * 128 + m;
+        const int copy = p.stack ? (m >> 6) : 0;                       // which dy copy this accumulator row belongs to
+        const int k = p.stack ? (m & 63) : ktile * 128 + m;
         bool ok = n_chunks > 0;
         if (ok) {
             ok = mbar_wait_bounded(&accum_bar, 0u, p.spin_limit, &abort_flag);
@@ -159,18 +207,34 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
             tc_fence_after();
         }
         if (ok) {
-            for (int tl = 0; tl < n_taps; ++tl) {
-                const int rs = p.taps.rs[tap0 + tl];
-                float* dst_row = p.dw + ((long long)k * p.rs_total + rs) * p.c_total + ctile * p.ct;
-                for (int c0 = 0; c0 < p.ct; c0 += 16) {
-                    uint32_t r[16];
-                    tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(tl * p.ct + c0), r);
-                    tmem_ld_wait();
-                    if (k < p.k_total) {
+            const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16);
+            const int n_ck = p.ct >> 4;
+            for (int b = 0; b < grp.nb; ++b) {
+                const int rs = grp.rs[copy][b];
+                const bool live = rs >= 0 && k < p.k_total;
+                float* dst_row = p.dw + ((long long)(live ? k : 0) * p.rs_total + (live ? rs : 0)) * p.c_total + ctile * p.ct;
+                // two chunks in flight: the next one is fetched while the current one is sent out
+                uint32_t ra[16], rb[16];
+                tmem_ld16(t_row + (uint32_t)(b * p.ct), ra);
+                tmem_ld_wait();
+                for (int ck = 0; ck < n_ck; ck += 2) {
+                    if (ck + 1 < n_ck) tmem_ld16(t_row + (uint32_t)(b * p.ct + (ck + 1) * 16), rb);
+                    if (live) {
 #pragma unroll
                         for (int i = 0; i < 16; i += 4)
-                            red_add_v4(dst_row + c0 + i, __uint_as_float(r[i]), __uint_as_float(r[i + 1]), __uint_as_float(r[i + 2]),
-                                       __uint_as_float(r[i + 3]));
+                            red_add_v4(dst_row + ck * 16 + i, __uint_as_float(ra[i]), __uint_as_float(ra[i + 1]), __uint_as_float(ra[i + 2]),
+                                       __uint_as_float(ra[i + 3]));
+                    }
+                    if (ck + 1 < n_ck) {
+                        tmem_ld_wait();
+                        if (ck + 2 < n_ck) tmem_ld16(t_row + (uint32_t)(b * p.ct + (ck + 2) * 16), ra);
+                        if (live) {
+#pragma unroll
+                            for (int i = 0; i < 16; i += 4)
+                                red_add_v4(dst_row + (ck + 1) * 16 + i, __uint_as_float(rb[i]), __uint_as_float(rb[i + 1]), __uint_as_float(rb[i + 2]),
+                                           __uint_as_float(rb[i + 3]));
+                        }
+                        if (ck + 2 < n_ck) tmem_ld_wait();
                     }
                 }
             }
@@ -210,28 +274,73 @@ b2c_status launch_conv_wgrad(b2c_ctx* ctx, const WgradProblem& pb, cudaStream_t 
     if (!b2c_is_pow2(pb.p) || !b2c_is_pow2(pb.q) || pb.p > 128 || pb.q > 128) return B2C_ERR_UNSUPPORTED_SHAPE;
     if (!b2c_aligned16(pb.dy) || !b2c_aligned16(pb.x) || !b2c_aligned16(pb.dw)) return B2C_ERR_MISALIGNED;
 
-    // channels per box: one swizzle row; both tensors use the same width so that one descriptor geometry serves both
-    p.cw = (pb.c % 64 == 0 && pb.k % 64 == 0) ? 64 : (pb.c % 32 == 0 && pb.k % 32 == 0) ? 32 : 16;
-    p.swz = p.cw == 64 ? SWZ_128B : p.cw == 32 ? SWZ_64B : SWZ_32B;
-    p.taps_per_group = R == 3 ? 3 : 1;
-    p.n_groups = R == 3 ? 3 : 1;
-    // x-channel tile: largest divisor of c that is a multiple of cw, at most 160 (three taps fit 512 TMEM columns)
-    p.ct = p.cw;
-    for (int cand = 160; cand >= p.cw; cand -= 16)
-        if (pb.c % cand == 0 && cand % p.cw == 0) { p.ct = cand; break; }
+    // channels per box = one swizzle row, chosen per tensor
+    p.cw_a = (pb.k % 64 == 0) ? 64 : (pb.k % 32 == 0) ? 32 : 16;
+    p.cw_b = (pb.c % 64 == 0) ? 64 : (pb.c % 32 == 0) ? 32 : 16;
+    p.swz_a = p.cw_a == 64 ? SWZ_128B : p.cw_a == 32 ? SWZ_64B : SWZ_32B;
+    p.swz_b = p.cw_b == 64 ? SWZ_128B : p.cw_b == 32 ? SWZ_64B : SWZ_32B;
+    // stacking needs chunks that stay inside one image (at least 64 pixels per image)
+    p.stack = (R == 3 && pb.stride == 1 && pb.k == 64 && pb.p * pb.q >= 64) ? 1 : 0;
+    // x-channel tile: largest divisor of c that is a multiple of cw_b, at most 160 (three shifts fit 512 TMEM columns)
+    p.ct = p.cw_b;
+    for (int cand = 160; cand >= p.cw_b; cand -= 16)
+        if (pb.c % cand == 0 && cand % p.cw_b == 0) { p.ct = cand; break; }
     p.n_ctiles = pb.c / p.ct;
-    p.n_ktiles = (pb.k + 127) / 128;
-    p.a_boxes = 128 / p.cw;
-    p.b_boxes = p.ct / p.cw;
+    p.n_ktiles = p.stack ? 1 : (pb.k + 127) / 128;
+    p.a_boxes = p.stack ? 2 : 128 / p.cw_a;
+    p.b_boxes = p.ct / p.cw_b;
+    const int shifts = R == 3 ? 3 : 1;
     p.tmem_cols = 32;
-    while (p.tmem_cols < p.taps_per_group * p.ct) p.tmem_cols *= 2;
+    while (p.tmem_cols < shifts * p.ct) p.tmem_cols *= 2;
     if (p.tmem_cols > 512) return B2C_ERR_UNSUPPORTED_SHAPE;
+    // MMAs per k-step: merge the column blocks of consecutive shifts while N stays within 256
+    if (shifts * p.ct <= 256) {
+        p.n_pieces = 1; p.piece_t0[0] = 0; p.piece_nt[0] = shifts;
+    } else if (2 * p.ct <= 256) {
+        p.n_pieces = 2; p.piece_t0[0] = 0; p.piece_nt[0] = 2; p.piece_t0[1] = 2; p.piece_nt[1] = 1;
+    } else {
+        p.n_pieces = shifts;
+        for (int i = 0; i < shifts; ++i) { p.piece_t0[i] = i; p.piece_nt[i] = 1; }
+    }
+
+    // tap groups
+    TapList fw;
+    forward_taps(fw, R, pb.stride, pb.pad);
+    if (R == 1) {
+        p.n_groups = 1;
+        WgGroup& g = p.groups[0];
+        g.nb = 1; g.map[0] = fw.map[0]; g.dh[0] = fw.dh[0]; g.dw[0] = fw.dw[0];
+        g.rs[0][0] = 0; g.rs[1][0] = -1;
+    } else if (!p.stack) {
+        p.n_groups = 3;   // one group per filter row
+        for (int r = 0; r < 3; ++r) {
+            WgGroup& g = p.groups[r];
+            g.nb = 3;
+            for (int s = 0; s < 3; ++s) {
+                g.map[s] = fw.map[r * 3 + s]; g.dh[s] = fw.dh[r * 3 + s]; g.dw[s] = fw.dw[r * 3 + s];
+                g.rs[0][s] = (int8_t)(r * 3 + s); g.rs[1][s] = -1;
+            }
+        }
+    } else {
+        p.n_groups = 2;   // rows {0,1} and {1,2}; the second group's copy 0 repeats row 1 and is dropped
+        for (int gi = 0; gi < 2; ++gi) {
+            WgGroup& g = p.groups[gi];
+            const int r0 = gi;   // x is gathered at filter row r0; dy copy a lands on row r0 + a
+            g.nb = 3;
+            for (int s = 0; s < 3; ++s) {
+                g.map[s] = fw.map[r0 * 3 + s]; g.dh[s] = fw.dh[r0 * 3 + s]; g.dw[s] = fw.dw[r0 * 3 + s];
+                g.rs[0][s] = gi == 0 ? (int8_t)(r0 * 3 + s) : (int8_t)-1;
+                g.rs[1][s] = (int8_t)((r0 + 1) * 3 + s);
+            }
+        }
+    }
 
     // pixel chunk: 64 pixels, or 32 when a 64-pixel stage would not leave room for three stages
     p.pb = 64;
     for (;;) {
-        p.box_bytes = p.pb * p.cw * 2;
-        p.stage_bytes = (p.a_boxes + p.taps_per_group * p.b_boxes) * p.box_bytes;
+        p.box_a = p.pb * p.cw_a * 2;
+        p.box_b = p.pb * p.cw_b * 2;
+        p.stage_bytes = p.a_boxes * p.box_a + shifts * p.b_boxes * p.box_b;
         if (p.stage_bytes * 3 <= 200 * 1024 || p.pb == 32) break;
         p.pb = 32;
     }
@@ -242,26 +351,26 @@ b2c_status launch_conv_wgrad(b2c_ctx* ctx, const WgradProblem& pb, cudaStream_t 
     p.bw = pb.q < p.pb ? pb.q : p.pb;
     p.bh = (p.pb / p.bw) < pb.p ? (p.pb / p.bw) : pb.p;
     p.bn = p.pb / (p.bw * p.bh);
+    if (p.stack && p.bn != 1) return B2C_ERR_UNSUPPORTED_SHAPE;   // cannot happen: 64 pixels per image guarantee bn == 1
     p.tiles_w = pb.q / p.bw;
-    p.tiles_h = pb.p / p.bh;
+    p.tiles_h = (pb.p + (p.stack ? 1 : 0) + p.bh - 1) / p.bh;   // stacked: dy copy 1 of row p-1 is met at chunk row p
     const int tiles_n = (pb.n + p.bn - 1) / p.bn;
     p.chunks_total = p.tiles_w * p.tiles_h * tiles_n;
     const int base = p.n_ktiles * p.n_ctiles * p.n_groups;
-    int n_splits = (2 * ctx->sm_count + base - 1) / base;
+    int n_splits = ctx->sm_count / base;   // one wave of one CTA per SM
     if (n_splits > p.chunks_total / 4) n_splits = p.chunks_total / 4;
     if (n_splits < 1) n_splits = 1;
     p.n_splits = n_splits;
 
-    if (!encode_activation_map(ctx, &p.tmDy, pb.dy, pb.n, pb.p, pb.q, pb.k, 1, 0, 0, p.cw, p.bw, p.bh, p.bn)) return B2C_ERR_CUDA;
+    if (!encode_activation_map(ctx, &p.tmDy, pb.dy, pb.n, pb.p, pb.q, pb.k, 1, 0, 0, p.cw_a, p.bw, p.bh, p.bn)) return B2C_ERR_CUDA;
     if (pb.stride == 2) {
         for (int ph = 0; ph < 2; ++ph)
             for (int pw = 0; pw < 2; ++pw)
-                if (!encode_activation_map(ctx, &p.tmX[ph * 2 + pw], pb.x, pb.n, pb.h, pb.w, pb.c, 2, ph, pw, p.cw, p.bw, p.bh, p.bn))
+                if (!encode_activation_map(ctx, &p.tmX[ph * 2 + pw], pb.x, pb.n, pb.h, pb.w, pb.c, 2, ph, pw, p.cw_b, p.bw, p.bh, p.bn))
                     return B2C_ERR_CUDA;
     } else {
-        if (!encode_activation_map(ctx, &p.tmX[0], pb.x, pb.n, pb.h, pb.w, pb.c, 1, 0, 0, p.cw, p.bw, p.bh, p.bn)) return B2C_ERR_CUDA;
+        if (!encode_activation_map(ctx, &p.tmX[0], pb.x, pb.n, pb.h, pb.w, pb.c, 1, 0, 0, p.cw_b, p.bw, p.bh, p.bn)) return B2C_ERR_CUDA;
     }
-    forward_taps(p.taps, R, pb.stride, pb.pad);
     p.k_total = pb.k;
     p.c_total = pb.c;
     p.rs_total = R * R;
@@ -270,7 +379,7 @@ b2c_status launch_conv_wgrad(b2c_ctx* ctx, const WgradProblem& pb, cudaStream_t 
     p.spin_limit = ctx->spin_limit;
 
     if (!attr_set) {
-        B2C_CUDA(cudaFuncSetAttribute(conv_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
+        B2C_CUDA(cudaFuncSetAttribute(conv_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 212 * 1024));
         attr_set = true;
     }
     const size_t smem_bytes = (size_t)p.stages * p.stage_bytes + 1024;
