@@ -226,3 +226,86 @@ def check_step(net, spec, images, labels, n, n_micro_scale=1, sample=None, seed=
                 if L["src"] != 0:
                     rep.add(f"{name} dgrad", grad(L["src"], s_slot), rb(oracle.conv2d_dgrad(dy, w, x.shape, L["stride"], L["pad"])))
     return rep
+
+
+def check_step_sampled(net, spec, images, labels, n, groups=1, samples=128, bn_channels=4, seed=0):
+    """Full-size variant of check_step: every layer of the pass left in the workspace is checked against the oracle
+    on its own device inputs, but only on what the oracle can compute one by one at this size -- `samples` random
+    outputs per convolution (forward, data gradient) and a few filter entries (weight gradient), `bn_channels` whole
+    channels per BatchNorm (statistics, outputs, both gradients), and the small head in full.  Host copies are fp32
+    (exact for bf16 data) and fetched on demand, so the largest workloads fit in host memory."""
+    rep = Report()
+    rng = np.random.default_rng(seed)
+    rb, rf = oracle.round_bf16, oracle.round_f32
+    wq, wm, g = net.unpack(net.w_bf16), net.unpack(net.w), net.unpack(net.g)
+    slots, n_contrib = grad_slots(spec)
+    per = n // groups
+
+    def host32(t):
+        return t.detach().float().cpu().numpy()
+
+    def act(t):
+        if t == 0:
+            return np.asarray(images, np.float32)
+        dt = torch.float32 if spec[t - 1]["kind"] == "fc" else torch.bfloat16
+        return host32(net.tensor_view(t, _shape(spec, t, n, net), dt))
+
+    def grad(t, slot):
+        return host32(net.tensor_view(t, _shape(spec, t, n, net), torch.bfloat16, True, slot))
+
+    def cols(a, chs):   # selected channels as a contiguous fp64 [rows, len(chs)] array per group
+        return np.ascontiguousarray(a.reshape(groups, -1, a.shape[-1])[:, :, chs], dtype=np.float64)
+
+    def tol(full, ref):
+        return MAX_REL * float(np.max(np.abs(full))) / max(float(np.max(np.abs(ref))), 1e-30)
+
+    for i, L in enumerate(spec):
+        k, name = L["kind"], L.get("name", str(i))
+        if k == "conv":
+            x, w, y = act(L["src"]), wq[f"w{i}"].astype(np.float64), act(i + 1)
+            idx, ref = _conv_samples(rng, x, w, y.shape, L["stride"], L["pad"], samples)
+            rep.add(f"{name} fwd (sampled)", y[tuple(idx.T)], rb(ref), 2 * REL_FRO, tol(y, ref))
+            dy = grad(i + 1, 0)
+            idx, ref = _wgrad_samples(rng, dy, x, L["R"], L["stride"], L["pad"], max(8, samples // 8))
+            rep.add(f"{name} wgrad (sampled)", g[f"w{i}"][tuple(idx.T)], ref, 2 * REL_FRO, tol(g[f"w{i}"], ref))
+            if L["src"] != 0:
+                dx = grad(L["src"], slots[i][0])
+                idx, ref = _dgrad_samples(rng, dy, w, x.shape, L["stride"], L["pad"], samples)
+                rep.add(f"{name} dgrad (sampled)", dx[tuple(idx.T)], rb(ref), 2 * REL_FRO, tol(dx, ref))
+        elif k == "bn":
+            C = L["C"]
+            chs = np.sort(rng.choice(C, size=min(bn_channels, C), replace=False))
+            y, a = cols(act(L["src"]), chs), cols(act(i + 1), chs)
+            res = cols(act(L["res"]), chs) if L["res"] >= 0 else None
+            g1 = cols(grad(i + 1, 0), chs)
+            g2 = cols(grad(i + 1, 1), chs) if n_contrib[i + 1] == 2 else None
+            gam, bet = wm[f"gamma{i}"][chs], wm[f"beta{i}"][chs]
+            a_ref, dy_ref, dres_ref, dg, db = [], [], [], 0.0, 0.0
+            for gi in range(groups):
+                mean, var, invstd = oracle.bn_stats(y[gi], 1e-5)
+                mean, invstd = rf(mean), rf(invstd)
+                a_ref.append(oracle.bn_relu_apply(y[gi], mean, invstd, gam, bet, None if res is None else res[gi], L["relu"]))
+                q = oracle.bn_relu_bwd(g1[gi], None if g2 is None else g2[gi], y[gi], a[gi], gam, mean, invstd, L["relu"], L["res"] >= 0)
+                dy_ref.append(q[0]); dres_ref.append(q[1]); dg = dg + q[2]; db = db + q[3]
+            rep.add(f"{name} fwd (channels)", a, rb(np.stack(a_ref)))
+            rep.add(f"{name} bwd dy (channels)", cols(grad(L["src"], slots[i][0]), chs), rb(np.stack(dy_ref)))
+            if L["res"] >= 0:
+                rep.add(f"{name} bwd dres (channels)", cols(grad(L["res"], slots[i][1]), chs), rb(np.stack(dres_ref)))
+            rep.add(f"{name} dgamma (channels)", g[f"gamma{i}"][chs], dg)
+            rep.add(f"{name} dbeta (channels)", g[f"beta{i}"][chs], db)
+        elif k == "avgpool":
+            rep.add(f"{name} fwd", act(i + 1), rb(oracle.avgpool_fwd(act(L["src"]))))
+            rep.add(f"{name} bwd", grad(L["src"], slots[i][0]), rb(oracle.avgpool_bwd(grad(i + 1, 0), L["H"], L["W"])))
+        elif k == "fc":
+            pooled, dz = act(L["src"]).astype(np.float64), grad(i + 1, 0).astype(np.float64)
+            z = pooled @ wq[f"w{i}"].astype(np.float64).T + wm[f"b{i}"].astype(np.float64)
+            rep.add(f"{name} fwd", act(i + 1)[:, :L["K"]], z)
+            rep.add(f"{name} wgrad", g[f"w{i}"], dz[:, :L["K"]].T @ pooled)
+            rep.add(f"{name} bias grad", g[f"b{i}"], dz[:, :L["K"]].sum(0), 1e-4, 1e-4)
+            rep.add(f"{name} dgrad", grad(L["src"], slots[i][0]), rb(dz[:, :L["K"]] @ wq[f"w{i}"].astype(np.float64)))
+        elif k == "xent":
+            z = act(L["src"])[:, :L["K"]].astype(np.float64)
+            loss, dz = oracle.softmax_xent(z, labels, 1.0 / per)
+            rep.add("loss", np.array([net.loss.item()]), np.array([loss]), 1e-5, 1e-5)
+            rep.add("dlogits", grad(L["src"], slots[i][0])[:, :L["K"]], rb(dz))
+    return rep

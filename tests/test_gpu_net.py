@@ -264,3 +264,59 @@ def test_concurrent_micro_batches_match_sequential(ctx):
     for name in sorted(params):
         assert_close(gp[name], gs[name], f"grad {name} (concurrent vs sequential)", 1e-2, 3e-2)
     seq.close(); par.close()
+
+
+def _full_size_sampled(ctx, spec, micro_batch, n_micro, seed):
+    """One pass of a full-size workload in the launch configuration bench.py times (all micro-batches side by side),
+    every layer checked on sampled outputs against the oracle; then the fused update against the oracle's update on
+    the device gradient sum, element by element."""
+    from paper_2503_23186_b200 import binding
+    from netcheck import check_step_sampled
+    params = wl.init_params(spec, seed)
+    images, labels = wl.image_batch(seed, micro_batch * n_micro)
+    net = binding.Net(ctx, spec, micro_batch, n_concurrent=n_micro)
+    net.load_params(params)
+    d_img, d_lab = dev_bf16(images), torch.from_numpy(labels).cuda()
+    net.train_step(d_img, d_lab, n_micro, LR, MU, WD, update=False)
+    assert ctx.device_status() == 0
+    rep = check_step_sampled(net, spec, images, labels, micro_batch * n_micro, groups=n_micro, samples=96, seed=seed)
+    worst = rep.worst()
+    print("full-size sampled check: %d comparisons, worst %s relF=%.3e max=%.3e" % (len(rep.rows), worst[0], worst[1], worst[2]))
+    rep.assert_ok()
+    # scale invariance of every convolution that feeds a BatchNorm: <w, dL/dw> ~ 0 (holds at any size)
+    g, w = net.unpack(net.g), net.unpack(net.w)
+    for i, L in enumerate(spec):
+        if L["kind"] == "conv":
+            assert abs(np.vdot(g[f"w{i}"], w[f"w{i}"])) <= 2e-2 * np.linalg.norm(g[f"w{i}"]) * np.linalg.norm(w[f"w{i}"]), L["name"]
+    # the update, on the device's own gradient sum
+    net.apply_update(n_micro, LR, MU, WD)
+    assert ctx.device_status() == 0
+    w_new, v_new = net.unpack(net.w), net.unpack(net.v)
+    for name in sorted(params):
+        rw, rv = oracle.sgd_momentum(params[name], np.zeros_like(params[name]), g[name], 1.0 / n_micro, LR, MU, WD)
+        assert_close(w_new[name], rw, f"w_new {name}", SGD_REL, 1e-5)
+        assert_close(v_new[name], rv, f"v_new {name}", SGD_REL, 1e-5)
+    assert torch.equal(net.w_bf16, net.w.to(torch.bfloat16))
+    net.close()
+
+
+def test_resnet18_batch1024_config4_full_size(ctx):
+    _full_size_sampled(ctx, wl.resnet18_spec(), 128, 8, 0)
+
+
+def test_wrn28_10_batch256_config5_full_size(ctx):
+    _full_size_sampled(ctx, wl.wrn28_10_spec(), 256, 1, 0)
+
+
+def test_wrn28_10_small_batch_layerwise(ctx):
+    """The WRN-28-10-shaped net at batch 8: every layer in full against the oracle (teacher-forced)."""
+    from paper_2503_23186_b200 import binding
+    from netcheck import check_step
+    spec = wl.wrn28_10_spec()
+    net = binding.Net(ctx, spec, 8)
+    net.load_params(wl.init_params(spec, 0))
+    images, labels = wl.image_batch(0, 8)
+    net.train_step(dev_bf16(images), torch.from_numpy(labels).cuda(), 1, LR, MU, WD, update=False)
+    assert ctx.device_status() == 0
+    check_step(net, spec, images, labels, 8).assert_ok()
+    net.close()
