@@ -91,14 +91,18 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                                          "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                                          "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             threading.Thread(target=self._pump, daemon=True).start()
         except OSError:
             self.proc = None
 
     def _pump(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.lines.append((time.time(), line.strip()))
+
+    def mark(self):
+        """Start of the window whose samples count (the sampler itself is started earlier: nvidia-smi is slow to start)."""
+        self.t0 = time.time()
 
     def stop(self):
         if self.proc is None:
@@ -110,7 +114,9 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in self.lines:
+        for stamp, line in self.lines:
+            if stamp < getattr(self, "t0", 0.0):
+                continue
             parts = [p.strip() for p in line.split(",")]
             if len(parts) < 6:
                 continue
@@ -180,7 +186,7 @@ def run_reference(args, spec, name):
 def run_b2c(args, spec, name, micro_batch, n_micro):
     import torch
     import torch.distributed as dist
-    from paper_2503_23186_b200 import binding
+    from paper_2503_23186_b200 import binding, data_parallel
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -200,21 +206,17 @@ def run_b2c(args, spec, name, micro_batch, n_micro):
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")   # larger than the 126 MB L2
 
     def step(img, lab):
-        if world == 1:
-            net.train_step(img, lab, n_micro, LR, MU, WD, update=True)
-        else:
-            # data parallel: replicas exchange the summed gradients, then every replica applies the same update
-            net.train_step(img, lab, n_micro, LR, MU, WD, update=False)
-            dist.all_reduce(net.g)
-            net.apply_update(n_micro * world, LR, MU, WD)
+        # one replica: the fused single-call step; several: backward, NCCL sum of the gradient arrays, same update everywhere
+        data_parallel.dp_train_step(net, img, lab, n_micro, LR, MU, WD)
 
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
     for _ in range(max(args.warmup, 3)):
         step(d_img, d_lab)
     ctx.check_device()
     net.profile_enable(True)
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
+    sampler.mark()
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
@@ -304,7 +306,7 @@ def run_b2c(args, spec, name, micro_batch, n_micro):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="b2c", choices=["b2c", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
