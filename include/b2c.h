@@ -89,11 +89,13 @@ b2c_status b2c_conv2d_fwd(b2c_ctx* ctx, const b2c_conv_desc* d, const void* x, c
  *            b2c_conv2d_fwd); otherwise the call zeroes it and computes them (scratch owned by caller)
  *   save_mean, save_invstd fp32 [c] (outputs, used by the backward pass)
  *   run_mean, run_var fp32 [c] or NULL: running statistics, updated with `momentum` and the
- *            unbiased variance.   c must be a multiple of 8. */
+ *            unbiased variance.   c must be a multiple of 8.
+ *   relu_mask  NULL, or n*h*w*c/8 bytes (output, only written when relu != 0): bit i of byte j is "a[8j+i] > 0".
+ *            b2c_bn_relu_bwd can read it in place of a (1/16 of the bytes). */
 b2c_status b2c_bn_relu_fwd(b2c_ctx* ctx, int n, int h, int w, int c, const void* y, double* ch_stats, int stats_ready,
                            const float* gamma, const float* beta, const void* residual, int relu, float eps, void* a,
                            float* save_mean, float* save_invstd, float* run_mean, float* run_var, float momentum,
-                           void* stream);
+                           void* relu_mask, void* stream);
 
 /* Global average pool: pooled[n,c] = mean over h*w of a[n,:,:,c]; bf16 in, bf16 out; c % 8 == 0. */
 b2c_status b2c_avgpool_fwd(b2c_ctx* ctx, int n, int hw, int c, const void* a, void* pooled, void* stream);
@@ -125,12 +127,13 @@ size_t b2c_bn_relu_bwd_workspace_bytes(int c);
  * dbeta = sum dz; dgamma = sum dz*xhat, xhat = (y-mean)*invstd;
  * dy = gamma*invstd*(dz - dbeta/m - xhat*dgamma/m);  dres = dz.
  *   da1 bf16; da2 bf16 or NULL; y, a bf16 (forward input / output); dy bf16; dres bf16 or NULL
+ *   relu_mask  NULL, or the bit mask b2c_bn_relu_fwd wrote: then a is not read and may be NULL
  *   dgamma, dbeta fp32 [c]: overwritten if acc == 0, accumulated into if acc != 0
  *   ws: scratch of b2c_bn_relu_bwd_workspace_bytes(c) bytes; the call zeroes it itself. */
 b2c_status b2c_bn_relu_bwd(b2c_ctx* ctx, int n, int h, int w, int c, const void* da1, const void* da2, const void* y,
                            const void* a, const float* gamma, const float* save_mean, const float* save_invstd,
-                           int relu, void* dy, void* dres, float* dgamma, float* dbeta, int acc, void* ws,
-                           size_t ws_bytes, void* stream);
+                           int relu, void* dy, void* dres, float* dgamma, float* dbeta, int acc,
+                           const void* relu_mask, void* ws, size_t ws_bytes, void* stream);
 
 /* (No counterpart in the paper: a packaging variant of b2c_bn_relu_bwd.)
  * The same computation, arguments and results as b2c_bn_relu_bwd, but without the `ws` argument: the per-channel

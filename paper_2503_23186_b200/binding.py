@@ -136,10 +136,10 @@ class Context:
                                     _ptr(bias), _ptr(ch_stats), _stream()), "b2c_conv2d_fwd")
 
     def bn_relu_fwd(self, n, h, w, c, y, ch_stats, stats_ready, gamma, beta, residual, relu, eps, a, save_mean, save_invstd,
-                    run_mean=None, run_var=None, momentum=0.1):
+                    run_mean=None, run_var=None, momentum=0.1, relu_mask=None):
         _check(lib().b2c_bn_relu_fwd(self.handle, n, h, w, c, _ptr(y), _ptr(ch_stats), c_int(int(stats_ready)), _ptr(gamma), _ptr(beta),
                                      _ptr(residual), c_int(int(relu)), c_float(eps), _ptr(a), _ptr(save_mean), _ptr(save_invstd),
-                                     _ptr(run_mean), _ptr(run_var), c_float(momentum), _stream()), "b2c_bn_relu_fwd")
+                                     _ptr(run_mean), _ptr(run_var), c_float(momentum), _ptr(relu_mask), _stream()), "b2c_bn_relu_fwd")
 
     def avgpool_fwd(self, n, hw, c, a, pooled):
         _check(lib().b2c_avgpool_fwd(self.handle, n, hw, c, _ptr(a), _ptr(pooled), _stream()), "b2c_avgpool_fwd")
@@ -160,10 +160,10 @@ class Context:
     def bn_relu_bwd_workspace_bytes(c) -> int:
         return lib().b2c_bn_relu_bwd_workspace_bytes(c_int(c))
 
-    def bn_relu_bwd(self, n, h, w, c, da1, da2, y, a, gamma, save_mean, save_invstd, relu, dy, dres, dgamma, dbeta, acc, ws):
+    def bn_relu_bwd(self, n, h, w, c, da1, da2, y, a, gamma, save_mean, save_invstd, relu, dy, dres, dgamma, dbeta, acc, ws, relu_mask=None):
         _check(lib().b2c_bn_relu_bwd(self.handle, n, h, w, c, _ptr(da1), _ptr(da2), _ptr(y), _ptr(a), _ptr(gamma), _ptr(save_mean),
                                      _ptr(save_invstd), c_int(int(relu)), _ptr(dy), _ptr(dres), _ptr(dgamma), _ptr(dbeta), c_int(int(acc)),
-                                     _ptr(ws), c_size_t(ws.numel() * ws.element_size()), _stream()), "b2c_bn_relu_bwd")
+                                     _ptr(relu_mask), _ptr(ws), c_size_t(ws.numel() * ws.element_size()), _stream()), "b2c_bn_relu_bwd")
 
     def bn_relu_bwd_static(self, n, h, w, c, da1, da2, y, a, gamma, save_mean, save_invstd, relu, dy, dres, dgamma, dbeta, acc):
         """b2c_bn_relu_bwd without a caller-provided workspace: the accumulators live inside the library, so the

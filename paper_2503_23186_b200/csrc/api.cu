@@ -170,7 +170,7 @@ struct LayerPlan {
     int c_pad = 0, k_pad = 0;      // stored input / output channels of conv and fc layers
     int p = 0, q = 0;
     long long w_off = -1, gamma_off = -1, beta_off = -1, bias_off = -1;   // elements into the flat parameter arrays
-    long long mean_off = -1, invstd_off = -1, bwd_ws_off = -1;            // bytes into the workspace
+    long long mean_off = -1, invstd_off = -1, bwd_ws_off = -1, mask_off = -1;   // bytes into the workspace
     int src_slot = -1, res_slot = -1;                                     // which gradient buffer of src / res this layer writes
 };
 
@@ -295,6 +295,7 @@ b2c_status b2c_net_create_concurrent(b2c_ctx* ctx, const b2c_layer_desc* layers,
                 }
                 o = in; o.producer = i; o.n_contrib = 0; o.grad_off[0] = o.grad_off[1] = -1; o.stats_off = -1; o.fused_stats = false;
                 o.act_off = alloc(o.elems() * 2);
+                if (d.relu) L.mask_off = alloc(o.elems() / 8);   // one bit per output for the backward pass
                 break;
             }
             case B2C_LAYER_AVGPOOL: {
@@ -507,7 +508,7 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
                     B2C_TRY(launch_bn_fwd(ctx, G, (long long)net->micro_batch * in.h * in.w, in.c, act(d.src), stats, ready, net->w + L.gamma_off,
                                           net->w + L.beta_off, d.res >= 0 ? act(d.res) : nullptr, d.relu, 1e-5f, act(i + 1),
                                           reinterpret_cast<float*>(net->ws + L.mean_off), reinterpret_cast<float*>(net->ws + L.invstd_off), nullptr,
-                                          nullptr, 0.f, stream));
+                                          nullptr, 0.f, L.mask_off >= 0 ? net->ws + L.mask_off : nullptr, stream));
                     break;
                 }
                 case B2C_LAYER_AVGPOOL: {
@@ -572,7 +573,8 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
                                           act(d.src), act(i + 1), net->w + L.gamma_off, reinterpret_cast<float*>(net->ws + L.mean_off),
                                           reinterpret_cast<float*>(net->ws + L.invstd_off), d.relu, grad(d.src, L.src_slot),
                                           d.res >= 0 ? grad(d.res, L.res_slot) : nullptr, net->g + L.gamma_off, net->g + L.beta_off, 1,
-                                          reinterpret_cast<double*>(net->ws + L.bwd_ws_off), stream));
+                                          reinterpret_cast<double*>(net->ws + L.bwd_ws_off), /*sums_zeroed=*/in.stats_off >= 0,
+                                          L.mask_off >= 0 ? net->ws + L.mask_off : nullptr, stream));
                     break;
                 }
                 case B2C_LAYER_CONV: {

@@ -103,7 +103,7 @@ __global__ void __launch_bounds__(kEwThreads, 2) bn_apply_kernel(const void* __r
                                                                  const float* __restrict__ gamma, const float* __restrict__ beta,
                                                                  const void* __restrict__ residual, int relu, float eps, void* __restrict__ a,
                                                                  float* save_mean, float* save_invstd, float* run_mean, float* run_var,
-                                                                 float momentum)
+                                                                 float momentum, uint8_t* __restrict__ relu_mask)
 {
     const RowWalk rw(c);
     const int g = threadIdx.x % rw.groups, rl = threadIdx.x / rw.groups;
@@ -156,7 +156,16 @@ __global__ void __launch_bounds__(kEwThreads, 2) bn_apply_kernel(const void* __r
                 if (residual != nullptr) z += res[i];
                 f[i] = (relu && z < 0.f) ? 0.f : z;
             }
-            reinterpret_cast<uint4*>(a)[base + (r + u * step) * rw.groups + g] = pack8(f);
+            const uint4 packed = pack8(f);
+            reinterpret_cast<uint4*>(a)[base + (r + u * step) * rw.groups + g] = packed;
+            if (relu_mask != nullptr) {   // one bit per stored output: "a > 0", read by the backward pass instead of a
+                float st[8];
+                unpack8(packed, st);
+                unsigned bits = 0;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) bits |= (st[i] > 0.f ? 1u : 0u) << i;
+                relu_mask[base + (r + u * step) * rw.groups + g] = (uint8_t)bits;
+            }
         }
     }
 }
@@ -165,7 +174,8 @@ __global__ void __launch_bounds__(kEwThreads, 2) bn_apply_kernel(const void* __r
 // Pass 1: S1 = sum dz, S2 = sum dz*y per channel (dgamma = invstd*(S2 - mean*S1) is formed in fp64 by pass 2).
 __global__ void __launch_bounds__(kEwThreads, 2) bn_bwd_reduce_kernel(const void* __restrict__ da1, const void* __restrict__ da2,
                                                                       const void* __restrict__ y, const void* __restrict__ a, long long m, int c,
-                                                                      int relu, double* __restrict__ sums_all /* [G][2c] */)
+                                                                      int relu, double* __restrict__ sums_all /* [G][2c] */,
+                                                                      const uint8_t* __restrict__ relu_mask)
 {
     extern __shared__ float s_acc[];
     for (int i = threadIdx.x; i < 2 * c; i += kEwThreads) s_acc[i] = 0.f;
@@ -181,6 +191,7 @@ __global__ void __launch_bounds__(kEwThreads, 2) bn_bwd_reduce_kernel(const void
         constexpr int U = 2;
         for (long long r = (long long)blockIdx.x * rw.rows_per_iter + rl; r < m; r += U * step) {
             uint4 v1[U], v2[U], vy[U], va[U];
+            unsigned mk[U];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const bool ok = r + u * step < m;
@@ -188,7 +199,11 @@ __global__ void __launch_bounds__(kEwThreads, 2) bn_bwd_reduce_kernel(const void
                 v1[u] = ld16_or_zero(da1, vi, ok);
                 if (da2 != nullptr) v2[u] = ld16_or_zero(da2, vi, ok);
                 vy[u] = ld16_or_zero(y, vi, ok);
-                if (relu) va[u] = ld16_or_zero(a, vi, ok);
+                mk[u] = 0xffu;
+                if (relu) {
+                    if (relu_mask != nullptr) mk[u] = ok ? (unsigned)__ldg(relu_mask + vi) : 0u;
+                    else va[u] = ld16_or_zero(a, vi, ok);
+                }
             }
 #pragma unroll
             for (int u = 0; u < U; ++u) {
@@ -196,12 +211,18 @@ __global__ void __launch_bounds__(kEwThreads, 2) bn_bwd_reduce_kernel(const void
                 unpack8(v1[u], d);
                 if (da2 != nullptr) unpack8(v2[u], d2);
                 unpack8(vy[u], fy);
-                if (relu) unpack8(va[u], fa);
+                if (relu && relu_mask == nullptr) {
+                    unpack8(va[u], fa);
+                    unsigned bits = 0;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) bits |= (fa[i] > 0.f ? 1u : 0u) << i;
+                    mk[u] = bits;
+                }
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
                     float dz = d[i];
                     if (da2 != nullptr) dz += d2[i];
-                    if (relu && !(fa[i] > 0.f)) dz = 0.f;
+                    if (!((mk[u] >> i) & 1u)) dz = 0.f;
                     sb[i] += dz;
                     sg[i] = fmaf(dz, fy[i], sg[i]);
                 }
@@ -224,7 +245,8 @@ __global__ void __launch_bounds__(kEwThreads, 2) bn_bwd_apply_kernel(const void*
                                                                      const float* __restrict__ gamma, const float* __restrict__ mean_all,
                                                                      const float* __restrict__ invstd_all, int relu,
                                                                      const double* __restrict__ sums_all, void* __restrict__ dy,
-                                                                     void* __restrict__ dres, float* dgamma, float* dbeta, int acc)
+                                                                     void* __restrict__ dres, float* dgamma, float* dbeta, int acc,
+                                                                     const uint8_t* __restrict__ relu_mask)
 {
     const RowWalk rw(c);
     const int g = threadIdx.x % rw.groups, rl = threadIdx.x / rw.groups;
@@ -262,6 +284,7 @@ __global__ void __launch_bounds__(kEwThreads, 2) bn_bwd_apply_kernel(const void*
     constexpr int U = 2;
     for (long long r = (long long)blockIdx.x * rw.rows_per_iter + rl; r < m; r += U * step) {
         uint4 v1[U], v2[U], vy[U], va[U];
+        unsigned mk[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const bool ok = r + u * step < m;
@@ -269,7 +292,11 @@ __global__ void __launch_bounds__(kEwThreads, 2) bn_bwd_apply_kernel(const void*
             v1[u] = ld16_or_zero(da1, vi, ok);
             if (da2 != nullptr) v2[u] = ld16_or_zero(da2, vi, ok);
             vy[u] = ld16_or_zero(y, vi, ok);
-            if (relu) va[u] = ld16_or_zero(a, vi, ok);
+            mk[u] = 0xffu;
+            if (relu) {
+                if (relu_mask != nullptr) mk[u] = ok ? (unsigned)__ldg(relu_mask + vi) : 0u;
+                else va[u] = ld16_or_zero(a, vi, ok);
+            }
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
@@ -278,12 +305,18 @@ __global__ void __launch_bounds__(kEwThreads, 2) bn_bwd_apply_kernel(const void*
             unpack8(v1[u], d);
             if (da2 != nullptr) unpack8(v2[u], d2);
             unpack8(vy[u], fy);
-            if (relu) unpack8(va[u], fa);
+            if (relu && relu_mask == nullptr) {
+                unpack8(va[u], fa);
+                unsigned bits = 0;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) bits |= (fa[i] > 0.f ? 1u : 0u) << i;
+                mk[u] = bits;
+            }
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 float dz = d[i];
                 if (da2 != nullptr) dz += d2[i];
-                if (relu && !(fa[i] > 0.f)) dz = 0.f;
+                if (!((mk[u] >> i) & 1u)) dz = 0.f;
                 d[i] = dz;
                 o[i] = k0[i] * (dz - kb[i] - (fy[i] - mu[i]) * kg[i]);
             }
@@ -383,13 +416,23 @@ __global__ void softmax_xent_kernel(const float* __restrict__ logits, int logits
     }
 }
 
-__global__ void bias_grad_kernel(const __nv_bfloat16* __restrict__ dz, int m, int k, int pitch, float* db, int accumulate)
+// db[ch] (+)= sum over rows of dz[row, ch]: a block per 32 channels x a slice of rows, warp-shuffle free (each thread
+// owns a channel and a row lane, partial sums meet in shared memory), one atomic per channel and block.
+__global__ void bias_grad_kernel(const __nv_bfloat16* __restrict__ dz, int m, int k, int pitch, float* db)
 {
-    const int ch = blockIdx.x * blockDim.x + threadIdx.x;
-    if (ch >= k) return;
+    __shared__ float part[8][33];
+    const int ch = blockIdx.x * 32 + threadIdx.x;        // blockDim = (32, 8)
     float s = 0.f;
-    for (int r = 0; r < m; ++r) s += __bfloat162float(dz[(long long)r * pitch + ch]);
-    db[ch] = accumulate ? db[ch] + s : s;
+    if (ch < k)
+        for (int r = blockIdx.y * 8 + threadIdx.y; r < m; r += gridDim.y * 8) s += __bfloat162float(dz[(long long)r * pitch + ch]);
+    part[threadIdx.y][threadIdx.x] = s;
+    __syncthreads();
+    if (threadIdx.y == 0 && ch < k) {
+        float t = 0.f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) t += part[j][threadIdx.x];
+        atomicAdd(db + ch, t);
+    }
 }
 
 // ------------------------------------------------------------------------------ update
@@ -420,17 +463,28 @@ __global__ void __launch_bounds__(kEwThreads) sgd_momentum_kernel(float4* __rest
 struct PackSegs {
     b2c_weight_seg seg[128];
 };
+// dst[c][rs-1-t][k] = src[k][t][c] per segment: for a fixed tap this is a k x c -> c x k transpose, done in 32 x 32
+// tiles through shared memory so that both the reads (c contiguous) and the writes (k contiguous) are coalesced.
+// blockIdx.z = segment, blockIdx.y = tap, blockIdx.x = tile of the (k, c) plane; blocks past a segment's extent exit.
 __global__ void weight_pack_dgrad_kernel(const __grid_constant__ PackSegs segs, const __nv_bfloat16* __restrict__ src,
                                          __nv_bfloat16* __restrict__ dst)
 {
-    const b2c_weight_seg sg = segs.seg[blockIdx.y];
-    const long long total = (long long)sg.k * sg.rs * sg.c;
-    const long long j = (long long)blockIdx.x * blockDim.x + threadIdx.x;   // destination index: [c][t][k]
-    if (j >= total) return;
-    const int k = (int)(j % sg.k);
-    const int t = (int)((j / sg.k) % sg.rs);
-    const int c = (int)(j / ((long long)sg.k * sg.rs));
-    dst[sg.offset + j] = src[sg.offset + ((long long)k * sg.rs + (sg.rs - 1 - t)) * sg.c + c];
+    __shared__ __nv_bfloat16 tile[32][33];
+    const b2c_weight_seg sg = segs.seg[blockIdx.z];
+    const int t = blockIdx.y;
+    if (t >= sg.rs) return;
+    const int tiles_c = (sg.c + 31) / 32, tiles_k = (sg.k + 31) / 32;
+    if ((int)blockIdx.x >= tiles_c * tiles_k) return;
+    const int k0 = ((int)blockIdx.x / tiles_c) * 32, c0 = ((int)blockIdx.x % tiles_c) * 32;
+    for (int j = threadIdx.y; j < 32; j += 8) {          // blockDim = (32, 8)
+        const int k = k0 + j, c = c0 + threadIdx.x;
+        tile[j][threadIdx.x] = (k < sg.k && c < sg.c) ? src[sg.offset + ((long long)k * sg.rs + t) * sg.c + c] : __float2bfloat16(0.f);
+    }
+    __syncthreads();
+    for (int j = threadIdx.y; j < 32; j += 8) {
+        const int c = c0 + j, k = k0 + threadIdx.x;
+        if (c < sg.c && k < sg.k) dst[sg.offset + ((long long)c * sg.rs + (sg.rs - 1 - t)) * sg.k + k] = tile[threadIdx.x][j];
+    }
 }
 
 // ------------------------------------------------------------------------------ launchers
@@ -445,7 +499,7 @@ static int ew_grid(b2c_ctx* ctx, int n_groups, long long m, int rows_per_iter)
 
 b2c_status launch_bn_fwd(b2c_ctx* ctx, int G, long long m, int c, const void* y, double* stats, bool stats_ready, const float* gamma,
                          const float* beta, const void* residual, int relu, float eps, void* a, float* save_mean, float* save_invstd,
-                         float* run_mean, float* run_var, float momentum, cudaStream_t stream)
+                         float* run_mean, float* run_var, float momentum, void* relu_mask, cudaStream_t stream)
 {
     const int rows_per_iter = kEwThreads / (c / 8);
     dim3 grid((unsigned)ew_grid(ctx, G, m, rows_per_iter), (unsigned)G);
@@ -454,21 +508,22 @@ b2c_status launch_bn_fwd(b2c_ctx* ctx, int G, long long m, int c, const void* y,
         bn_stats_kernel<<<grid, kEwThreads, sizeof(float) * 2 * c, stream>>>(y, m, c, stats);
     }
     bn_apply_kernel<<<grid, kEwThreads, 0, stream>>>(y, m, c, stats, gamma, beta, residual, relu, eps, a, save_mean, save_invstd, run_mean, run_var,
-                                                     momentum);
+                                                     momentum, relu ? reinterpret_cast<uint8_t*>(relu_mask) : nullptr);
     B2C_CUDA(cudaGetLastError());
     return B2C_OK;
 }
 
 b2c_status launch_bn_bwd(b2c_ctx* ctx, int G, long long m, int c, const void* da1, const void* da2, const void* y, const void* a,
                          const float* gamma, const float* save_mean, const float* save_invstd, int relu, void* dy, void* dres, float* dgamma,
-                         float* dbeta, int acc, double* sums, cudaStream_t stream)
+                         float* dbeta, int acc, double* sums, bool sums_zeroed, const void* relu_mask, cudaStream_t stream)
 {
     const int rows_per_iter = kEwThreads / (c / 8);
     dim3 grid((unsigned)ew_grid(ctx, G, m, rows_per_iter), (unsigned)G);
-    B2C_CUDA(cudaMemsetAsync(sums, 0, sizeof(double) * 2 * c * G, stream));
-    bn_bwd_reduce_kernel<<<grid, kEwThreads, sizeof(float) * 2 * c, stream>>>(da1, da2, y, a, m, c, relu, sums);
+    const uint8_t* mask = relu ? reinterpret_cast<const uint8_t*>(relu_mask) : nullptr;
+    if (!sums_zeroed) B2C_CUDA(cudaMemsetAsync(sums, 0, sizeof(double) * 2 * c * G, stream));
+    bn_bwd_reduce_kernel<<<grid, kEwThreads, sizeof(float) * 2 * c, stream>>>(da1, da2, y, a, m, c, relu, sums, mask);
     bn_bwd_apply_kernel<<<grid, kEwThreads, 0, stream>>>(da1, da2, y, a, m, c, gamma, save_mean, save_invstd, relu, sums, dy, dres, dgamma, dbeta,
-                                                         acc);
+                                                         acc, mask);
     B2C_CUDA(cudaGetLastError());
     return B2C_OK;
 }
@@ -481,7 +536,7 @@ extern "C" {
 
 b2c_status b2c_bn_relu_fwd(b2c_ctx* ctx, int n, int h, int w, int c, const void* y, double* ch_stats, int stats_ready, const float* gamma,
                            const float* beta, const void* residual, int relu, float eps, void* a, float* save_mean, float* save_invstd,
-                           float* run_mean, float* run_var, float momentum, void* stream_)
+                           float* run_mean, float* run_var, float momentum, void* relu_mask, void* stream_)
 {
     cudaStream_t stream = (cudaStream_t)stream_;
     if (!ctx || !y || !ch_stats || !gamma || !beta || !a || !save_mean || !save_invstd) return B2C_ERR_INVALID_ARG;
@@ -490,25 +545,25 @@ b2c_status b2c_bn_relu_fwd(b2c_ctx* ctx, int n, int h, int w, int c, const void*
     if (!b2c_aligned16(y) || !b2c_aligned16(a) || (residual && !b2c_aligned16(residual)) || (reinterpret_cast<uintptr_t>(ch_stats) & 7u))
         return B2C_ERR_MISALIGNED;
     return launch_bn_fwd(ctx, 1, (long long)n * h * w, c, y, ch_stats, stats_ready != 0, gamma, beta, residual, relu, eps, a, save_mean, save_invstd,
-                         run_mean, run_var, momentum, stream);
+                         run_mean, run_var, momentum, relu_mask, stream);
 }
 
 size_t b2c_bn_relu_bwd_workspace_bytes(int c) { return c > 0 ? sizeof(double) * 2 * (size_t)c : 0; }
 
 b2c_status b2c_bn_relu_bwd(b2c_ctx* ctx, int n, int h, int w, int c, const void* da1, const void* da2, const void* y, const void* a,
                            const float* gamma, const float* save_mean, const float* save_invstd, int relu, void* dy, void* dres, float* dgamma,
-                           float* dbeta, int acc, void* ws, size_t ws_bytes, void* stream_)
+                           float* dbeta, int acc, const void* relu_mask, void* ws, size_t ws_bytes, void* stream_)
 {
     cudaStream_t stream = (cudaStream_t)stream_;
     if (!ctx || !da1 || !y || !gamma || !save_mean || !save_invstd || !dy || !dgamma || !dbeta || !ws) return B2C_ERR_INVALID_ARG;
-    if (relu && !a) return B2C_ERR_INVALID_ARG;
+    if (relu && !a && !relu_mask) return B2C_ERR_INVALID_ARG;
     if (n < 1 || h < 1 || w < 1 || c < 8 || c % 8 || c > 2048) return B2C_ERR_UNSUPPORTED_SHAPE;
     if (ws_bytes < b2c_bn_relu_bwd_workspace_bytes(c)) return B2C_ERR_WORKSPACE_TOO_SMALL;
     if (!b2c_aligned16(da1) || (da2 && !b2c_aligned16(da2)) || !b2c_aligned16(y) || (a && !b2c_aligned16(a)) || !b2c_aligned16(dy) ||
         (dres && !b2c_aligned16(dres)) || (reinterpret_cast<uintptr_t>(ws) & 7u))
         return B2C_ERR_MISALIGNED;
     return launch_bn_bwd(ctx, 1, (long long)n * h * w, c, da1, da2, y, a, gamma, save_mean, save_invstd, relu, dy, dres, dgamma, dbeta, acc,
-                         reinterpret_cast<double*>(ws), stream);
+                         reinterpret_cast<double*>(ws), false, relu_mask, stream);
 }
 
 b2c_status b2c_avgpool_fwd(b2c_ctx* ctx, int n, int hw, int c, const void* a, void* pooled, void* stream_)
@@ -563,7 +618,11 @@ b2c_status b2c_bias_grad(b2c_ctx* ctx, int m, int k, int pitch, const void* dz, 
 {
     if (!ctx || !dz || !db) return B2C_ERR_INVALID_ARG;
     if (m < 1 || k < 1 || pitch < k) return B2C_ERR_UNSUPPORTED_SHAPE;
-    bias_grad_kernel<<<(k + 127) / 128, 128, 0, (cudaStream_t)stream_>>>(reinterpret_cast<const __nv_bfloat16*>(dz), m, k, pitch, db, accumulate);
+    if (!accumulate) B2C_CUDA(cudaMemsetAsync(db, 0, sizeof(float) * (size_t)k, (cudaStream_t)stream_));
+    int row_blocks = (m + 63) / 64;
+    if (row_blocks > 64) row_blocks = 64;
+    bias_grad_kernel<<<dim3((unsigned)((k + 31) / 32), (unsigned)row_blocks), dim3(32, 8), 0, (cudaStream_t)stream_>>>(
+        reinterpret_cast<const __nv_bfloat16*>(dz), m, k, pitch, db);
     B2C_CUDA(cudaGetLastError());
     return B2C_OK;
 }
@@ -591,16 +650,17 @@ b2c_status b2c_weight_pack_dgrad(b2c_ctx* ctx, const b2c_weight_seg* segs, int n
     if (!ctx || !segs || !src_bf16 || !dst_bf16) return B2C_ERR_INVALID_ARG;
     if (n_segs < 1 || n_segs > 128) return B2C_ERR_UNSUPPORTED_SHAPE;
     PackSegs ps;
-    long long biggest = 0;
+    int max_tiles = 0, max_rs = 0;
     for (int i = 0; i < n_segs; ++i) {
         if (segs[i].k < 1 || segs[i].rs < 1 || segs[i].c < 1 || segs[i].offset < 0) return B2C_ERR_INVALID_ARG;
         ps.seg[i] = segs[i];
-        const long long sz = (long long)segs[i].k * segs[i].rs * segs[i].c;
-        biggest = sz > biggest ? sz : biggest;
+        const int tiles = ((segs[i].k + 31) / 32) * ((segs[i].c + 31) / 32);
+        max_tiles = tiles > max_tiles ? tiles : max_tiles;
+        max_rs = segs[i].rs > max_rs ? segs[i].rs : max_rs;
     }
-    dim3 grid((unsigned)((biggest + 255) / 256), (unsigned)n_segs);
-    weight_pack_dgrad_kernel<<<grid, 256, 0, (cudaStream_t)stream_>>>(ps, reinterpret_cast<const __nv_bfloat16*>(src_bf16),
-                                                                      reinterpret_cast<__nv_bfloat16*>(dst_bf16));
+    dim3 grid((unsigned)max_tiles, (unsigned)max_rs, (unsigned)n_segs);
+    weight_pack_dgrad_kernel<<<grid, dim3(32, 8), 0, (cudaStream_t)stream_>>>(ps, reinterpret_cast<const __nv_bfloat16*>(src_bf16),
+                                                                              reinterpret_cast<__nv_bfloat16*>(dst_bf16));
     B2C_CUDA(cudaGetLastError());
     return B2C_OK;
 }
@@ -637,7 +697,7 @@ b2c_status b2c_bn_relu_bwd_static(b2c_ctx* ctx, int n, int h, int w, int c, cons
     }
     // the array keeps the previous call's sums: the launcher clears the part this call uses
     return launch_bn_bwd(ctx, 1, (long long)n * h * w, c, da1, da2, y, a, gamma, save_mean, save_invstd, relu, dy, dres, dgamma, dbeta, acc,
-                         g_bn_bwd_static_ptr[current], stream);
+                         g_bn_bwd_static_ptr[current], false, nullptr, stream);
 }
 
 }  // extern "C"

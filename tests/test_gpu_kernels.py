@@ -174,8 +174,12 @@ def test_bn_relu_fwd_bwd(ctx, shape, relu, use_res):
     stats = torch.full((2 * C,), 7.0, dtype=torch.float64, device="cuda")   # stale contents must not matter
     sm, si = torch.empty(C, device="cuda"), torch.empty(C, device="cuda")
     rm, rv = torch.zeros(C, device="cuda"), torch.ones(C, device="cuda")
+    mask = torch.full((M * C // 8,), 0xAA, dtype=torch.uint8, device="cuda")
     ctx.bn_relu_fwd(N, H, W, C, dy_, stats, False, dev_f32(gamma), dev_f32(beta), None if res is None else dev_bf16(res), relu, 1e-5, a, sm, si,
-                    rm, rv, 0.1)
+                    rm, rv, 0.1, relu_mask=mask)
+    if relu:   # bit i of byte j says whether stored output 8j+i is positive
+        bits = np.unpackbits(mask.cpu().numpy(), bitorder="little").astype(bool)
+        assert np.array_equal(bits, host(a).reshape(-1) > 0)
     assert_close(sm, mean, "mean", 1e-5, 1e-5)
     assert_close(si, invstd, "invstd", 1e-4, 1e-4)
     assert_close(a, a_ref, "a")
@@ -195,6 +199,15 @@ def test_bn_relu_fwd_bwd(ctx, shape, relu, use_res):
     assert_close(db, db_ref - 2.0, "dbeta (accumulated)", 2e-3, 2e-3)
     if use_res:
         assert_close(dres, oracle.round_bf16(dres_ref), "dres", 1e-6, 1e-6)
+    if relu:
+        # the same backward pass reading the bit mask of the oracle's stored output instead of the output tensor
+        mask_ref = torch.from_numpy(np.packbits((a_ref.reshape(-1) > 0), bitorder="little")).cuda()
+        dyo2 = torch.empty_like(dyo)
+        dg2, db2 = torch.zeros(C, device="cuda"), torch.zeros(C, device="cuda")
+        ctx.bn_relu_bwd(N, H, W, C, dev_bf16(da1), None if da2 is None else dev_bf16(da2), dy_, None, dev_f32(gamma), dev_f32(mean32),
+                        dev_f32(invstd32), relu, dyo2, None, dg2, db2, False, ws, relu_mask=mask_ref)
+        assert_close(dyo2, host(dyo), "dy (mask)", 1e-5, 1e-2)   # same arithmetic; the channel sums differ in summation order only
+        assert_close(dg2, dg_ref, "dgamma (mask)", 2e-3, 2e-3)
     assert ctx.device_status() == 0
 
 
