@@ -106,6 +106,12 @@ b2c_status b2c_avgpool_bwd(b2c_ctx* ctx, int n, int hw, int c, const void* dpool
  * Used for the 3-channel image batch (TMA rows must be multiples of 16 bytes). c_out % 8 == 0. */
 b2c_status b2c_pad_channels(b2c_ctx* ctx, long m, int c_in, int c_out, const void* x, void* y, void* stream);
 
+/* Patch matrix of a 3x3, stride 1, pad 1 convolution: y[m, (r*3+s)*c_in + ch] = x[n, h+r-1, w+s-1, ch] (zero outside the
+ * image) for every pixel m = (n,h,w); columns 9*c_in .. c_out-1 are zero.  bf16 in, bf16 out; c_in <= 3, c_out >= 32, c_out % 8 == 0.
+ * With it the first convolution of a network (3 input channels) is the 1x1 convolution of the patch matrix with the
+ * filter bank viewed as [k][9*c_in] rows padded to c_out. */
+b2c_status b2c_im2col_3x3(b2c_ctx* ctx, int n, int h, int w, int c_in, int c_out, const void* x, void* y, void* stream);
+
 /* ---- Loss (Algorithm 1, "Compute loss") ------------------------------------------------- */
 
 /* Softmax cross-entropy over rows of logits fp32 [n, logits_pitch] (first `classes` columns used,
@@ -220,8 +226,12 @@ size_t b2c_net_param_count(const b2c_net* net);
 /* Element offset of a layer's parameter inside the flat arrays.  which: 0 = weight (conv: [k,r,s,c_padded],
  * fc: [k,c]), 1 = BN gamma, 2 = BN beta, 3 = fc bias.  Returns -1 if the layer has no such parameter. */
 long long b2c_net_param_offset(const b2c_net* net, int layer, int which);
-/* Input channels of the first convolution after padding (what the weight layout uses). */
+/* Stored input width of the first convolution (what its weight layout uses): the image channels rounded up to 16,
+ * or 32 when b2c_net_first_conv_im2col() is non-zero. */
 int b2c_net_padded_image_channels(const b2c_net* net);
+/* Non-zero if the first convolution (3x3, stride 1, at most 3 image channels) runs on the 3x3 patch matrix of the
+ * image batch: its filter bank is then stored as [k][32] rows holding the [r][s][c] taps flattened (27 used). */
+int b2c_net_first_conv_im2col(const b2c_net* net);
 /* Bytes of activation/gradient workspace one micro-batch needs. */
 size_t b2c_net_workspace_bytes(const b2c_net* net);
 /* Byte offset inside the workspace of tensor t's activation (bf16; logits fp32), or of its

@@ -28,7 +28,7 @@ EXPORTS = [
     "b2c_softmax_xent_fwd_bwd", "b2c_bn_relu_bwd_workspace_bytes", "b2c_bn_relu_bwd", "b2c_bn_relu_bwd_static", "b2c_conv2d_dgrad",
     "b2c_conv2d_wgrad", "b2c_bias_grad", "b2c_grad_accum_sgd_momentum", "b2c_weight_pack_dgrad",
     "b2c_net_create", "b2c_net_create_concurrent", "b2c_net_destroy", "b2c_net_param_count", "b2c_net_param_offset",
-    "b2c_net_padded_image_channels", "b2c_net_workspace_bytes", "b2c_net_tensor_offset", "b2c_net_bind",
+    "b2c_net_padded_image_channels", "b2c_net_first_conv_im2col", "b2c_im2col_3x3", "b2c_net_workspace_bytes", "b2c_net_tensor_offset", "b2c_net_bind",
     "b2c_net_sync_weights", "b2c_train_step", "b2c_net_apply_update", "b2c_net_profile_enable", "b2c_net_profile_read",
 ]
 PROF_KINDS = ["conv_fwd", "conv_dgrad", "conv_wgrad", "bn_fwd", "bn_bwd", "other", "update"]
@@ -147,6 +147,9 @@ class Context:
     def avgpool_bwd(self, n, hw, c, dpooled, da):
         _check(lib().b2c_avgpool_bwd(self.handle, n, hw, c, _ptr(dpooled), _ptr(da), _stream()), "b2c_avgpool_bwd")
 
+    def im2col_3x3(self, n, h, w, c_in, c_out, x, y):
+        _check(lib().b2c_im2col_3x3(self.handle, n, h, w, c_in, c_out, _ptr(x), _ptr(y), _stream()), "b2c_im2col_3x3")
+
     def pad_channels(self, m, c_in, c_out, x, y):
         _check(lib().b2c_pad_channels(self.handle, c_long(m), c_in, c_out, _ptr(x), _ptr(y), _stream()), "b2c_pad_channels")
 
@@ -208,6 +211,7 @@ class Net:
         self.param_count = lib().b2c_net_param_count(self.handle)
         self.workspace_bytes = lib().b2c_net_workspace_bytes(self.handle)
         self.image_c_pad = lib().b2c_net_padded_image_channels(self.handle)
+        self.first_conv_im2col = bool(lib().b2c_net_first_conv_im2col(self.handle))
         dev = torch.device("cuda")
         self.w = torch.zeros(self.param_count, dtype=torch.float32, device=dev)
         self.v = torch.zeros_like(self.w)
@@ -238,9 +242,12 @@ class Net:
 
     # ---- flat-array <-> per-layer parameter dictionaries (host-side layout bookkeeping)
     def _slots(self):
-        """Yield (name, offset, stored_shape, logical_shape)."""
+        """Yield (name, offset, stored_shape, logical_shape as laid out inside the stored array)."""
         for i, L in enumerate(self.spec):
             if L["kind"] == "conv":
+                if i == 0 and self.first_conv_im2col:   # [k][r][s][c] taps flattened into rows of the patch-matrix GEMM
+                    yield f"w{i}", self.param_offset(i, 0), (L["K"], self.image_c_pad), (L["K"], L["R"] * L["R"] * L["C"])
+                    continue
                 cpad = -(-L["C"] // 16) * 16
                 yield f"w{i}", self.param_offset(i, 0), (L["K"], L["R"], L["R"], cpad), (L["K"], L["R"], L["R"], L["C"])
             elif L["kind"] == "fc":
@@ -251,11 +258,17 @@ class Net:
                 yield f"gamma{i}", self.param_offset(i, 1), (L["C"],), (L["C"],)
                 yield f"beta{i}", self.param_offset(i, 2), (L["C"],), (L["C"],)
 
+    def _logical_shape(self, name):
+        L = self.spec[int(name.lstrip("wbgamet"))]
+        if name.startswith("w"):
+            return (L["K"], L["R"], L["R"], L["C"]) if L["kind"] == "conv" else (L["K"], L["C"])
+        return (L["K"],) if name.startswith("b") and not name.startswith("beta") else (L["C"],)
+
     def pack(self, params: dict) -> np.ndarray:
         flat = np.zeros(self.param_count, np.float32)
         for name, off, stored, logical in self._slots():
             buf = np.zeros(stored, np.float32)
-            buf[tuple(slice(0, s) for s in logical)] = params[name]
+            buf[tuple(slice(0, s) for s in logical)] = np.asarray(params[name]).reshape(logical)
             flat[off:off + buf.size] = buf.reshape(-1)
         return flat
 
@@ -264,7 +277,7 @@ class Net:
         out = {}
         for name, off, stored, logical in self._slots():
             size = int(np.prod(stored))
-            out[name] = flat[off:off + size].reshape(stored)[tuple(slice(0, s) for s in logical)].copy()
+            out[name] = flat[off:off + size].reshape(stored)[tuple(slice(0, s) for s in logical)].copy().reshape(self._logical_shape(name))
         return out
 
     def load_params(self, params: dict, velocity: dict | None = None):

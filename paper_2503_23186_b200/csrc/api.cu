@@ -168,6 +168,7 @@ struct TensorPlan {
 struct LayerPlan {
     b2c_layer_desc d;
     int c_pad = 0, k_pad = 0;      // stored input / output channels of conv and fc layers
+    int gemm_r = 0;                // filter size the convolution kernels see (1 for the patch-matrix stem)
     int p = 0, q = 0;
     long long w_off = -1, gamma_off = -1, beta_off = -1, bias_off = -1;   // elements into the flat parameter arrays
     long long mean_off = -1, invstd_off = -1, bwd_ws_off = -1, mask_off = -1;   // bytes into the workspace
@@ -183,6 +184,7 @@ struct b2c_net {
     int micro_batch = 0;
     int n_conc = 1;            // micro-batches processed side by side in one pass
     int image_h = 0, image_w = 0, image_c = 0, image_c_pad = 0;
+    bool stem_im2col = false;   // the first convolution runs as a 1x1 GEMM on the 3x3 patch matrix of the images
     std::vector<LayerPlan> layers;
     std::vector<TensorPlan> tensors;
     std::vector<b2c_weight_seg> segs;
@@ -257,6 +259,8 @@ b2c_status b2c_net_create_concurrent(b2c_ctx* ctx, const b2c_layer_desc* layers,
     if (layers[0].kind != B2C_LAYER_CONV || layers[0].src != 0) return fail(B2C_ERR_INVALID_ARG);
     net->image_h = layers[0].h; net->image_w = layers[0].w; net->image_c = layers[0].c;
     net->image_c_pad = round_up(layers[0].c, 16);
+    net->stem_im2col = layers[0].r == 3 && layers[0].stride == 1 && layers[0].c * 9 <= 32;
+    if (net->stem_im2col) net->image_c_pad = 32;
     {
         TensorPlan& t0 = net->tensors[0];
         t0.n = batch; t0.h = net->image_h; t0.w = net->image_w; t0.c = net->image_c_pad; t0.exists = true;
@@ -273,7 +277,8 @@ b2c_status b2c_net_create_concurrent(b2c_ctx* ctx, const b2c_layer_desc* layers,
         o.producer = i;
         switch (d.kind) {
             case B2C_LAYER_CONV: {
-                if (in.f32 || d.h != in.h || d.w != in.w || round_up(d.c, 16) != in.c) return fail(B2C_ERR_INVALID_ARG);
+                const bool patch = net->stem_im2col && i == 0;   // this layer reads the patch matrix: a 1x1 GEMM over 32 columns
+                if (in.f32 || d.h != in.h || d.w != in.w || (!patch && round_up(d.c, 16) != in.c)) return fail(B2C_ERR_INVALID_ARG);
                 if (d.k % 16 || !(d.r == 1 || d.r == 3) || !(d.stride == 1 || d.stride == 2)) return fail(B2C_ERR_UNSUPPORTED_SHAPE);
                 if (d.src != 0 && d.c % 16) return fail(B2C_ERR_UNSUPPORTED_SHAPE);
                 const int pad = (d.r - 1) / 2;
@@ -282,8 +287,9 @@ b2c_status b2c_net_create_concurrent(b2c_ctx* ctx, const b2c_layer_desc* layers,
                 if (L.p * d.stride != d.h || L.q * d.stride != d.w || !b2c_is_pow2(L.p) || !b2c_is_pow2(L.q)) return fail(B2C_ERR_UNSUPPORTED_SHAPE);
                 o.n = batch; o.h = L.p; o.w = L.q; o.c = d.k; o.exists = true;
                 o.act_off = alloc(o.elems() * 2);
-                L.w_off = palloc((size_t)d.k * d.r * d.r * L.c_pad);
-                net->segs.push_back(b2c_weight_seg{L.w_off, d.k, d.r * d.r, L.c_pad});
+                L.gemm_r = patch ? 1 : d.r;
+                L.w_off = palloc((size_t)d.k * L.gemm_r * L.gemm_r * L.c_pad);
+                net->segs.push_back(b2c_weight_seg{L.w_off, d.k, L.gemm_r * L.gemm_r, L.c_pad});
                 break;
             }
             case B2C_LAYER_BN: {
@@ -379,6 +385,7 @@ void b2c_net_destroy(b2c_net* net) { delete net; }
 size_t b2c_net_param_count(const b2c_net* net) { return net ? net->param_count : 0; }
 size_t b2c_net_workspace_bytes(const b2c_net* net) { return net ? net->ws_bytes : 0; }
 int b2c_net_padded_image_channels(const b2c_net* net) { return net ? net->image_c_pad : 0; }
+int b2c_net_first_conv_im2col(const b2c_net* net) { return net && net->stem_im2col ? 1 : 0; }
 
 long long b2c_net_param_offset(const b2c_net* net, int layer, int which)
 {
@@ -475,7 +482,10 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
         const void* t0;
         if (net->tensors[0].act_off >= 0) {
             ProfScope ps_(net, stream, B2C_PROF_OTHER, 1);
-            B2C_TRY(b2c_pad_channels(ctx, (long)N * net->image_h * net->image_w, net->image_c, net->image_c_pad, img, act(0), stream));
+            if (net->stem_im2col)
+                B2C_TRY(b2c_im2col_3x3(ctx, N, net->image_h, net->image_w, net->image_c, net->image_c_pad, img, act(0), stream));
+            else
+                B2C_TRY(b2c_pad_channels(ctx, (long)N * net->image_h * net->image_w, net->image_c, net->image_c_pad, img, act(0), stream));
             t0 = act(0);
         } else {
             t0 = img;
@@ -492,7 +502,7 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
                 case B2C_LAYER_CONV: {
                     KMajorProblem pb{};
                     pb.n = N; pb.ih = d.h; pb.iw = d.w; pb.ic = L.c_pad; pb.oh = L.p; pb.ow = L.q; pb.oc = d.k;
-                    pb.r = d.r; pb.stride = d.stride; pb.pad = (d.r - 1) / 2; pb.dgrad = false;
+                    pb.r = L.gemm_r; pb.stride = d.stride; pb.pad = (L.gemm_r - 1) / 2; pb.dgrad = false;
                     pb.in = act_in(d.src); pb.wt = w_bf16 + L.w_off; pb.out = act(i + 1);
                     pb.stats = o.fused_stats ? reinterpret_cast<double*>(net->ws + o.stats_off) : nullptr;
                     pb.stats_group_images = net->micro_batch;
@@ -581,7 +591,7 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
                     const void* dy = grad(i + 1, 0);
                     WgradProblem wp{};
                     wp.n = N; wp.h = d.h; wp.w = d.w; wp.c = L.c_pad; wp.p = L.p; wp.q = L.q; wp.k = d.k;
-                    wp.r = d.r; wp.stride = d.stride; wp.pad = (d.r - 1) / 2;
+                    wp.r = L.gemm_r; wp.stride = d.stride; wp.pad = (L.gemm_r - 1) / 2;
                     wp.dy = dy; wp.x = act_in(d.src); wp.dw = net->g + L.w_off;
                     {
                         ProfScope ps_(net, stream, B2C_PROF_CONV_WGRAD, 1);

@@ -381,6 +381,44 @@ __global__ void pad_channels_kernel(const __nv_bfloat16* __restrict__ x, long lo
     reinterpret_cast<uint4*>(y)[idx] = pack8(f);
 }
 
+// Patch matrix of a 3x3, stride 1, pad 1 convolution over a narrow image: y[pixel, (r*3+s)*c_in + ch] = x[n, h+r-1, w+s-1, ch]
+// (zero outside the image), columns 9*c_in .. c_out-1 zero.  Turns the first convolution into a 1x1-shaped GEMM.
+template <int C_IN>
+__global__ void im2col3x3_kernel(const __nv_bfloat16* __restrict__ x, int n, int h, int w, int c_out, void* __restrict__ y)
+{
+    // one thread per pixel: 9*C_IN (<= 32) values gathered with static tap offsets, written as whole 16-byte vectors
+    const long long pix = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (pix >= (long long)n * h * w) return;
+    const int ww = (int)(pix % w);
+    const int hh = (int)((pix / w) % h);
+    const long long img = pix / ((long long)w * h);
+    float f[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) f[i] = 0.f;
+#pragma unroll
+    for (int r = 0; r < 3; ++r) {
+        const int ih = hh + r - 1;
+#pragma unroll
+        for (int q = 0; q < 3; ++q) {
+            const int iw = ww + q - 1;
+            if (ih >= 0 && ih < h && iw >= 0 && iw < w) {
+                const __nv_bfloat16* src = x + ((img * h + ih) * w + iw) * C_IN;
+#pragma unroll
+                for (int ch = 0; ch < C_IN; ++ch) f[(r * 3 + q) * C_IN + ch] = __bfloat162float(src[ch]);
+            }
+        }
+    }
+    uint4* dst = reinterpret_cast<uint4*>(y) + pix * (c_out >> 3);
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+        float v[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = f[g * 8 + i];
+        dst[g] = pack8(v);
+    }
+    for (int g = 4; g < (c_out >> 3); ++g) dst[g] = make_uint4(0u, 0u, 0u, 0u);
+}
+
 // ------------------------------------------------------------------------------ loss
 // One warp per row.
 __global__ void softmax_xent_kernel(const float* __restrict__ logits, int logits_pitch, const int32_t* __restrict__ labels, int n, int classes,
@@ -596,6 +634,22 @@ b2c_status b2c_pad_channels(b2c_ctx* ctx, long m, int c_in, int c_out, const voi
     const long long total = (long long)m * (c_out / 8);
     pad_channels_kernel<<<(unsigned)((total + 255) / 256), 256, 0, (cudaStream_t)stream_>>>(reinterpret_cast<const __nv_bfloat16*>(x), m, c_in,
                                                                                             c_out, y);
+    B2C_CUDA(cudaGetLastError());
+    return B2C_OK;
+}
+
+b2c_status b2c_im2col_3x3(b2c_ctx* ctx, int n, int h, int w, int c_in, int c_out, const void* x, void* y, void* stream_)
+{
+    if (!ctx || !x || !y) return B2C_ERR_INVALID_ARG;
+    if (n < 1 || h < 1 || w < 1 || c_in < 1 || c_out < 32 || c_out % 8) return B2C_ERR_UNSUPPORTED_SHAPE;
+    if (!b2c_aligned16(y) || (reinterpret_cast<uintptr_t>(x) & 1u)) return B2C_ERR_MISALIGNED;
+    if (c_in > 3) return B2C_ERR_UNSUPPORTED_SHAPE;
+    const long long total = (long long)n * h * w;
+    const unsigned blocks = (unsigned)((total + 127) / 128);
+    const __nv_bfloat16* xs = reinterpret_cast<const __nv_bfloat16*>(x);
+    if (c_in == 3) im2col3x3_kernel<3><<<blocks, 128, 0, (cudaStream_t)stream_>>>(xs, n, h, w, c_out, y);
+    else if (c_in == 2) im2col3x3_kernel<2><<<blocks, 128, 0, (cudaStream_t)stream_>>>(xs, n, h, w, c_out, y);
+    else im2col3x3_kernel<1><<<blocks, 128, 0, (cudaStream_t)stream_>>>(xs, n, h, w, c_out, y);
     B2C_CUDA(cudaGetLastError());
     return B2C_OK;
 }

@@ -256,6 +256,16 @@ def test_avgpool_pad_bias(ctx):
     xp = torch.full((7, 5, 5, 16), float("nan"), dtype=torch.bfloat16, device="cuda")
     ctx.pad_channels(7 * 25, 3, 16, dev_bf16(x), xp)
     assert np.array_equal(host(xp)[..., :3], x) and np.all(host(xp)[..., 3:] == 0)
+    # patch matrix of the 3x3 / pad 1 window: column (r*3+s)*3 + ch holds x[h+r-1, w+s-1, ch]
+    xc = torch.full((7, 5, 5, 32), float("nan"), dtype=torch.bfloat16, device="cuda")
+    ctx.im2col_3x3(7, 5, 5, 3, 32, dev_bf16(x), xc)
+    xpad = np.zeros((7, 7, 7, 3), np.float32)
+    xpad[:, 1:6, 1:6, :] = x
+    ref = np.zeros((7, 5, 5, 32), np.float32)
+    for rr in range(3):
+        for ss in range(3):
+            ref[..., (rr * 3 + ss) * 3:(rr * 3 + ss) * 3 + 3] = xpad[:, rr:rr + 5, ss:ss + 5, :]
+    assert np.array_equal(host(xc), ref)
     dz = wl.to_bf16_grid(r.standard_normal((130, 128)))
     db = torch.ones(100, device="cuda")
     ctx.bias_grad(130, 100, 128, dev_bf16(dz), db, True)
