@@ -26,6 +26,10 @@ b2c_status b2c_create(b2c_ctx** out, int device)
     ctx->sm_count = prop.multiProcessorCount;
     ctx->spin_limit = 1u << 22;
     ctx->stall_counters = nullptr;
+    {
+        const char* env = std::getenv("B2C_CTA_PAIRS");
+        ctx->use_pairs = (env && env[0] == '1') ? 1 : 0;
+    }
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || fn == nullptr ||

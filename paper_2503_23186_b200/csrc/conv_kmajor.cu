@@ -42,6 +42,7 @@ struct alignas(64) ConvKParams {
     int a_bytes, b_bytes;            // shared-memory footprint of the A tile / one B tile (multiples of 1 KB)
     int tx_a, tx_b;                  // bytes one A / B load delivers
     int a_step;                      // byte offset of one image row inside the A tile (vreuse)
+    int pair;                        // CTA pairs (cta_group::2): M = 256 per MMA, each CTA holds half of every B tile
     int resident;                    // filter bank of this CTA's channel tile stays in shared memory
     int resident_bytes;
     int n_valid, oc_valid;           // images / output channels that exist
@@ -78,6 +79,21 @@ __device__ __forceinline__ UnitCoord decode_unit(const ConvKParams& p, int u)
     c.par = u / p.tiles_n;
     return c;
 }
+// Units of this CTA: plain kernels walk units blockIdx.x, +gridDim.x, ...; CTA pairs walk pair-units (two pixel tiles
+// next to each other, same channel tile) and CTA `rank` of the pair takes tile 2*m + rank.
+struct UnitWalk {
+    int first, stride, count, rank, pair;
+    __device__ UnitWalk(const ConvKParams& p, int rank_) : rank(rank_), pair(p.pair)
+    {
+        first = pair ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+        stride = pair ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+        count = pair ? p.total_units >> 1 : p.total_units;
+    }
+    __device__ int unit(const ConvKParams& p, int pu) const
+    {
+        return pair ? (2 * (pu / p.n_ktiles) + rank) * p.n_ktiles + pu % p.n_ktiles : pu;
+    }
+};
 __device__ __forceinline__ int unit_iters(const ConvKParams& p, int par)
 {
     const int taps = p.taps[par].count;
@@ -110,8 +126,12 @@ __device__ __forceinline__ void butterfly16(float (&a)[16], float (&b)[16], int 
 // are reduced over rows per unit into a per-warp shared-memory array.
 template <int NCH>
 __device__ __forceinline__ void epilogue_loop(const ConvKParams& p, uint32_t tmem_base, uint64_t* acc_full, uint64_t* acc_empty,
-                                              uint32_t* abort_flag, float* my_stats, int e, int lane)
+                                              uint32_t* abort_flag, float* my_stats, int e, int lane, int rank)
 {
+    const UnitWalk walk(p, rank);
+    // the accumulator-free barrier lives in the leader CTA of a pair: the peer's warps arrive on it remotely
+    const uint32_t remote_empty0 = (p.pair && rank != 0) ? map_to_cta(smem_u32(&acc_empty[0]), 0) : 0u;
+    const uint32_t remote_empty1 = (p.pair && rank != 0) ? map_to_cta(smem_u32(&acc_empty[1]), 0) : 0u;
     const int q = (e + 2) & 3;       // TMEM lane quarter this warp may read: (warp index in the CTA) % 4, epilogue warps start at 2
     const int m = q * 32 + lane;     // accumulator row = pixel of the tile (w fastest, then h, then image)
     const int lw = m % p.bw, lh = (m / p.bw) % p.bh, ln = m / (p.bw * p.bh);
@@ -166,8 +186,8 @@ __device__ __forceinline__ void epilogue_loop(const ConvKParams& p, uint32_t tme
         }
     };
 
-    for (int u = (int)blockIdx.x; u < p.total_units; u += (int)gridDim.x) {
-        const UnitCoord c = decode_unit(p, u);
+    for (int pu = walk.first; pu < walk.count; pu += walk.stride) {
+        const UnitCoord c = decode_unit(p, walk.unit(p, pu));
         const int n_it = unit_iters(p, c.par);
         const bool row_valid = (c.n0 + ln) < p.n_valid;
         const long long row_off = (long long)(c.n0 + ln) * p.os_n + (long long)(c.oh0 + lh) * p.os_h + (long long)(c.ow0 + lw) * p.os_w + p.off[c.par];
@@ -199,7 +219,10 @@ __device__ __forceinline__ void epilogue_loop(const ConvKParams& p, uint32_t tme
             if (n_it > 0) {
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&acc_empty[buf]);
+                if (lane == 0) {
+                    if (remote_empty0 != 0u) mbar_arrive_cluster(buf ? remote_empty1 : remote_empty0);
+                    else mbar_arrive(&acc_empty[buf]);
+                }
             }
         };
         // bias, rounding and stores of one 16-column chunk; returns the values as stored in pk
@@ -321,7 +344,7 @@ __device__ __forceinline__ void epilogue_loop(const ConvKParams& p, uint32_t tme
 // the issuing thread spends a handful of independent instructions per MMA (its own dependent-issue latency, not the
 // tensor pipe, bounds small-N tiles otherwise).  Descriptor low words advance by 32 bytes per k-step inside the
 // swizzle atom and by a_step / b_step per sub-tile.
-template <int KS, int NB>
+template <int KS, int NB, bool PAIR>
 __device__ __forceinline__ void issue_stage(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc,
                                             uint32_t a_step16, uint32_t b_step16, uint32_t accumulate_first)
 {
@@ -331,13 +354,16 @@ __device__ __forceinline__ void issue_stage(uint32_t d_tmem, uint32_t a_lo, uint
         for (int k = 0; k < KS; ++k) {
             const uint64_t ad = ((uint64_t)desc_hi << 32) | (uint64_t)(a_lo + (uint32_t)j * a_step16 + 2u * k);
             const uint64_t bd = ((uint64_t)desc_hi << 32) | (uint64_t)(b_lo + (uint32_t)j * b_step16 + 2u * k);
-            umma_bf16(d_tmem, ad, bd, idesc, (j == 0 && k == 0) ? accumulate_first : 1u);
+            if constexpr (PAIR) umma_bf16_pair(d_tmem, ad, bd, idesc, (j == 0 && k == 0) ? accumulate_first : 1u);
+            else umma_bf16(d_tmem, ad, bd, idesc, (j == 0 && k == 0) ? accumulate_first : 1u);
         }
     }
 }
 
+template <bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_constant__ ConvKParams p)
 {
+    const int rank = PAIR ? (int)cluster_ctarank() : 0;   // 0 = leader of the pair: issues the MMAs, owns the barriers the pair shares
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], acc_full[2], acc_empty[2], w_bar, drain_bar;
     __shared__ uint32_t tmem_slot;
@@ -357,7 +383,7 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(&acc_full[b], 1);
-            mbar_init(&acc_empty[b], kEpiWarps);   // one arrival per epilogue warp
+            mbar_init(&acc_empty[b], PAIR ? 2 * kEpiWarps : kEpiWarps);   // one arrival per epilogue warp (of both CTAs of a pair)
         }
         mbar_init(&w_bar, 1);
         mbar_init(&drain_bar, 1);
@@ -365,14 +391,21 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
         fence_mbar_init();
     }
     if (warp == 1) {
-        tmem_alloc(&tmem_slot, (uint32_t)p.tmem_cols);
-        tmem_relinquish();
+        if constexpr (PAIR) {
+            tmem_alloc_pair(&tmem_slot, (uint32_t)p.tmem_cols);
+            tmem_relinquish_pair();
+        } else {
+            tmem_alloc(&tmem_slot, (uint32_t)p.tmem_cols);
+            tmem_relinquish();
+        }
     }
     tc_fence_before();
     __syncthreads();
+    if constexpr (PAIR) cluster_sync_all();   // the peer's barriers exist before anything arrives on them
     tc_fence_after();
     const uint32_t tmem_base = tmem_slot;
     const long long t_start = clock64();
+    const UnitWalk walk(p, rank);
     int issued = 0;  // producer lane: stages whose loads were issued
 
     if (warp == 0) {
@@ -380,18 +413,24 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
             // ------------------------------------------------------------ TMA producer
             prefetch_tensormap(&p.tmB);
             prefetch_tensormap(&p.tmA[0]);
+            // a pair counts the bytes of both CTAs on the leader's barriers; b_row = first filter row this CTA fetches
+            const int b_rows = PAIR ? p.n_tile >> 1 : p.n_tile;
+            const uint32_t w_bar_cl = PAIR ? map_to_cta(smem_u32(&w_bar), 0) : 0u;
             if (p.resident) {
-                const int ktile = (int)blockIdx.x % p.n_ktiles;   // the grid is a multiple of n_ktiles: fixed per CTA
+                const int ktile = walk.first % p.n_ktiles;   // the walk stride is a multiple of n_ktiles: fixed per CTA
                 const TapList& tl = p.taps[0];
-                mbar_expect_tx(&w_bar, (uint32_t)(tl.count * p.c_blocks * p.tx_b));
+                if (rank == 0) mbar_expect_tx(&w_bar, (uint32_t)((PAIR ? 2 : 1) * tl.count * p.c_blocks * p.tx_b));
                 for (int t = 0; t < tl.count; ++t)
-                    for (int cb = 0; cb < p.c_blocks; ++cb)
-                        tma_load_3d(smem + (size_t)(t * p.c_blocks + cb) * p.b_bytes, &p.tmB, &w_bar, cb * p.kb, tl.rs[t], ktile * p.n_tile);
+                    for (int cb = 0; cb < p.c_blocks; ++cb) {
+                        uint8_t* dst = smem + (size_t)(t * p.c_blocks + cb) * p.b_bytes;
+                        if constexpr (PAIR) tma_load_3d_pair(dst, &p.tmB, w_bar_cl, cb * p.kb, tl.rs[t], ktile * p.n_tile + rank * b_rows);
+                        else tma_load_3d(dst, &p.tmB, &w_bar, cb * p.kb, tl.rs[t], ktile * p.n_tile);
+                    }
             }
             bool ok = true;
             long long waited = 0;
-            for (int u = (int)blockIdx.x; ok && u < p.total_units; u += (int)gridDim.x) {
-                const UnitCoord c = decode_unit(p, u);
+            for (int pu = walk.first; ok && pu < walk.count; pu += walk.stride) {
+                const UnitCoord c = decode_unit(p, walk.unit(p, pu));
                 const TapList& tl = p.taps[c.par];
                 const int n_it = unit_iters(p, c.par);
                 for (int it = 0; it < n_it; ++it, ++issued) {
@@ -406,25 +445,37 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
                     waited += clock64() - w0;
                     const int t0 = it / p.c_blocks, cb = it - t0 * p.c_blocks;   // tap (or horizontal shift) and channel block
                     uint8_t* a_dst = ring + (size_t)s * stage_bytes;
-                    mbar_expect_tx(&full_bar[s], (uint32_t)(p.tx_a + (p.resident ? 0 : p.nb * p.tx_b)));
+                    const uint32_t stage_tx = (uint32_t)(p.tx_a + (p.resident ? 0 : p.nb * p.tx_b));
                     // with vreuse the table entry of vertical tap 0 carries the shift of the whole haloed tile
-                    tma_load_4d(a_dst, &p.tmA[tl.map[t0]], &full_bar[s], cb * p.kb, c.ow0 + tl.dw[t0], c.oh0 + tl.dh[t0], c.n0);
-                    if (!p.resident) {
-                        for (int j = 0; j < p.nb; ++j)
-                            tma_load_3d(a_dst + p.a_bytes + (size_t)j * p.b_bytes, &p.tmB, &full_bar[s], cb * p.kb, tl.rs[t0 + 3 * j],
-                                        c.ktile * p.n_tile);
+                    if constexpr (PAIR) {
+                        const uint32_t full_cl = map_to_cta(smem_u32(&full_bar[s]), 0);
+                        if (rank == 0) mbar_expect_tx(&full_bar[s], 2u * stage_tx);
+                        tma_load_4d_pair(a_dst, &p.tmA[tl.map[t0]], full_cl, cb * p.kb, c.ow0 + tl.dw[t0], c.oh0 + tl.dh[t0], c.n0);
+                        if (!p.resident) {
+                            for (int j = 0; j < p.nb; ++j)
+                                tma_load_3d_pair(a_dst + p.a_bytes + (size_t)j * p.b_bytes, &p.tmB, full_cl, cb * p.kb, tl.rs[t0 + 3 * j],
+                                                 c.ktile * p.n_tile + rank * b_rows);
+                        }
+                    } else {
+                        mbar_expect_tx(&full_bar[s], stage_tx);
+                        tma_load_4d(a_dst, &p.tmA[tl.map[t0]], &full_bar[s], cb * p.kb, c.ow0 + tl.dw[t0], c.oh0 + tl.dh[t0], c.n0);
+                        if (!p.resident) {
+                            for (int j = 0; j < p.nb; ++j)
+                                tma_load_3d(a_dst + p.a_bytes + (size_t)j * p.b_bytes, &p.tmB, &full_bar[s], cb * p.kb, tl.rs[t0 + 3 * j],
+                                            c.ktile * p.n_tile);
+                        }
                     }
                 }
             }
-            if (p.stall != nullptr) {
+            if (p.stall != nullptr && rank == 0) {
                 atomicAdd(p.stall + 0, (unsigned long long)waited);
                 atomicAdd(p.stall + 4, (unsigned long long)(clock64() - t_start));
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            // ------------------------------------------------------------ MMA issuer
-            const uint32_t idesc = make_idesc_bf16(128, p.n_tile, false, false);
+        if (lane == 0 && rank == 0) {
+            // ------------------------------------------------------------ MMA issuer (the leader CTA of a pair)
+            const uint32_t idesc = make_idesc_bf16(PAIR ? 256 : 128, p.n_tile, false, false);
             const uint32_t sbo = 8u * (uint32_t)p.kb * 2u;  // eight rows of kb bf16
             const int ksteps = p.kb >> 4;
             const uint64_t desc_proto = make_smem_desc(0u, 16u, sbo, (uint32_t)p.swz);
@@ -440,8 +491,8 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
             }
             int consumed = 0, jacc = 0;
             long long wait_ring = 0, wait_acc = 0;
-            for (int u = (int)blockIdx.x; ok && u < p.total_units; u += (int)gridDim.x) {
-                const UnitCoord c = decode_unit(p, u);
+            for (int pu = walk.first; ok && pu < walk.count; pu += walk.stride) {
+                const UnitCoord c = decode_unit(p, walk.unit(p, pu));
                 const int n_it = unit_iters(p, c.par);
                 if (n_it == 0) continue;
                 const int buf = jacc & 1;
@@ -476,19 +527,22 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
                     }
                     const uint32_t acc0 = it != 0 ? 1u : 0u;
                     if (p.nb == 3) {
-                        if (ksteps == 4) issue_stage<4, 3>(d_tmem, a_lo, b_lo, desc_hi, idesc, a_step16, b_step16, acc0);
-                        else if (ksteps == 2) issue_stage<2, 3>(d_tmem, a_lo, b_lo, desc_hi, idesc, a_step16, b_step16, acc0);
-                        else issue_stage<1, 3>(d_tmem, a_lo, b_lo, desc_hi, idesc, a_step16, b_step16, acc0);
+                        if (ksteps == 4) issue_stage<4, 3, PAIR>(d_tmem, a_lo, b_lo, desc_hi, idesc, a_step16, b_step16, acc0);
+                        else if (ksteps == 2) issue_stage<2, 3, PAIR>(d_tmem, a_lo, b_lo, desc_hi, idesc, a_step16, b_step16, acc0);
+                        else issue_stage<1, 3, PAIR>(d_tmem, a_lo, b_lo, desc_hi, idesc, a_step16, b_step16, acc0);
                     } else {
-                        if (ksteps == 4) issue_stage<4, 1>(d_tmem, a_lo, b_lo, desc_hi, idesc, a_step16, b_step16, acc0);
-                        else if (ksteps == 2) issue_stage<2, 1>(d_tmem, a_lo, b_lo, desc_hi, idesc, a_step16, b_step16, acc0);
-                        else issue_stage<1, 1>(d_tmem, a_lo, b_lo, desc_hi, idesc, a_step16, b_step16, acc0);
+                        if (ksteps == 4) issue_stage<4, 1, PAIR>(d_tmem, a_lo, b_lo, desc_hi, idesc, a_step16, b_step16, acc0);
+                        else if (ksteps == 2) issue_stage<2, 1, PAIR>(d_tmem, a_lo, b_lo, desc_hi, idesc, a_step16, b_step16, acc0);
+                        else issue_stage<1, 1, PAIR>(d_tmem, a_lo, b_lo, desc_hi, idesc, a_step16, b_step16, acc0);
                     }
                     if (++cur_cb == p.c_blocks) { cur_cb = 0; ++cur_t0; }
-                    umma_commit(&empty_bar[s]);  // frees the stage once these MMAs have read it
+                    // frees the stage (in both CTAs of a pair) once these MMAs have read it
+                    if constexpr (PAIR) umma_commit_pair(&empty_bar[s], (uint16_t)3);
+                    else umma_commit(&empty_bar[s]);
                 }
                 if (!ok) break;
-                umma_commit(&acc_full[buf]);
+                if constexpr (PAIR) umma_commit_pair(&acc_full[buf], (uint16_t)3);
+                else umma_commit(&acc_full[buf]);
                 ++jacc;
             }
             if (p.stall != nullptr) {
@@ -500,18 +554,20 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
         // ---------------------------------------------------------------- epilogue (8 warps)
         const int e = warp - 2;
         if (p.stats != nullptr && p.n_tile <= 32)
-            epilogue_loop<1>(p, tmem_base, acc_full, acc_empty, &abort_flag, s_stats[e], e, lane);
+            epilogue_loop<1>(p, tmem_base, acc_full, acc_empty, &abort_flag, s_stats[e], e, lane, rank);
         else if (p.stats != nullptr && p.n_tile <= 64)
-            epilogue_loop<2>(p, tmem_base, acc_full, acc_empty, &abort_flag, s_stats[e], e, lane);
+            epilogue_loop<2>(p, tmem_base, acc_full, acc_empty, &abort_flag, s_stats[e], e, lane, rank);
         else
-            epilogue_loop<0>(p, tmem_base, acc_full, acc_empty, &abort_flag, s_stats[e], e, lane);
+            epilogue_loop<0>(p, tmem_base, acc_full, acc_empty, &abort_flag, s_stats[e], e, lane, rank);
     }
     tc_fence_before();
     __syncthreads();
+    if constexpr (PAIR) cluster_sync_all();   // both CTAs have left their loops: nothing new will be issued
     if (abort_flag) {
         // A wait gave up.  Before the CTA may exit, let every bulk copy it issued land and every
         // MMA it issued retire (both finish on their own; the polls here only bound the wait).
-        if (warp == 0 && lane == 0) {
+        // In a pair the leader's barriers count the peer's copies too.
+        if (warp == 0 && lane == 0 && rank == 0) {
             if (p.resident)
                 for (uint32_t i = 0; i < kDrainPolls && !mbar_try_wait(&w_bar, 0u); ++i) {}
             for (int back = 0; back < S && back < issued; ++back) {
@@ -519,15 +575,18 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
                 for (uint32_t i = 0; i < kDrainPolls && !mbar_try_wait(&full_bar[it % S], (uint32_t)(it / S) & 1u); ++i) {}
             }
         }
-        if (warp == 1 && lane == 0) {
-            umma_commit(&drain_bar);
+        if (warp == 1 && lane == 0 && rank == 0) {
+            if constexpr (PAIR) umma_commit_pair(&drain_bar, (uint16_t)1);
+            else umma_commit(&drain_bar);
             for (uint32_t i = 0; i < kDrainPolls && !mbar_try_wait(&drain_bar, 0u); ++i) {}
         }
         __syncthreads();
     }
+    if constexpr (PAIR) cluster_sync_all();   // the peer must not exit while the leader still drains copies into it
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
+        if constexpr (PAIR) tmem_dealloc_pair(tmem_base, (uint32_t)p.tmem_cols);
+        else tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
     }
 }
 
@@ -614,11 +673,22 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
     while (p.tmem_cols < 2 * p.acc_cols) p.tmem_cols *= 2;
     p.total_units = n_par * p.tiles_n * p.tiles_h * p.tiles_w * p.n_ktiles;
 
-    // launch shape: one persistent CTA per SM; a multiple of n_ktiles so that a CTA keeps its channel tile
-    int grid = ctx->sm_count < p.total_units ? ctx->sm_count : p.total_units;
-    grid -= grid % p.n_ktiles;
-    if (grid < p.n_ktiles) grid = p.n_ktiles;
-    const int units_per_cta = (p.total_units + grid - 1) / grid;
+    // CTA pairs (cta_group::2): two neighbouring pixel tiles share every filter tile, each CTA holding half of its
+    // rows, which halves the shared-memory operand traffic per MMA.  Needs an even number of pixel tiles and a channel
+    // tile that splits into two multiples of 16; the fp32 / bias / multi-parity cases stay on single CTAs.
+    const int m_tiles = p.tiles_n * p.tiles_h * p.tiles_w;
+    p.pair = (ctx->use_pairs && n_par == 1 && !pb.out_f32 && pb.bias == nullptr && n_tile % 32 == 0 && m_tiles % 2 == 0 && ctx->sm_count >= 2) ? 1 : 0;
+    const int b_rows = p.pair ? n_tile / 2 : n_tile;   // filter rows one CTA fetches per tile
+
+    // launch shape: one persistent CTA per SM; the unit walk stride (CTAs, or pairs) is a multiple of n_ktiles so that a
+    // CTA keeps its channel tile
+    const int walkers_max = p.pair ? ctx->sm_count / 2 : ctx->sm_count;
+    const int walk_units = p.pair ? p.total_units / 2 : p.total_units;
+    int walkers = walkers_max < walk_units ? walkers_max : walk_units;
+    walkers -= walkers % p.n_ktiles;
+    if (walkers < p.n_ktiles) walkers = p.n_ktiles;
+    const int grid = p.pair ? 2 * walkers : walkers;
+    const int units_per_cta = (walk_units + walkers - 1) / walkers;
 
     // shared-memory plan.  Preference: haloed stages (vertical tap reuse) with 64-channel k-blocks, then with
     // 32-channel k-blocks (smaller stages, so that a ring of at least four still fits), else one tap per stage.
@@ -635,8 +705,8 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
         p.c_blocks = pb.ic / kb;
         p.swz = kb == 64 ? SWZ_128B : kb == 32 ? SWZ_64B : SWZ_32B;
         p.vreuse = vr;
-        p.b_bytes = ((n_tile * kb * 2) + 1023) & ~1023;
-        p.tx_b = n_tile * kb * 2;
+        p.b_bytes = ((b_rows * kb * 2) + 1023) & ~1023;
+        p.tx_b = b_rows * kb * 2;
         const int a_rows = vr ? (p.bh + 2) * p.bw : 128;
         p.tx_a = a_rows * kb * 2;
         p.a_bytes = (p.tx_a + 1023) & ~1023;
@@ -668,7 +738,7 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
     {
         cuuint64_t dims[3] = {(cuuint64_t)pb.ic, (cuuint64_t)(R * R), (cuuint64_t)pb.oc};
         cuuint64_t str[2] = {(cuuint64_t)pb.ic * 2, (cuuint64_t)R * R * pb.ic * 2};
-        cuuint32_t box[3] = {(cuuint32_t)p.kb, 1u, (cuuint32_t)n_tile};
+        cuuint32_t box[3] = {(cuuint32_t)p.kb, 1u, (cuuint32_t)b_rows};
         if (!encode_map(ctx, &p.tmB, pb.wt, 3, dims, str, box, p.kb * 2)) return B2C_ERR_CUDA;
     }
 
@@ -715,10 +785,27 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
     p.stall = ctx->stall_counters;
 
     if (!attr_set) {
-        B2C_CUDA(cudaFuncSetAttribute(conv_kmajor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 212 * 1024));
+        B2C_CUDA(cudaFuncSetAttribute(conv_kmajor_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 212 * 1024));
+        B2C_CUDA(cudaFuncSetAttribute(conv_kmajor_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 212 * 1024));
         attr_set = true;
     }
-    conv_kmajor_kernel<<<grid, kThreads, smem_bytes, stream>>>(p);
+    if (p.pair) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)grid);
+        cfg.blockDim = dim3(kThreads);
+        cfg.dynamicSmemBytes = smem_bytes;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        B2C_CUDA(cudaLaunchKernelEx(&cfg, conv_kmajor_kernel<true>, p));
+    } else {
+        conv_kmajor_kernel<false><<<grid, kThreads, smem_bytes, stream>>>(p);
+    }
     B2C_CUDA(cudaGetLastError());
     return B2C_OK;
 }
