@@ -677,7 +677,11 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
     // rows, which halves the shared-memory operand traffic per MMA.  Needs an even number of pixel tiles and a channel
     // tile that splits into two multiples of 16; the fp32 / bias / multi-parity cases stay on single CTAs.
     const int m_tiles = p.tiles_n * p.tiles_h * p.tiles_w;
-    p.pair = (ctx->use_pairs && n_par == 1 && !pb.out_f32 && pb.bias == nullptr && n_tile % 32 == 0 && m_tiles % 2 == 0 && ctx->sm_count >= 2) ? 1 : 0;
+    // Measured on B200 (1024-image layers, isolated launches): pairs gain ~20 % at 128-channel tiles and lose ~10 % at 64
+    // and 256; inside the whole step the gain disappears, so pairs are off by default (use_pairs: 1 = 128-channel tiles
+    // only, 2 = every eligible problem).
+    const bool pair_ok = n_par == 1 && !pb.out_f32 && pb.bias == nullptr && n_tile % 32 == 0 && m_tiles % 2 == 0 && ctx->sm_count >= 2;
+    p.pair = (pair_ok && (ctx->use_pairs == 2 || (ctx->use_pairs == 1 && n_tile == 128))) ? 1 : 0;
     const int b_rows = p.pair ? n_tile / 2 : n_tile;   // filter rows one CTA fetches per tile
 
     // launch shape: one persistent CTA per SM; the unit walk stride (CTAs, or pairs) is a multiple of n_ktiles so that a

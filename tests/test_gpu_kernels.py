@@ -341,3 +341,30 @@ def test_bounded_wait_reports_timeout(ctx):
     ctx.conv2d_fwd(_desc(*shape), dev_bf16(x), dev_bf16(w), y)
     assert ctx.device_status() == 0
     assert_close(y, oracle.conv2d_fwd(x, w, 1, 1), "y after recovery")
+
+
+@pytest.mark.parametrize("mode", ["0", "2"])
+def test_conv_cta_pairs_forced_on_and_off(mode, monkeypatch):
+    """The forward / data-gradient kernel on single CTAs only (0) and on CTA pairs wherever possible (2): same results."""
+    from paper_2503_23186_b200 import binding
+    monkeypatch.setenv("B2C_CTA_PAIRS", mode)
+    c = binding.Context(0)
+    try:
+        for shape in [(8, 32, 32, 64, 64, 3, 1), (4, 16, 16, 128, 256, 3, 1), (4, 16, 16, 256, 128, 3, 1), (8, 32, 32, 64, 128, 3, 2),
+                      (2, 16, 16, 160, 160, 3, 1), (6, 4, 4, 128, 64, 3, 1)]:
+            N, H, W, C, K, R, st = shape
+            x, w, g = wl.conv_problem(11, *shape)
+            ref = oracle.conv2d_fwd(x, w, st, (R - 1) // 2)
+            y = torch.full(ref.shape, float("nan"), dtype=torch.bfloat16, device="cuda")
+            stats = torch.zeros(2 * K, dtype=torch.float64, device="cuda")
+            c.conv2d_fwd(_desc(*shape), dev_bf16(x), dev_bf16(w), y, ch_stats=stats)
+            assert c.device_status() == 0
+            assert_close(y, ref, f"y {shape} pairs={mode}")
+            ys = host(y).reshape(-1, K)
+            np.testing.assert_allclose(host(stats)[:K], ys.sum(0), rtol=1e-5, atol=1e-3 * np.sqrt(ys.shape[0]))
+            dx = torch.full(x.shape, float("nan"), dtype=torch.bfloat16, device="cuda")
+            c.conv2d_dgrad(_desc(*shape), dev_bf16(g), _dgrad_weights(c, w), dx)
+            assert c.device_status() == 0
+            assert_close(dx, oracle.conv2d_dgrad(g, w, x.shape, st, (R - 1) // 2), f"dx {shape} pairs={mode}")
+    finally:
+        c.close()
