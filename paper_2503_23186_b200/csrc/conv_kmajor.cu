@@ -18,8 +18,10 @@
 //     offsets of one image row (a multiple of the swizzle period), so the input is fetched three
 //     times instead of nine.
 //   * Small filter banks stay resident in shared memory for the whole launch.
-// Warp roles: warp 0 = TMA producer (one lane), warp 1 = TMEM owner + MMA issuer (one lane),
-// warps 2..9 = epilogue (two per TMEM lane quarter, splitting the columns).  Every mbarrier wait is bounded.
+// Warp roles: warp 0 = first TMA producer (one lane), warp 1 = TMEM owner + first MMA issuer (one lane),
+// warps 2..9 = epilogue (two per TMEM lane quarter, splitting the columns), warp 10 = second MMA issuer (one lane;
+// the two issuers take alternate units), warp 11 = second TMA producer (one lane; the two producers take alternate
+// stages).  Every mbarrier wait is bounded.
 #include "common.h"
 #include "ptx.cuh"
 
@@ -39,9 +41,12 @@ struct alignas(64) ConvKParams {
     int tmem_cols, acc_cols;         // allocation, columns per accumulator
     int vreuse;                      // a stage serves the three vertical taps of one horizontal shift
     int nb;                          // B tiles per stage (1, or 3 with vreuse)
+    int b_merged;                    // the three B tiles of a stage come with one load (box of three filter rows)
+    int r_filter;                    // filter height = width
     int a_bytes, b_bytes;            // shared-memory footprint of the A tile / one B tile (multiples of 1 KB)
     int tx_a, tx_b;                  // bytes one A / B load delivers
     int a_step;                      // byte offset of one image row inside the A tile (vreuse)
+    int issuers;                     // MMA-issuing threads at work (1 or 2)
     int pair;                        // CTA pairs (cta_group::2): M = 256 per MMA, each CTA holds half of every B tile
     int resident;                    // filter bank of this CTA's channel tile stays in shared memory
     int resident_bytes;
@@ -60,7 +65,10 @@ struct alignas(64) ConvKParams {
 
 static constexpr int kMaxStages = 8;
 static constexpr int kEpiWarps = 8;
-static constexpr int kThreads = 64 + 32 * kEpiWarps;
+static constexpr int kIssuers = 2;       // MMA-issuing threads: warp 1 and the warps after the epilogue warps
+static constexpr int kProducers = 2;     // TMA-issuing threads: warp 0 and the warp after the issuer warps; they take alternate stages
+static constexpr int kThreads = 64 + 32 * kEpiWarps + 32 * (kIssuers - 1) + 32 * (kProducers - 1);
+static constexpr int kProducerWarp1 = 2 + kEpiWarps + (kIssuers - 1);   // warp index of the second producer
 static constexpr uint32_t kDrainPolls = 1u << 22;
 
 struct UnitCoord {
@@ -195,7 +203,8 @@ __device__ __forceinline__ void epilogue_loop(const ConvKParams& p, uint32_t tme
         if (n_it > 0) {
             buf = jacc & 1;
             const long long w3 = clock64();
-            ok = mbar_wait_bounded(&acc_full[buf], (uint32_t)(jacc >> 1) & 1u, p.spin_limit, abort_flag);
+            ok = true;
+            if (lane == 0) ok = mbar_wait_bounded(&acc_full[buf], (uint32_t)(jacc >> 1) & 1u, p.spin_limit, abort_flag);   // one poller per warp
             epi_wait += clock64() - w3;
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) {
@@ -360,6 +369,104 @@ __device__ __forceinline__ void issue_stage(uint32_t d_tmem, uint32_t a_lo, uint
     }
 }
 
+// One MMA-issuing thread.  The CTA runs kIssuers of them (in different warps): issuer `my` accumulates the CTA's units
+// my, my + kIssuers, ... (unit j always into accumulator j & 1) and steps over the ring stages of the others.  A single
+// thread cannot keep the tensor pipe busy on narrow tiles: it pays roughly 45 cycles per tcgen05.mma, 180 per barrier
+// wait and 55 per commit, all serial, against 48-64 cycles the pipe needs per MMA at N <= 128; two threads working on
+// different accumulators can.
+template <int KS, int NB, bool PAIR>
+__device__ __forceinline__ void mma_issuer(const ConvKParams& p, const UnitWalk& walk, int my, uint32_t tmem_base, uint32_t smem_addr,
+                                           uint32_t ring_addr, int stage_bytes, uint64_t* full_bar, uint64_t* empty_bar, uint64_t* acc_full,
+                                           uint64_t* acc_empty, uint64_t* w_bar, uint32_t* abort_flag, const int* slot_stage)
+{
+    const uint32_t idesc = make_idesc_bf16(PAIR ? 256 : 128, p.n_tile, false, false);
+    const uint32_t sbo = 8u * (uint32_t)p.kb * 2u;  // eight rows of kb bf16
+    const uint64_t desc_proto = make_smem_desc(0u, 16u, sbo, (uint32_t)p.swz);
+    const uint32_t desc_hi = (uint32_t)(desc_proto >> 32), desc_lo_base = (uint32_t)desc_proto;
+    const uint32_t a_to_b16 = (uint32_t)p.a_bytes >> 4, a_step16 = (uint32_t)p.a_step >> 4;
+    // B tiles of consecutive vertical taps are adjacent, in a stage and in the resident bank alike
+    const uint32_t b_step16 = (uint32_t)p.b_bytes >> 4;
+    const uint32_t b_cb16 = (uint32_t)(p.nb * p.b_bytes) >> 4, stage16 = (uint32_t)stage_bytes >> 4;
+    const uint32_t ring_lo = desc_lo_base + (ring_addr >> 4), bank_lo = desc_lo_base + (smem_addr >> 4);
+    const int S = p.stages;
+    const bool timed = p.stall != nullptr;
+    const int units_per_par = p.n_par > 1 ? p.total_units / p.n_par : 1;
+    const int n_it_fixed = unit_iters(p, 0);
+    bool ok = true;
+    if (p.resident && !mbar_wait_bounded(w_bar, 0u, p.spin_limit, abort_flag)) {
+        atomicOr(p.status, B2C_DEV_TIMEOUT);
+        ok = false;
+    }
+    int s = 0, j = 0, i_stage = 0;   // ring slot and index of the next stage in CTA order, count of units that have stages
+    uint32_t ph = 0;
+    long long wait_ring = 0, wait_acc = 0;
+    for (int pu = walk.first; ok && pu < walk.count; pu += walk.stride) {
+        int n_it = n_it_fixed;
+        if (p.n_par > 1) n_it = unit_iters(p, walk.unit(p, pu) / units_per_par);
+        if (n_it == 0) continue;   // a parity without taps: the epilogue stores zeros without an accumulator
+        if ((j % p.issuers) != my) {   // another issuer's unit: step over its stages
+            i_stage += n_it;
+            s += n_it;
+            while (s >= S) { s -= S; ph ^= 1u; }
+            ++j;
+            continue;
+        }
+        const int buf = j & 1;
+        const long long w1 = timed ? clock64() : 0;
+        if (!mbar_wait_bounded(&acc_empty[buf], ((uint32_t)(j >> 1) & 1u) ^ 1u, p.spin_limit, abort_flag)) {
+            atomicOr(p.status, B2C_DEV_TIMEOUT);
+            ok = false;
+            break;
+        }
+        if (timed) wait_acc += clock64() - w1;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * p.acc_cols);
+        uint32_t b_res = bank_lo;   // resident bank: B tile of (tap or horizontal shift, channel block), consecutive per stage
+        for (int it = 0; it < n_it; ++it) {
+            const long long w2 = timed ? clock64() : 0;
+            // A parity wait tells a barrier's phases apart only modulo two, and with two issuers this thread may reach a
+            // slot before the slot's previous stage (another issuer's) was even loaded.  A producer issues the load of
+            // stage i only after the previous stage in that slot was consumed, and then stamps the slot with i + 1:
+            // seeing the stamp pass i makes the parity wait unambiguous.
+            if (p.issuers > 1) {
+                uint32_t polls = 0;
+                while (ld_acquire_shared(&slot_stage[s]) <= i_stage) {
+                    if (++polls > p.spin_limit || *(volatile uint32_t*)abort_flag != 0u) {
+                        ok = false;
+                        break;
+                    }
+                }
+            }
+            if (!ok || !mbar_wait_bounded(&full_bar[s], ph, p.spin_limit, abort_flag)) {
+                *(volatile uint32_t*)abort_flag = 1u;
+                atomicOr(p.status, B2C_DEV_TIMEOUT);
+                ok = false;
+                break;
+            }
+            if (timed) wait_ring += clock64() - w2;
+            tc_fence_after();
+            // descriptors differ from stage to stage only in the 14-bit address field: add offsets to the low word
+            const uint32_t a_lo = ring_lo + (uint32_t)s * stage16;
+            const uint32_t b_lo = p.resident ? b_res : a_lo + a_to_b16;
+            issue_stage<KS, NB, PAIR>(d_tmem, a_lo, b_lo, desc_hi, idesc, a_step16, b_step16, it != 0 ? 1u : 0u);
+            b_res += b_cb16;
+            // frees the stage (in both CTAs of a pair) once these MMAs have read it
+            if constexpr (PAIR) umma_commit_pair(&empty_bar[s], (uint16_t)3);
+            else umma_commit(&empty_bar[s]);
+            ++i_stage;
+            if (++s == S) { s = 0; ph ^= 1u; }
+        }
+        if (!ok) break;
+        if constexpr (PAIR) umma_commit_pair(&acc_full[buf], (uint16_t)3);
+        else umma_commit(&acc_full[buf]);
+        ++j;
+    }
+    if (timed) {
+        atomicAdd(p.stall + 1, (unsigned long long)wait_ring);
+        atomicAdd(p.stall + 2, (unsigned long long)wait_acc);
+    }
+}
+
 template <bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_constant__ ConvKParams p)
 {
@@ -368,6 +475,7 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
     __shared__ uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], acc_full[2], acc_empty[2], w_bar, drain_bar;
     __shared__ uint32_t tmem_slot;
     __shared__ uint32_t abort_flag;
+    __shared__ int slot_stage[kMaxStages];   // per ring slot: 1 + index of the stage whose loads were issued into it last
     __shared__ float s_stats[kEpiWarps][256];   // per epilogue warp (128 columns at most): [0,128) sums, [128,256) sums of squares
 
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023u) & ~uintptr_t(1023));
@@ -386,8 +494,9 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
             mbar_init(&acc_empty[b], PAIR ? 2 * kEpiWarps : kEpiWarps);   // one arrival per epilogue warp (of both CTAs of a pair)
         }
         mbar_init(&w_bar, 1);
-        mbar_init(&drain_bar, 1);
+        mbar_init(&drain_bar, kIssuers);
         abort_flag = 0;
+        for (int i = 0; i < kMaxStages; ++i) slot_stage[i] = 0;
         fence_mbar_init();
     }
     if (warp == 1) {
@@ -406,148 +515,115 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
     const uint32_t tmem_base = tmem_slot;
     const long long t_start = clock64();
     const UnitWalk walk(p, rank);
-    int issued = 0;  // producer lane: stages whose loads were issued
+    int issued = 0, last_issued = -1;  // producer lanes: own stages whose loads were issued, index of the last one
 
-    if (warp == 0) {
+    if (warp == 0 || warp == kProducerWarp1) {
         if (lane == 0) {
-            // ------------------------------------------------------------ TMA producer
+            // ------------------------------------------------------------ TMA producers
+            // Producer w stages every kProducers-th stage of the CTA's sequence: the chain wait -> expect -> issue of one
+            // thread (several hundred cycles) would otherwise bound short stages.
+            const int w = warp == 0 ? 0 : 1;
             prefetch_tensormap(&p.tmB);
             prefetch_tensormap(&p.tmA[0]);
             // a pair counts the bytes of both CTAs on the leader's barriers; b_row = first filter row this CTA fetches
             const int b_rows = PAIR ? p.n_tile >> 1 : p.n_tile;
+            const int R = p.r_filter;
             const uint32_t w_bar_cl = PAIR ? map_to_cta(smem_u32(&w_bar), 0) : 0u;
-            if (p.resident) {
+            if (p.resident && w == 0) {
+                // bank order: [tap or horizontal shift][channel block][vertical tap]
                 const int ktile = walk.first % p.n_ktiles;   // the walk stride is a multiple of n_ktiles: fixed per CTA
                 const TapList& tl = p.taps[0];
+                const int oc0 = ktile * p.n_tile + rank * b_rows;
                 if (rank == 0) mbar_expect_tx(&w_bar, (uint32_t)((PAIR ? 2 : 1) * tl.count * p.c_blocks * p.tx_b));
-                for (int t = 0; t < tl.count; ++t)
+                const int groups = p.vreuse ? tl.count / 3 : tl.count;
+                for (int t = 0; t < groups; ++t)
                     for (int cb = 0; cb < p.c_blocks; ++cb) {
-                        uint8_t* dst = smem + (size_t)(t * p.c_blocks + cb) * p.b_bytes;
-                        if constexpr (PAIR) tma_load_3d_pair(dst, &p.tmB, w_bar_cl, cb * p.kb, tl.rs[t], ktile * p.n_tile + rank * b_rows);
-                        else tma_load_3d(dst, &p.tmB, &w_bar, cb * p.kb, tl.rs[t], ktile * p.n_tile);
+                        uint8_t* dst = smem + (size_t)(t * p.c_blocks + cb) * p.nb * p.b_bytes;
+                        const int n_loads = p.b_merged ? 1 : p.nb;
+                        for (int v = 0; v < n_loads; ++v) {
+                            const int rs = tl.rs[t + 3 * v];
+                            if constexpr (PAIR) tma_load_4d_pair(dst + (size_t)v * p.b_bytes, &p.tmB, w_bar_cl, cb * p.kb, rs % R, oc0, rs / R);
+                            else tma_load_4d(dst + (size_t)v * p.b_bytes, &p.tmB, &w_bar, cb * p.kb, rs % R, oc0, rs / R);
+                        }
                     }
             }
             bool ok = true;
             long long waited = 0;
+            const bool timed = p.stall != nullptr;
+            int i = w, i_base = 0;   // this producer's next stage and the first stage of the current unit, in CTA order
+            int s = w % S;
+            uint32_t ph = (uint32_t)(w / S) & 1u;
+            const uint32_t stage_tx = (uint32_t)(p.tx_a + (p.resident ? 0 : p.nb * p.tx_b));
+            const int n_b_loads = p.resident ? 0 : (p.b_merged ? 1 : p.nb);
             for (int pu = walk.first; ok && pu < walk.count; pu += walk.stride) {
-                const UnitCoord c = decode_unit(p, walk.unit(p, pu));
+                const int u = walk.unit(p, pu);
+                const int n_it = unit_iters(p, p.n_par > 1 ? u / (p.total_units / p.n_par) : 0);
+                if (i >= i_base + n_it) {   // no stage of this unit is mine
+                    i_base += n_it;
+                    continue;
+                }
+                const UnitCoord c = decode_unit(p, u);
                 const TapList& tl = p.taps[c.par];
-                const int n_it = unit_iters(p, c.par);
-                for (int it = 0; it < n_it; ++it, ++issued) {
-                    const int s = issued % S;
-                    const uint32_t ph = (uint32_t)(issued / S) & 1u;
-                    const long long w0 = clock64();
+                const int oc0 = c.ktile * p.n_tile + rank * b_rows;
+                for (; i < i_base + n_it; i += kProducers) {
+                    const int it = i - i_base;
+                    const long long w0 = timed ? clock64() : 0;
                     if (!mbar_wait_bounded(&empty_bar[s], ph ^ 1u, p.spin_limit, &abort_flag)) {
                         atomicOr(p.status, B2C_DEV_TIMEOUT);
                         ok = false;
                         break;
                     }
-                    waited += clock64() - w0;
+                    if (timed) waited += clock64() - w0;
                     const int t0 = it / p.c_blocks, cb = it - t0 * p.c_blocks;   // tap (or horizontal shift) and channel block
                     uint8_t* a_dst = ring + (size_t)s * stage_bytes;
-                    const uint32_t stage_tx = (uint32_t)(p.tx_a + (p.resident ? 0 : p.nb * p.tx_b));
                     // with vreuse the table entry of vertical tap 0 carries the shift of the whole haloed tile
                     if constexpr (PAIR) {
                         const uint32_t full_cl = map_to_cta(smem_u32(&full_bar[s]), 0);
                         if (rank == 0) mbar_expect_tx(&full_bar[s], 2u * stage_tx);
                         tma_load_4d_pair(a_dst, &p.tmA[tl.map[t0]], full_cl, cb * p.kb, c.ow0 + tl.dw[t0], c.oh0 + tl.dh[t0], c.n0);
-                        if (!p.resident) {
-                            for (int j = 0; j < p.nb; ++j)
-                                tma_load_3d_pair(a_dst + p.a_bytes + (size_t)j * p.b_bytes, &p.tmB, full_cl, cb * p.kb, tl.rs[t0 + 3 * j],
-                                                 c.ktile * p.n_tile + rank * b_rows);
+                        for (int v = 0; v < n_b_loads; ++v) {
+                            const int rs = tl.rs[t0 + 3 * v];
+                            tma_load_4d_pair(a_dst + p.a_bytes + (size_t)v * p.b_bytes, &p.tmB, full_cl, cb * p.kb, rs % R, oc0, rs / R);
                         }
                     } else {
                         mbar_expect_tx(&full_bar[s], stage_tx);
                         tma_load_4d(a_dst, &p.tmA[tl.map[t0]], &full_bar[s], cb * p.kb, c.ow0 + tl.dw[t0], c.oh0 + tl.dh[t0], c.n0);
-                        if (!p.resident) {
-                            for (int j = 0; j < p.nb; ++j)
-                                tma_load_3d(a_dst + p.a_bytes + (size_t)j * p.b_bytes, &p.tmB, &full_bar[s], cb * p.kb, tl.rs[t0 + 3 * j],
-                                            c.ktile * p.n_tile);
+                        for (int v = 0; v < n_b_loads; ++v) {
+                            const int rs = tl.rs[t0 + 3 * v];
+                            tma_load_4d(a_dst + p.a_bytes + (size_t)v * p.b_bytes, &p.tmB, &full_bar[s], cb * p.kb, rs % R, oc0, rs / R);
                         }
                     }
+                    ++issued;
+                    last_issued = i;
+                    if (p.issuers > 1) st_release_shared(&slot_stage[s], i + 1);   // lets the issuers tell this slot's phases apart
+                    s += kProducers;
+                    if (s >= S) { s -= S; ph ^= 1u; }
                 }
+                i_base += n_it;
             }
-            if (p.stall != nullptr && rank == 0) {
+            if (p.stall != nullptr && rank == 0 && w == 0) {
                 atomicAdd(p.stall + 0, (unsigned long long)waited);
                 atomicAdd(p.stall + 4, (unsigned long long)(clock64() - t_start));
             }
         }
-    } else if (warp == 1) {
+    } else if (warp == 1 || (warp >= 2 + kEpiWarps && warp < kProducerWarp1)) {
         if (lane == 0 && rank == 0) {
-            // ------------------------------------------------------------ MMA issuer (the leader CTA of a pair)
-            const uint32_t idesc = make_idesc_bf16(PAIR ? 256 : 128, p.n_tile, false, false);
-            const uint32_t sbo = 8u * (uint32_t)p.kb * 2u;  // eight rows of kb bf16
-            const int ksteps = p.kb >> 4;
-            const uint64_t desc_proto = make_smem_desc(0u, 16u, sbo, (uint32_t)p.swz);
-            const uint32_t desc_hi = (uint32_t)(desc_proto >> 32), desc_lo_base = (uint32_t)desc_proto;
+            // ------------------------------------------------------------ MMA issuers (in the leader CTA of a pair)
+            const int my = warp == 1 ? 0 : warp - (2 + kEpiWarps) + 1;
+            if (my < p.issuers) {
             const uint32_t smem_addr = smem_u32(smem), ring_addr = smem_u32(ring);
-            const uint32_t a_to_b16 = (uint32_t)p.a_bytes >> 4, a_step16 = (uint32_t)p.a_step >> 4;
-            // B tiles of consecutive vertical taps: adjacent in a stage, three table rows apart in the resident bank
-            const uint32_t b_step16 = (uint32_t)(p.resident ? 3 * p.c_blocks * p.b_bytes : p.b_bytes) >> 4;
-            bool ok = true;
-            if (p.resident && !mbar_wait_bounded(&w_bar, 0u, p.spin_limit, &abort_flag)) {
-                atomicOr(p.status, B2C_DEV_TIMEOUT);
-                ok = false;
+            const int ksteps = p.kb >> 4;
+#define B2C_ISSUER(KS, NB) mma_issuer<KS, NB, PAIR>(p, walk, my, tmem_base, smem_addr, ring_addr, stage_bytes, full_bar, empty_bar, acc_full, acc_empty, &w_bar, &abort_flag, slot_stage)
+            if (p.nb == 3) {
+                if (ksteps == 4) B2C_ISSUER(4, 3);
+                else if (ksteps == 2) B2C_ISSUER(2, 3);
+                else B2C_ISSUER(1, 3);
+            } else {
+                if (ksteps == 4) B2C_ISSUER(4, 1);
+                else if (ksteps == 2) B2C_ISSUER(2, 1);
+                else B2C_ISSUER(1, 1);
             }
-            int consumed = 0, jacc = 0;
-            long long wait_ring = 0, wait_acc = 0;
-            for (int pu = walk.first; ok && pu < walk.count; pu += walk.stride) {
-                const UnitCoord c = decode_unit(p, walk.unit(p, pu));
-                const int n_it = unit_iters(p, c.par);
-                if (n_it == 0) continue;
-                const int buf = jacc & 1;
-                const long long w1 = clock64();
-                if (!mbar_wait_bounded(&acc_empty[buf], ((uint32_t)(jacc >> 1) & 1u) ^ 1u, p.spin_limit, &abort_flag)) {
-                    atomicOr(p.status, B2C_DEV_TIMEOUT);
-                    ok = false;
-                    break;
-                }
-                wait_acc += clock64() - w1;
-                tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * p.acc_cols);
-                int cur_t0 = 0, cur_cb = 0;   // tap (or horizontal shift) and channel block of the stage
-                for (int it = 0; it < n_it; ++it, ++consumed) {
-                    const int s = consumed % S;
-                    const uint32_t ph = (uint32_t)(consumed / S) & 1u;
-                    const long long w2 = clock64();
-                    if (!mbar_wait_bounded(&full_bar[s], ph, p.spin_limit, &abort_flag)) {
-                        atomicOr(p.status, B2C_DEV_TIMEOUT);
-                        ok = false;
-                        break;
-                    }
-                    wait_ring += clock64() - w2;
-                    tc_fence_after();
-                    // descriptors differ from stage to stage only in the 14-bit address field: add offsets to the low word
-                    const uint32_t a_lo = desc_lo_base + ((ring_addr + (uint32_t)(s * stage_bytes)) >> 4);
-                    uint32_t b_lo;
-                    if (p.resident) {
-                        b_lo = desc_lo_base + ((smem_addr + (uint32_t)((cur_t0 * p.c_blocks + cur_cb) * p.b_bytes)) >> 4);
-                    } else {
-                        b_lo = a_lo + a_to_b16;
-                    }
-                    const uint32_t acc0 = it != 0 ? 1u : 0u;
-                    if (p.nb == 3) {
-                        if (ksteps == 4) issue_stage<4, 3, PAIR>(d_tmem, a_lo, b_lo, desc_hi, idesc, a_step16, b_step16, acc0);
-                        else if (ksteps == 2) issue_stage<2, 3, PAIR>(d_tmem, a_lo, b_lo, desc_hi, idesc, a_step16, b_step16, acc0);
-                        else issue_stage<1, 3, PAIR>(d_tmem, a_lo, b_lo, desc_hi, idesc, a_step16, b_step16, acc0);
-                    } else {
-                        if (ksteps == 4) issue_stage<4, 1, PAIR>(d_tmem, a_lo, b_lo, desc_hi, idesc, a_step16, b_step16, acc0);
-                        else if (ksteps == 2) issue_stage<2, 1, PAIR>(d_tmem, a_lo, b_lo, desc_hi, idesc, a_step16, b_step16, acc0);
-                        else issue_stage<1, 1, PAIR>(d_tmem, a_lo, b_lo, desc_hi, idesc, a_step16, b_step16, acc0);
-                    }
-                    if (++cur_cb == p.c_blocks) { cur_cb = 0; ++cur_t0; }
-                    // frees the stage (in both CTAs of a pair) once these MMAs have read it
-                    if constexpr (PAIR) umma_commit_pair(&empty_bar[s], (uint16_t)3);
-                    else umma_commit(&empty_bar[s]);
-                }
-                if (!ok) break;
-                if constexpr (PAIR) umma_commit_pair(&acc_full[buf], (uint16_t)3);
-                else umma_commit(&acc_full[buf]);
-                ++jacc;
-            }
-            if (p.stall != nullptr) {
-                atomicAdd(p.stall + 1, (unsigned long long)wait_ring);
-                atomicAdd(p.stall + 2, (unsigned long long)wait_acc);
+#undef B2C_ISSUER
             }
         }
     } else {
@@ -567,18 +643,21 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
         // A wait gave up.  Before the CTA may exit, let every bulk copy it issued land and every
         // MMA it issued retire (both finish on their own; the polls here only bound the wait).
         // In a pair the leader's barriers count the peer's copies too.
-        if (warp == 0 && lane == 0 && rank == 0) {
-            if (p.resident)
+        if ((warp == 0 || warp == kProducerWarp1) && lane == 0 && rank == 0) {
+            if (p.resident && warp == 0)
                 for (uint32_t i = 0; i < kDrainPolls && !mbar_try_wait(&w_bar, 0u); ++i) {}
-            for (int back = 0; back < S && back < issued; ++back) {
-                const int it = issued - 1 - back;
+            // own stages among the last S of the CTA (older ones were consumed, so they had landed)
+            for (int back = 0; back < S && back < issued * kProducers; back += kProducers) {
+                const int it = last_issued - back;
+                if (it < 0) break;
                 for (uint32_t i = 0; i < kDrainPolls && !mbar_try_wait(&full_bar[it % S], (uint32_t)(it / S) & 1u); ++i) {}
             }
         }
-        if (warp == 1 && lane == 0 && rank == 0) {
+        if ((warp == 1 || (warp >= 2 + kEpiWarps && warp < kProducerWarp1)) && lane == 0 && rank == 0) {   // a commit covers the MMAs of the thread that makes it
             if constexpr (PAIR) umma_commit_pair(&drain_bar, (uint16_t)1);
             else umma_commit(&drain_bar);
-            for (uint32_t i = 0; i < kDrainPolls && !mbar_try_wait(&drain_bar, 0u); ++i) {}
+            if (warp == 1)
+                for (uint32_t i = 0; i < kDrainPolls && !mbar_try_wait(&drain_bar, 0u); ++i) {}
         }
         __syncthreads();
     }
@@ -709,8 +788,9 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
         p.c_blocks = pb.ic / kb;
         p.swz = kb == 64 ? SWZ_128B : kb == 32 ? SWZ_64B : SWZ_32B;
         p.vreuse = vr;
-        p.b_bytes = ((b_rows * kb * 2) + 1023) & ~1023;
         p.tx_b = b_rows * kb * 2;
+        p.b_merged = (vr && p.tx_b % 1024 == 0) ? 1 : 0;   // tiles of one load lie back to back: they must keep the swizzle alignment
+        p.b_bytes = (p.tx_b + 1023) & ~1023;
         const int a_rows = vr ? (p.bh + 2) * p.bw : 128;
         p.tx_a = a_rows * kb * 2;
         p.a_bytes = (p.tx_a + 1023) & ~1023;
@@ -726,6 +806,8 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
         if (stages >= 4 || !vr) break;
     }
     if (p.stages < 2) return B2C_ERR_UNSUPPORTED_SHAPE;
+    // Two issuing threads where one cannot keep the tensor pipe busy: tiles of at most 128 channels.
+    p.issuers = p.n_tile <= 128 ? kIssuers : 1;
     const int stage_bytes = p.a_bytes + (p.resident ? 0 : p.nb * p.b_bytes);
     const size_t smem_bytes = (size_t)p.resident_bytes + (size_t)p.stages * stage_bytes + 1024;
 
@@ -740,10 +822,11 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
         if (!encode_activation_map(ctx, &p.tmA[0], pb.in, pb.n, pb.ih, pb.iw, pb.ic, 1, 0, 0, p.kb, p.bw, box_h, p.bn)) return B2C_ERR_CUDA;
     }
     {
-        cuuint64_t dims[3] = {(cuuint64_t)pb.ic, (cuuint64_t)(R * R), (cuuint64_t)pb.oc};
-        cuuint64_t str[2] = {(cuuint64_t)pb.ic * 2, (cuuint64_t)R * R * pb.ic * 2};
-        cuuint32_t box[3] = {(cuuint32_t)p.kb, 1u, (cuuint32_t)b_rows};
-        if (!encode_map(ctx, &p.tmB, pb.wt, 3, dims, str, box, p.kb * 2)) return B2C_ERR_CUDA;
+        // weights [out][r][s][in] viewed as (in, s, out, r): a box of three filter rows lands as three tiles [r][out][in]
+        cuuint64_t dims[4] = {(cuuint64_t)pb.ic, (cuuint64_t)R, (cuuint64_t)pb.oc, (cuuint64_t)R};
+        cuuint64_t str[3] = {(cuuint64_t)pb.ic * 2, (cuuint64_t)R * R * pb.ic * 2, (cuuint64_t)R * pb.ic * 2};
+        cuuint32_t box[4] = {(cuuint32_t)p.kb, 1u, (cuuint32_t)b_rows, p.b_merged ? 3u : 1u};
+        if (!encode_map(ctx, &p.tmB, pb.wt, 4, dims, str, box, p.kb * 2)) return B2C_ERR_CUDA;
     }
 
     // tap tables (row-major over (r, s); with vreuse entry s of row 0 carries the shift of the haloed tile)
@@ -776,6 +859,7 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
             }
         p.os_n = (long long)pb.oh * pb.ow * pb.oc; p.os_h = 2ll * pb.ow * pb.oc; p.os_w = 2ll * pb.oc;
     }
+    p.r_filter = R;
     p.n_valid = pb.n;
     p.oc_valid = pb.oc;
     p.out = pb.out;

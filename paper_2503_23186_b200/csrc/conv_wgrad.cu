@@ -201,7 +201,7 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
         const int k = p.stack ? (m & 63) : ktile * 128 + m;
         bool ok = n_chunks > 0;
         if (ok) {
-            ok = mbar_wait_bounded(&accum_bar, 0u, p.spin_limit, &abort_flag);
+            if (lane == 0) ok = mbar_wait_bounded(&accum_bar, 0u, p.spin_limit, &abort_flag);   // one poller per warp
             ok = __all_sync(0xffffffffu, ok);
             if (!ok && lane == 0) atomicOr(p.status, B2C_DEV_TIMEOUT);
             tc_fence_after();
