@@ -10,9 +10,9 @@
 // B is a box (kb channels, one tap, n_tile output channels) of the [out][tap][in] weights.
 //
 // The kernel is persistent: one CTA per SM walks a list of (pixel tile, channel tile) units.
-//   * Two accumulators in TMEM: while the four epilogue warps drain unit i (bias, bf16 rounding,
-//     BatchNorm sums, stores), the MMA thread already accumulates unit i+1 into the other one, and
-//     the TMA producer runs ahead through the shared-memory ring across unit boundaries.
+//   * Two or four accumulators in TMEM (four where 4 x n_tile columns fit): while the epilogue warps drain unit i
+//     (bias, bf16 rounding, BatchNorm sums, stores), the MMA threads already accumulate the next units into the
+//     others, and the TMA producers run ahead through the shared-memory ring across unit boundaries.
 //   * Vertical tap reuse (3x3, stride 1, tile inside one image): a stage holds the tile plus one
 //     halo row above and below for one horizontal shift; the three vertical taps read it at row
 //     offsets of one image row (a multiple of the swizzle period), so the input is fetched three
@@ -33,12 +33,14 @@ struct alignas(64) ConvKParams {
     TapList taps[4];
     int bw, bh, bn;                  // pixel box of an output tile; bw*bh*bn == 128
     int tiles_w, tiles_h, tiles_n;   // tiles of the output grid
+    int tw_shift, th_shift, nk_shift, grp_shift;   // log2 of tiles_w, tiles_h, n_ktiles, stats_group_images (-1: not a power of two)
     int n_ktiles, n_tile;            // output-channel tiles, UMMA N
     int n_par;                       // output parities (stride-2 data gradient: 4)
     int total_units;
     int kb, c_blocks;                // channels per k-block, k-blocks per tap
     int stages, swz;
     int tmem_cols, acc_cols;         // allocation, columns per accumulator
+    int acc_bufs, acc_shift;         // accumulators in TMEM (2 or 4) and log2 of that: unit j uses accumulator j % acc_bufs
     int vreuse;                      // a stage serves the three vertical taps of one horizontal shift
     int nb;                          // B tiles per stage (1, or 3 with vreuse)
     int b_merged;                    // the three B tiles of a stage come with one load (box of three filter rows)
@@ -64,6 +66,7 @@ struct alignas(64) ConvKParams {
 };
 
 static constexpr int kMaxStages = 8;
+static constexpr int kMaxAccBufs = 4;
 static constexpr int kEpiWarps = 8;
 static constexpr int kIssuers = 2;       // MMA-issuing threads: warp 1 and the warps after the epilogue warps
 static constexpr int kProducers = 2;     // TMA-issuing threads: warp 0 and the warp after the issuer warps; they take alternate stages
@@ -74,17 +77,28 @@ static constexpr uint32_t kDrainPolls = 1u << 22;
 struct UnitCoord {
     int par, ktile, ow0, oh0, n0;
 };
+// tiles_w and tiles_h are powers of two (the grid sides are); the channel-tile count and the stats group size usually are
 __device__ __forceinline__ UnitCoord decode_unit(const ConvKParams& p, int u)
 {
     UnitCoord c;
-    c.ktile = u % p.n_ktiles;
-    u /= p.n_ktiles;
-    c.ow0 = (u % p.tiles_w) * p.bw;
-    u /= p.tiles_w;
-    c.oh0 = (u % p.tiles_h) * p.bh;
-    u /= p.tiles_h;
-    c.n0 = (u % p.tiles_n) * p.bn;
-    c.par = u / p.tiles_n;
+    if (p.nk_shift >= 0) {
+        c.ktile = u & (p.n_ktiles - 1);
+        u >>= p.nk_shift;
+    } else {
+        c.ktile = u % p.n_ktiles;
+        u /= p.n_ktiles;
+    }
+    c.ow0 = (u & (p.tiles_w - 1)) * p.bw;
+    u >>= p.tw_shift;
+    c.oh0 = (u & (p.tiles_h - 1)) * p.bh;
+    u >>= p.th_shift;
+    if (p.n_par > 1) {
+        c.n0 = (u % p.tiles_n) * p.bn;
+        c.par = u / p.tiles_n;
+    } else {
+        c.n0 = u * p.bn;
+        c.par = 0;
+    }
     return c;
 }
 // Units of this CTA: plain kernels walk units blockIdx.x, +gridDim.x, ...; CTA pairs walk pair-units (two pixel tiles
@@ -138,8 +152,7 @@ __device__ __forceinline__ void epilogue_loop(const ConvKParams& p, uint32_t tme
 {
     const UnitWalk walk(p, rank);
     // the accumulator-free barrier lives in the leader CTA of a pair: the peer's warps arrive on it remotely
-    const uint32_t remote_empty0 = (p.pair && rank != 0) ? map_to_cta(smem_u32(&acc_empty[0]), 0) : 0u;
-    const uint32_t remote_empty1 = (p.pair && rank != 0) ? map_to_cta(smem_u32(&acc_empty[1]), 0) : 0u;
+    const bool remote_empty = p.pair && rank != 0;
     const int q = (e + 2) & 3;       // TMEM lane quarter this warp may read: (warp index in the CTA) % 4, epilogue warps start at 2
     const int m = q * 32 + lane;     // accumulator row = pixel of the tile (w fastest, then h, then image)
     const int lw = m % p.bw, lh = (m / p.bw) % p.bh, ln = m / (p.bw * p.bh);
@@ -201,10 +214,10 @@ __device__ __forceinline__ void epilogue_loop(const ConvKParams& p, uint32_t tme
         const long long row_off = (long long)(c.n0 + ln) * p.os_n + (long long)(c.oh0 + lh) * p.os_h + (long long)(c.ow0 + lw) * p.os_w + p.off[c.par];
         int buf = 0;
         if (n_it > 0) {
-            buf = jacc & 1;
+            buf = jacc & (p.acc_bufs - 1);
             const long long w3 = clock64();
             ok = true;
-            if (lane == 0) ok = mbar_wait_bounded(&acc_full[buf], (uint32_t)(jacc >> 1) & 1u, p.spin_limit, abort_flag);   // one poller per warp
+            if (lane == 0) ok = mbar_wait_bounded(&acc_full[buf], (uint32_t)(jacc >> p.acc_shift) & 1u, p.spin_limit, abort_flag);   // one poller per warp
             epi_wait += clock64() - w3;
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) {
@@ -215,7 +228,7 @@ __device__ __forceinline__ void epilogue_loop(const ConvKParams& p, uint32_t tme
             ++jacc;
         }
         if (do_stats) {
-            const int grp = p.stats_group_images > 0 ? c.n0 / p.stats_group_images : 0;
+            const int grp = p.stats_group_images > 0 ? (p.grp_shift >= 0 ? c.n0 >> p.grp_shift : c.n0 / p.stats_group_images) : 0;
             if (grp != cur_group) {
                 if (cur_group >= 0) flush_stats();
                 cur_group = grp;
@@ -229,7 +242,7 @@ __device__ __forceinline__ void epilogue_loop(const ConvKParams& p, uint32_t tme
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) {
-                    if (remote_empty0 != 0u) mbar_arrive_cluster(buf ? remote_empty1 : remote_empty0);
+                    if (remote_empty) mbar_arrive_cluster(map_to_cta(smem_u32(&acc_empty[buf]), 0));
                     else mbar_arrive(&acc_empty[buf]);
                 }
             }
@@ -370,7 +383,7 @@ __device__ __forceinline__ void issue_stage(uint32_t d_tmem, uint32_t a_lo, uint
 }
 
 // One MMA-issuing thread.  The CTA runs kIssuers of them (in different warps): issuer `my` accumulates the CTA's units
-// my, my + kIssuers, ... (unit j always into accumulator j & 1) and steps over the ring stages of the others.  A single
+// my, my + kIssuers, ... (unit j always into accumulator j % acc_bufs) and steps over the ring stages of the others.  A single
 // thread cannot keep the tensor pipe busy on narrow tiles: it pays roughly 45 cycles per tcgen05.mma, 180 per barrier
 // wait and 55 per commit, all serial, against 48-64 cycles the pipe needs per MMA at N <= 128; two threads working on
 // different accumulators can.
@@ -411,9 +424,9 @@ __device__ __forceinline__ void mma_issuer(const ConvKParams& p, const UnitWalk&
             ++j;
             continue;
         }
-        const int buf = j & 1;
+        const int buf = j & (p.acc_bufs - 1);
         const long long w1 = timed ? clock64() : 0;
-        if (!mbar_wait_bounded(&acc_empty[buf], ((uint32_t)(j >> 1) & 1u) ^ 1u, p.spin_limit, abort_flag)) {
+        if (!mbar_wait_bounded(&acc_empty[buf], ((uint32_t)(j >> p.acc_shift) & 1u) ^ 1u, p.spin_limit, abort_flag)) {
             atomicOr(p.status, B2C_DEV_TIMEOUT);
             ok = false;
             break;
@@ -472,7 +485,7 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
 {
     const int rank = PAIR ? (int)cluster_ctarank() : 0;   // 0 = leader of the pair: issues the MMAs, owns the barriers the pair shares
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], acc_full[2], acc_empty[2], w_bar, drain_bar;
+    __shared__ uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], acc_full[kMaxAccBufs], acc_empty[kMaxAccBufs], w_bar, drain_bar;
     __shared__ uint32_t tmem_slot;
     __shared__ uint32_t abort_flag;
     __shared__ int slot_stage[kMaxStages];   // per ring slot: 1 + index of the stage whose loads were issued into it last
@@ -489,7 +502,7 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], 1);
         }
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < kMaxAccBufs; ++b) {
             mbar_init(&acc_full[b], 1);
             mbar_init(&acc_empty[b], PAIR ? 2 * kEpiWarps : kEpiWarps);   // one arrival per epilogue warp (of both CTAs of a pair)
         }
@@ -691,6 +704,14 @@ bool encode_activation_map(b2c_ctx* ctx, CUtensorMap* tm, const void* base, int 
     return encode_map(ctx, tm, b, 4, dims, str, box, box_c * 2);
 }
 
+static int log2_exact(int v)
+{
+    if (v <= 0 || (v & (v - 1)) != 0) return -1;
+    int l = 0;
+    while ((1 << l) < v) ++l;
+    return l;
+}
+
 static int floordiv2(int e) { return (e >= 0) ? e / 2 : -((-e + 1) / 2); }
 
 void forward_taps(TapList& tl, int R, int stride, int pad)
@@ -748,8 +769,11 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
     p.n_tile = n_tile;
     p.n_ktiles = pb.oc / n_tile;
     p.acc_cols = ((n_tile + 31) / 32) * 32;
+    // four accumulators where TMEM has room: the issuers then run a unit or two ahead of the epilogue
+    p.acc_bufs = (4 * p.acc_cols <= 512) ? 4 : 2;
+    p.acc_shift = p.acc_bufs == 4 ? 2 : 1;
     p.tmem_cols = 32;
-    while (p.tmem_cols < 2 * p.acc_cols) p.tmem_cols *= 2;
+    while (p.tmem_cols < p.acc_bufs * p.acc_cols) p.tmem_cols *= 2;
     p.total_units = n_par * p.tiles_n * p.tiles_h * p.tiles_w * p.n_ktiles;
 
     // CTA pairs (cta_group::2): two neighbouring pixel tiles share every filter tile, each CTA holding half of its
@@ -867,6 +891,10 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
     p.bias = pb.bias;
     p.stats = pb.out_f32 ? nullptr : pb.stats;
     p.stats_group_images = pb.stats_group_images;
+    p.tw_shift = log2_exact(p.tiles_w);
+    p.th_shift = log2_exact(p.tiles_h);
+    p.nk_shift = log2_exact(p.n_ktiles);
+    p.grp_shift = log2_exact(p.stats_group_images);
     if (p.stats && p.stats_group_images > 0 && (p.stats_group_images % p.bn) != 0) return B2C_ERR_UNSUPPORTED_SHAPE;  // a tile must not straddle groups
     p.status = ctx->d_status;
     p.spin_limit = ctx->spin_limit;
