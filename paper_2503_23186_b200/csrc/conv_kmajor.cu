@@ -528,13 +528,14 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
     const uint32_t tmem_base = tmem_slot;
     const long long t_start = clock64();
     const UnitWalk walk(p, rank);
-    int issued = 0, last_issued = -1;  // producer lanes: own stages whose loads were issued, index of the last one
+    int last_issued = -1;  // producer lanes: index of the last stage whose loads this lane issued
 
     if (warp == 0 || warp == kProducerWarp1) {
         if (lane == 0) {
             // ------------------------------------------------------------ TMA producers
-            // Producer w stages every kProducers-th stage of the CTA's sequence: the chain wait -> expect -> issue of one
-            // thread (several hundred cycles) would otherwise bound short stages.
+            // Producer w fills the ring slots w, w + kProducers, ...: the chain wait -> expect -> issue of one thread
+            // (several hundred cycles) would otherwise bound short stages.  Splitting by slot (not by stage) keeps
+            // every slot with one producer that uses it strictly in order, which a parity wait on its barrier needs.
             const int w = warp == 0 ? 0 : 1;
             prefetch_tensormap(&p.tmB);
             prefetch_tensormap(&p.tmA[0]);
@@ -564,8 +565,8 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
             long long waited = 0;
             const bool timed = p.stall != nullptr;
             int i = w, i_base = 0;   // this producer's next stage and the first stage of the current unit, in CTA order
-            int s = w % S;
-            uint32_t ph = (uint32_t)(w / S) & 1u;
+            int s = w;   // w < kProducers <= S
+            uint32_t ph = 0u;
             const uint32_t stage_tx = (uint32_t)(p.tx_a + (p.resident ? 0 : p.nb * p.tx_b));
             const int n_b_loads = p.resident ? 0 : (p.b_merged ? 1 : p.nb);
             for (int pu = walk.first; ok && pu < walk.count; pu += walk.stride) {
@@ -578,7 +579,7 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
                 const UnitCoord c = decode_unit(p, u);
                 const TapList& tl = p.taps[c.par];
                 const int oc0 = c.ktile * p.n_tile + rank * b_rows;
-                for (; i < i_base + n_it; i += kProducers) {
+                while (i < i_base + n_it) {
                     const int it = i - i_base;
                     const long long w0 = timed ? clock64() : 0;
                     if (!mbar_wait_bounded(&empty_bar[s], ph ^ 1u, p.spin_limit, &abort_flag)) {
@@ -606,11 +607,16 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
                             tma_load_4d(a_dst + p.a_bytes + (size_t)v * p.b_bytes, &p.tmB, &full_bar[s], cb * p.kb, rs % R, oc0, rs / R);
                         }
                     }
-                    ++issued;
                     last_issued = i;
                     if (p.issuers > 1) st_release_shared(&slot_stage[s], i + 1);   // lets the issuers tell this slot's phases apart
-                    s += kProducers;
-                    if (s >= S) { s -= S; ph ^= 1u; }
+                    if (s + kProducers < S) {
+                        i += kProducers;
+                        s += kProducers;
+                    } else {   // wrap to this producer's first slot
+                        i += S - s + w;
+                        s = w;
+                        ph ^= 1u;
+                    }
                 }
                 i_base += n_it;
             }
@@ -659,11 +665,12 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
         if ((warp == 0 || warp == kProducerWarp1) && lane == 0 && rank == 0) {
             if (p.resident && warp == 0)
                 for (uint32_t i = 0; i < kDrainPolls && !mbar_try_wait(&w_bar, 0u); ++i) {}
-            // own stages among the last S of the CTA (older ones were consumed, so they had landed)
-            for (int back = 0; back < S && back < issued * kProducers; back += kProducers) {
-                const int it = last_issued - back;
-                if (it < 0) break;
-                for (uint32_t i = 0; i < kDrainPolls && !mbar_try_wait(&full_bar[it % S], (uint32_t)(it / S) & 1u); ++i) {}
+            // the last stage issued into each of the own slots (older ones were consumed, so they had landed)
+            const int w = warp == 0 ? 0 : 1;
+            for (int sl = w; sl < S; sl += kProducers) {
+                if (last_issued < sl) continue;
+                const int it = last_issued - ((last_issued - sl) % S);   // largest stage index <= last_issued in slot sl
+                for (uint32_t i = 0; i < kDrainPolls && !mbar_try_wait(&full_bar[sl], (uint32_t)(it / S) & 1u); ++i) {}
             }
         }
         if ((warp == 1 || (warp >= 2 + kEpiWarps && warp < kProducerWarp1)) && lane == 0 && rank == 0) {   // a commit covers the MMAs of the thread that makes it

@@ -39,6 +39,8 @@ struct alignas(64) WgradParams {
     int chunks_total;
     int stages, tmem_cols;
     int box_a, box_b, a_boxes, b_boxes;   // bytes per dy / x box; dy boxes per stage; x boxes per shift
+    int a_bytes, a_lbo;                   // dy bytes per stage; byte distance between the two 64-row halves of the A operand
+    int tw_shift;                         // log2(tiles_w)
     int stage_bytes;
     int n_pieces, piece_t0[3], piece_nt[3];   // MMAs per k-step: first shift and number of shifts each covers
     int k_total, c_total, rs_total;
@@ -48,7 +50,9 @@ struct alignas(64) WgradParams {
 };
 
 static constexpr int kWgStages = 6;
-static constexpr int kWgThreads = 192;
+static constexpr int kWgProducers = 2;   // warp 0 and the warp after the epilogue warps; they fill alternate ring slots
+static constexpr int kWgProducerWarp1 = 6;
+static constexpr int kWgThreads = 224;
 static constexpr uint32_t kWgDrainPolls = 1u << 22;
 
 __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d)
@@ -110,45 +114,59 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_slot;
-    int issued = 0;  // producer lane: chunks whose loads were issued
+    int last_issued = -1;  // producer lanes: last chunk whose loads this lane issued
 
-    if (warp == 0) {
+    if (warp == 0 || warp == kWgProducerWarp1) {
         if (lane == 0) {
+            // Producer w fills the ring slots w, w + 2, ...: one thread's wait -> expect -> issue chain is longer than
+            // the MMAs of a stage take.  Each slot keeps one producer, which uses it strictly in order.
+            const int w = warp == 0 ? 0 : 1;
             prefetch_tensormap(&p.tmDy);
             prefetch_tensormap(&p.tmX[0]);
-            const uint32_t tx = (uint32_t)(p.a_boxes * p.box_a + grp.nb * p.b_boxes * p.box_b);
-            for (int it = 0; it < n_chunks; ++it, ++issued) {
-                const int s = it % S;
-                const uint32_t ph = (uint32_t)(it / S) & 1u;
+            const uint32_t tx = (uint32_t)(p.a_bytes + grp.nb * p.b_boxes * p.box_b);
+            int it = w, s = w;
+            uint32_t ph = 0u;
+            while (it < n_chunks) {
                 if (!mbar_wait_bounded(&empty_bar[s], ph ^ 1u, p.spin_limit, &abort_flag)) {
                     atomicOr(p.status, B2C_DEV_TIMEOUT);
                     break;
                 }
                 int ch = chunk_begin + it;
-                const int ow0 = (ch % p.tiles_w) * p.bw;
-                ch /= p.tiles_w;
-                const int oh0 = (ch % p.tiles_h) * p.bh;
-                const int n0 = (ch / p.tiles_h) * p.bn;
+                const int ow0 = (ch & (p.tiles_w - 1)) * p.bw;
+                ch >>= p.tw_shift;
+                const int th = ch / p.tiles_h;
+                const int oh0 = (ch - th * p.tiles_h) * p.bh;
+                const int n0 = th * p.bn;
                 uint8_t* dst = smem + (size_t)s * p.stage_bytes;
                 mbar_expect_tx(&full_bar[s], tx);
                 if (p.stack) {
-                    for (int a = 0; a < 2; ++a)   // copy a of dy is gathered a rows higher
-                        tma_load_4d(dst + (size_t)a * p.box_a, &p.tmDy, &full_bar[s], 0, ow0, oh0 - a, n0);
+                    // one box with a halo row on top: copy 1 of dy (gathered one row higher) is its first pb pixels,
+                    // copy 0 starts one image row further down
+                    tma_load_4d(dst, &p.tmDy, &full_bar[s], 0, ow0, oh0 - 1, n0);
                 } else {
                     for (int j = 0; j < p.a_boxes; ++j)  // boxes past the last channel are zero-filled
                         tma_load_4d(dst + (size_t)j * p.box_a, &p.tmDy, &full_bar[s], ktile * 128 + j * p.cw_a, ow0, oh0, n0);
                 }
-                dst += (size_t)p.a_boxes * p.box_a;
+                dst += p.a_bytes;
                 for (int b = 0; b < grp.nb; ++b)
                     for (int j = 0; j < p.b_boxes; ++j)
                         tma_load_4d(dst + (size_t)(b * p.b_boxes + j) * p.box_b, &p.tmX[grp.map[b]], &full_bar[s], ctile * p.ct + j * p.cw_b,
                                     ow0 + grp.dw[b], oh0 + grp.dh[b], n0);
+                last_issued = it;
+                if (s + kWgProducers < S) {
+                    it += kWgProducers;
+                    s += kWgProducers;
+                } else {   // wrap to this producer's first slot
+                    it += S - s + w;
+                    s = w;
+                    ph ^= 1u;
+                }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
             // SBO = eight pixel rows, LBO = next block of cw channels (the next box)
-            const uint64_t proto_a = make_smem_desc(0u, (uint32_t)p.box_a, 16u * (uint32_t)p.cw_a, (uint32_t)p.swz_a);
+            const uint64_t proto_a = make_smem_desc(0u, (uint32_t)p.a_lbo, 16u * (uint32_t)p.cw_a, (uint32_t)p.swz_a);
             const uint64_t proto_b = make_smem_desc(0u, (uint32_t)p.box_b, 16u * (uint32_t)p.cw_b, (uint32_t)p.swz_b);
             const uint32_t a_hi = (uint32_t)(proto_a >> 32), a_lo_base = (uint32_t)proto_a;
             const uint32_t b_hi = (uint32_t)(proto_b >> 32), b_lo_base = (uint32_t)proto_b;
@@ -161,7 +179,7 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
                 if (p.piece_t0[i] >= grp.nb) break;
                 const int nt = min(p.piece_nt[i], grp.nb - p.piece_t0[i]);
                 const uint32_t id = make_idesc_bf16(128, nt * p.ct, true, true);
-                const uint32_t bo = (uint32_t)(p.a_boxes * p.box_a + p.piece_t0[i] * p.b_boxes * p.box_b) >> 4;
+                const uint32_t bo = (uint32_t)(p.a_bytes + p.piece_t0[i] * p.b_boxes * p.box_b) >> 4;
                 const uint32_t dc = (uint32_t)(p.piece_t0[i] * p.ct);
                 if (i == 0) { idesc0 = id; boff0 = bo; dcol0 = dc; }
                 else if (i == 1) { idesc1 = id; boff1 = bo; dcol1 = dc; }
@@ -197,7 +215,7 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
     } else {
         const int q = warp & 3;
         const int m = q * 32 + lane;
-        const int copy = p.stack ? (m >> 6) : 0;                       // which dy copy this accumulator row belongs to
+        const int copy = p.stack ? 1 - (m >> 6) : 0;                   // which dy copy this accumulator row belongs to (copy 1 comes first)
         const int k = p.stack ? (m & 63) : ktile * 128 + m;
         bool ok = n_chunks > 0;
         if (ok) {
@@ -244,10 +262,12 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
     __syncthreads();
     if (abort_flag) {
         // A wait gave up: let the issued bulk copies land and the issued MMAs retire before exit.
-        if (warp == 0 && lane == 0) {
-            for (int back = 0; back < S && back < issued; ++back) {
-                const int it = issued - 1 - back;
-                for (uint32_t i = 0; i < kWgDrainPolls && !mbar_try_wait(&full_bar[it % S], (uint32_t)(it / S) & 1u); ++i) {}
+        if ((warp == 0 || warp == kWgProducerWarp1) && lane == 0) {
+            const int w = warp == 0 ? 0 : 1;
+            for (int sl = w; sl < S; sl += kWgProducers) {   // the last chunk issued into each of the own slots
+                if (last_issued < sl) continue;
+                const int it = last_issued - ((last_issued - sl) % S);
+                for (uint32_t i = 0; i < kWgDrainPolls && !mbar_try_wait(&full_bar[sl], (uint32_t)(it / S) & 1u); ++i) {}
             }
         }
         if (warp == 1 && lane == 0) {
@@ -280,7 +300,7 @@ b2c_status launch_conv_wgrad(b2c_ctx* ctx, const WgradProblem& pb, cudaStream_t 
     p.swz_a = p.cw_a == 64 ? SWZ_128B : p.cw_a == 32 ? SWZ_64B : SWZ_32B;
     p.swz_b = p.cw_b == 64 ? SWZ_128B : p.cw_b == 32 ? SWZ_64B : SWZ_32B;
     // stacking needs chunks that stay inside one image (at least 64 pixels per image)
-    p.stack = (R == 3 && pb.stride == 1 && pb.k == 64 && pb.p * pb.q >= 64) ? 1 : 0;
+    p.stack = (R == 3 && pb.stride == 1 && pb.k == 64 && pb.p * pb.q >= 64 && pb.q >= 8) ? 1 : 0;   // q >= 8: the second copy starts on a swizzle-atom boundary
     // x-channel tile: largest divisor of c that is a multiple of cw_b, at most 160 (three shifts fit 512 TMEM columns)
     p.ct = p.cw_b;
     for (int cand = 160; cand >= p.cw_b; cand -= 16)
@@ -340,7 +360,8 @@ b2c_status launch_conv_wgrad(b2c_ctx* ctx, const WgradProblem& pb, cudaStream_t 
     for (;;) {
         p.box_a = p.pb * p.cw_a * 2;
         p.box_b = p.pb * p.cw_b * 2;
-        p.stage_bytes = p.a_boxes * p.box_a + shifts * p.b_boxes * p.box_b;
+        p.a_bytes = p.stack ? (p.pb + (pb.q < p.pb ? pb.q : p.pb)) * p.cw_a * 2 : p.a_boxes * p.box_a;   // stacked: one box with a halo row
+        p.stage_bytes = p.a_bytes + shifts * p.b_boxes * p.box_b;
         if (p.stage_bytes * 3 <= 200 * 1024 || p.pb == 32) break;
         p.pb = 32;
     }
@@ -353,6 +374,9 @@ b2c_status launch_conv_wgrad(b2c_ctx* ctx, const WgradProblem& pb, cudaStream_t 
     p.bn = p.pb / (p.bw * p.bh);
     if (p.stack && p.bn != 1) return B2C_ERR_UNSUPPORTED_SHAPE;   // cannot happen: 64 pixels per image guarantee bn == 1
     p.tiles_w = pb.q / p.bw;
+    p.tw_shift = 0;
+    while ((1 << p.tw_shift) < p.tiles_w) ++p.tw_shift;
+    p.a_lbo = p.stack ? p.bw * p.cw_a * 2 : p.box_a;   // stacked: copy 0 starts one image row below copy 1
     p.tiles_h = (pb.p + (p.stack ? 1 : 0) + p.bh - 1) / p.bh;   // stacked: dy copy 1 of row p-1 is met at chunk row p
     const int tiles_n = (pb.n + p.bn - 1) / p.bn;
     p.chunks_total = p.tiles_w * p.tiles_h * tiles_n;
@@ -362,7 +386,7 @@ b2c_status launch_conv_wgrad(b2c_ctx* ctx, const WgradProblem& pb, cudaStream_t 
     if (n_splits < 1) n_splits = 1;
     p.n_splits = n_splits;
 
-    if (!encode_activation_map(ctx, &p.tmDy, pb.dy, pb.n, pb.p, pb.q, pb.k, 1, 0, 0, p.cw_a, p.bw, p.bh, p.bn)) return B2C_ERR_CUDA;
+    if (!encode_activation_map(ctx, &p.tmDy, pb.dy, pb.n, pb.p, pb.q, pb.k, 1, 0, 0, p.cw_a, p.bw, p.stack ? p.bh + 1 : p.bh, p.bn)) return B2C_ERR_CUDA;
     if (pb.stride == 2) {
         for (int ph = 0; ph < 2; ++ph)
             for (int pw = 0; pw < 2; ++pw)
