@@ -33,7 +33,7 @@ struct alignas(64) ConvKParams {
     TapList taps[4];
     int bw, bh, bn;                  // pixel box of an output tile; bw*bh*bn == 128
     int tiles_w, tiles_h, tiles_n;   // tiles of the output grid
-    int tw_shift, th_shift, nk_shift, grp_shift;   // log2 of tiles_w, tiles_h, n_ktiles, stats_group_images (-1: not a power of two)
+    int tw_shift, th_shift, nk_shift, grp_shift, cb_shift;   // log2 of tiles_w, tiles_h, n_ktiles, stats_group_images, c_blocks (-1: not a power of two)
     int n_ktiles, n_tile;            // output-channel tiles, UMMA N
     int n_par;                       // output parities (stride-2 data gradient: 4)
     int total_units;
@@ -443,7 +443,7 @@ __device__ __forceinline__ void mma_issuer(const ConvKParams& p, const UnitWalk&
             // seeing the stamp pass i makes the parity wait unambiguous.
             if (p.issuers > 1) {
                 uint32_t polls = 0;
-                while (ld_acquire_shared(&slot_stage[s]) <= i_stage) {
+                while (ld_volatile_shared(&slot_stage[s]) <= i_stage) {
                     if (++polls > p.spin_limit || *(volatile uint32_t*)abort_flag != 0u) {
                         ok = false;
                         break;
@@ -588,7 +588,11 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
                         break;
                     }
                     if (timed) waited += clock64() - w0;
-                    const int t0 = it / p.c_blocks, cb = it - t0 * p.c_blocks;   // tap (or horizontal shift) and channel block
+                    // The previous stage in this slot has been consumed, so its barrier phase is over: the stamp lets the
+                    // issuers tell this slot's phases apart (a relaxed store: the wait above orders it).
+                    if (p.issuers > 1) st_volatile_shared(&slot_stage[s], i + 1);
+                    const int t0 = p.cb_shift >= 0 ? it >> p.cb_shift : it / p.c_blocks;   // tap (or horizontal shift)
+                    const int cb = it - t0 * p.c_blocks;                                     // channel block
                     uint8_t* a_dst = ring + (size_t)s * stage_bytes;
                     // with vreuse the table entry of vertical tap 0 carries the shift of the whole haloed tile
                     if constexpr (PAIR) {
@@ -596,19 +600,18 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
                         if (rank == 0) mbar_expect_tx(&full_bar[s], 2u * stage_tx);
                         tma_load_4d_pair(a_dst, &p.tmA[tl.map[t0]], full_cl, cb * p.kb, c.ow0 + tl.dw[t0], c.oh0 + tl.dh[t0], c.n0);
                         for (int v = 0; v < n_b_loads; ++v) {
-                            const int rs = tl.rs[t0 + 3 * v];
-                            tma_load_4d_pair(a_dst + p.a_bytes + (size_t)v * p.b_bytes, &p.tmB, full_cl, cb * p.kb, rs % R, oc0, rs / R);
+                            const int rs = tl.rs[t0 + 3 * v], fr = (rs * 11) >> 5;   // rs / 3 for rs < 9 (R is 1 or 3)
+                            tma_load_4d_pair(a_dst + p.a_bytes + (size_t)v * p.b_bytes, &p.tmB, full_cl, cb * p.kb, rs - fr * R, oc0, fr);
                         }
                     } else {
                         mbar_expect_tx(&full_bar[s], stage_tx);
                         tma_load_4d(a_dst, &p.tmA[tl.map[t0]], &full_bar[s], cb * p.kb, c.ow0 + tl.dw[t0], c.oh0 + tl.dh[t0], c.n0);
                         for (int v = 0; v < n_b_loads; ++v) {
-                            const int rs = tl.rs[t0 + 3 * v];
-                            tma_load_4d(a_dst + p.a_bytes + (size_t)v * p.b_bytes, &p.tmB, &full_bar[s], cb * p.kb, rs % R, oc0, rs / R);
+                            const int rs = tl.rs[t0 + 3 * v], fr = (rs * 11) >> 5;   // rs / 3 for rs < 9 (R is 1 or 3)
+                            tma_load_4d(a_dst + p.a_bytes + (size_t)v * p.b_bytes, &p.tmB, &full_bar[s], cb * p.kb, rs - fr * R, oc0, fr);
                         }
                     }
                     last_issued = i;
-                    if (p.issuers > 1) st_release_shared(&slot_stage[s], i + 1);   // lets the issuers tell this slot's phases apart
                     if (s + kProducers < S) {
                         i += kProducers;
                         s += kProducers;
@@ -902,6 +905,7 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
     p.th_shift = log2_exact(p.tiles_h);
     p.nk_shift = log2_exact(p.n_ktiles);
     p.grp_shift = log2_exact(p.stats_group_images);
+    p.cb_shift = log2_exact(p.c_blocks);
     if (p.stats && p.stats_group_images > 0 && (p.stats_group_images % p.bn) != 0) return B2C_ERR_UNSUPPORTED_SHAPE;  // a tile must not straddle groups
     p.status = ctx->d_status;
     p.spin_limit = ctx->spin_limit;

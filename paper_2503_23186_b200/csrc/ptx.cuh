@@ -27,15 +27,16 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-// A counter in shared memory that one thread publishes and others poll.
-__device__ __forceinline__ void st_release_shared(int* p, int v)
+// A word in shared memory that one thread publishes and others poll (relaxed: callers order it through the
+// barrier operations that precede the store and follow the load).
+__device__ __forceinline__ void st_volatile_shared(int* p, int v)
 {
-    asm volatile("st.release.cta.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
+    asm volatile("st.volatile.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
 }
-__device__ __forceinline__ int ld_acquire_shared(const int* p)
+__device__ __forceinline__ int ld_volatile_shared(const int* p)
 {
     int v;
-    asm volatile("ld.acquire.cta.shared::cta.b32 %0, [%1];" : "=r"(v) : "r"(smem_u32(p)) : "memory");
+    asm volatile("ld.volatile.shared::cta.b32 %0, [%1];" : "=r"(v) : "r"(smem_u32(p)) : "memory");
     return v;
 }
 
