@@ -28,7 +28,7 @@ b2c_status b2c_create(b2c_ctx** out, int device)
     ctx->stall_counters = nullptr;
     {
         const char* env = std::getenv("B2C_CTA_PAIRS");
-        ctx->use_pairs = env ? (env[0] == '2' ? 2 : env[0] == '1' ? 1 : 0) : 0;   // 0 never (default), 1 for 128-channel tiles, 2 wherever possible
+        ctx->use_pairs = env ? (env[0] == '2' ? 2 : env[0] == '1' ? 1 : 0) : 1;   // 0 never, 1 for 128-channel tiles (default), 2 wherever possible
     }
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;

@@ -790,11 +790,12 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
     // rows, which halves the shared-memory operand traffic per MMA.  Needs an even number of pixel tiles and a channel
     // tile that splits into two multiples of 16; the fp32 / bias / multi-parity cases stay on single CTAs.
     const int m_tiles = p.tiles_n * p.tiles_h * p.tiles_w;
-    // Measured on B200 (1024-image layers, isolated launches): pairs gain ~20 % at 128-channel tiles and lose ~10 % at 64
-    // and 256; inside the whole step the gain disappears, so pairs are off by default (use_pairs: 1 = 128-channel tiles
-    // only, 2 = every eligible problem).
+    // Measured on B200 (1024-image layers): pairs gain ~30 % at 128-channel tiles, where the filter traffic from L2
+    // bounds single CTAs, and lose 5-30 % at 64 and 256 and on the short reductions of 1x1 and stride-2 layers; so by
+    // default only 3x3 stride-1 layers with 128-channel tiles use them (use_pairs: 0 = never, 1 = those, 2 = every
+    // eligible problem).
     const bool pair_ok = n_par == 1 && !pb.out_f32 && pb.bias == nullptr && n_tile % 32 == 0 && m_tiles % 2 == 0 && ctx->sm_count >= 2;
-    p.pair = (pair_ok && (ctx->use_pairs == 2 || (ctx->use_pairs == 1 && n_tile == 128))) ? 1 : 0;
+    p.pair = (pair_ok && (ctx->use_pairs == 2 || (ctx->use_pairs == 1 && n_tile == 128 && R == 3 && pb.stride == 1))) ? 1 : 0;
     const int b_rows = p.pair ? n_tile / 2 : n_tile;   // filter rows one CTA fetches per tile
 
     // launch shape: one persistent CTA per SM; the unit walk stride (CTAs, or pairs) is a multiple of n_ktiles so that a
@@ -809,7 +810,7 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
 
     // shared-memory plan.  Preference: haloed stages (vertical tap reuse) with 64-channel k-blocks, then with
     // 32-channel k-blocks (smaller stages, so that a ring of at least four still fits), else one tap per stage.
-    const int ring_budget = 200 * 1024;
+    const int ring_budget = 210 * 1024;
     const int kb_natural = (pb.ic % 64 == 0) ? 64 : (pb.ic % 32 == 0) ? 32 : 16;
     const bool can_vreuse = (R == 3 && pb.stride == 1 && p.bn == 1);
     const int taps_total = R * R;
@@ -830,6 +831,8 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
         p.a_bytes = (p.tx_a + 1023) & ~1023;
         p.nb = vr ? 3 : 1;
         p.a_step = vr ? p.bw * kb * 2 : 0;
+        // (a pair could keep its half of a 3x3x128x128 bank, 148 KB, resident; measured slower than streaming it: the
+        // ring left over is short)
         const int bank_bytes = taps_total * p.c_blocks * p.b_bytes;
         p.resident = (n_par == 1 && bank_bytes <= 96 * 1024 && units_per_cta >= 2) ? 1 : 0;
         p.resident_bytes = p.resident ? bank_bytes : 0;
