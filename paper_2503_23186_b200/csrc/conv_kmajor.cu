@@ -57,6 +57,7 @@ struct alignas(64) ConvKParams {
     long long off[4];                // output element offset per parity
     void* out;
     int out_is_f32;
+    int out_v8;                      // the output base is 32-byte aligned: bf16 chunks go out as one 256-bit store per lane
     const float* bias;
     double* stats;
     int stats_group_images;          // images per BatchNorm statistics group (0: one group)
@@ -270,8 +271,12 @@ __device__ __forceinline__ void epilogue_loop(const ConvKParams& p, uint32_t tme
             for (int i = 0; i < 8; ++i) pk[i] = pack_bf16x2(v[2 * i], v[2 * i + 1]);
             if (row_valid) {
                 __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + row_off + ch0;
-                if (ch0 < p.oc_valid) *reinterpret_cast<uint4*>(dst) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                if (ch0 + 8 < p.oc_valid) *reinterpret_cast<uint4*>(dst + 8) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                if (p.out_v8 && ch0 + 8 < p.oc_valid) {
+                    st_global_v8(dst, pk);   // one full 32-byte sector per lane
+                } else {
+                    if (ch0 < p.oc_valid) *reinterpret_cast<uint4*>(dst) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    if (ch0 + 8 < p.oc_valid) *reinterpret_cast<uint4*>(dst + 8) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                }
             }
         };
 
@@ -901,6 +906,7 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
     p.oc_valid = pb.oc;
     p.out = pb.out;
     p.out_is_f32 = pb.out_f32 ? 1 : 0;
+    p.out_v8 = (reinterpret_cast<uintptr_t>(pb.out) % 32 == 0) ? 1 : 0;   // row pitches are multiples of 32 bytes (16 channels)
     p.bias = pb.bias;
     p.stats = pb.out_f32 ? nullptr : pb.stats;
     p.stats_group_images = pb.stats_group_images;

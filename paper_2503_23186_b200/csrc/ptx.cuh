@@ -27,6 +27,14 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+// 256-bit store to a 32-byte aligned global address.
+__device__ __forceinline__ void st_global_v8(void* p, const uint32_t (&v)[8])
+{
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]),
+                 "r"(v[6]), "r"(v[7])
+                 : "memory");
+}
+
 // A word in shared memory that one thread publishes and others poll (relaxed: callers order it through the
 // barrier operations that precede the store and follow the load).
 __device__ __forceinline__ void st_volatile_shared(int* p, int v)
