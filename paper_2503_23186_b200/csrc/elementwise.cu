@@ -327,6 +327,283 @@ __global__ void __launch_bounds__(kEwThreads, 2) bn_bwd_apply_kernel(const void*
     }
 }
 
+// ------------------------------------------------------------------------------ BN backward, staged through shared memory
+// The same two passes fed by bulk copies: a producer thread streams chunks of every input tensor (and of the ReLU bit
+// mask) into a ring of shared-memory stages with cp.async.bulk, eight consumer warps work from shared memory.  A
+// register-staged row walk keeps two 16-byte loads per tensor and thread in flight, too few bytes to hide the DRAM
+// latency at two blocks per SM; the ring keeps kStStages x ~25 KB per block in flight and costs no registers.
+//   chunk = 2 * rows_per_iter rows = 2 vectors per active thread and tensor (about 8 KB per tensor); chunk k of a group
+//   goes to block k % gridDim.x; a ragged last chunk is read with plain loads.
+static constexpr int kStStages = 4;
+static constexpr int kStThreads = kEwThreads + 32;   // consumer warps + the producer warp
+
+struct StagedWalk {
+    int groups, rpi, active, chunk_rows, chunk_vecs, nt, mask_stride, stage_bytes;
+    long long n_full;
+    __device__ StagedWalk(int c, long long m, int n_tensors, bool has_mask)
+    {
+        groups = c >> 3;
+        rpi = kEwThreads / groups;
+        active = rpi * groups;
+        chunk_rows = 2 * rpi;
+        chunk_vecs = 2 * active;
+        nt = n_tensors;
+        mask_stride = has_mask ? ((chunk_vecs + 127) & ~127) : 0;
+        stage_bytes = nt * chunk_vecs * 16 + mask_stride;
+        n_full = m / chunk_rows;
+    }
+};
+
+// Producer side: one thread.  Returns the number of chunks it issued (for the drain after an aborted wait).
+__device__ __forceinline__ int staged_produce(const StagedWalk& sw, uint8_t* ring, uint64_t* full, uint64_t* empty, const void* t0, const void* t1,
+                                              const void* t2, const uint8_t* mask, long long base_vec, unsigned spin_limit, uint32_t* abort_flag,
+                                              unsigned* status)
+{
+    int i = 0;
+    const uint32_t tbytes = (uint32_t)sw.chunk_vecs * 16u;
+    const uint32_t tx = (uint32_t)sw.nt * tbytes + (mask != nullptr ? (uint32_t)sw.chunk_vecs : 0u);
+    for (long long k = blockIdx.x; k < sw.n_full; k += gridDim.x, ++i) {
+        const int s = i % kStStages;
+        if (!mbar_wait_bounded(&empty[s], (((uint32_t)(i / kStStages)) & 1u) ^ 1u, spin_limit, abort_flag)) {
+            atomicOr(status, B2C_DEV_TIMEOUT);
+            break;
+        }
+        uint8_t* dst = ring + (size_t)s * sw.stage_bytes;
+        const long long v0 = base_vec + k * sw.chunk_vecs;
+        mbar_expect_tx(&full[s], tx);
+        bulk_load(dst, reinterpret_cast<const uint4*>(t0) + v0, tbytes, &full[s]);
+        bulk_load(dst + tbytes, reinterpret_cast<const uint4*>(t1) + v0, tbytes, &full[s]);
+        if (sw.nt > 2) bulk_load(dst + 2 * tbytes, reinterpret_cast<const uint4*>(t2) + v0, tbytes, &full[s]);
+        if (mask != nullptr) bulk_load(dst + sw.nt * tbytes, mask + v0, (uint32_t)sw.chunk_vecs, &full[s]);
+    }
+    return i;
+}
+// After an aborted wait: the copies already issued must land before the block may exit.
+__device__ __forceinline__ void staged_drain(int issued, uint64_t* full)
+{
+    for (int back = 0; back < kStStages && back < issued; ++back) {
+        const int it = issued - 1 - back;
+        for (uint32_t i = 0; i < (1u << 22) && !mbar_try_wait(&full[it % kStStages], (uint32_t)(it / kStStages) & 1u); ++i) {}
+    }
+}
+// Consumer side of one chunk: wait (one poller per warp), then the caller reads its two vectors per tensor.
+__device__ __forceinline__ bool staged_wait(uint64_t* full, int i, int lane, unsigned spin_limit, uint32_t* abort_flag, unsigned* status)
+{
+    bool ok = true;
+    if (lane == 0) {
+        ok = mbar_wait_bounded(&full[i % kStStages], (uint32_t)(i / kStStages) & 1u, spin_limit, abort_flag);
+        if (!ok) atomicOr(status, B2C_DEV_TIMEOUT);
+    }
+    return __all_sync(0xffffffffu, ok);
+}
+__device__ __forceinline__ void staged_release(uint64_t* empty, int i, int lane)
+{
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&empty[i % kStStages]);
+}
+__device__ __forceinline__ void staged_init(uint64_t* full, uint64_t* empty, uint32_t* abort_flag)
+{
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStStages; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], kEwThreads / 32);
+        }
+        *abort_flag = 0;
+        fence_mbar_init();
+    }
+}
+
+__global__ void __launch_bounds__(kStThreads, 2) bn_bwd_reduce_staged_kernel(const void* __restrict__ da1, const void* __restrict__ da2,
+                                                                             const void* __restrict__ y, long long m, int c, int relu,
+                                                                             double* __restrict__ sums_all, const uint8_t* __restrict__ relu_mask,
+                                                                             unsigned spin_limit, unsigned* status)
+{
+    extern __shared__ uint8_t st_raw[];
+    __shared__ uint64_t full[kStStages], empty[kStStages];
+    __shared__ uint32_t abort_flag;
+    uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(st_raw) + 127u) & ~uintptr_t(127));
+    const StagedWalk sw(c, m, da2 != nullptr ? 3 : 2, relu != 0);
+    float* s_acc = reinterpret_cast<float*>(ring + (size_t)kStStages * sw.stage_bytes);
+    for (int i = threadIdx.x; i < 2 * c; i += kStThreads) s_acc[i] = 0.f;
+    staged_init(full, empty, &abort_flag);
+    __syncthreads();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long base = (long long)blockIdx.y * m * sw.groups;
+    const uint8_t* mask = relu ? relu_mask : nullptr;
+    int issued = 0;
+    if (warp == kEwThreads / 32) {
+        if (lane == 0) issued = staged_produce(sw, ring, full, empty, da1, y, da2, mask, base, spin_limit, &abort_flag, status);
+    } else {
+        const int g = threadIdx.x % sw.groups;
+        const bool act = threadIdx.x < sw.active;
+        const uint32_t tbytes = (uint32_t)sw.chunk_vecs * 16u;
+        float sb[8], sg[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) sb[i] = sg[i] = 0.f;
+        auto accumulate = [&](const uint4& v1, const uint4& vy, const uint4& v2, bool two, unsigned mk) {
+            float d[8], d2[8], fy[8];
+            unpack8(v1, d);
+            if (two) unpack8(v2, d2);
+            unpack8(vy, fy);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                float dz = d[i];
+                if (two) dz += d2[i];
+                if (!((mk >> i) & 1u)) dz = 0.f;
+                sb[i] += dz;
+                sg[i] = fmaf(dz, fy[i], sg[i]);
+            }
+        };
+        int i = 0;
+        bool ok = true;
+        for (long long k = blockIdx.x; k < sw.n_full; k += gridDim.x, ++i) {
+            ok = staged_wait(full, i, lane, spin_limit, &abort_flag, status);
+            if (!ok) break;
+            if (act) {
+                const uint8_t* st = ring + (size_t)(i % kStStages) * sw.stage_bytes;
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int v = u * sw.active + threadIdx.x;
+                    const uint4 v1 = reinterpret_cast<const uint4*>(st)[v];
+                    const uint4 vy = reinterpret_cast<const uint4*>(st + tbytes)[v];
+                    uint4 v2 = make_uint4(0u, 0u, 0u, 0u);
+                    if (sw.nt > 2) v2 = reinterpret_cast<const uint4*>(st + 2 * tbytes)[v];
+                    const unsigned mk = mask != nullptr ? (unsigned)st[sw.nt * tbytes + v] : 0xffu;
+                    accumulate(v1, vy, v2, sw.nt > 2, mk);
+                }
+            }
+            staged_release(empty, i, lane);
+        }
+        // ragged tail of the group: plain loads, by the block whose turn it would be
+        if (ok && act && (long long)sw.n_full * sw.chunk_rows < m && (sw.n_full % gridDim.x) == blockIdx.x) {
+            for (long long r = sw.n_full * sw.chunk_rows + threadIdx.x / sw.groups; r < m; r += sw.rpi) {
+                const long long vi = base + r * sw.groups + g;
+                const uint4 v1 = ld16(da1, vi), vy = ld16(y, vi);
+                const uint4 v2 = da2 != nullptr ? ld16(da2, vi) : make_uint4(0u, 0u, 0u, 0u);
+                const unsigned mk = mask != nullptr ? (unsigned)__ldg(mask + vi) : 0xffu;
+                accumulate(v1, vy, v2, da2 != nullptr, mk);
+            }
+        }
+        if (act) {
+#pragma unroll
+            for (int i2 = 0; i2 < 8; ++i2) {
+                atomicAdd(&s_acc[g * 8 + i2], sb[i2]);
+                atomicAdd(&s_acc[c + g * 8 + i2], sg[i2]);
+            }
+        }
+    }
+    __syncthreads();
+    if (abort_flag && warp == kEwThreads / 32 && lane == 0) staged_drain(issued, full);
+    double* out = sums_all + (size_t)blockIdx.y * 2 * c;
+    for (int i = threadIdx.x; i < 2 * c; i += kStThreads) atomicAdd(out + i, (double)s_acc[i]);
+    __syncthreads();
+}
+
+__global__ void __launch_bounds__(kStThreads, 2) bn_bwd_apply_staged_kernel(const void* __restrict__ da1, const void* __restrict__ da2,
+                                                                            const void* __restrict__ y, long long m, int c,
+                                                                            const float* __restrict__ gamma, const float* __restrict__ mean_all,
+                                                                            const float* __restrict__ invstd_all, int relu,
+                                                                            const double* __restrict__ sums_all, void* __restrict__ dy,
+                                                                            void* __restrict__ dres, float* dgamma, float* dbeta, int acc,
+                                                                            const uint8_t* __restrict__ relu_mask, unsigned spin_limit,
+                                                                            unsigned* status)
+{
+    extern __shared__ uint8_t st_raw[];
+    __shared__ uint64_t full[kStStages], empty[kStStages];
+    __shared__ uint32_t abort_flag;
+    uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(st_raw) + 127u) & ~uintptr_t(127));
+    const StagedWalk sw(c, m, da2 != nullptr ? 3 : 2, relu != 0);
+    staged_init(full, empty, &abort_flag);
+    __syncthreads();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const double* sums = sums_all + (size_t)blockIdx.y * 2 * c;
+    const float* mean = mean_all + (size_t)blockIdx.y * c;
+    const float* invstd = invstd_all + (size_t)blockIdx.y * c;
+    const long long base = (long long)blockIdx.y * m * sw.groups;
+    const uint8_t* mask = relu ? relu_mask : nullptr;
+    int issued = 0;
+    if (warp == kEwThreads / 32) {
+        if (lane == 0) issued = staged_produce(sw, ring, full, empty, da1, y, da2, mask, base, spin_limit, &abort_flag, status);
+    } else {
+        if (blockIdx.x == 0) {
+            for (int ch = threadIdx.x; ch < c; ch += kEwThreads) {
+                const double s1 = sums[ch], s2 = sums[c + ch];
+                const float db = (float)s1, dg = (float)((double)invstd[ch] * (s2 - (double)mean[ch] * s1));
+                if (gridDim.y == 1) {
+                    dbeta[ch] = acc ? dbeta[ch] + db : db;
+                    dgamma[ch] = acc ? dgamma[ch] + dg : dg;
+                } else {   // several groups add into the same gradient (always accumulating)
+                    atomicAdd(dbeta + ch, db);
+                    atomicAdd(dgamma + ch, dg);
+                }
+            }
+        }
+        const int g = threadIdx.x % sw.groups;
+        const bool act = threadIdx.x < sw.active;
+        const uint32_t tbytes = (uint32_t)sw.chunk_vecs * 16u;
+        const double inv_m = 1.0 / (double)m;
+        float mu[8], k0[8], kb[8], kg[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int ch = g * 8 + i;
+            const double s1 = sums[ch], s2 = sums[c + ch];
+            const double is = (double)invstd[ch], dgam = is * (s2 - (double)mean[ch] * s1);
+            mu[i] = mean[ch];
+            k0[i] = gamma[ch] * invstd[ch];                        // gamma*invstd
+            kb[i] = (float)(s1 * inv_m);                           // dbeta/m
+            kg[i] = (float)(dgam * inv_m * is);                    // (dgamma/m)*invstd, multiplies (y-mean)
+        }
+        auto emit = [&](const uint4& v1, const uint4& vy, const uint4& v2, bool two, unsigned mk, long long vi) {
+            float d[8], d2[8], fy[8], o[8];
+            unpack8(v1, d);
+            if (two) unpack8(v2, d2);
+            unpack8(vy, fy);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                float dz = d[i];
+                if (two) dz += d2[i];
+                if (!((mk >> i) & 1u)) dz = 0.f;
+                d[i] = dz;
+                o[i] = k0[i] * (dz - kb[i] - (fy[i] - mu[i]) * kg[i]);
+            }
+            reinterpret_cast<uint4*>(dy)[vi] = pack8(o);
+            if (dres != nullptr) reinterpret_cast<uint4*>(dres)[vi] = pack8(d);
+        };
+        int i = 0;
+        bool ok = true;
+        for (long long k = blockIdx.x; k < sw.n_full; k += gridDim.x, ++i) {
+            ok = staged_wait(full, i, lane, spin_limit, &abort_flag, status);
+            if (!ok) break;
+            if (act) {
+                const uint8_t* st = ring + (size_t)(i % kStStages) * sw.stage_bytes;
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int v = u * sw.active + threadIdx.x;
+                    const uint4 v1 = reinterpret_cast<const uint4*>(st)[v];
+                    const uint4 vy = reinterpret_cast<const uint4*>(st + tbytes)[v];
+                    uint4 v2 = make_uint4(0u, 0u, 0u, 0u);
+                    if (sw.nt > 2) v2 = reinterpret_cast<const uint4*>(st + 2 * tbytes)[v];
+                    const unsigned mk = mask != nullptr ? (unsigned)st[sw.nt * tbytes + v] : 0xffu;
+                    emit(v1, vy, v2, sw.nt > 2, mk, base + k * sw.chunk_vecs + v);
+                }
+            }
+            staged_release(empty, i, lane);
+        }
+        if (ok && act && (long long)sw.n_full * sw.chunk_rows < m && (sw.n_full % gridDim.x) == blockIdx.x) {
+            for (long long r = sw.n_full * sw.chunk_rows + threadIdx.x / sw.groups; r < m; r += sw.rpi) {
+                const long long vi = base + r * sw.groups + g;
+                const uint4 v1 = ld16(da1, vi), vy = ld16(y, vi);
+                const uint4 v2 = da2 != nullptr ? ld16(da2, vi) : make_uint4(0u, 0u, 0u, 0u);
+                const unsigned mk = mask != nullptr ? (unsigned)__ldg(mask + vi) : 0xffu;
+                emit(v1, vy, v2, da2 != nullptr, mk, vi);
+            }
+        }
+    }
+    __syncthreads();
+    if (abort_flag && warp == kEwThreads / 32 && lane == 0) staged_drain(issued, full);
+    __syncthreads();
+}
+
 // ------------------------------------------------------------------------------ pooling, padding
 __global__ void avgpool_fwd_kernel(const void* __restrict__ a, int n, int hw, int c, void* __restrict__ pooled)
 {
@@ -559,6 +836,29 @@ b2c_status launch_bn_bwd(b2c_ctx* ctx, int G, long long m, int c, const void* da
     dim3 grid((unsigned)ew_grid(ctx, G, m, rows_per_iter), (unsigned)G);
     const uint8_t* mask = relu ? reinterpret_cast<const uint8_t*>(relu_mask) : nullptr;
     if (!sums_zeroed) B2C_CUDA(cudaMemsetAsync(sums, 0, sizeof(double) * 2 * c * G, stream));
+    // The staged kernels need the ReLU mask (not the activation), chunk offsets that keep the mask copies 16-byte
+    // aligned, and at least one full chunk per block to be worth their set-up.
+    const int groups = c / 8, active = rows_per_iter * groups, chunk_vecs = 2 * active;
+    const bool staged = (!relu || mask != nullptr) && chunk_vecs % 16 == 0 && (m * groups) % 16 == 0 && m >= 2ll * rows_per_iter * grid.x &&
+                        reinterpret_cast<uintptr_t>(mask) % 16 == 0;
+    if (staged) {
+        static bool attr_set = false;
+        const int nt = da2 != nullptr ? 3 : 2;
+        const size_t stage = (size_t)nt * chunk_vecs * 16 + (relu ? ((chunk_vecs + 127) & ~127) : 0);
+        const size_t smem = kStStages * stage + sizeof(float) * 2 * c + 128;
+        if (smem <= 110 * 1024) {
+            if (!attr_set) {
+                B2C_CUDA(cudaFuncSetAttribute(bn_bwd_reduce_staged_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024));
+                B2C_CUDA(cudaFuncSetAttribute(bn_bwd_apply_staged_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024));
+                attr_set = true;
+            }
+            bn_bwd_reduce_staged_kernel<<<grid, kStThreads, smem, stream>>>(da1, da2, y, m, c, relu, sums, mask, ctx->spin_limit, ctx->d_status);
+            bn_bwd_apply_staged_kernel<<<grid, kStThreads, smem, stream>>>(da1, da2, y, m, c, gamma, save_mean, save_invstd, relu, sums, dy, dres,
+                                                                            dgamma, dbeta, acc, mask, ctx->spin_limit, ctx->d_status);
+            B2C_CUDA(cudaGetLastError());
+            return B2C_OK;
+        }
+    }
     bn_bwd_reduce_kernel<<<grid, kEwThreads, sizeof(float) * 2 * c, stream>>>(da1, da2, y, a, m, c, relu, sums, mask);
     bn_bwd_apply_kernel<<<grid, kEwThreads, 0, stream>>>(da1, da2, y, a, m, c, gamma, save_mean, save_invstd, relu, sums, dy, dres, dgamma, dbeta,
                                                          acc, mask);
