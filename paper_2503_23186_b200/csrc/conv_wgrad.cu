@@ -50,9 +50,9 @@ struct alignas(64) WgradParams {
 };
 
 static constexpr int kWgStages = 6;
-static constexpr int kWgProducers = 2;   // warp 0 and the warp after the epilogue warps; they fill alternate ring slots
+static constexpr int kWgProducers = 3;   // warp 0 and the warps after the epilogue warps; producer w fills ring slots w, w + 3, ...
 static constexpr int kWgProducerWarp1 = 6;
-static constexpr int kWgThreads = 224;
+static constexpr int kWgThreads = 256;
 static constexpr uint32_t kWgDrainPolls = 1u << 22;
 
 __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d)
@@ -116,11 +116,11 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
     const uint32_t tmem_base = tmem_slot;
     int last_issued = -1;  // producer lanes: last chunk whose loads this lane issued
 
-    if (warp == 0 || warp == kWgProducerWarp1) {
-        if (lane == 0) {
-            // Producer w fills the ring slots w, w + 2, ...: one thread's wait -> expect -> issue chain is longer than
-            // the MMAs of a stage take.  Each slot keeps one producer, which uses it strictly in order.
-            const int w = warp == 0 ? 0 : 1;
+    if (warp == 0 || warp >= kWgProducerWarp1) {
+        const int w = warp == 0 ? 0 : warp - kWgProducerWarp1 + 1;
+        if (lane == 0 && w < S) {
+            // Producer w fills the ring slots w, w + kWgProducers, ...: one thread's wait -> expect -> issue chain is
+            // longer than the MMAs of a stage take.  Each slot keeps one producer, which uses it strictly in order.
             prefetch_tensormap(&p.tmDy);
             prefetch_tensormap(&p.tmX[0]);
             const uint32_t tx = (uint32_t)(p.a_bytes + grp.nb * p.b_boxes * p.box_b);
@@ -262,8 +262,8 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
     __syncthreads();
     if (abort_flag) {
         // A wait gave up: let the issued bulk copies land and the issued MMAs retire before exit.
-        if ((warp == 0 || warp == kWgProducerWarp1) && lane == 0) {
-            const int w = warp == 0 ? 0 : 1;
+        if ((warp == 0 || warp >= kWgProducerWarp1) && lane == 0) {
+            const int w = warp == 0 ? 0 : warp - kWgProducerWarp1 + 1;
             for (int sl = w; sl < S; sl += kWgProducers) {   // the last chunk issued into each of the own slots
                 if (last_issued < sl) continue;
                 const int it = last_issued - ((last_issued - sl) % S);
