@@ -30,6 +30,10 @@ b2c_status b2c_create(b2c_ctx** out, int device)
         const char* env = std::getenv("B2C_CTA_PAIRS");
         ctx->use_pairs = env ? (env[0] == '2' ? 2 : env[0] == '1' ? 1 : 0) : 1;   // 0 never, 1 for 128-channel tiles (default), 2 wherever possible
     }
+    {
+        const char* env = std::getenv("B2C_FULL_HALO");
+        ctx->use_full_halo = env ? (env[0] != '0') : 1;
+    }
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || fn == nullptr ||

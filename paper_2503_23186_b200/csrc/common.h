@@ -21,6 +21,7 @@ struct b2c_ctx {
     unsigned* d_status;  // one device word
     unsigned spin_limit;
     b2c_encode_tiled_fn encode_tiled;
+    int use_full_halo;                   // 3x3 stride-1 convolutions with a resident filter bank stage one framed tile for all nine taps
     int use_pairs;                       // forward / data-gradient convolutions may run on CTA pairs (cta_group::2)
     unsigned long long* stall_counters;  // optional device array the convolution kernels add their wait cycles to
 };

@@ -42,6 +42,7 @@ struct alignas(64) ConvKParams {
     int tmem_cols, acc_cols;         // allocation, columns per accumulator
     int acc_bufs, acc_shift;         // accumulators in TMEM (2 or 4) and log2 of that: unit j uses accumulator j % acc_bufs
     int vreuse;                      // a stage serves the three vertical taps of one horizontal shift
+    int fh;                          // full halo: a stage holds the tile with a one-pixel frame and serves all nine taps
     int nb;                          // B tiles per stage (1, or 3 with vreuse)
     int b_merged;                    // the three B tiles of a stage come with one load (box of three filter rows)
     int r_filter;                    // filter height = width
@@ -120,6 +121,7 @@ struct UnitWalk {
 __device__ __forceinline__ int unit_iters(const ConvKParams& p, int par)
 {
     const int taps = p.taps[par].count;
+    if (p.fh) return p.c_blocks;
     return (p.vreuse ? taps / 3 : taps) * p.c_blocks;
 }
 
@@ -387,6 +389,32 @@ __device__ __forceinline__ void issue_stage(uint32_t d_tmem, uint32_t a_lo, uint
     }
 }
 
+// Full-halo stage: the A tile is a box of (bw + 2) x (bh + 2) pixels with bw = 8, so every image row of the tile is
+// one 8-row group of the K-major operand and the group stride (SBO) is bw + 2 rows.  Tap (r, s) reads the same box
+// starting r image rows and s pixels further in: a start address that is a whole number of 128-byte rows off the
+// swizzle atom, which works because the swizzle is keyed on absolute shared-memory address bits (measured: exact
+// results for arbitrary row offsets and group strides).  B tiles come from the resident bank, order [s][cb][r].
+template <int KS, bool PAIR>
+__device__ __forceinline__ void issue_stage_fh(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t a_hi, uint32_t b_hi, uint32_t idesc,
+                                               uint32_t a_row16, uint32_t a_rowpitch16, uint32_t b_tile16, uint32_t b_s16,
+                                               uint32_t accumulate_first)
+{
+#pragma unroll
+    for (int sft = 0; sft < 3; ++sft) {
+#pragma unroll
+        for (int r = 0; r < 3; ++r) {
+#pragma unroll
+            for (int k = 0; k < KS; ++k) {
+                const uint64_t ad = ((uint64_t)a_hi << 32) | (uint64_t)(a_lo + (uint32_t)r * a_rowpitch16 + (uint32_t)sft * a_row16 + 2u * k);
+                const uint64_t bd = ((uint64_t)b_hi << 32) | (uint64_t)(b_lo + (uint32_t)sft * b_s16 + (uint32_t)r * b_tile16 + 2u * k);
+                const uint32_t acc = (sft == 0 && r == 0 && k == 0) ? accumulate_first : 1u;
+                if constexpr (PAIR) umma_bf16_pair(d_tmem, ad, bd, idesc, acc);
+                else umma_bf16(d_tmem, ad, bd, idesc, acc);
+            }
+        }
+    }
+}
+
 // One MMA-issuing thread.  The CTA runs kIssuers of them (in different warps): issuer `my` accumulates the CTA's units
 // my, my + kIssuers, ... (unit j always into accumulator j % acc_bufs) and steps over the ring stages of the others.  A single
 // thread cannot keep the tensor pipe busy on narrow tiles: it pays roughly 45 cycles per tcgen05.mma, 180 per barrier
@@ -401,6 +429,10 @@ __device__ __forceinline__ void mma_issuer(const ConvKParams& p, const UnitWalk&
     const uint32_t sbo = 8u * (uint32_t)p.kb * 2u;  // eight rows of kb bf16
     const uint64_t desc_proto = make_smem_desc(0u, 16u, sbo, (uint32_t)p.swz);
     const uint32_t desc_hi = (uint32_t)(desc_proto >> 32), desc_lo_base = (uint32_t)desc_proto;
+    // full halo: A groups are (bw + 2) rows apart
+    const uint32_t a_hi_fh = (uint32_t)(make_smem_desc(0u, 16u, (uint32_t)(p.bw + 2) * (uint32_t)p.kb * 2u, (uint32_t)p.swz) >> 32);
+    const uint32_t a_row16 = ((uint32_t)p.kb * 2u) >> 4, a_rowpitch16 = (uint32_t)(p.bw + 2) * a_row16;
+    const uint32_t b_s16 = (uint32_t)(p.c_blocks * 3 * p.b_bytes) >> 4;
     const uint32_t a_to_b16 = (uint32_t)p.a_bytes >> 4, a_step16 = (uint32_t)p.a_step >> 4;
     // B tiles of consecutive vertical taps are adjacent, in a stage and in the resident bank alike
     const uint32_t b_step16 = (uint32_t)p.b_bytes >> 4;
@@ -466,7 +498,8 @@ __device__ __forceinline__ void mma_issuer(const ConvKParams& p, const UnitWalk&
             // descriptors differ from stage to stage only in the 14-bit address field: add offsets to the low word
             const uint32_t a_lo = ring_lo + (uint32_t)s * stage16;
             const uint32_t b_lo = p.resident ? b_res : a_lo + a_to_b16;
-            issue_stage<KS, NB, PAIR>(d_tmem, a_lo, b_lo, desc_hi, idesc, a_step16, b_step16, it != 0 ? 1u : 0u);
+            if (p.fh) issue_stage_fh<KS, PAIR>(d_tmem, a_lo, b_lo, a_hi_fh, desc_hi, idesc, a_row16, a_rowpitch16, b_step16, b_s16, it != 0 ? 1u : 0u);
+            else issue_stage<KS, NB, PAIR>(d_tmem, a_lo, b_lo, desc_hi, idesc, a_step16, b_step16, it != 0 ? 1u : 0u);
             b_res += b_cb16;
             // frees the stage (in both CTAs of a pair) once these MMAs have read it
             if constexpr (PAIR) umma_commit_pair(&empty_bar[s], (uint16_t)3);
@@ -554,7 +587,7 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
                 const TapList& tl = p.taps[0];
                 const int oc0 = ktile * p.n_tile + rank * b_rows;
                 if (rank == 0) mbar_expect_tx(&w_bar, (uint32_t)((PAIR ? 2 : 1) * tl.count * p.c_blocks * p.tx_b));
-                const int groups = p.vreuse ? tl.count / 3 : tl.count;
+                const int groups = (p.vreuse || p.fh) ? tl.count / 3 : tl.count;
                 for (int t = 0; t < groups; ++t)
                     for (int cb = 0; cb < p.c_blocks; ++cb) {
                         uint8_t* dst = smem + (size_t)(t * p.c_blocks + cb) * p.nb * p.b_bytes;
@@ -596,8 +629,9 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
                     // The previous stage in this slot has been consumed, so its barrier phase is over: the stamp lets the
                     // issuers tell this slot's phases apart (a relaxed store: the wait above orders it).
                     if (p.issuers > 1) st_volatile_shared(&slot_stage[s], i + 1);
-                    const int t0 = p.cb_shift >= 0 ? it >> p.cb_shift : it / p.c_blocks;   // tap (or horizontal shift)
-                    const int cb = it - t0 * p.c_blocks;                                     // channel block
+                    int t0 = p.cb_shift >= 0 ? it >> p.cb_shift : it / p.c_blocks;   // tap (or horizontal shift)
+                    const int cb = it - t0 * p.c_blocks;                               // channel block
+                    if (p.fh) t0 = 0;   // one framed box per channel block: the entry of tap (0, 0) carries its origin
                     uint8_t* a_dst = ring + (size_t)s * stage_bytes;
                     // with vreuse the table entry of vertical tap 0 carries the shift of the whole haloed tile
                     if constexpr (PAIR) {
@@ -813,6 +847,11 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
     const int grid = p.pair ? 2 * walkers : walkers;
     const int units_per_cta = (walk_units + walkers - 1) / walkers;
 
+    // Full-halo plan (3x3, stride 1, 64-channel k-blocks, images of at least 8 x 16 pixels, filter bank resident): tiles
+    // of 8 x 16 pixels, one framed box per channel block serves all nine taps, so the input crosses L2 -> SM once
+    // (three times with vertical tap reuse, nine without) and a ring slot holds a whole channel block of a unit.
+    const bool fh_ok = R == 3 && pb.stride == 1 && n_par == 1 && pb.ic % 64 == 0 && gw >= 8 && gh >= 16 && !p.pair && ctx->use_full_halo &&
+                       9 * (pb.ic / 64) * (((n_tile * 64 * 2) + 1023) & ~1023) <= 96 * 1024;
     // shared-memory plan.  Preference: haloed stages (vertical tap reuse) with 64-channel k-blocks, then with
     // 32-channel k-blocks (smaller stages, so that a ring of at least four still fits), else one tap per stage.
     const int ring_budget = 210 * 1024;
@@ -820,7 +859,24 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
     const bool can_vreuse = (R == 3 && pb.stride == 1 && p.bn == 1);
     const int taps_total = R * R;
     const int attempts[3][2] = {{kb_natural, 1}, {32, 1}, {kb_natural, 0}};   // (kb, vreuse)
-    for (int a = 0; a < 3; ++a) {
+    bool planned = false;
+    if (fh_ok && units_per_cta >= 2) {
+        const int tx_b = b_rows * 64 * 2, bank = taps_total * (pb.ic / 64) * tx_b, a_bytes = ((10 * 18 * 128) + 1023) & ~1023;
+        int stages = (ring_budget - bank) / a_bytes;
+        if (stages > kMaxStages) stages = kMaxStages;
+        if (stages >= 3) {
+            p.bw = 8; p.bh = 16; p.bn = 1;
+            p.tiles_w = gw / 8; p.tiles_h = gh / 16; p.tiles_n = pb.n;
+            p.fh = 1; p.vreuse = 0;
+            p.kb = 64; p.c_blocks = pb.ic / 64; p.swz = SWZ_128B;
+            p.tx_b = tx_b; p.b_bytes = tx_b; p.b_merged = 1; p.nb = 3;   // bank order [s][cb][r], three filter rows per load
+            p.tx_a = 10 * 18 * 128; p.a_bytes = a_bytes; p.a_step = 0;
+            p.resident = 1; p.resident_bytes = bank;
+            p.stages = stages;
+            planned = true;
+        }
+    }
+    for (int a = 0; a < 3 && !planned; ++a) {
         const int kb = attempts[a][0], vr = attempts[a][1];
         if (vr && !can_vreuse) continue;
         if (kb > kb_natural) continue;
@@ -854,14 +910,15 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
     const size_t smem_bytes = (size_t)p.resident_bytes + (size_t)p.stages * stage_bytes + 1024;
 
     // tensor maps
-    const int box_h = p.vreuse ? p.bh + 2 : p.bh;
+    const int box_h = (p.vreuse || p.fh) ? p.bh + 2 : p.bh;
+    const int box_w = p.fh ? p.bw + 2 : p.bw;
     if (!pb.dgrad && pb.stride == 2) {
         for (int ph = 0; ph < 2; ++ph)
             for (int pw = 0; pw < 2; ++pw)
-                if (!encode_activation_map(ctx, &p.tmA[ph * 2 + pw], pb.in, pb.n, pb.ih, pb.iw, pb.ic, 2, ph, pw, p.kb, p.bw, box_h, p.bn))
+                if (!encode_activation_map(ctx, &p.tmA[ph * 2 + pw], pb.in, pb.n, pb.ih, pb.iw, pb.ic, 2, ph, pw, p.kb, box_w, box_h, p.bn))
                     return B2C_ERR_CUDA;
     } else {
-        if (!encode_activation_map(ctx, &p.tmA[0], pb.in, pb.n, pb.ih, pb.iw, pb.ic, 1, 0, 0, p.kb, p.bw, box_h, p.bn)) return B2C_ERR_CUDA;
+        if (!encode_activation_map(ctx, &p.tmA[0], pb.in, pb.n, pb.ih, pb.iw, pb.ic, 1, 0, 0, p.kb, box_w, box_h, p.bn)) return B2C_ERR_CUDA;
     }
     {
         // weights [out][r][s][in] viewed as (in, s, out, r): a box of three filter rows lands as three tiles [r][out][in]
