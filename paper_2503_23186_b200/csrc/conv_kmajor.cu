@@ -301,7 +301,7 @@ __device__ __forceinline__ void epilogue_loop(const ConvKParams& p, uint32_t tme
                 if (ck < n_chunks) {
                     uint32_t pk[8];
                     store_chunk(r[ck], ck * 16, pk);
-                    if (row_valid) {   // sums of the values as stored, kept per row in registers
+                    if (do_stats && row_valid) {   // sums of the values as stored, kept per row in registers
 #pragma unroll
                         for (int i = 0; i < 8; ++i) {
                             __nv_bfloat162 h = *reinterpret_cast<__nv_bfloat162*>(&pk[i]);
@@ -690,9 +690,9 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
     } else {
         // ---------------------------------------------------------------- epilogue (8 warps)
         const int e = warp - 2;
-        if (p.stats != nullptr && p.n_tile <= 32)
+        if (p.n_tile <= 32 && !p.out_is_f32)
             epilogue_loop<1>(p, tmem_base, acc_full, acc_empty, &abort_flag, s_stats[e], e, lane, rank);
-        else if (p.stats != nullptr && p.n_tile <= 64)
+        else if (p.n_tile <= 64 && !p.out_is_f32)
             epilogue_loop<2>(p, tmem_base, acc_full, acc_empty, &abort_flag, s_stats[e], e, lane, rank);
         else
             epilogue_loop<0>(p, tmem_base, acc_full, acc_empty, &abort_flag, s_stats[e], e, lane, rank);
