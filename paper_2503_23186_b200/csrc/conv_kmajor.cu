@@ -850,8 +850,8 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
     // Full-halo plan (3x3, stride 1, 64-channel k-blocks, images of at least 8 x 16 pixels, filter bank resident): tiles
     // of 8 x 16 pixels, one framed box per channel block serves all nine taps, so the input crosses L2 -> SM once
     // (three times with vertical tap reuse, nine without) and a ring slot holds a whole channel block of a unit.
-    const bool fh_ok = R == 3 && pb.stride == 1 && n_par == 1 && pb.ic % 64 == 0 && gw >= 8 && gh >= 16 && !p.pair && ctx->use_full_halo &&
-                       9 * (pb.ic / 64) * (((n_tile * 64 * 2) + 1023) & ~1023) <= 96 * 1024;
+    const bool fh_ok = R == 3 && pb.stride == 1 && n_par == 1 && pb.ic % 64 == 0 && gw >= 8 && gh >= 16 && ctx->use_full_halo &&
+                       9 * (pb.ic / 64) * b_rows * 64 * 2 <= (p.pair ? 148 : 96) * 1024;
     // shared-memory plan.  Preference: haloed stages (vertical tap reuse) with 64-channel k-blocks, then with
     // 32-channel k-blocks (smaller stages, so that a ring of at least four still fits), else one tap per stage.
     const int ring_budget = 210 * 1024;
@@ -864,7 +864,7 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
         const int tx_b = b_rows * 64 * 2, bank = taps_total * (pb.ic / 64) * tx_b, a_bytes = ((10 * 18 * 128) + 1023) & ~1023;
         int stages = (ring_budget - bank) / a_bytes;
         if (stages > kMaxStages) stages = kMaxStages;
-        if (stages >= 3) {
+        if (stages >= (p.pair ? 2 : 3)) {
             p.bw = 8; p.bh = 16; p.bn = 1;
             p.tiles_w = gw / 8; p.tiles_h = gh / 16; p.tiles_n = pb.n;
             p.fh = 1; p.vreuse = 0;
