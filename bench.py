@@ -42,6 +42,11 @@ FALLBACK_BF16_TFLOPS, FALLBACK_HBM_GBS = 1590.0, 6650.0
 # ------------------------------------------------------------------------------------------------
 # algorithmic work of one micro-batch (what the method must do; padding and halos not counted)
 # ------------------------------------------------------------------------------------------------
+# DRAM traffic of conv_kmajor_kernel from one ncu capture of all its launches in one step of the named workload
+# (profiles/conv_kmajor_resnet18_b1024.md); None for workloads that were not captured.
+KMAJOR_DRAM_BYTES_PER_LAUNCH = {"resnet18_cifar_b1024_8x128": 91.08e6}
+
+
 def algorithmic_work(spec, n):
     """Returns dict family -> (flops, bytes) for one micro-batch of n images."""
     w = {k: [0.0, 0.0] for k in ("conv_fwd", "conv_dgrad", "conv_wgrad", "bn_fwd", "bn_bwd", "update")}
@@ -283,9 +288,13 @@ def run_b2c(args, spec, name, micro_batch, n_micro):
     km_ms = fam_ms["conv_fwd"] + fam_ms["conv_dgrad"]
     km_flops = (work["conv_fwd"][0] + work["conv_dgrad"][0]) * reps
     km_tf = km_flops / (km_ms * 1e-3) / 1e12 if km_ms > 0 else None
+    km_launches = fam_launches["conv_fwd"] + fam_launches["conv_dgrad"]
+    km_bytes = (work["conv_fwd"][1] + work["conv_dgrad"][1]) * reps
     roofline = {"kernel": "conv_kmajor_kernel (forward + data-gradient launches)", "bound": "tensor", "achieved": km_tf,
                 "peak": peaks["bf16"], "unit": "TFLOP/s", "frac": km_tf / peaks["bf16"] if km_tf else None,
-                "peak_source": f"{peaks['source']} (sustained bf16 GEMM; kernel timed inside a long step)", "traffic": None,
+                "peak_source": f"{peaks['source']} (sustained bf16 GEMM; kernel timed inside a long step)", "traffic": KMAJOR_DRAM_BYTES_PER_LAUNCH.get(name),
+                "traffic_unit": "bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum, mean over the kernel's launches of one step)",
+                "algorithmic_bytes_per_launch": km_bytes / km_launches if km_launches else None,
                 "all_conv_tflops": conv_tf, "all_conv_frac_of_measured": conv_tf / peaks["bf16"] if conv_tf else None,
                 "all_conv_frac_of_nominal": conv_tf / NOMINAL_BF16_TFLOPS if conv_tf else None}
     sample = 32
