@@ -150,7 +150,9 @@ def test_conv_rejects_bad_arguments(ctx):
 
 
 # ------------------------------------------------------------------------------ BatchNorm
-BN_SHAPES = [(8, 32, 32, 64), (3, 8, 8, 160), (128, 4, 4, 512), (5, 16, 16, 8), (2, 16, 16, 640)]
+# the last two are large enough for the bulk-copy ring of the backward kernels (with a ragged last chunk; 160 channels
+# leave 16 threads of a block without a channel group)
+BN_SHAPES = [(8, 32, 32, 64), (3, 8, 8, 160), (128, 4, 4, 512), (5, 16, 16, 8), (2, 16, 16, 640), (33, 31, 32, 64), (20, 32, 33, 160)]
 
 
 @pytest.mark.parametrize("shape", BN_SHAPES, ids=lambda s: "x".join(map(str, s)))
@@ -341,6 +343,34 @@ def test_bounded_wait_reports_timeout(ctx):
     ctx.conv2d_fwd(_desc(*shape), dev_bf16(x), dev_bf16(w), y)
     assert ctx.device_status() == 0
     assert_close(y, oracle.conv2d_fwd(x, w, 1, 1), "y after recovery")
+
+
+@pytest.mark.parametrize("mode", ["0", "1"])
+def test_conv_full_halo_on_and_off(mode, monkeypatch):
+    """3x3 stride-1 layers large enough for full-halo stages (one framed 8x16 tile per channel block serves all nine
+    taps; single CTAs at 64 channels, CTA pairs at 128), with the mode switched off and on: same results."""
+    from paper_2503_23186_b200 import binding
+    monkeypatch.setenv("B2C_FULL_HALO", mode)
+    c = binding.Context(0)
+    try:
+        for shape in [(64, 32, 32, 64, 64, 3, 1), (160, 16, 16, 128, 128, 3, 1), (40, 16, 32, 64, 64, 3, 1)]:
+            N, H, W, C, K, R, st = shape
+            x, w, g = wl.conv_problem(13, *shape)
+            ref = oracle.conv2d_fwd(x, w, st, 1)
+            y = torch.full(ref.shape, float("nan"), dtype=torch.bfloat16, device="cuda")
+            stats = torch.zeros(2 * K, dtype=torch.float64, device="cuda")
+            c.conv2d_fwd(_desc(*shape), dev_bf16(x), dev_bf16(w), y, ch_stats=stats)
+            assert c.device_status() == 0
+            assert_close(y, ref, f"y {shape} full_halo={mode}")
+            ys = host(y).reshape(-1, K)
+            np.testing.assert_allclose(host(stats)[:K], ys.sum(0), rtol=1e-5, atol=1e-3 * np.sqrt(ys.shape[0]))
+            np.testing.assert_allclose(host(stats)[K:], (ys * ys).sum(0), rtol=1e-4)
+            dx = torch.full(x.shape, float("nan"), dtype=torch.bfloat16, device="cuda")
+            c.conv2d_dgrad(_desc(*shape), dev_bf16(g), _dgrad_weights(c, w), dx)
+            assert c.device_status() == 0
+            assert_close(dx, oracle.conv2d_dgrad(g, w, x.shape, st, 1), f"dx {shape} full_halo={mode}")
+    finally:
+        c.close()
 
 
 @pytest.mark.parametrize("mode", ["0", "2"])
