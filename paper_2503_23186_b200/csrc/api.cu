@@ -34,6 +34,10 @@ b2c_status b2c_create(b2c_ctx** out, int device)
         const char* env = std::getenv("B2C_FULL_HALO");
         ctx->use_full_halo = env ? (env[0] != '0') : 1;
     }
+    {
+        const char* env = std::getenv("B2C_PDL");
+        ctx->use_pdl = env ? (env[0] != '0') : 1;
+    }
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || fn == nullptr ||

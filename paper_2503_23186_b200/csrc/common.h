@@ -24,6 +24,7 @@ struct b2c_ctx {
     int use_full_halo;                   // 3x3 stride-1 convolutions with a resident filter bank stage one framed tile for all nine taps
     int use_pairs;                       // forward / data-gradient convolutions may run on CTA pairs (cta_group::2)
     unsigned long long* stall_counters;  // optional device array the convolution kernels add their wait cycles to
+    int use_pdl;                         // kernels are launched with programmatic stream serialization (their set-up overlaps the previous kernel's tail)
 };
 
 #define B2C_CUDA(call)                               \
@@ -31,6 +32,37 @@ struct b2c_ctx {
         cudaError_t e_ = (call);                     \
         if (e_ != cudaSuccess) return B2C_ERR_CUDA;  \
     } while (0)
+
+// Kernel launch.  With ctx->use_pdl the launch carries the programmatic-stream-serialization attribute: the kernel may be
+// scheduled while the previous kernel of the stream drains, and it orders itself behind that kernel with pdl_wait()
+// (every kernel of the library calls it before its first global access).  cluster > 1 launches thread-block clusters.
+template <typename... KArgs, typename... Args>
+static inline cudaError_t b2c_launch(const b2c_ctx* ctx, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                     unsigned cluster, Args&&... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    unsigned n = 0;
+    if (ctx->use_pdl) {
+        attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n].val.programmaticStreamSerializationAllowed = 1;
+        ++n;
+    }
+    if (cluster > 1) {
+        attr[n].id = cudaLaunchAttributeClusterDimension;
+        attr[n].val.clusterDim.x = cluster;
+        attr[n].val.clusterDim.y = 1;
+        attr[n].val.clusterDim.z = 1;
+        ++n;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = n;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
 
 static inline bool b2c_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 static inline bool b2c_is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }

@@ -564,6 +564,9 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
     if constexpr (PAIR) cluster_sync_all();   // the peer's barriers exist before anything arrives on them
     tc_fence_after();
     const uint32_t tmem_base = tmem_slot;
+    // set-up done (it touched no global data): order behind the previous kernel of the stream, then let the next one in
+    pdl_wait();
+    pdl_launch_dependents();
     const long long t_start = clock64();
     const UnitWalk walk(p, rank);
     int last_issued = -1;  // producer lanes: index of the last stage whose loads this lane issued
@@ -982,23 +985,8 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
         B2C_CUDA(cudaFuncSetAttribute(conv_kmajor_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 212 * 1024));
         attr_set = true;
     }
-    if (p.pair) {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)grid);
-        cfg.blockDim = dim3(kThreads);
-        cfg.dynamicSmemBytes = smem_bytes;
-        cfg.stream = stream;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = 2;
-        attr[0].val.clusterDim.y = 1;
-        attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        B2C_CUDA(cudaLaunchKernelEx(&cfg, conv_kmajor_kernel<true>, p));
-    } else {
-        conv_kmajor_kernel<false><<<grid, kThreads, smem_bytes, stream>>>(p);
-    }
+    if (p.pair) B2C_CUDA(b2c_launch(ctx, conv_kmajor_kernel<true>, dim3((unsigned)grid), dim3(kThreads), smem_bytes, stream, 2u, p));
+    else B2C_CUDA(b2c_launch(ctx, conv_kmajor_kernel<false>, dim3((unsigned)grid), dim3(kThreads), smem_bytes, stream, 1u, p));
     B2C_CUDA(cudaGetLastError());
     return B2C_OK;
 }

@@ -114,6 +114,9 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_slot;
+    // set-up done (it touched no global data): order behind the previous kernel of the stream, then let the next one in
+    pdl_wait();
+    pdl_launch_dependents();
     int last_issued = -1;  // producer lanes: last chunk whose loads this lane issued
 
     if (warp == 0 || warp >= kWgProducerWarp1) {
@@ -408,7 +411,7 @@ b2c_status launch_conv_wgrad(b2c_ctx* ctx, const WgradProblem& pb, cudaStream_t 
     }
     const size_t smem_bytes = (size_t)p.stages * p.stage_bytes + 1024;
     dim3 grid((unsigned)(base * n_splits));
-    conv_wgrad_kernel<<<grid, kWgThreads, smem_bytes, stream>>>(p);
+    B2C_CUDA(b2c_launch(ctx, conv_wgrad_kernel, grid, dim3(kWgThreads), smem_bytes, stream, 1u, p));
     B2C_CUDA(cudaGetLastError());
     return B2C_OK;
 }

@@ -51,6 +51,8 @@ __device__ __forceinline__ uint4 ld16_or_zero(const void* base, long long vec_in
 // ------------------------------------------------------------------------------ BN forward
 __global__ void __launch_bounds__(kEwThreads, 2) bn_stats_kernel(const void* __restrict__ y, long long m, int c, double* __restrict__ stats)
 {
+    pdl_wait();   // first global access comes after the previous kernel of the stream
+    pdl_launch_dependents();
     extern __shared__ float s_acc[];  // [2*c]
     for (int i = threadIdx.x; i < 2 * c; i += kEwThreads) s_acc[i] = 0.f;
     __syncthreads();
@@ -105,6 +107,8 @@ __global__ void __launch_bounds__(kEwThreads, 2) bn_apply_kernel(const void* __r
                                                                  float* save_mean, float* save_invstd, float* run_mean, float* run_var,
                                                                  float momentum, uint8_t* __restrict__ relu_mask)
 {
+    pdl_wait();   // first global access comes after the previous kernel of the stream
+    pdl_launch_dependents();
     const RowWalk rw(c);
     const int g = threadIdx.x % rw.groups, rl = threadIdx.x / rw.groups;
     const double inv_m = 1.0 / (double)m;
@@ -177,6 +181,8 @@ __global__ void __launch_bounds__(kEwThreads, 2) bn_bwd_reduce_kernel(const void
                                                                       int relu, double* __restrict__ sums_all /* [G][2c] */,
                                                                       const uint8_t* __restrict__ relu_mask)
 {
+    pdl_wait();   // first global access comes after the previous kernel of the stream
+    pdl_launch_dependents();
     extern __shared__ float s_acc[];
     for (int i = threadIdx.x; i < 2 * c; i += kEwThreads) s_acc[i] = 0.f;
     __syncthreads();
@@ -248,6 +254,8 @@ __global__ void __launch_bounds__(kEwThreads, 2) bn_bwd_apply_kernel(const void*
                                                                      void* __restrict__ dres, float* dgamma, float* dbeta, int acc,
                                                                      const uint8_t* __restrict__ relu_mask)
 {
+    pdl_wait();   // first global access comes after the previous kernel of the stream
+    pdl_launch_dependents();
     const RowWalk rw(c);
     const int g = threadIdx.x % rw.groups, rl = threadIdx.x / rw.groups;
     const double* sums = sums_all + (size_t)blockIdx.y * 2 * c;
@@ -418,6 +426,8 @@ __global__ void __launch_bounds__(kStThreads, 2) bn_bwd_reduce_staged_kernel(con
                                                                              double* __restrict__ sums_all, const uint8_t* __restrict__ relu_mask,
                                                                              unsigned spin_limit, unsigned* status)
 {
+    pdl_wait();   // first global access comes after the previous kernel of the stream
+    pdl_launch_dependents();
     extern __shared__ uint8_t st_raw[];
     __shared__ uint64_t full[kStStages], empty[kStStages];
     __shared__ uint32_t abort_flag;
@@ -508,6 +518,8 @@ __global__ void __launch_bounds__(kStThreads, 2) bn_bwd_apply_staged_kernel(cons
                                                                             const uint8_t* __restrict__ relu_mask, unsigned spin_limit,
                                                                             unsigned* status)
 {
+    pdl_wait();   // first global access comes after the previous kernel of the stream
+    pdl_launch_dependents();
     extern __shared__ uint8_t st_raw[];
     __shared__ uint64_t full[kStStages], empty[kStStages];
     __shared__ uint32_t abort_flag;
@@ -607,6 +619,8 @@ __global__ void __launch_bounds__(kStThreads, 2) bn_bwd_apply_staged_kernel(cons
 // ------------------------------------------------------------------------------ pooling, padding
 __global__ void avgpool_fwd_kernel(const void* __restrict__ a, int n, int hw, int c, void* __restrict__ pooled)
 {
+    pdl_wait();   // first global access comes after the previous kernel of the stream
+    pdl_launch_dependents();
     const int groups = c >> 3;
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (long long)n * groups) return;
@@ -629,6 +643,8 @@ __global__ void avgpool_fwd_kernel(const void* __restrict__ a, int n, int hw, in
 
 __global__ void avgpool_bwd_kernel(const void* __restrict__ dpooled, int n, int hw, int c, void* __restrict__ da)
 {
+    pdl_wait();   // first global access comes after the previous kernel of the stream
+    pdl_launch_dependents();
     const int groups = c >> 3;
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (long long)n * hw * groups) return;
@@ -644,6 +660,8 @@ __global__ void avgpool_bwd_kernel(const void* __restrict__ dpooled, int n, int 
 
 __global__ void pad_channels_kernel(const __nv_bfloat16* __restrict__ x, long long m, int c_in, int c_out, void* __restrict__ y)
 {
+    pdl_wait();   // first global access comes after the previous kernel of the stream
+    pdl_launch_dependents();
     const int groups = c_out >> 3;
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= m * groups) return;
@@ -663,6 +681,8 @@ __global__ void pad_channels_kernel(const __nv_bfloat16* __restrict__ x, long lo
 template <int C_IN>
 __global__ void im2col3x3_kernel(const __nv_bfloat16* __restrict__ x, int n, int h, int w, int c_out, void* __restrict__ y)
 {
+    pdl_wait();   // first global access comes after the previous kernel of the stream
+    pdl_launch_dependents();
     // one thread per pixel: 9*C_IN (<= 32) values gathered with static tap offsets, written as whole 16-byte vectors
     const long long pix = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (pix >= (long long)n * h * w) return;
@@ -702,6 +722,8 @@ __global__ void softmax_xent_kernel(const float* __restrict__ logits, int logits
                                     float loss_scale, float grad_scale, float* loss, __nv_bfloat16* __restrict__ dlogits, int pitch,
                                     unsigned* status)
 {
+    pdl_wait();   // first global access comes after the previous kernel of the stream
+    pdl_launch_dependents();
     const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (row >= n) return;
@@ -735,6 +757,8 @@ __global__ void softmax_xent_kernel(const float* __restrict__ logits, int logits
 // owns a channel and a row lane, partial sums meet in shared memory), one atomic per channel and block.
 __global__ void bias_grad_kernel(const __nv_bfloat16* __restrict__ dz, int m, int k, int pitch, float* db)
 {
+    pdl_wait();   // first global access comes after the previous kernel of the stream
+    pdl_launch_dependents();
     __shared__ float part[8][33];
     const int ch = blockIdx.x * 32 + threadIdx.x;        // blockDim = (32, 8)
     float s = 0.f;
@@ -755,6 +779,8 @@ __global__ void __launch_bounds__(kEwThreads) sgd_momentum_kernel(float4* __rest
                                                                   long long count4, float inv_n, float lr, float mu, float wd,
                                                                   uint2* __restrict__ w_bf16, int zero_grad)
 {
+    pdl_wait();   // first global access comes after the previous kernel of the stream
+    pdl_launch_dependents();
     const long long step = (long long)gridDim.x * blockDim.x;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < count4; i += step) {
         float4 wi = w[i], vi = v[i];
@@ -784,6 +810,8 @@ struct PackSegs {
 __global__ void weight_pack_dgrad_kernel(const __grid_constant__ PackSegs segs, const __nv_bfloat16* __restrict__ src,
                                          __nv_bfloat16* __restrict__ dst)
 {
+    pdl_wait();   // first global access comes after the previous kernel of the stream
+    pdl_launch_dependents();
     __shared__ __nv_bfloat16 tile[32][33];
     const b2c_weight_seg sg = segs.seg[blockIdx.z];
     const int t = blockIdx.y;
@@ -820,10 +848,10 @@ b2c_status launch_bn_fwd(b2c_ctx* ctx, int G, long long m, int c, const void* y,
     dim3 grid((unsigned)ew_grid(ctx, G, m, rows_per_iter), (unsigned)G);
     if (!stats_ready) {
         B2C_CUDA(cudaMemsetAsync(stats, 0, sizeof(double) * 2 * c * G, stream));
-        bn_stats_kernel<<<grid, kEwThreads, sizeof(float) * 2 * c, stream>>>(y, m, c, stats);
+        B2C_CUDA(b2c_launch(ctx, bn_stats_kernel, dim3(grid), dim3(kEwThreads), sizeof(float) * 2 * c, stream, 1u, y, m, c, stats));
     }
-    bn_apply_kernel<<<grid, kEwThreads, 0, stream>>>(y, m, c, stats, gamma, beta, residual, relu, eps, a, save_mean, save_invstd, run_mean, run_var,
-                                                     momentum, relu ? reinterpret_cast<uint8_t*>(relu_mask) : nullptr);
+    B2C_CUDA(b2c_launch(ctx, bn_apply_kernel, dim3(grid), dim3(kEwThreads), 0, stream, 1u, y, m, c, stats, gamma, beta, residual, relu, eps, a, save_mean, save_invstd, run_mean, run_var,
+                                                     momentum, relu ? reinterpret_cast<uint8_t*>(relu_mask) : nullptr));
     B2C_CUDA(cudaGetLastError());
     return B2C_OK;
 }
@@ -852,16 +880,16 @@ b2c_status launch_bn_bwd(b2c_ctx* ctx, int G, long long m, int c, const void* da
                 B2C_CUDA(cudaFuncSetAttribute(bn_bwd_apply_staged_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024));
                 attr_set = true;
             }
-            bn_bwd_reduce_staged_kernel<<<grid, kStThreads, smem, stream>>>(da1, da2, y, m, c, relu, sums, mask, ctx->spin_limit, ctx->d_status);
-            bn_bwd_apply_staged_kernel<<<grid, kStThreads, smem, stream>>>(da1, da2, y, m, c, gamma, save_mean, save_invstd, relu, sums, dy, dres,
-                                                                            dgamma, dbeta, acc, mask, ctx->spin_limit, ctx->d_status);
+            B2C_CUDA(b2c_launch(ctx, bn_bwd_reduce_staged_kernel, dim3(grid), dim3(kStThreads), smem, stream, 1u, da1, da2, y, m, c, relu, sums, mask, ctx->spin_limit, ctx->d_status));
+            B2C_CUDA(b2c_launch(ctx, bn_bwd_apply_staged_kernel, dim3(grid), dim3(kStThreads), smem, stream, 1u, da1, da2, y, m, c, gamma, save_mean, save_invstd, relu, sums, dy, dres,
+                                                                            dgamma, dbeta, acc, mask, ctx->spin_limit, ctx->d_status));
             B2C_CUDA(cudaGetLastError());
             return B2C_OK;
         }
     }
-    bn_bwd_reduce_kernel<<<grid, kEwThreads, sizeof(float) * 2 * c, stream>>>(da1, da2, y, a, m, c, relu, sums, mask);
-    bn_bwd_apply_kernel<<<grid, kEwThreads, 0, stream>>>(da1, da2, y, a, m, c, gamma, save_mean, save_invstd, relu, sums, dy, dres, dgamma, dbeta,
-                                                         acc, mask);
+    B2C_CUDA(b2c_launch(ctx, bn_bwd_reduce_kernel, dim3(grid), dim3(kEwThreads), sizeof(float) * 2 * c, stream, 1u, da1, da2, y, a, m, c, relu, sums, mask));
+    B2C_CUDA(b2c_launch(ctx, bn_bwd_apply_kernel, dim3(grid), dim3(kEwThreads), 0, stream, 1u, da1, da2, y, a, m, c, gamma, save_mean, save_invstd, relu, sums, dy, dres, dgamma, dbeta,
+                                                         acc, mask));
     B2C_CUDA(cudaGetLastError());
     return B2C_OK;
 }
@@ -910,7 +938,7 @@ b2c_status b2c_avgpool_fwd(b2c_ctx* ctx, int n, int hw, int c, const void* a, vo
     if (n < 1 || hw < 1 || c < 8 || c % 8) return B2C_ERR_UNSUPPORTED_SHAPE;
     if (!b2c_aligned16(a) || !b2c_aligned16(pooled)) return B2C_ERR_MISALIGNED;
     const long long total = (long long)n * (c / 8);
-    avgpool_fwd_kernel<<<(unsigned)((total + 127) / 128), 128, 0, (cudaStream_t)stream_>>>(a, n, hw, c, pooled);
+    B2C_CUDA(b2c_launch(ctx, avgpool_fwd_kernel, dim3((unsigned)((total + 127) / 128)), dim3(128), 0, (cudaStream_t)stream_, 1u, a, n, hw, c, pooled));
     B2C_CUDA(cudaGetLastError());
     return B2C_OK;
 }
@@ -921,7 +949,7 @@ b2c_status b2c_avgpool_bwd(b2c_ctx* ctx, int n, int hw, int c, const void* dpool
     if (n < 1 || hw < 1 || c < 8 || c % 8) return B2C_ERR_UNSUPPORTED_SHAPE;
     if (!b2c_aligned16(dpooled) || !b2c_aligned16(da)) return B2C_ERR_MISALIGNED;
     const long long total = (long long)n * hw * (c / 8);
-    avgpool_bwd_kernel<<<(unsigned)((total + 255) / 256), 256, 0, (cudaStream_t)stream_>>>(dpooled, n, hw, c, da);
+    B2C_CUDA(b2c_launch(ctx, avgpool_bwd_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, (cudaStream_t)stream_, 1u, dpooled, n, hw, c, da));
     B2C_CUDA(cudaGetLastError());
     return B2C_OK;
 }
@@ -932,8 +960,8 @@ b2c_status b2c_pad_channels(b2c_ctx* ctx, long m, int c_in, int c_out, const voi
     if (m < 1 || c_in < 1 || c_out < c_in || c_out % 8) return B2C_ERR_UNSUPPORTED_SHAPE;
     if (!b2c_aligned16(y) || (reinterpret_cast<uintptr_t>(x) & 1u)) return B2C_ERR_MISALIGNED;
     const long long total = (long long)m * (c_out / 8);
-    pad_channels_kernel<<<(unsigned)((total + 255) / 256), 256, 0, (cudaStream_t)stream_>>>(reinterpret_cast<const __nv_bfloat16*>(x), m, c_in,
-                                                                                            c_out, y);
+    B2C_CUDA(b2c_launch(ctx, pad_channels_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, (cudaStream_t)stream_, 1u, reinterpret_cast<const __nv_bfloat16*>(x), m, c_in,
+                                                                                            c_out, y));
     B2C_CUDA(cudaGetLastError());
     return B2C_OK;
 }
@@ -947,9 +975,9 @@ b2c_status b2c_im2col_3x3(b2c_ctx* ctx, int n, int h, int w, int c_in, int c_out
     const long long total = (long long)n * h * w;
     const unsigned blocks = (unsigned)((total + 127) / 128);
     const __nv_bfloat16* xs = reinterpret_cast<const __nv_bfloat16*>(x);
-    if (c_in == 3) im2col3x3_kernel<3><<<blocks, 128, 0, (cudaStream_t)stream_>>>(xs, n, h, w, c_out, y);
-    else if (c_in == 2) im2col3x3_kernel<2><<<blocks, 128, 0, (cudaStream_t)stream_>>>(xs, n, h, w, c_out, y);
-    else im2col3x3_kernel<1><<<blocks, 128, 0, (cudaStream_t)stream_>>>(xs, n, h, w, c_out, y);
+    if (c_in == 3) B2C_CUDA(b2c_launch(ctx, im2col3x3_kernel<3>, dim3(blocks), dim3(128), 0, (cudaStream_t)stream_, 1u, xs, n, h, w, c_out, y));
+    else if (c_in == 2) B2C_CUDA(b2c_launch(ctx, im2col3x3_kernel<2>, dim3(blocks), dim3(128), 0, (cudaStream_t)stream_, 1u, xs, n, h, w, c_out, y));
+    else B2C_CUDA(b2c_launch(ctx, im2col3x3_kernel<1>, dim3(blocks), dim3(128), 0, (cudaStream_t)stream_, 1u, xs, n, h, w, c_out, y));
     B2C_CUDA(cudaGetLastError());
     return B2C_OK;
 }
@@ -961,9 +989,9 @@ b2c_status b2c_softmax_xent_fwd_bwd(b2c_ctx* ctx, int n, int classes, const floa
     if (n < 1 || classes < 1 || logits_pitch < classes || pitch < classes || pitch % 8) return B2C_ERR_UNSUPPORTED_SHAPE;
     if (!b2c_aligned16(dlogits)) return B2C_ERR_MISALIGNED;
     const int warps = 4;
-    softmax_xent_kernel<<<(n + warps - 1) / warps, warps * 32, 0, (cudaStream_t)stream_>>>(logits, logits_pitch, labels, n, classes, loss_scale,
+    B2C_CUDA(b2c_launch(ctx, softmax_xent_kernel, dim3((n + warps - 1) / warps), dim3(warps * 32), 0, (cudaStream_t)stream_, 1u, logits, logits_pitch, labels, n, classes, loss_scale,
                                                                                           grad_scale, loss, reinterpret_cast<__nv_bfloat16*>(dlogits),
-                                                                                          pitch, ctx->d_status);
+                                                                                          pitch, ctx->d_status));
     B2C_CUDA(cudaGetLastError());
     return B2C_OK;
 }
@@ -975,8 +1003,8 @@ b2c_status b2c_bias_grad(b2c_ctx* ctx, int m, int k, int pitch, const void* dz, 
     if (!accumulate) B2C_CUDA(cudaMemsetAsync(db, 0, sizeof(float) * (size_t)k, (cudaStream_t)stream_));
     int row_blocks = (m + 63) / 64;
     if (row_blocks > 64) row_blocks = 64;
-    bias_grad_kernel<<<dim3((unsigned)((k + 31) / 32), (unsigned)row_blocks), dim3(32, 8), 0, (cudaStream_t)stream_>>>(
-        reinterpret_cast<const __nv_bfloat16*>(dz), m, k, pitch, db);
+    B2C_CUDA(b2c_launch(ctx, bias_grad_kernel, dim3(dim3((unsigned)((k + 31) / 32), (unsigned)row_blocks)), dim3(dim3(32, 8)), 0, (cudaStream_t)stream_, 1u, 
+        reinterpret_cast<const __nv_bfloat16*>(dz), m, k, pitch, db));
     B2C_CUDA(cudaGetLastError());
     return B2C_OK;
 }
@@ -992,9 +1020,9 @@ b2c_status b2c_grad_accum_sgd_momentum(b2c_ctx* ctx, size_t count, float* w, flo
     long long blocks = (count4 + kEwThreads - 1) / kEwThreads;
     const long long cap = (long long)ctx->sm_count * 8;
     if (blocks > cap) blocks = cap;
-    sgd_momentum_kernel<<<(unsigned)blocks, kEwThreads, 0, (cudaStream_t)stream_>>>(reinterpret_cast<float4*>(w), reinterpret_cast<float4*>(v),
+    B2C_CUDA(b2c_launch(ctx, sgd_momentum_kernel, dim3((unsigned)blocks), dim3(kEwThreads), 0, (cudaStream_t)stream_, 1u, reinterpret_cast<float4*>(w), reinterpret_cast<float4*>(v),
                                                                                    reinterpret_cast<float4*>(g_accum), count4, inv_n_micro, lr,
-                                                                                   momentum, wd, reinterpret_cast<uint2*>(w_bf16), zero_grad);
+                                                                                   momentum, wd, reinterpret_cast<uint2*>(w_bf16), zero_grad));
     B2C_CUDA(cudaGetLastError());
     return B2C_OK;
 }
@@ -1013,8 +1041,8 @@ b2c_status b2c_weight_pack_dgrad(b2c_ctx* ctx, const b2c_weight_seg* segs, int n
         max_rs = segs[i].rs > max_rs ? segs[i].rs : max_rs;
     }
     dim3 grid((unsigned)max_tiles, (unsigned)max_rs, (unsigned)n_segs);
-    weight_pack_dgrad_kernel<<<grid, dim3(32, 8), 0, (cudaStream_t)stream_>>>(ps, reinterpret_cast<const __nv_bfloat16*>(src_bf16),
-                                                                              reinterpret_cast<__nv_bfloat16*>(dst_bf16));
+    B2C_CUDA(b2c_launch(ctx, weight_pack_dgrad_kernel, dim3(grid), dim3(dim3(32, 8)), 0, (cudaStream_t)stream_, 1u, ps, reinterpret_cast<const __nv_bfloat16*>(src_bf16),
+                                                                              reinterpret_cast<__nv_bfloat16*>(dst_bf16)));
     B2C_CUDA(cudaGetLastError());
     return B2C_OK;
 }

@@ -10,6 +10,14 @@
 
 namespace b2c {
 
+// Programmatic dependent launch.  A kernel launched with the programmatic-serialization attribute may start while the
+// previous kernel of the stream still runs; pdl_wait() blocks until that kernel has completed and its writes are
+// visible, so everything before it must touch no global data (barrier set-up, TMEM allocation, descriptor prefetch).
+// pdl_launch_dependents() lets the next kernel of the stream be scheduled as SMs free up.  Both are no-ops in a launch
+// without the attribute.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 // ---------------------------------------------------------------- mbarrier

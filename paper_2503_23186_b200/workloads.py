@@ -71,6 +71,25 @@ def _basic_block(spec, t_in, C, K, stride, H, W, name):
     return t, Ho, Wo
 
 
+def _bottleneck_block(spec, t_in, C, width, stride, H, W, name, expansion=4):
+    """a1 = relu(bn(conv1x1(x))); a2 = relu(bn(conv3x3 stride(a1))); out = relu(bn(conv1x1(a2)) + shortcut(x)),
+    the last 1x1 widening to expansion*width channels.  shortcut as in the basic block."""
+    K = expansion * width
+    Ho, Wo = (H + 2 - 3) // stride + 1, (W + 2 - 3) // stride + 1
+    t = _conv(spec, t_in, C, width, 1, 1, H, W, name + "c1")
+    t = _bn(spec, t, width, H, W, True, name=name + "bn1")
+    if stride != 1 or C != K:
+        ts = _conv(spec, t_in, C, K, 1, stride, H, W, name + "sc")
+        ts = _bn(spec, ts, K, Ho, Wo, False, name=name + "scbn")
+    else:
+        ts = t_in
+    t = _conv(spec, t, width, width, 3, stride, H, W, name + "c2")
+    t = _bn(spec, t, width, Ho, Wo, True, name=name + "bn2")
+    t = _conv(spec, t, width, K, 1, 1, Ho, Wo, name + "c3")
+    t = _bn(spec, t, K, Ho, Wo, True, res=ts, name=name + "bn3")
+    return t, Ho, Wo
+
+
 def _head(spec, t, C, H, W, classes):
     spec.append(dict(kind="avgpool", src=t, C=C, H=H, W=W, name="pool"))
     spec.append(dict(kind="fc", src=len(spec), C=C, K=classes, name="fc"))
@@ -91,6 +110,20 @@ def residual_net_spec(stem_width, widths, strides, blocks_per_stage, classes=100
     return spec
 
 
+def bottleneck_net_spec(stem_width, widths, strides, blocks, classes=100, image_hw=32, image_c=3, expansion=4):
+    spec = []
+    H = W = image_hw
+    t = _conv(spec, 0, image_c, stem_width, 3, 1, H, W, "stem")
+    t = _bn(spec, t, stem_width, H, W, True, name="stembn")
+    C = stem_width
+    for si, (width, st, nb) in enumerate(zip(widths, strides, blocks), 1):
+        for b in range(nb):
+            t, H, W = _bottleneck_block(spec, t, C, width, st if b == 0 else 1, H, W, f"s{si}b{b + 1}", expansion)
+            C = expansion * width
+    _head(spec, t, C, H, W, classes)
+    return spec
+
+
 def resnet18_spec(classes=100):
     """ResNet-18-shaped CIFAR net: stem 3->64, stages 64/128/256/512 x 2 basic blocks."""
     return residual_net_spec(64, (64, 128, 256, 512), (1, 2, 2, 2), 2, classes)
@@ -99,6 +132,17 @@ def resnet18_spec(classes=100):
 def wrn28_10_spec(classes=100):
     """Wide-ResNet-28-10-shaped net: stem 3->16, stages 160/320/640 x 4 basic blocks."""
     return residual_net_spec(16, (160, 320, 640), (1, 2, 2), 4, classes)
+
+
+def resnet50_spec(classes=100):
+    """ResNet-50-shaped CIFAR net (the paper's convolutional workload, Section IV-A, at CIFAR resolution):
+    stem 3->64, stages of 3/4/6/3 bottleneck blocks with widths 64/128/256/512 (outputs 256..2048)."""
+    return bottleneck_net_spec(64, (64, 128, 256, 512), (1, 2, 2, 2), (3, 4, 6, 3), classes)
+
+
+def tiny_bottleneck_spec(classes=10, hw=8, c=16, width=16):
+    """Small bottleneck net: one projection block at stride 1, one identity block, one stride-2 block."""
+    return bottleneck_net_spec(width, (width, 2 * width), (1, 2), (2, 1), classes, image_hw=hw, image_c=c, expansion=2)
 
 
 def tiny_net_spec(classes=10, hw=8, c=16, width=16, width2=32):
