@@ -31,6 +31,7 @@ WORKLOADS = {
     "resnet18_cifar_b1024_8x128": (wl.resnet18_spec, 128, 8),
     "resnet18_cifar_b128": (wl.resnet18_spec, 128, 1),
     "wrn28_10_cifar_b256": (wl.wrn28_10_spec, 256, 1),
+    "resnet50_cifar_b1024_8x128": (wl.resnet50_spec, 128, 8),
 }
 DEFAULT_WORKLOAD = "resnet18_cifar_b1024_8x128"
 LR, MU, WD = 0.1, 0.9, 5e-4

@@ -8,6 +8,11 @@
 
 using namespace b2c;
 
+// Default L2 budget (MB) for the largest tensor of a layer per launch inside b2c_train_step; 0 = whole passes.
+#ifndef B2C_DEFAULT_CHUNK_MB
+#define B2C_DEFAULT_CHUNK_MB 0
+#endif
+
 extern "C" {
 
 b2c_status b2c_create(b2c_ctx** out, int device)
@@ -185,6 +190,7 @@ struct LayerPlan {
     long long w_off = -1, gamma_off = -1, beta_off = -1, bias_off = -1;   // elements into the flat parameter arrays
     long long mean_off = -1, invstd_off = -1, bwd_ws_off = -1, mask_off = -1;   // bytes into the workspace
     int src_slot = -1, res_slot = -1;                                     // which gradient buffer of src / res this layer writes
+    int chunk_groups = 1;          // micro-batches of a pass this layer takes per launch (divides n_conc)
 };
 
 inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
@@ -389,6 +395,27 @@ b2c_status b2c_net_create_concurrent(b2c_ctx* ctx, const b2c_layer_desc* layers,
     }
     net->stats_end = (long long)ws;
     net->ws_bytes = ws;
+    // Chunking for L2: a layer takes as many micro-batches per launch as keep its largest tensor under the budget (a
+    // power-of-two divisor of the pass; B2C_CHUNK_MB sets the budget in MB, 0 = whole passes).
+    {
+        const char* cenv = std::getenv("B2C_CHUNK_MB");
+        const double budget = (cenv ? std::atof(cenv) : (double)B2C_DEFAULT_CHUNK_MB) * 1e6;
+        for (int i = 0; i < n_layers; ++i) {
+            LayerPlan& L = net->layers[i];
+            int gc = n_concurrent;
+            if (budget > 0.0) {
+                const TensorPlan& a = net->tensors[L.d.src];
+                const TensorPlan& b = net->tensors[i + 1];
+                double per_mb = (double)micro_batch * a.h * a.w * a.c * (a.f32 ? 4 : 2);
+                if (b.exists) {
+                    const double pb = (double)micro_batch * b.h * b.w * b.c * (b.f32 ? 4 : 2);
+                    if (pb > per_mb) per_mb = pb;
+                }
+                while (gc > 1 && (gc * per_mb > budget || n_concurrent % gc != 0)) --gc;
+            }
+            L.chunk_groups = gc;
+        }
+    }
     *out = net;
     return B2C_OK;
 }
@@ -481,43 +508,54 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
     const int n_layers = (int)net->layers.size();
     const __nv_bfloat16* w_bf16 = reinterpret_cast<const __nv_bfloat16*>(net->w_bf16);
     const __nv_bfloat16* w_dg = reinterpret_cast<const __nv_bfloat16*>(net->w_dgrad);
-    auto act = [&](int t) -> void* { return net->ws + net->tensors[t].act_off; };
-    auto grad = [&](int t, int slot) -> void* { return slot >= 0 && net->tensors[t].grad_off[slot] >= 0 ? net->ws + net->tensors[t].grad_off[slot] : nullptr; };
+    // Tensors hold the images of a pass back to back, so a run of whole micro-batches (statistics groups g0 .. g0 + Gc) of any
+    // tensor or per-group array is the same array at an offset: img0 = first image of the run.
+    auto act = [&](int t, int img0) -> void* {
+        const TensorPlan& T = net->tensors[t];
+        return net->ws + T.act_off + (long long)img0 * T.h * T.w * T.c * (T.f32 ? 4 : 2);
+    };
+    auto grad = [&](int t, int slot, int img0) -> void* {
+        const TensorPlan& T = net->tensors[t];
+        return slot >= 0 && T.grad_off[slot] >= 0 ? net->ws + T.grad_off[slot] + (long long)img0 * T.h * T.w * T.c * 2 : nullptr;
+    };
 
     B2C_CUDA(cudaMemsetAsync(loss_dev, 0, sizeof(float), stream));
     const size_t image_bytes = (size_t)N * net->image_h * net->image_w * net->image_c * 2;
     if (image_bytes % 16) return B2C_ERR_MISALIGNED;
+    const int mbs = net->micro_batch;
 
     for (int mb = 0; mb < n_passes; ++mb) {
         const char* img = reinterpret_cast<const char*>(images) + (size_t)mb * image_bytes;
         const int32_t* lab = labels + (size_t)mb * N;
-        const void* t0;
-        if (net->tensors[0].act_off >= 0) {
-            ProfScope ps_(net, stream, B2C_PROF_OTHER, 1);
-            if (net->stem_im2col)
-                B2C_TRY(b2c_im2col_3x3(ctx, N, net->image_h, net->image_w, net->image_c, net->image_c_pad, img, act(0), stream));
-            else
-                B2C_TRY(b2c_pad_channels(ctx, (long)N * net->image_h * net->image_w, net->image_c, net->image_c_pad, img, act(0), stream));
-            t0 = act(0);
-        } else {
-            t0 = img;
-        }
-        auto act_in = [&](int t) -> const void* { return t == 0 ? t0 : act(t); };
+        const bool staged_input = net->tensors[0].act_off >= 0;
+        auto act_in = [&](int t, int img0) -> const void* {
+            if (t == 0 && !staged_input) return img + (size_t)img0 * net->image_h * net->image_w * net->image_c * 2;
+            return act(t, img0);
+        };
         B2C_CUDA(cudaMemsetAsync(net->ws + net->stats_begin, 0, (size_t)(net->stats_end - net->stats_begin), stream));
 
-        // ---------------- forward pass and loss
-        for (int i = 0; i < n_layers; ++i) {
+        // forward pass of layer i over the micro-batches g0 .. g0 + Gc of the pass
+        auto forward_layer = [&](int i, int g0, int Gc) -> b2c_status {
             const LayerPlan& L = net->layers[i];
             const b2c_layer_desc& d = L.d;
             const TensorPlan& o = net->tensors[i + 1];
+            const int img0 = g0 * mbs, Nc = Gc * mbs;
+            if (i == 0 && staged_input) {   // the first layer's chunk of the image batch, expanded on the device
+                ProfScope ps_(net, stream, B2C_PROF_OTHER, 1);
+                const char* src = img + (size_t)img0 * net->image_h * net->image_w * net->image_c * 2;
+                if (net->stem_im2col)
+                    B2C_TRY(b2c_im2col_3x3(ctx, Nc, net->image_h, net->image_w, net->image_c, net->image_c_pad, src, act(0, img0), stream));
+                else
+                    B2C_TRY(b2c_pad_channels(ctx, (long)Nc * net->image_h * net->image_w, net->image_c, net->image_c_pad, src, act(0, img0), stream));
+            }
             switch (d.kind) {
                 case B2C_LAYER_CONV: {
                     KMajorProblem pb{};
-                    pb.n = N; pb.ih = d.h; pb.iw = d.w; pb.ic = L.c_pad; pb.oh = L.p; pb.ow = L.q; pb.oc = d.k;
+                    pb.n = Nc; pb.ih = d.h; pb.iw = d.w; pb.ic = L.c_pad; pb.oh = L.p; pb.ow = L.q; pb.oc = d.k;
                     pb.r = L.gemm_r; pb.stride = d.stride; pb.pad = (L.gemm_r - 1) / 2; pb.dgrad = false;
-                    pb.in = act_in(d.src); pb.wt = w_bf16 + L.w_off; pb.out = act(i + 1);
-                    pb.stats = o.fused_stats ? reinterpret_cast<double*>(net->ws + o.stats_off) : nullptr;
-                    pb.stats_group_images = net->micro_batch;
+                    pb.in = act_in(d.src, img0); pb.wt = w_bf16 + L.w_off; pb.out = act(i + 1, img0);
+                    pb.stats = o.fused_stats ? reinterpret_cast<double*>(net->ws + o.stats_off) + (size_t)g0 * 2 * d.k : nullptr;
+                    pb.stats_group_images = mbs;
                     ProfScope ps_(net, stream, B2C_PROF_CONV_FWD, 1);
                     B2C_TRY(launch_conv_kmajor(ctx, pb, stream));
                     break;
@@ -525,25 +563,26 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
                 case B2C_LAYER_BN: {
                     const TensorPlan& in = net->tensors[d.src];
                     const bool ready = in.fused_stats;
-                    double* stats = reinterpret_cast<double*>(net->ws + (in.stats_off >= 0 ? in.stats_off : L.bwd_ws_off));
+                    double* stats = reinterpret_cast<double*>(net->ws + (in.stats_off >= 0 ? in.stats_off : L.bwd_ws_off)) + (size_t)g0 * 2 * in.c;
                     ProfScope ps_(net, stream, B2C_PROF_BN_FWD, ready ? 1 : 2);
-                    B2C_TRY(launch_bn_fwd(ctx, G, (long long)net->micro_batch * in.h * in.w, in.c, act(d.src), stats, ready, net->w + L.gamma_off,
-                                          net->w + L.beta_off, d.res >= 0 ? act(d.res) : nullptr, d.relu, 1e-5f, act(i + 1),
-                                          reinterpret_cast<float*>(net->ws + L.mean_off), reinterpret_cast<float*>(net->ws + L.invstd_off), nullptr,
-                                          nullptr, 0.f, L.mask_off >= 0 ? net->ws + L.mask_off : nullptr, stream));
+                    B2C_TRY(launch_bn_fwd(ctx, Gc, (long long)mbs * in.h * in.w, in.c, act(d.src, img0), stats, ready, net->w + L.gamma_off,
+                                          net->w + L.beta_off, d.res >= 0 ? act(d.res, img0) : nullptr, d.relu, 1e-5f, act(i + 1, img0),
+                                          reinterpret_cast<float*>(net->ws + L.mean_off) + (size_t)g0 * in.c,
+                                          reinterpret_cast<float*>(net->ws + L.invstd_off) + (size_t)g0 * in.c, nullptr, nullptr, 0.f,
+                                          L.mask_off >= 0 ? net->ws + L.mask_off + (long long)img0 * in.h * in.w * in.c / 8 : nullptr, stream));
                     break;
                 }
                 case B2C_LAYER_AVGPOOL: {
                     const TensorPlan& in = net->tensors[d.src];
                     ProfScope ps_(net, stream, B2C_PROF_OTHER, 1);
-                    B2C_TRY(b2c_avgpool_fwd(ctx, N, in.h * in.w, in.c, act(d.src), act(i + 1), stream));
+                    B2C_TRY(b2c_avgpool_fwd(ctx, Nc, in.h * in.w, in.c, act(d.src, img0), act(i + 1, img0), stream));
                     break;
                 }
                 case B2C_LAYER_FC: {
                     KMajorProblem pb{};
-                    pb.n = N; pb.ih = 1; pb.iw = 1; pb.ic = L.c_pad; pb.oh = 1; pb.ow = 1; pb.oc = L.k_pad;
+                    pb.n = Nc; pb.ih = 1; pb.iw = 1; pb.ic = L.c_pad; pb.oh = 1; pb.ow = 1; pb.oc = L.k_pad;
                     pb.r = 1; pb.stride = 1; pb.pad = 0; pb.dgrad = false;
-                    pb.in = act(d.src); pb.wt = w_bf16 + L.w_off; pb.out = act(i + 1);
+                    pb.in = act(d.src, img0); pb.wt = w_bf16 + L.w_off; pb.out = act(i + 1, img0);
                     pb.out_f32 = true; pb.bias = net->w + L.bias_off;
                     ProfScope ps_(net, stream, B2C_PROF_OTHER, 1);
                     B2C_TRY(launch_conv_kmajor(ctx, pb, stream));
@@ -552,74 +591,99 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
                 case B2C_LAYER_XENT: {
                     const TensorPlan& in = net->tensors[d.src];
                     ProfScope ps_(net, stream, B2C_PROF_OTHER, 1);
-                    B2C_TRY(b2c_softmax_xent_fwd_bwd(ctx, N, d.k, reinterpret_cast<const float*>(act(d.src)), in.c, lab,
-                                                     1.f / ((float)net->micro_batch * (float)n_micro), 1.f / (float)net->micro_batch, loss_dev,
-                                                     grad(d.src, L.src_slot), in.c,
-                                                     stream));
+                    B2C_TRY(b2c_softmax_xent_fwd_bwd(ctx, Nc, d.k, reinterpret_cast<const float*>(act(d.src, img0)), in.c, lab + img0,
+                                                     1.f / ((float)mbs * (float)n_micro), 1.f / (float)mbs, loss_dev,
+                                                     grad(d.src, L.src_slot, img0), in.c, stream));
                     break;
                 }
             }
-        }
-        // ---------------- backward pass, gradients summed into the flat gradient array
-        for (int i = n_layers - 1; i >= 0; --i) {
+            return B2C_OK;
+        };
+
+        // backward pass of layer i over the same kind of run; parameter gradients are summed into the flat gradient array
+        auto backward_layer = [&](int i, int g0, int Gc) -> b2c_status {
             const LayerPlan& L = net->layers[i];
             const b2c_layer_desc& d = L.d;
             const TensorPlan& o = net->tensors[i + 1];
+            const int img0 = g0 * mbs, Nc = Gc * mbs;
             switch (d.kind) {
                 case B2C_LAYER_XENT: break;
                 case B2C_LAYER_FC: {
-                    const void* dz = grad(i + 1, 0);
+                    const void* dz = grad(i + 1, 0, img0);
                     WgradProblem wp{};
-                    wp.n = N; wp.h = 1; wp.w = 1; wp.c = L.c_pad; wp.p = 1; wp.q = 1; wp.k = L.k_pad; wp.r = 1; wp.stride = 1; wp.pad = 0;
-                    wp.dy = dz; wp.x = act(d.src); wp.dw = net->g + L.w_off;
+                    wp.n = Nc; wp.h = 1; wp.w = 1; wp.c = L.c_pad; wp.p = 1; wp.q = 1; wp.k = L.k_pad; wp.r = 1; wp.stride = 1; wp.pad = 0;
+                    wp.dy = dz; wp.x = act(d.src, img0); wp.dw = net->g + L.w_off;
                     ProfScope ps_(net, stream, B2C_PROF_OTHER, 3);
                     B2C_TRY(launch_conv_wgrad(ctx, wp, stream));
-                    B2C_TRY(b2c_bias_grad(ctx, N, L.k_pad, L.k_pad, dz, net->g + L.bias_off, 1, stream));
+                    B2C_TRY(b2c_bias_grad(ctx, Nc, L.k_pad, L.k_pad, dz, net->g + L.bias_off, 1, stream));
                     KMajorProblem pb{};
-                    pb.n = N; pb.ih = 1; pb.iw = 1; pb.ic = L.k_pad; pb.oh = 1; pb.ow = 1; pb.oc = L.c_pad;
+                    pb.n = Nc; pb.ih = 1; pb.iw = 1; pb.ic = L.k_pad; pb.oh = 1; pb.ow = 1; pb.oc = L.c_pad;
                     pb.r = 1; pb.stride = 1; pb.pad = 0; pb.dgrad = true;
-                    pb.in = dz; pb.wt = w_dg + L.w_off; pb.out = grad(d.src, L.src_slot);
+                    pb.in = dz; pb.wt = w_dg + L.w_off; pb.out = grad(d.src, L.src_slot, img0);
                     B2C_TRY(launch_conv_kmajor(ctx, pb, stream));
                     break;
                 }
                 case B2C_LAYER_AVGPOOL: {
                     const TensorPlan& in = net->tensors[d.src];
                     ProfScope ps_(net, stream, B2C_PROF_OTHER, 1);
-                    B2C_TRY(b2c_avgpool_bwd(ctx, N, in.h * in.w, in.c, grad(i + 1, 0), grad(d.src, L.src_slot), stream));
+                    B2C_TRY(b2c_avgpool_bwd(ctx, Nc, in.h * in.w, in.c, grad(i + 1, 0, img0), grad(d.src, L.src_slot, img0), stream));
                     break;
                 }
                 case B2C_LAYER_BN: {
                     const TensorPlan& in = net->tensors[d.src];
                     ProfScope ps_(net, stream, B2C_PROF_BN_BWD, 2);
-                    B2C_TRY(launch_bn_bwd(ctx, G, (long long)net->micro_batch * in.h * in.w, in.c, grad(i + 1, 0), o.n_contrib > 1 ? grad(i + 1, 1) : nullptr,
-                                          act(d.src), act(i + 1), net->w + L.gamma_off, reinterpret_cast<float*>(net->ws + L.mean_off),
-                                          reinterpret_cast<float*>(net->ws + L.invstd_off), d.relu, grad(d.src, L.src_slot),
-                                          d.res >= 0 ? grad(d.res, L.res_slot) : nullptr, net->g + L.gamma_off, net->g + L.beta_off, 1,
-                                          reinterpret_cast<double*>(net->ws + L.bwd_ws_off), /*sums_zeroed=*/in.stats_off >= 0,
-                                          L.mask_off >= 0 ? net->ws + L.mask_off : nullptr, stream));
+                    B2C_TRY(launch_bn_bwd(ctx, Gc, (long long)mbs * in.h * in.w, in.c, grad(i + 1, 0, img0),
+                                          o.n_contrib > 1 ? grad(i + 1, 1, img0) : nullptr, act(d.src, img0), act(i + 1, img0), net->w + L.gamma_off,
+                                          reinterpret_cast<float*>(net->ws + L.mean_off) + (size_t)g0 * in.c,
+                                          reinterpret_cast<float*>(net->ws + L.invstd_off) + (size_t)g0 * in.c, d.relu, grad(d.src, L.src_slot, img0),
+                                          d.res >= 0 ? grad(d.res, L.res_slot, img0) : nullptr, net->g + L.gamma_off, net->g + L.beta_off, 1,
+                                          reinterpret_cast<double*>(net->ws + L.bwd_ws_off) + (size_t)g0 * 2 * in.c, /*sums_zeroed=*/in.stats_off >= 0,
+                                          L.mask_off >= 0 ? net->ws + L.mask_off + (long long)img0 * in.h * in.w * in.c / 8 : nullptr, stream));
                     break;
                 }
                 case B2C_LAYER_CONV: {
-                    const void* dy = grad(i + 1, 0);
+                    const void* dy = grad(i + 1, 0, img0);
                     WgradProblem wp{};
-                    wp.n = N; wp.h = d.h; wp.w = d.w; wp.c = L.c_pad; wp.p = L.p; wp.q = L.q; wp.k = d.k;
+                    wp.n = Nc; wp.h = d.h; wp.w = d.w; wp.c = L.c_pad; wp.p = L.p; wp.q = L.q; wp.k = d.k;
                     wp.r = L.gemm_r; wp.stride = d.stride; wp.pad = (L.gemm_r - 1) / 2;
-                    wp.dy = dy; wp.x = act_in(d.src); wp.dw = net->g + L.w_off;
+                    wp.dy = dy; wp.x = act_in(d.src, img0); wp.dw = net->g + L.w_off;
                     {
                         ProfScope ps_(net, stream, B2C_PROF_CONV_WGRAD, 1);
                         B2C_TRY(launch_conv_wgrad(ctx, wp, stream));
                     }
                     if (d.src != 0) {
                         KMajorProblem pb{};
-                        pb.n = N; pb.ih = L.p; pb.iw = L.q; pb.ic = d.k; pb.oh = d.h; pb.ow = d.w; pb.oc = L.c_pad;
+                        pb.n = Nc; pb.ih = L.p; pb.iw = L.q; pb.ic = d.k; pb.oh = d.h; pb.ow = d.w; pb.oc = L.c_pad;
                         pb.r = d.r; pb.stride = d.stride; pb.pad = (d.r - 1) / 2; pb.dgrad = true;
-                        pb.in = dy; pb.wt = w_dg + L.w_off; pb.out = grad(d.src, L.src_slot);
+                        pb.in = dy; pb.wt = w_dg + L.w_off; pb.out = grad(d.src, L.src_slot, img0);
                         ProfScope ps_(net, stream, B2C_PROF_CONV_DGRAD, 1);
                         B2C_TRY(launch_conv_kmajor(ctx, pb, stream));
                     }
                     break;
                 }
             }
+            return B2C_OK;
+        };
+
+        // Layers whose tensors exceed the L2 budget run in segments: a run of consecutive layers with the same chunk size
+        // is taken chunk by chunk (a few micro-batches at a time), so that a tensor is still in L2 when its consumer (and
+        // the second pass of the BatchNorm backward) reads it.  Every layer acts on images independently except through the
+        // per-micro-batch BatchNorm statistics, so any run of whole micro-batches is a valid chunk.
+        for (int seg = 0; seg < n_layers;) {
+            const int Gc = net->layers[seg].chunk_groups;
+            int seg_end = seg + 1;
+            while (seg_end < n_layers && net->layers[seg_end].chunk_groups == Gc) ++seg_end;
+            for (int g0 = 0; g0 < G; g0 += Gc)
+                for (int i = seg; i < seg_end; ++i) B2C_TRY(forward_layer(i, g0, Gc));
+            seg = seg_end;
+        }
+        for (int seg_end = n_layers; seg_end > 0;) {
+            const int Gc = net->layers[seg_end - 1].chunk_groups;
+            int seg = seg_end - 1;
+            while (seg > 0 && net->layers[seg - 1].chunk_groups == Gc) --seg;
+            for (int g0 = 0; g0 < G; g0 += Gc)
+                for (int i = seg_end - 1; i >= seg; --i) B2C_TRY(backward_layer(i, g0, Gc));
+            seg_end = seg;
         }
     }
     // ---------------- gradient average + parameter update, refresh of both bf16 weight copies

@@ -266,6 +266,35 @@ def test_concurrent_micro_batches_match_sequential(ctx):
     seq.close(); par.close()
 
 
+def test_chunked_schedule_matches_oracle(ctx, monkeypatch):
+    """b2c_train_step with an L2 budget (B2C_CHUNK_MB): runs of layers are taken a few micro-batches at a time.  The budget
+    here puts the wide early layers on chunks of one and two micro-batches and leaves the late layers whole."""
+    from paper_2503_23186_b200 import binding
+    from netcheck import check_step
+    spec = wl.tiny_net_spec(classes=10, hw=16, c=3, width=64, width2=128)
+    params = wl.perturb_bn_params(wl.init_params(spec, 6), 6)
+    images, labels = wl.image_batch(6, 4 * 8, hw=16, c=3, classes=10)
+    d_img, d_lab = dev_bf16(images), torch.from_numpy(labels).cuda()
+    whole = binding.Net(ctx, spec, 8, n_concurrent=4)
+    whole.load_params(params)
+    loss_whole = whole.train_step(d_img, d_lab, 4, LR, MU, WD, update=False).item()
+    monkeypatch.setenv("B2C_CHUNK_MB", "0.3")   # 64 x 16 x 16 x 8 images x 2 bytes = 0.26 MB per micro-batch
+    chunked = binding.Net(ctx, spec, 8, n_concurrent=4)
+    monkeypatch.delenv("B2C_CHUNK_MB")
+    chunked.load_params(params)
+    loss_chunked = chunked.train_step(d_img, d_lab, 4, LR, MU, WD, update=False).item()
+    assert ctx.device_status() == 0
+    _, launches_whole = whole.profile_read()
+    _, launches_chunked = chunked.profile_read()
+    assert sum(launches_chunked.values()) > sum(launches_whole.values())   # the budget did split layers
+    check_step(chunked, spec, images, labels, 32, groups=4).assert_ok()
+    assert abs(loss_chunked - loss_whole) <= 1e-5 * abs(loss_whole)
+    gw, gc = whole.unpack(whole.g), chunked.unpack(chunked.g)
+    for name in sorted(params):
+        assert_close(gc[name], gw[name], f"grad {name} (chunked vs whole passes)", 1e-4, 1e-3)
+    whole.close(); chunked.close()
+
+
 def _full_size_sampled(ctx, spec, micro_batch, n_micro, seed):
     """One pass of a full-size workload in the launch configuration bench.py times (all micro-batches side by side),
     every layer checked on sampled outputs against the oracle; then the fused update against the oracle's update on
@@ -306,6 +335,35 @@ def test_resnet18_batch1024_config4_full_size(ctx):
 
 def test_wrn28_10_batch256_config5_full_size(ctx):
     _full_size_sampled(ctx, wl.wrn28_10_spec(), 256, 1, 0)
+
+
+def test_tiny_bottleneck_net(ctx):
+    """Bottleneck blocks (1x1 -> 3x3 -> 1x1 with expansion, projection and identity shortcuts, a stride-2 block): the
+    whole step against the oracle, two micro-batches.  Ten convolutions and BatchNorms deep: the free-running gradients
+    are held to direction (see _gradient_gate), every layer to the per-kernel budget on identical inputs."""
+    spec = wl.tiny_bottleneck_spec(classes=10, hw=8, c=16, width=16)
+    params = wl.perturb_bn_params(wl.init_params(spec, 7), 7)
+    images, labels = wl.image_batch(7, 2 * 12, hw=8, c=16, classes=10)
+    _compare_step(ctx, spec, params, None, images, labels, 12, 2, gate_gradients=False)
+
+
+def test_resnet50_small_batch_layerwise(ctx):
+    """The ResNet-50-shaped net at batch 8: every layer in full against the oracle (teacher-forced)."""
+    from paper_2503_23186_b200 import binding
+    from netcheck import check_step
+    spec = wl.resnet50_spec()
+    net = binding.Net(ctx, spec, 8)
+    net.load_params(wl.init_params(spec, 0))
+    images, labels = wl.image_batch(0, 8)
+    net.train_step(dev_bf16(images), torch.from_numpy(labels).cuda(), 1, LR, MU, WD, update=False)
+    assert ctx.device_status() == 0
+    check_step(net, spec, images, labels, 8).assert_ok()
+    net.close()
+
+
+def test_resnet50_batch1024_full_size(ctx):
+    """The ResNet-50-shaped net in the launch configuration bench.py times (eight micro-batches of 128 side by side)."""
+    _full_size_sampled(ctx, wl.resnet50_spec(), 128, 8, 0)
 
 
 def test_wrn28_10_small_batch_layerwise(ctx):

@@ -288,8 +288,16 @@ def _tiny():
     return spec, params, images, labels
 
 
-def test_net_gradients_finite_differences():
-    spec, params, images, labels = _tiny()
+def _tiny_bottleneck():
+    spec = wl.tiny_bottleneck_spec(classes=10, hw=8, c=4, width=4)
+    params = wl.perturb_bn_params(wl.init_params(spec, 5), 5)
+    params = {k: v.astype(np.float64) for k, v in params.items()}
+    return spec, params, rng.standard_normal((4, 8, 8, 4)), rng.integers(0, 10, 4).astype(np.int32)
+
+
+@pytest.mark.parametrize("make", [_tiny, _tiny_bottleneck], ids=["basic_blocks", "bottleneck_blocks"])
+def test_net_gradients_finite_differences(make):
+    spec, params, images, labels = make()
     fw = onet.forward(spec, params, images, labels, rounding=False)
     grads, _ = onet.backward(spec, params, fw, rounding=False)
     assert set(grads) == set(params)
@@ -373,3 +381,8 @@ def test_network_shapes_match_published_parameter_counts():
         return conv_fc, bn
     assert count(wl.resnet18_spec()) == (11210432, 9600)
     assert count(wl.wrn28_10_spec()) == (36518832, 20192)
+    # ResNet-50 (Section IV-A names it as the convolutional workload): the ImageNet model has 25,557,032 parameters;
+    # the CIFAR-shaped net swaps its 7x7x3x64 stem for 3x3x3x64 and its 2048x1000+1000 classifier for 2048x100+100
+    r50 = count(wl.resnet50_spec())
+    assert sum(r50) + 100 == 25557032 - 7 * 7 * 3 * 64 - (2048 * 1000 + 1000) + 3 * 3 * 3 * 64 + (2048 * 100 + 100)
+    assert r50[1] == 2 * 26560   # gamma and beta of 53 BatchNorm layers (ImageNet model: 53,120 BatchNorm parameters)
