@@ -803,22 +803,30 @@ __global__ void __launch_bounds__(kEwThreads) sgd_momentum_kernel(float4* __rest
 
 struct PackSegs {
     b2c_weight_seg seg[128];
+    int first_block[129];   // running total of (taps x tiles) per segment: block b belongs to the segment with first_block[s] <= b < first_block[s + 1]
+    int n_segs;
 };
 // dst[c][rs-1-t][k] = src[k][t][c] per segment: for a fixed tap this is a k x c -> c x k transpose, done in 32 x 32
 // tiles through shared memory so that both the reads (c contiguous) and the writes (k contiguous) are coalesced.
-// blockIdx.z = segment, blockIdx.y = tap, blockIdx.x = tile of the (k, c) plane; blocks past a segment's extent exit.
+// One block per (segment, tap, tile of the (k, c) plane), numbered consecutively over all segments.
 __global__ void weight_pack_dgrad_kernel(const __grid_constant__ PackSegs segs, const __nv_bfloat16* __restrict__ src,
                                          __nv_bfloat16* __restrict__ dst)
 {
     pdl_wait();   // first global access comes after the previous kernel of the stream
     pdl_launch_dependents();
     __shared__ __nv_bfloat16 tile[32][33];
-    const b2c_weight_seg sg = segs.seg[blockIdx.z];
-    const int t = blockIdx.y;
-    if (t >= sg.rs) return;
+    int lo = 0, hi = segs.n_segs;   // binary search for the segment of this block
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if ((int)blockIdx.x >= segs.first_block[mid]) lo = mid;
+        else hi = mid;
+    }
+    const b2c_weight_seg sg = segs.seg[lo];
+    const int local = (int)blockIdx.x - segs.first_block[lo];
     const int tiles_c = (sg.c + 31) / 32, tiles_k = (sg.k + 31) / 32;
-    if ((int)blockIdx.x >= tiles_c * tiles_k) return;
-    const int k0 = ((int)blockIdx.x / tiles_c) * 32, c0 = ((int)blockIdx.x % tiles_c) * 32;
+    const int t = local / (tiles_c * tiles_k), tile_id = local - t * (tiles_c * tiles_k);
+    if (t >= sg.rs) return;
+    const int k0 = (tile_id / tiles_c) * 32, c0 = (tile_id % tiles_c) * 32;
     for (int j = threadIdx.y; j < 32; j += 8) {          // blockDim = (32, 8)
         const int k = k0 + j, c = c0 + threadIdx.x;
         tile[j][threadIdx.x] = (k < sg.k && c < sg.c) ? src[sg.offset + ((long long)k * sg.rs + t) * sg.c + c] : __float2bfloat16(0.f);
@@ -1032,15 +1040,17 @@ b2c_status b2c_weight_pack_dgrad(b2c_ctx* ctx, const b2c_weight_seg* segs, int n
     if (!ctx || !segs || !src_bf16 || !dst_bf16) return B2C_ERR_INVALID_ARG;
     if (n_segs < 1 || n_segs > 128) return B2C_ERR_UNSUPPORTED_SHAPE;
     PackSegs ps;
-    int max_tiles = 0, max_rs = 0;
+    long long blocks = 0;
     for (int i = 0; i < n_segs; ++i) {
         if (segs[i].k < 1 || segs[i].rs < 1 || segs[i].c < 1 || segs[i].offset < 0) return B2C_ERR_INVALID_ARG;
         ps.seg[i] = segs[i];
-        const int tiles = ((segs[i].k + 31) / 32) * ((segs[i].c + 31) / 32);
-        max_tiles = tiles > max_tiles ? tiles : max_tiles;
-        max_rs = segs[i].rs > max_rs ? segs[i].rs : max_rs;
+        ps.first_block[i] = (int)blocks;
+        blocks += (long long)segs[i].rs * ((segs[i].k + 31) / 32) * ((segs[i].c + 31) / 32);
+        if (blocks > 0x7fffffffll) return B2C_ERR_UNSUPPORTED_SHAPE;
     }
-    dim3 grid((unsigned)max_tiles, (unsigned)max_rs, (unsigned)n_segs);
+    ps.first_block[n_segs] = (int)blocks;
+    ps.n_segs = n_segs;
+    dim3 grid((unsigned)blocks);
     B2C_CUDA(b2c_launch(ctx, weight_pack_dgrad_kernel, dim3(grid), dim3(dim3(32, 8)), 0, (cudaStream_t)stream_, 1u, ps, reinterpret_cast<const __nv_bfloat16*>(src_bf16),
                                                                               reinterpret_cast<__nv_bfloat16*>(dst_bf16)));
     B2C_CUDA(cudaGetLastError());
