@@ -101,6 +101,9 @@ __device__ __forceinline__ void bn_moments(const double* stats, int c, int ch, d
     invstd = rsqrtf((float)v + eps);
 }
 
+// UNROLL independent 16-byte loads per tensor and thread are in flight: without a residual the kernel reads one tensor,
+// so it takes twice the rows per step to keep as many bytes in flight as the residual variant (HBM latency x bandwidth).
+template <int UNROLL, bool RES>
 __global__ void __launch_bounds__(kEwThreads, 2) bn_apply_kernel(const void* __restrict__ y, long long m, int c, const double* __restrict__ stats_all,
                                                                  const float* __restrict__ gamma, const float* __restrict__ beta,
                                                                  const void* __restrict__ residual, int relu, float eps, void* __restrict__ a,
@@ -139,25 +142,25 @@ __global__ void __launch_bounds__(kEwThreads, 2) bn_apply_kernel(const void* __r
         bt[i] = beta[g * 8 + i];
     }
     const long long step = (long long)gridDim.x * rw.rows_per_iter;
-    for (long long r = (long long)blockIdx.x * rw.rows_per_iter + rl; r < m; r += kRowsUnroll * step) {
-        uint4 vy[kRowsUnroll], vr[kRowsUnroll];
+    for (long long r = (long long)blockIdx.x * rw.rows_per_iter + rl; r < m; r += UNROLL * step) {
+        uint4 vy[UNROLL], vr[RES ? UNROLL : 1];
 #pragma unroll
-        for (int u = 0; u < kRowsUnroll; ++u) {
+        for (int u = 0; u < UNROLL; ++u) {
             const bool ok = r + u * step < m;
             const long long vi = base + (r + u * step) * rw.groups + g;
             vy[u] = ld16_or_zero(y, vi, ok);
-            if (residual != nullptr) vr[u] = ld16_or_zero(residual, vi, ok);
+            if constexpr (RES) vr[u] = ld16_or_zero(residual, vi, ok);
         }
 #pragma unroll
-        for (int u = 0; u < kRowsUnroll; ++u) {
+        for (int u = 0; u < UNROLL; ++u) {
             if (r + u * step >= m) break;
             float f[8], res[8];
             unpack8(vy[u], f);
-            if (residual != nullptr) unpack8(vr[u], res);
+            if constexpr (RES) unpack8(vr[u], res);
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 float z = fmaf(f[i] - shift[i], scale[i], bt[i]);
-                if (residual != nullptr) z += res[i];
+                if constexpr (RES) z += res[i];
                 f[i] = (relu && z < 0.f) ? 0.f : z;
             }
             const uint4 packed = pack8(f);
@@ -858,8 +861,13 @@ b2c_status launch_bn_fwd(b2c_ctx* ctx, int G, long long m, int c, const void* y,
         B2C_CUDA(cudaMemsetAsync(stats, 0, sizeof(double) * 2 * c * G, stream));
         B2C_CUDA(b2c_launch(ctx, bn_stats_kernel, dim3(grid), dim3(kEwThreads), sizeof(float) * 2 * c, stream, 1u, y, m, c, stats));
     }
-    B2C_CUDA(b2c_launch(ctx, bn_apply_kernel, dim3(grid), dim3(kEwThreads), 0, stream, 1u, y, m, c, stats, gamma, beta, residual, relu, eps, a, save_mean, save_invstd, run_mean, run_var,
-                                                     momentum, relu ? reinterpret_cast<uint8_t*>(relu_mask) : nullptr));
+    uint8_t* mask_out = relu ? reinterpret_cast<uint8_t*>(relu_mask) : nullptr;
+    if (residual != nullptr)
+        B2C_CUDA(b2c_launch(ctx, bn_apply_kernel<4, true>, dim3(grid), dim3(kEwThreads), 0, stream, 1u, y, m, c, stats, gamma, beta, residual, relu, eps, a,
+                            save_mean, save_invstd, run_mean, run_var, momentum, mask_out));
+    else
+        B2C_CUDA(b2c_launch(ctx, bn_apply_kernel<8, false>, dim3(grid), dim3(kEwThreads), 0, stream, 1u, y, m, c, stats, gamma, beta, residual, relu, eps, a,
+                            save_mean, save_invstd, run_mean, run_var, momentum, mask_out));
     B2C_CUDA(cudaGetLastError());
     return B2C_OK;
 }
