@@ -65,9 +65,7 @@ void b2c_set_spin_limit(b2c_ctx* ctx, unsigned limit);
 /* Pipeline diagnostics of the convolution kernels.  `counters` is a DEVICE array of 8 unsigned 64-bit words owned
  * by the caller (NULL switches the feature off, the default).  Every CTA of the forward / data-gradient kernel adds
  * the SM clock cycles its roles spent waiting: [0] TMA producer for a free ring stage, [1] MMA thread for a loaded
- * stage, [2] MMA thread for a free accumulator, [3] first epilogue warp for a finished accumulator, [4] CTA lifetime
- * (first producer), [5] / [6] first epilogue warp inside its TMEM loads / its pack-store-sum code (tiles of up to 64
- * channels); [7] receives the MAXIMUM over CTAs of the time at which the first epilogue warp finished. */
+ * stage, [2] MMA thread for a free accumulator, [3] first epilogue warp for a finished accumulator, [4] CTA lifetime. */
 void b2c_set_stall_counters(b2c_ctx* ctx, unsigned long long* counters);
 
 /* ---- Forward pass (Algorithm 1, "Perform forward pass") -------------------------------- */

@@ -18,11 +18,10 @@
 //     offsets of one image row (a multiple of the swizzle period), so the input is fetched three
 //     times instead of nine.
 //   * Small filter banks stay resident in shared memory for the whole launch.
-// Warp roles: warpgroup 0 = control (warp 0 = first TMA producer, warp 1 = TMEM owner + first MMA issuer, warp 2 =
-// second MMA issuer, warp 3 = second TMA producer; one lane at work in each; the two issuers take alternate units, the
-// two producers alternate stages), warps 4..11 = epilogue (two per TMEM lane quarter, splitting the columns).  The
-// control warpgroup hands most of its registers to the epilogue warpgroups (setmaxnreg), which use them to fetch the
-// next accumulator from TMEM while they pack, store and sum the current one.  Every mbarrier wait is bounded.
+// Warp roles: warp 0 = first TMA producer (one lane), warp 1 = TMEM owner + first MMA issuer (one lane),
+// warps 2..9 = epilogue (two per TMEM lane quarter, splitting the columns), warp 10 = second MMA issuer (one lane;
+// the two issuers take alternate units), warp 11 = second TMA producer (one lane; the two producers take alternate
+// stages).  Every mbarrier wait is bounded.
 #include "common.h"
 #include "ptx.cuh"
 
@@ -65,20 +64,16 @@ struct alignas(64) ConvKParams {
     int stats_group_images;          // images per BatchNorm statistics group (0: one group)
     unsigned* status;
     unsigned spin_limit;
-    unsigned long long* stall;       // optional [8]: cycles waited by producer / MMA (ring) / MMA (accumulator) / epilogue, CTA lifetime, epilogue warp 0 in TMEM loads / in pack-store-sum (narrow tiles)
+    unsigned long long* stall;       // optional [5]: cycles waited by producer / MMA (ring) / MMA (accumulator) / epilogue, CTA lifetime
 };
 
 static constexpr int kMaxStages = 8;
 static constexpr int kMaxAccBufs = 4;
 static constexpr int kEpiWarps = 8;
-static constexpr int kIssuers = 2;       // MMA-issuing threads: warps 1 and 2
-static constexpr int kProducers = 2;     // TMA-issuing threads: warps 0 and 3; they take alternate stages
-static constexpr int kCtrlWarps = 4;     // warpgroup 0
-static constexpr int kThreads = 32 * (kCtrlWarps + kEpiWarps);
-static constexpr int kProducerWarp1 = 3;   // warp index of the second producer
-// Registers per thread after the split: launched with 168 x 384 = 64512; 128 x 80 + 256 x 208 = 63488 fit.
-static constexpr int kCtrlRegs = 80, kEpiRegs = 208;
-static_assert(kThreads == 384 && 128 * kCtrlRegs + 256 * kEpiRegs <= 384 * 168, "register split exceeds the launch allocation");
+static constexpr int kIssuers = 2;       // MMA-issuing threads: warp 1 and the warps after the epilogue warps
+static constexpr int kProducers = 2;     // TMA-issuing threads: warp 0 and the warp after the issuer warps; they take alternate stages
+static constexpr int kThreads = 64 + 32 * kEpiWarps + 32 * (kIssuers - 1) + 32 * (kProducers - 1);
+static constexpr int kProducerWarp1 = 2 + kEpiWarps + (kIssuers - 1);   // warp index of the second producer
 static constexpr uint32_t kDrainPolls = 1u << 22;
 
 struct UnitCoord {
@@ -156,12 +151,12 @@ __device__ __forceinline__ void butterfly16(float (&a)[16], float (&b)[16], int 
 // are reduced over rows per unit into a per-warp shared-memory array.
 template <int NCH>
 __device__ __forceinline__ void epilogue_loop(const ConvKParams& p, uint32_t tmem_base, uint64_t* acc_full, uint64_t* acc_empty,
-                                              uint32_t* abort_flag, float* my_stats, int e, int lane, int rank, long long t_start)
+                                              uint32_t* abort_flag, float* my_stats, int e, int lane, int rank)
 {
     const UnitWalk walk(p, rank);
     // the accumulator-free barrier lives in the leader CTA of a pair: the peer's warps arrive on it remotely
     const bool remote_empty = p.pair && rank != 0;
-    const int q = e & 3;             // TMEM lane quarter this warp may read: (warp index in the CTA) % 4, epilogue warps start at 4
+    const int q = (e + 2) & 3;       // TMEM lane quarter this warp may read: (warp index in the CTA) % 4, epilogue warps start at 2
     const int m = q * 32 + lane;     // accumulator row = pixel of the tile (w fastest, then h, then image)
     const int lw = m % p.bw, lh = (m / p.bw) % p.bh, ln = m / (p.bw * p.bh);
     const bool do_stats = p.stats != nullptr;
@@ -215,8 +210,26 @@ __device__ __forceinline__ void epilogue_loop(const ConvKParams& p, uint32_t tme
         }
     };
 
-    // Per-unit pieces shared by both paths below.
-    auto enter_group = [&](const UnitCoord& c) {   // statistics bookkeeping before a unit's values are summed
+    for (int pu = walk.first; pu < walk.count; pu += walk.stride) {
+        const UnitCoord c = decode_unit(p, walk.unit(p, pu));
+        const int n_it = unit_iters(p, c.par);
+        const bool row_valid = (c.n0 + ln) < p.n_valid;
+        const long long row_off = (long long)(c.n0 + ln) * p.os_n + (long long)(c.oh0 + lh) * p.os_h + (long long)(c.ow0 + lw) * p.os_w + p.off[c.par];
+        int buf = 0;
+        if (n_it > 0) {
+            buf = jacc & (p.acc_bufs - 1);
+            const long long w3 = clock64();
+            ok = true;
+            if (lane == 0) ok = mbar_wait_bounded(&acc_full[buf], (uint32_t)(jacc >> p.acc_shift) & 1u, p.spin_limit, abort_flag);   // one poller per warp
+            epi_wait += clock64() - w3;
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) {
+                if (lane == 0) atomicOr(p.status, B2C_DEV_TIMEOUT);
+                break;
+            }
+            tc_fence_after();
+            ++jacc;
+        }
         if (do_stats) {
             const int grp = p.stats_group_images > 0 ? (p.grp_shift >= 0 ? c.n0 >> p.grp_shift : c.n0 / p.stats_group_images) : 0;
             if (grp != cur_group) {
@@ -225,89 +238,52 @@ __device__ __forceinline__ void epilogue_loop(const ConvKParams& p, uint32_t tme
             }
             cur_ktile = c.ktile;
         }
-    };
-    // the accumulator is handed back to the MMA thread as soon as this warp has read its last column
-    auto release = [&](int n_it, int buf) {
-        if (n_it > 0) {
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) {
-                if (remote_empty) mbar_arrive_cluster(map_to_cta(smem_u32(&acc_empty[buf]), 0));
-                else mbar_arrive(&acc_empty[buf]);
+        const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * p.acc_cols + col_begin);
+        // the accumulator is handed back to the MMA thread as soon as this warp has read its last column
+        auto release = [&]() {
+            if (n_it > 0) {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    if (remote_empty) mbar_arrive_cluster(map_to_cta(smem_u32(&acc_empty[buf]), 0));
+                    else mbar_arrive(&acc_empty[buf]);
+                }
             }
-        }
-    };
-    // bias, rounding and stores of one 16-column chunk; returns the values as stored in pk
-    auto store_chunk = [&](const UnitCoord& c, bool row_valid, long long row_off, const uint32_t (&r)[16], int c0, uint32_t (&pk)[8]) {
-        const int ch0 = c.ktile * p.n_tile + col_begin + c0;  // first output channel of this chunk
-        float v[16];
+        };
+        // bias, rounding and stores of one 16-column chunk; returns the values as stored in pk
+        auto store_chunk = [&](const uint32_t (&r)[16], int c0, uint32_t (&pk)[8]) {
+            const int ch0 = c.ktile * p.n_tile + col_begin + c0;  // first output channel of this chunk
+            float v[16];
 #pragma unroll
-        for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
-        if (p.bias != nullptr) {
+            for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+            if (p.bias != nullptr) {
 #pragma unroll
-            for (int i = 0; i < 16; ++i) v[i] += (ch0 + i < p.oc_valid) ? __ldg(p.bias + ch0 + i) : 0.f;
-        }
-        if (p.out_is_f32) {
+                for (int i = 0; i < 16; ++i) v[i] += (ch0 + i < p.oc_valid) ? __ldg(p.bias + ch0 + i) : 0.f;
+            }
+            if (p.out_is_f32) {
+                if (row_valid) {
+                    float* dst = reinterpret_cast<float*>(p.out) + row_off + ch0;
+#pragma unroll
+                    for (int i = 0; i < 16; i += 4)
+                        if (ch0 + i < p.oc_valid) *reinterpret_cast<float4*>(dst + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                }
+                return;
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) pk[i] = pack_bf16x2(v[2 * i], v[2 * i + 1]);
             if (row_valid) {
-                float* dst = reinterpret_cast<float*>(p.out) + row_off + ch0;
-#pragma unroll
-                for (int i = 0; i < 16; i += 4)
-                    if (ch0 + i < p.oc_valid) *reinterpret_cast<float4*>(dst + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + row_off + ch0;
+                if (p.out_v8 && ch0 + 8 < p.oc_valid) {
+                    st_global_v8(dst, pk);   // one full 32-byte sector per lane
+                } else {
+                    if (ch0 < p.oc_valid) *reinterpret_cast<uint4*>(dst) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    if (ch0 + 8 < p.oc_valid) *reinterpret_cast<uint4*>(dst + 8) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                }
             }
-            return;
-        }
-#pragma unroll
-        for (int i = 0; i < 8; ++i) pk[i] = pack_bf16x2(v[2 * i], v[2 * i + 1]);
-        if (row_valid) {
-            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + row_off + ch0;
-            if (p.out_v8 && ch0 + 8 < p.oc_valid) {
-                st_global_v8(dst, pk);   // one full 32-byte sector per lane
-            } else {
-                if (ch0 < p.oc_valid) *reinterpret_cast<uint4*>(dst) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                if (ch0 + 8 < p.oc_valid) *reinterpret_cast<uint4*>(dst + 8) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
-            }
-        }
-    };
-    // Waits for the accumulator of the CTA's next unit (blocking == false: one probe) and reports it.
-    // Returns 1 = ready (n_it, buf set; n_it == 0: a unit without taps, nothing to wait for), 0 = not yet, -1 = the wait gave up.
-    auto acquire = [&](int pu, bool blocking, int& n_it, int& buf) -> int {
-        n_it = p.n_par > 1 ? unit_iters(p, decode_unit(p, walk.unit(p, pu)).par) : unit_iters(p, 0);
-        buf = 0;
-        if (n_it == 0) return 1;
-        buf = jacc & (p.acc_bufs - 1);
-        const uint32_t parity = (uint32_t)(jacc >> p.acc_shift) & 1u;
-        bool got = true;
-        if (blocking) {
-            const long long w3 = clock64();
-            if (lane == 0) got = mbar_wait_bounded(&acc_full[buf], parity, p.spin_limit, abort_flag);   // one poller per warp
-            epi_wait += clock64() - w3;
-            if (!__all_sync(0xffffffffu, got)) return -1;
-        } else {
-            if (lane == 0) got = mbar_test_wait(&acc_full[buf], parity);
-            if (!__all_sync(0xffffffffu, got)) return 0;
-        }
-        tc_fence_after();
-        ++jacc;
-        return 1;
-    };
+        };
 
-    if constexpr (NCH > 0) {
-        // Narrow tiles: read all of this warp's columns at once, free the accumulator, then work from registers.
-        long long t_ld = 0, t_proc = 0;
-        const bool timed = p.stall != nullptr;
-        for (int pu = walk.first; pu < walk.count; pu += walk.stride) {
-            const UnitCoord c = decode_unit(p, walk.unit(p, pu));
-            const bool row_valid = (c.n0 + ln) < p.n_valid;
-            const long long row_off = (long long)(c.n0 + ln) * p.os_n + (long long)(c.oh0 + lh) * p.os_h + (long long)(c.ow0 + lw) * p.os_w + p.off[c.par];
-            int n_it = 0, buf = 0;
-            if (acquire(pu, true, n_it, buf) < 0) {
-                ok = false;
-                if (lane == 0) atomicOr(p.status, B2C_DEV_TIMEOUT);
-                break;
-            }
-            enter_group(c);
-            const long long t0 = timed ? clock64() : 0;
-            const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * p.acc_cols + col_begin);
+        if constexpr (NCH > 0) {
+            // narrow tiles: read all of this warp's columns at once, free the accumulator, then work from registers
             uint32_t r[NCH][16];
 #pragma unroll
             for (int ck = 0; ck < NCH; ++ck) {
@@ -319,13 +295,12 @@ __device__ __forceinline__ void epilogue_loop(const ConvKParams& p, uint32_t tme
                 }
             }
             if (n_it > 0) tmem_ld_wait();
-            release(n_it, buf);
-            const long long t1 = timed ? clock64() : 0;
+            release();
 #pragma unroll
             for (int ck = 0; ck < NCH; ++ck) {
                 if (ck < n_chunks) {
                     uint32_t pk[8];
-                    store_chunk(c, row_valid, row_off, r[ck], ck * 16, pk);
+                    store_chunk(r[ck], ck * 16, pk);
                     if (do_stats && row_valid) {   // sums of the values as stored, kept per row in registers
 #pragma unroll
                         for (int i = 0; i < 8; ++i) {
@@ -339,31 +314,10 @@ __device__ __forceinline__ void epilogue_loop(const ConvKParams& p, uint32_t tme
                     }
                 }
             }
-            if (timed) {
-                t_ld += t1 - t0;
-                t_proc += clock64() - t1;
-            }
-        }
-        if (timed && e == 0 && lane == 0) {
-            atomicAdd(p.stall + 5, (unsigned long long)t_ld);
-            atomicAdd(p.stall + 6, (unsigned long long)t_proc);
-        }
-    } else {
-        for (int pu = walk.first; pu < walk.count; pu += walk.stride) {
-            const UnitCoord c = decode_unit(p, walk.unit(p, pu));
-            const bool row_valid = (c.n0 + ln) < p.n_valid;
-            const long long row_off = (long long)(c.n0 + ln) * p.os_n + (long long)(c.oh0 + lh) * p.os_h + (long long)(c.ow0 + lw) * p.os_w + p.off[c.par];
-            int n_it = 0, buf = 0;
-            if (acquire(pu, true, n_it, buf) < 0) {
-                ok = false;
-                if (lane == 0) atomicOr(p.status, B2C_DEV_TIMEOUT);
-                break;
-            }
-            enter_group(c);
-            const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * p.acc_cols + col_begin);
+        } else {
             auto process = [&](const uint32_t (&r)[16], int c0) {
                 uint32_t pk[8];
-                store_chunk(c, row_valid, row_off, r, c0, pk);
+                store_chunk(r, c0, pk);
                 if (do_stats && !p.out_is_f32) {
                     float a[16], b[16];
 #pragma unroll
@@ -391,7 +345,7 @@ __device__ __forceinline__ void epilogue_loop(const ConvKParams& p, uint32_t tme
 #pragma unroll
                 for (int i = 0; i < 16; ++i) ra[i] = rb[i] = 0u;
             }
-            if (n_chunks <= 1) release(n_it, buf);
+            if (n_chunks <= 1) release();
             for (int ck = 0; ck < n_chunks; ck += 2) {
                 // chunk ck is in ra; fetch ck+1 into rb while ra is processed, then ck+2 into ra while rb is processed
                 if (n_it > 0 && ck + 1 < n_chunks) tmem_ld16(t_row + (uint32_t)((ck + 1) * 16), rb);
@@ -399,23 +353,20 @@ __device__ __forceinline__ void epilogue_loop(const ConvKParams& p, uint32_t tme
                 if (ck + 1 < n_chunks) {
                     if (n_it > 0) {
                         tmem_ld_wait();
-                        if (ck + 2 == n_chunks) release(n_it, buf);
+                        if (ck + 2 == n_chunks) release();
                         if (ck + 2 < n_chunks) tmem_ld16(t_row + (uint32_t)((ck + 2) * 16), ra);
                     }
                     process(rb, (ck + 1) * 16);
                     if (n_it > 0 && ck + 2 < n_chunks) {
                         tmem_ld_wait();
-                        if (ck + 3 == n_chunks) release(n_it, buf);
+                        if (ck + 3 == n_chunks) release();
                     }
                 }
             }
         }
     }
     if (do_stats && cur_group >= 0 && ok) flush_stats();
-    if (p.stall != nullptr && e == 0 && lane == 0) {
-        atomicAdd(p.stall + 3, (unsigned long long)epi_wait);
-        atomicMax(p.stall + 7, (unsigned long long)(clock64() - t_start));   // the slowest CTA bounds the launch
-    }
+    if (p.stall != nullptr && e == 0 && lane == 0) atomicAdd(p.stall + 3, (unsigned long long)epi_wait);
 }
 
 // Issues the MMAs of one stage: NB sub-tiles (vertical taps) x KS k-steps of 16 channels, fully unrolled so that
@@ -621,7 +572,6 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
     int last_issued = -1;  // producer lanes: index of the last stage whose loads this lane issued
 
     if (warp == 0 || warp == kProducerWarp1) {
-        setmaxnreg_dec<kCtrlRegs>();   // every warp of the control warpgroup gives up registers (here and in the issuer branch)
         if (lane == 0) {
             // ------------------------------------------------------------ TMA producers
             // Producer w fills the ring slots w, w + kProducers, ...: the chain wait -> expect -> issue of one thread
@@ -720,11 +670,10 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
                 atomicAdd(p.stall + 4, (unsigned long long)(clock64() - t_start));
             }
         }
-    } else if (warp == 1 || warp == 2) {
-        setmaxnreg_dec<kCtrlRegs>();
+    } else if (warp == 1 || (warp >= 2 + kEpiWarps && warp < kProducerWarp1)) {
         if (lane == 0 && rank == 0) {
             // ------------------------------------------------------------ MMA issuers (in the leader CTA of a pair)
-            const int my = warp - 1;
+            const int my = warp == 1 ? 0 : warp - (2 + kEpiWarps) + 1;
             if (my < p.issuers) {
             const uint32_t smem_addr = smem_u32(smem), ring_addr = smem_u32(ring);
             const int ksteps = p.kb >> 4;
@@ -743,14 +692,13 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
         }
     } else {
         // ---------------------------------------------------------------- epilogue (8 warps)
-        setmaxnreg_inc<kEpiRegs>();   // both epilogue warpgroups take what the control warpgroup released
-        const int e = warp - kCtrlWarps;
+        const int e = warp - 2;
         if (p.n_tile <= 32 && !p.out_is_f32)
-            epilogue_loop<1>(p, tmem_base, acc_full, acc_empty, &abort_flag, s_stats[e], e, lane, rank, t_start);
+            epilogue_loop<1>(p, tmem_base, acc_full, acc_empty, &abort_flag, s_stats[e], e, lane, rank);
         else if (p.n_tile <= 64 && !p.out_is_f32)
-            epilogue_loop<2>(p, tmem_base, acc_full, acc_empty, &abort_flag, s_stats[e], e, lane, rank, t_start);
+            epilogue_loop<2>(p, tmem_base, acc_full, acc_empty, &abort_flag, s_stats[e], e, lane, rank);
         else
-            epilogue_loop<0>(p, tmem_base, acc_full, acc_empty, &abort_flag, s_stats[e], e, lane, rank, t_start);
+            epilogue_loop<0>(p, tmem_base, acc_full, acc_empty, &abort_flag, s_stats[e], e, lane, rank);
     }
     tc_fence_before();
     __syncthreads();
@@ -770,7 +718,7 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
                 for (uint32_t i = 0; i < kDrainPolls && !mbar_try_wait(&full_bar[sl], (uint32_t)(it / S) & 1u); ++i) {}
             }
         }
-        if ((warp == 1 || warp == 2) && lane == 0 && rank == 0) {   // a commit covers the MMAs of the thread that makes it
+        if ((warp == 1 || (warp >= 2 + kEpiWarps && warp < kProducerWarp1)) && lane == 0 && rank == 0) {   // a commit covers the MMAs of the thread that makes it
             if constexpr (PAIR) umma_commit_pair(&drain_bar, (uint16_t)1);
             else umma_commit(&drain_bar);
             if (warp == 1)
