@@ -14,6 +14,14 @@
 // second gathered one row higher, are stacked on M: with x gathered at (r0 - pad, s - pad) the rows of
 // copy a accumulate tap (r0 + a, s), since sum_p dy[p - (a,0)] x[p + t] = sum_p dy[p] x[p + t + (a,0)].
 // Partial sums of the pixel ranges are added to dw with vector fp32 reductions.
+//
+// Framed x stages (3x3, stride 1, image rows of at least 8 pixels, 64-channel x boxes): instead of one x box per
+// horizontal shift, a stage holds each 64-channel block of the chunk once, with one extra pixel left and right of every
+// image row (box of bw + 2 pixels).  The operand of shift s is the same box read from a start address s pixel rows
+// (s x 128 bytes) further in: the k-step of 16 pixels starts at row h * (bw + 2) + w0 + s, and the three shifts are the
+// three 64-column blocks of one N = 192 MMA whose block stride (LBO) is one pixel row.  The 128-byte swizzle is keyed on
+// absolute shared-memory address bits, so a start that is not a multiple of the 8-row atom reads the right data
+// (the parity tests cover it).  The x tensor crosses L2 -> SM once per filter row instead of three times.
 #include "common.h"
 #include "ptx.cuh"
 
@@ -43,6 +51,10 @@ struct alignas(64) WgradParams {
     int tw_shift;                         // log2(tiles_w)
     int stage_bytes;
     int n_pieces, piece_t0[3], piece_nt[3];   // MMAs per k-step: first shift and number of shifts each covers
+    int fx;                               // framed x stages: one box of (bw + 2) x bh pixels per 64-channel block serves the three shifts
+    int fx_box, fx_tx;                    // shared-memory footprint (1 KB multiple) and bytes delivered per framed box
+    uint32_t fx_koff[4];                  // start of k-step kk inside a framed box, in 16-byte units
+    uint32_t fx_sbo;                      // byte distance between the two 8-pixel groups of a k-step
     int k_total, c_total, rs_total;
     float* dw;
     unsigned* status;
@@ -61,6 +73,19 @@ __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float 
 }
 
 // One MMA per k-step of 16 pixels, unrolled: descriptors differ only in their low (address) word.
+// Framed x: the B operand of k-step kk starts at its own row offset inside the framed box.
+template <int KS>
+__device__ __forceinline__ void wg_issue_framed(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t a_hi, uint32_t b_hi, uint32_t idesc,
+                                                uint32_t kstep_a, uint32_t k0, uint32_t k1, uint32_t k2, uint32_t k3, uint32_t accumulate_first)
+{
+#pragma unroll
+    for (int kk = 0; kk < KS; ++kk) {
+        const uint32_t koff = kk == 0 ? k0 : kk == 1 ? k1 : kk == 2 ? k2 : k3;
+        const uint64_t ad = ((uint64_t)a_hi << 32) | (uint64_t)(a_lo + (uint32_t)kk * kstep_a);
+        const uint64_t bd = ((uint64_t)b_hi << 32) | (uint64_t)(b_lo + koff);
+        umma_bf16(d_tmem, ad, bd, idesc, kk == 0 ? accumulate_first : 1u);
+    }
+}
 template <int KS>
 __device__ __forceinline__ void wg_issue(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t a_hi, uint32_t b_hi, uint32_t idesc,
                                          uint32_t kstep_a, uint32_t kstep_b, uint32_t accumulate_first)
@@ -126,7 +151,7 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
             // longer than the MMAs of a stage take.  Each slot keeps one producer, which uses it strictly in order.
             prefetch_tensormap(&p.tmDy);
             prefetch_tensormap(&p.tmX[0]);
-            const uint32_t tx = (uint32_t)(p.a_bytes + grp.nb * p.b_boxes * p.box_b);
+            const uint32_t tx = p.fx ? (uint32_t)(p.a_bytes + p.b_boxes * p.fx_tx) : (uint32_t)(p.a_bytes + grp.nb * p.b_boxes * p.box_b);
             int it = w, s = w;
             uint32_t ph = 0u;
             while (it < n_chunks) {
@@ -151,6 +176,11 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
                         tma_load_4d(dst + (size_t)j * p.box_a, &p.tmDy, &full_bar[s], ktile * 128 + j * p.cw_a, ow0, oh0, n0);
                 }
                 dst += p.a_bytes;
+                if (p.fx) {   // one framed box per channel block, gathered at the first shift (one pixel to the left)
+                    for (int j = 0; j < p.b_boxes; ++j)
+                        tma_load_4d(dst + (size_t)j * p.fx_box, &p.tmX[grp.map[0]], &full_bar[s], ctile * p.ct + j * p.cw_b, ow0 + grp.dw[0],
+                                    oh0 + grp.dh[0], n0);
+                } else
                 for (int b = 0; b < grp.nb; ++b)
                     for (int j = 0; j < p.b_boxes; ++j)
                         tma_load_4d(dst + (size_t)(b * p.b_boxes + j) * p.box_b, &p.tmX[grp.map[b]], &full_bar[s], ctile * p.ct + j * p.cw_b,
@@ -170,7 +200,9 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
         if (lane == 0) {
             // SBO = eight pixel rows, LBO = next block of cw channels (the next box)
             const uint64_t proto_a = make_smem_desc(0u, (uint32_t)p.a_lbo, 16u * (uint32_t)p.cw_a, (uint32_t)p.swz_a);
-            const uint64_t proto_b = make_smem_desc(0u, (uint32_t)p.box_b, 16u * (uint32_t)p.cw_b, (uint32_t)p.swz_b);
+            // framed x: the 64-column blocks of an MMA are the three shifts, one pixel row (128 bytes) apart
+            const uint64_t proto_b = p.fx ? make_smem_desc(0u, 128u, p.fx_sbo, (uint32_t)p.swz_b)
+                                          : make_smem_desc(0u, (uint32_t)p.box_b, 16u * (uint32_t)p.cw_b, (uint32_t)p.swz_b);
             const uint32_t a_hi = (uint32_t)(proto_a >> 32), a_lo_base = (uint32_t)proto_a;
             const uint32_t b_hi = (uint32_t)(proto_b >> 32), b_lo_base = (uint32_t)proto_b;
             const uint32_t kstep_a = (uint32_t)(16 * p.cw_a * 2) >> 4, kstep_b = (uint32_t)(16 * p.cw_b * 2) >> 4;   // 16 pixel rows
@@ -179,11 +211,12 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
             uint32_t idesc0 = 0, idesc1 = 0, idesc2 = 0, boff0 = 0, boff1 = 0, boff2 = 0, dcol0 = 0, dcol1 = 0, dcol2 = 0;
             int n_pieces = 0;
             for (int i = 0; i < p.n_pieces; ++i) {
-                if (p.piece_t0[i] >= grp.nb) break;
+                if (!p.fx && p.piece_t0[i] >= grp.nb) break;
                 const int nt = min(p.piece_nt[i], grp.nb - p.piece_t0[i]);
-                const uint32_t id = make_idesc_bf16(128, nt * p.ct, true, true);
-                const uint32_t bo = (uint32_t)(p.a_bytes + p.piece_t0[i] * p.b_boxes * p.box_b) >> 4;
-                const uint32_t dc = (uint32_t)(p.piece_t0[i] * p.ct);
+                // framed x: piece i = channel block i, N = three shifts x 64 channels
+                const uint32_t id = p.fx ? make_idesc_bf16(128, 192, true, true) : make_idesc_bf16(128, nt * p.ct, true, true);
+                const uint32_t bo = p.fx ? (uint32_t)(p.a_bytes + i * p.fx_box) >> 4 : (uint32_t)(p.a_bytes + p.piece_t0[i] * p.b_boxes * p.box_b) >> 4;
+                const uint32_t dc = p.fx ? (uint32_t)(i * 192) : (uint32_t)(p.piece_t0[i] * p.ct);
                 if (i == 0) { idesc0 = id; boff0 = bo; dcol0 = dc; }
                 else if (i == 1) { idesc1 = id; boff1 = bo; dcol1 = dc; }
                 else { idesc2 = id; boff2 = bo; dcol2 = dc; }
@@ -202,7 +235,11 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
                 const uint32_t st16 = smem_u32(smem + (size_t)s * p.stage_bytes) >> 4;
                 const uint32_t a_lo = a_lo_base + st16, b_lo = b_lo_base + st16;
                 const uint32_t acc0 = it != 0 ? 1u : 0u;
-                if (ksteps == 4) {
+                if (p.fx) {   // chunks of 64 pixels: four k-steps
+                    wg_issue_framed<4>(tmem_base + dcol0, a_lo, b_lo + boff0, a_hi, b_hi, idesc0, kstep_a, p.fx_koff[0], p.fx_koff[1], p.fx_koff[2], p.fx_koff[3], acc0);
+                    if (n_pieces > 1)
+                        wg_issue_framed<4>(tmem_base + dcol1, a_lo, b_lo + boff1, a_hi, b_hi, idesc1, kstep_a, p.fx_koff[0], p.fx_koff[1], p.fx_koff[2], p.fx_koff[3], acc0);
+                } else if (ksteps == 4) {
                     wg_issue<4>(tmem_base + dcol0, a_lo, b_lo + boff0, a_hi, b_hi, idesc0, kstep_a, kstep_b, acc0);
                     if (n_pieces > 1) wg_issue<4>(tmem_base + dcol1, a_lo, b_lo + boff1, a_hi, b_hi, idesc1, kstep_a, kstep_b, acc0);
                     if (n_pieces > 2) wg_issue<4>(tmem_base + dcol2, a_lo, b_lo + boff2, a_hi, b_hi, idesc2, kstep_a, kstep_b, acc0);
@@ -235,11 +272,15 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
                 const bool live = rs >= 0 && k < p.k_total;
                 float* dst_row = p.dw + ((long long)(live ? k : 0) * p.rs_total + (live ? rs : 0)) * p.c_total + ctile * p.ct;
                 // two chunks in flight: the next one is fetched while the current one is sent out
+                // accumulator column of 16-channel chunk ck of shift b (framed x: [channel block][shift][64 channels])
+                auto col = [&](int ck) -> uint32_t {
+                    return p.fx ? (uint32_t)((ck >> 2) * 192 + b * 64 + (ck & 3) * 16) : (uint32_t)(b * p.ct + ck * 16);
+                };
                 uint32_t ra[16], rb[16];
-                tmem_ld16(t_row + (uint32_t)(b * p.ct), ra);
+                tmem_ld16(t_row + col(0), ra);
                 tmem_ld_wait();
                 for (int ck = 0; ck < n_ck; ck += 2) {
-                    if (ck + 1 < n_ck) tmem_ld16(t_row + (uint32_t)(b * p.ct + (ck + 1) * 16), rb);
+                    if (ck + 1 < n_ck) tmem_ld16(t_row + col(ck + 1), rb);
                     if (live) {
 #pragma unroll
                         for (int i = 0; i < 16; i += 4)
@@ -248,7 +289,7 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
                     }
                     if (ck + 1 < n_ck) {
                         tmem_ld_wait();
-                        if (ck + 2 < n_ck) tmem_ld16(t_row + (uint32_t)(b * p.ct + (ck + 2) * 16), ra);
+                        if (ck + 2 < n_ck) tmem_ld16(t_row + col(ck + 2), ra);
                         if (live) {
 #pragma unroll
                             for (int i = 0; i < 16; i += 4)
@@ -308,16 +349,22 @@ b2c_status launch_conv_wgrad(b2c_ctx* ctx, const WgradProblem& pb, cudaStream_t 
     p.ct = p.cw_b;
     for (int cand = 160; cand >= p.cw_b; cand -= 16)
         if (pb.c % cand == 0 && cand % p.cw_b == 0) { p.ct = cand; break; }
+    // framed x stages: 64 pixels of one image per chunk, 64-channel x boxes, at most two of them per CTA (2 x 192 TMEM columns)
+    p.fx = (R == 3 && pb.stride == 1 && pb.q >= 8 && pb.p * pb.q >= 64 && p.cw_b == 64 && ctx->use_wgrad_frame) ? 1 : 0;
+    if (p.fx) p.ct = (pb.c % 128 == 0) ? 128 : 64;
     p.n_ctiles = pb.c / p.ct;
     p.n_ktiles = p.stack ? 1 : (pb.k + 127) / 128;
     p.a_boxes = p.stack ? 2 : 128 / p.cw_a;
     p.b_boxes = p.ct / p.cw_b;
     const int shifts = R == 3 ? 3 : 1;
     p.tmem_cols = 32;
-    while (p.tmem_cols < shifts * p.ct) p.tmem_cols *= 2;
+    while (p.tmem_cols < (p.fx ? p.b_boxes * 192 : shifts * p.ct)) p.tmem_cols *= 2;
     if (p.tmem_cols > 512) return B2C_ERR_UNSUPPORTED_SHAPE;
     // MMAs per k-step: merge the column blocks of consecutive shifts while N stays within 256
-    if (shifts * p.ct <= 256) {
+    if (p.fx) {
+        p.n_pieces = p.b_boxes;   // one N = 192 MMA per 64-channel block
+        for (int i = 0; i < p.n_pieces; ++i) { p.piece_t0[i] = 0; p.piece_nt[i] = 3; }
+    } else if (shifts * p.ct <= 256) {
         p.n_pieces = 1; p.piece_t0[0] = 0; p.piece_nt[0] = shifts;
     } else if (2 * p.ct <= 256) {
         p.n_pieces = 2; p.piece_t0[0] = 0; p.piece_nt[0] = 2; p.piece_t0[1] = 2; p.piece_nt[1] = 1;
@@ -365,9 +412,16 @@ b2c_status launch_conv_wgrad(b2c_ctx* ctx, const WgradProblem& pb, cudaStream_t 
         p.box_b = p.pb * p.cw_b * 2;
         p.a_bytes = p.stack ? (p.pb + (pb.q < p.pb ? pb.q : p.pb)) * p.cw_a * 2 : p.a_boxes * p.box_a;   // stacked: one box with a halo row
         p.stage_bytes = p.a_bytes + shifts * p.b_boxes * p.box_b;
+        if (p.fx) {
+            const int bw = pb.q < p.pb ? pb.q : p.pb, bh = p.pb / bw;
+            p.fx_tx = (bw + 2) * bh * 128;
+            p.fx_box = (p.fx_tx + 1023) & ~1023;
+            p.stage_bytes = p.a_bytes + p.b_boxes * p.fx_box;
+        }
         if (p.stage_bytes * 3 <= 200 * 1024 || p.pb == 32) break;
         p.pb = 32;
     }
+    if (p.fx && p.pb != 64) return B2C_ERR_UNSUPPORTED_SHAPE;   // cannot happen: a framed stage is under 40 KB
     int stages = (200 * 1024) / p.stage_bytes;
     if (stages > kWgStages) stages = kWgStages;
     if (stages < 2) return B2C_ERR_UNSUPPORTED_SHAPE;
@@ -376,6 +430,14 @@ b2c_status launch_conv_wgrad(b2c_ctx* ctx, const WgradProblem& pb, cudaStream_t 
     p.bh = (p.pb / p.bw) < pb.p ? (p.pb / p.bw) : pb.p;
     p.bn = p.pb / (p.bw * p.bh);
     if (p.stack && p.bn != 1) return B2C_ERR_UNSUPPORTED_SHAPE;   // cannot happen: 64 pixels per image guarantee bn == 1
+    if (p.fx) {
+        if (p.bn != 1) return B2C_ERR_UNSUPPORTED_SHAPE;   // cannot happen: at least 64 pixels per image
+        for (int kk = 0; kk < 4; ++kk) {
+            const int pix = 16 * kk, h = pix / p.bw, w0 = pix % p.bw;   // bw == 8: a k-step covers image rows 2kk and 2kk + 1
+            p.fx_koff[kk] = (uint32_t)((h * (p.bw + 2) + w0) * 128) >> 4;
+        }
+        p.fx_sbo = p.bw == 8 ? 10u * 128u : 1024u;
+    }
     p.tiles_w = pb.q / p.bw;
     p.tw_shift = 0;
     while ((1 << p.tw_shift) < p.tiles_w) ++p.tw_shift;
@@ -396,7 +458,7 @@ b2c_status launch_conv_wgrad(b2c_ctx* ctx, const WgradProblem& pb, cudaStream_t 
                 if (!encode_activation_map(ctx, &p.tmX[ph * 2 + pw], pb.x, pb.n, pb.h, pb.w, pb.c, 2, ph, pw, p.cw_b, p.bw, p.bh, p.bn))
                     return B2C_ERR_CUDA;
     } else {
-        if (!encode_activation_map(ctx, &p.tmX[0], pb.x, pb.n, pb.h, pb.w, pb.c, 1, 0, 0, p.cw_b, p.bw, p.bh, p.bn)) return B2C_ERR_CUDA;
+        if (!encode_activation_map(ctx, &p.tmX[0], pb.x, pb.n, pb.h, pb.w, pb.c, 1, 0, 0, p.cw_b, p.fx ? p.bw + 2 : p.bw, p.bh, p.bn)) return B2C_ERR_CUDA;
     }
     p.k_total = pb.k;
     p.c_total = pb.c;
