@@ -65,7 +65,10 @@ void b2c_set_spin_limit(b2c_ctx* ctx, unsigned limit);
 /* Pipeline diagnostics of the convolution kernels.  `counters` is a DEVICE array of 8 unsigned 64-bit words owned
  * by the caller (NULL switches the feature off, the default).  Every CTA of the forward / data-gradient kernel adds
  * the SM clock cycles its roles spent waiting: [0] TMA producer for a free ring stage, [1] MMA thread for a loaded
- * stage, [2] MMA thread for a free accumulator, [3] first epilogue warp for a finished accumulator, [4] CTA lifetime. */
+ * stage, [2] MMA thread for a free accumulator, [3] first epilogue warp for a finished accumulator, [4] CTA lifetime.
+ * The weight-gradient kernel adds [0] first producer waiting, [1] first MMA thread waiting, [4] that thread's lifetime,
+ * [5] time at which warp 2 finished its reductions, [6] cycles the first MMA thread spent issuing, and keeps in [7] the
+ * MAXIMUM over CTAs and warps of the finishing time (zero the array between launches that should not mix). */
 void b2c_set_stall_counters(b2c_ctx* ctx, unsigned long long* counters);
 
 /* ---- Forward pass (Algorithm 1, "Perform forward pass") -------------------------------- */

@@ -55,16 +55,23 @@ struct alignas(64) WgradParams {
     int fx_box, fx_tx;                    // shared-memory footprint (1 KB multiple) and bytes delivered per framed box
     uint32_t fx_koff[4];                  // start of k-step kk inside a framed box, in 16-byte units
     uint32_t fx_sbo;                      // byte distance between the two 8-pixel groups of a k-step
+    int issuers;                          // MMA-issuing threads at work: 2 with an even ring depth, else 1
     int k_total, c_total, rs_total;
     float* dw;
     unsigned* status;
     unsigned spin_limit;
+    unsigned long long* stall;            // optional [8]: wait and lifetime cycles of the roles (see b2c_set_stall_counters)
 };
 
 static constexpr int kWgStages = 6;
 static constexpr int kWgProducers = 3;   // warp 0 and the warps after the epilogue warps; producer w fills ring slots w, w + 3, ...
 static constexpr int kWgProducerWarp1 = 6;
 static constexpr int kWgThreads = 256;
+// MMA-issuing threads (lane 0 of warps 1 and 2).  They take alternate chunks and accumulate into the same TMEM tile: one
+// thread pays about 100 cycles per MMA with a wait and a commit every four, against 96 the pipe needs at N = 192.  The
+// second thread starts once the first chunk (the one that overwrites instead of accumulating) has completed.  The ring
+// depth is even, so a slot always returns to the same thread and its barrier phases stay unambiguous.
+static constexpr int kWgIssuers = 2;
 static constexpr uint32_t kWgDrainPolls = 1u << 22;
 
 __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d)
@@ -101,7 +108,7 @@ __device__ __forceinline__ void wg_issue(uint32_t d_tmem, uint32_t a_lo, uint32_
 __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_constant__ WgradParams p)
 {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t full_bar[kWgStages], empty_bar[kWgStages], accum_bar, drain_bar;
+    __shared__ uint64_t full_bar[kWgStages], empty_bar[kWgStages], accum_bar, drain_bar, init_bar;
     __shared__ uint32_t tmem_slot;
     __shared__ uint32_t abort_flag;
 
@@ -126,8 +133,9 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], 1);
         }
-        mbar_init(&accum_bar, 1);
-        mbar_init(&drain_bar, 1);
+        mbar_init(&accum_bar, (uint32_t)p.issuers);   // one commit per MMA-issuing thread
+        mbar_init(&drain_bar, (uint32_t)p.issuers);
+        mbar_init(&init_bar, 1);
         abort_flag = 0;
         fence_mbar_init();
     }
@@ -142,6 +150,7 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
     // set-up done (it touched no global data): order behind the previous kernel of the stream, then let the next one in
     pdl_wait();
     pdl_launch_dependents();
+    const long long t_kernel = clock64();
     int last_issued = -1;  // producer lanes: last chunk whose loads this lane issued
 
     if (warp == 0 || warp >= kWgProducerWarp1) {
@@ -154,11 +163,15 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
             const uint32_t tx = p.fx ? (uint32_t)(p.a_bytes + p.b_boxes * p.fx_tx) : (uint32_t)(p.a_bytes + grp.nb * p.b_boxes * p.box_b);
             int it = w, s = w;
             uint32_t ph = 0u;
+            const bool timed = p.stall != nullptr && w == 0;
+            long long waited = 0;
             while (it < n_chunks) {
+                const long long w0 = timed ? clock64() : 0;
                 if (!mbar_wait_bounded(&empty_bar[s], ph ^ 1u, p.spin_limit, &abort_flag)) {
                     atomicOr(p.status, B2C_DEV_TIMEOUT);
                     break;
                 }
+                if (timed) waited += clock64() - w0;
                 int ch = chunk_begin + it;
                 const int ow0 = (ch & (p.tiles_w - 1)) * p.bw;
                 ch >>= p.tw_shift;
@@ -195,9 +208,11 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
                     ph ^= 1u;
                 }
             }
+            if (timed) atomicAdd(p.stall + 0, (unsigned long long)waited);
         }
-    } else if (warp == 1) {
-        if (lane == 0) {
+    } else if (warp == 1 || warp == 2) {
+        if (lane == 0 && warp - 1 < p.issuers) {
+            const int my = warp - 1;
             // SBO = eight pixel rows, LBO = next block of cw channels (the next box)
             const uint64_t proto_a = make_smem_desc(0u, (uint32_t)p.a_lbo, 16u * (uint32_t)p.cw_a, (uint32_t)p.swz_a);
             // framed x: the 64-column blocks of an MMA are the three shifts, one pixel row (128 bytes) apart
@@ -223,14 +238,25 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
                 ++n_pieces;
             }
             bool ok = true;
-            for (int it = 0; it < n_chunks; ++it) {
+            const bool timed = p.stall != nullptr;
+            const long long t_begin = timed ? clock64() : 0;
+            long long waited = 0, issuing = 0;
+            if (my != 0 && n_chunks > 1 && !mbar_wait_bounded(&init_bar, 0u, p.spin_limit, &abort_flag)) {   // chunk 0 has initialised the accumulator
+                atomicOr(p.status, B2C_DEV_TIMEOUT);
+                ok = false;
+            }
+            if (my != 0) tc_fence_after();
+            for (int it = my; ok && it < n_chunks; it += p.issuers) {
                 const int s = it % S;
                 const uint32_t ph = (uint32_t)(it / S) & 1u;
+                const long long w0 = timed ? clock64() : 0;
                 if (!mbar_wait_bounded(&full_bar[s], ph, p.spin_limit, &abort_flag)) {
                     atomicOr(p.status, B2C_DEV_TIMEOUT);
                     ok = false;
                     break;
                 }
+                const long long w1 = timed ? clock64() : 0;
+                waited += w1 - w0;
                 tc_fence_after();
                 const uint32_t st16 = smem_u32(smem + (size_t)s * p.stage_bytes) >> 4;
                 const uint32_t a_lo = a_lo_base + st16, b_lo = b_lo_base + st16;
@@ -249,14 +275,26 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
                     if (n_pieces > 2) wg_issue<2>(tmem_base + dcol2, a_lo, b_lo + boff2, a_hi, b_hi, idesc2, kstep_a, kstep_b, acc0);
                 }
                 umma_commit(&empty_bar[s]);
+                if (it == 0) umma_commit(&init_bar);
+                if (timed) issuing += clock64() - w1;
             }
             if (ok && n_chunks > 0) umma_commit(&accum_bar);
+            if (timed && my == 0) {
+                atomicAdd(p.stall + 1, (unsigned long long)waited);
+                atomicAdd(p.stall + 4, (unsigned long long)(clock64() - t_begin));
+                atomicAdd(p.stall + 6, (unsigned long long)issuing);
+            }
         }
-    } else {
-        const int q = warp & 3;
+    }
+    // ------------------------------------------------------------------ epilogue: all eight warps
+    // The producer and MMA warps have nothing left to do once their loops end, so they help the four epilogue warps:
+    // two warps per TMEM lane quarter, each sending half of the channel chunks of every shift to dw.
+    {
+        const int q = warp & 3, part = warp >> 2;
         const int m = q * 32 + lane;
         const int copy = p.stack ? 1 - (m >> 6) : 0;                   // which dy copy this accumulator row belongs to (copy 1 comes first)
         const int k = p.stack ? (m & 63) : ktile * 128 + m;
+        __syncwarp();
         bool ok = n_chunks > 0;
         if (ok) {
             if (lane == 0) ok = mbar_wait_bounded(&accum_bar, 0u, p.spin_limit, &abort_flag);   // one poller per warp
@@ -267,40 +305,41 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
         if (ok) {
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16);
             const int n_ck = p.ct >> 4;
-            for (int b = 0; b < grp.nb; ++b) {
+            const int ck_begin = part == 0 ? 0 : (n_ck + 1) >> 1, ck_end = part == 0 ? (n_ck + 1) >> 1 : n_ck;   // this warp's chunks
+            for (int b = 0; b < grp.nb && ck_begin < ck_end; ++b) {
                 const int rs = grp.rs[copy][b];
                 const bool live = rs >= 0 && k < p.k_total;
                 float* dst_row = p.dw + ((long long)(live ? k : 0) * p.rs_total + (live ? rs : 0)) * p.c_total + ctile * p.ct;
-                // two chunks in flight: the next one is fetched while the current one is sent out
                 // accumulator column of 16-channel chunk ck of shift b (framed x: [channel block][shift][64 channels])
                 auto col = [&](int ck) -> uint32_t {
                     return p.fx ? (uint32_t)((ck >> 2) * 192 + b * 64 + (ck & 3) * 16) : (uint32_t)(b * p.ct + ck * 16);
                 };
-                uint32_t ra[16], rb[16];
-                tmem_ld16(t_row + col(0), ra);
-                tmem_ld_wait();
-                for (int ck = 0; ck < n_ck; ck += 2) {
-                    if (ck + 1 < n_ck) tmem_ld16(t_row + col(ck + 1), rb);
+                auto send = [&](const uint32_t (&r)[16], int ck) {
                     if (live) {
 #pragma unroll
                         for (int i = 0; i < 16; i += 4)
-                            red_add_v4(dst_row + ck * 16 + i, __uint_as_float(ra[i]), __uint_as_float(ra[i + 1]), __uint_as_float(ra[i + 2]),
-                                       __uint_as_float(ra[i + 3]));
+                            red_add_v4(dst_row + ck * 16 + i, __uint_as_float(r[i]), __uint_as_float(r[i + 1]), __uint_as_float(r[i + 2]),
+                                       __uint_as_float(r[i + 3]));
                     }
-                    if (ck + 1 < n_ck) {
+                };
+                // two chunks in flight: the next one is fetched while the current one is sent out
+                uint32_t ra[16], rb[16];
+                tmem_ld16(t_row + col(ck_begin), ra);
+                tmem_ld_wait();
+                for (int ck = ck_begin; ck < ck_end; ck += 2) {
+                    if (ck + 1 < ck_end) tmem_ld16(t_row + col(ck + 1), rb);
+                    send(ra, ck);
+                    if (ck + 1 < ck_end) {
                         tmem_ld_wait();
-                        if (ck + 2 < n_ck) tmem_ld16(t_row + col(ck + 2), ra);
-                        if (live) {
-#pragma unroll
-                            for (int i = 0; i < 16; i += 4)
-                                red_add_v4(dst_row + (ck + 1) * 16 + i, __uint_as_float(rb[i]), __uint_as_float(rb[i + 1]), __uint_as_float(rb[i + 2]),
-                                           __uint_as_float(rb[i + 3]));
-                        }
-                        if (ck + 2 < n_ck) tmem_ld_wait();
+                        if (ck + 2 < ck_end) tmem_ld16(t_row + col(ck + 2), ra);
+                        send(rb, ck + 1);
+                        if (ck + 2 < ck_end) tmem_ld_wait();
                     }
                 }
             }
         }
+        if (p.stall != nullptr && lane == 0) atomicMax(p.stall + 7, (unsigned long long)(clock64() - t_kernel));   // the slowest warp of the slowest CTA
+        if (p.stall != nullptr && warp == 2 && lane == 0) atomicAdd(p.stall + 5, (unsigned long long)(clock64() - t_kernel));
     }
     tc_fence_before();
     __syncthreads();
@@ -314,9 +353,10 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
                 for (uint32_t i = 0; i < kWgDrainPolls && !mbar_try_wait(&full_bar[sl], (uint32_t)(it / S) & 1u); ++i) {}
             }
         }
-        if (warp == 1 && lane == 0) {
+        if ((warp == 1 || warp == 2) && lane == 0 && warp - 1 < p.issuers) {   // a commit covers the MMAs of the thread that makes it
             umma_commit(&drain_bar);
-            for (uint32_t i = 0; i < kWgDrainPolls && !mbar_try_wait(&drain_bar, 0u); ++i) {}
+            if (warp == 1)
+                for (uint32_t i = 0; i < kWgDrainPolls && !mbar_try_wait(&drain_bar, 0u); ++i) {}
         }
         __syncthreads();
     }
@@ -425,6 +465,10 @@ b2c_status launch_conv_wgrad(b2c_ctx* ctx, const WgradProblem& pb, cudaStream_t 
     int stages = (200 * 1024) / p.stage_bytes;
     if (stages > kWgStages) stages = kWgStages;
     if (stages < 2) return B2C_ERR_UNSUPPORTED_SHAPE;
+    // Two issuing threads need an even ring.  Measured: four stages with two threads beat five with one (128 -> 128:
+    // 67 us against 79 us), three stages with one thread beat two with two (512 -> 512 at 4x4: 79 us against 106 us).
+    if (stages >= 4) stages &= ~1;
+    p.issuers = (stages % 2 == 0) ? kWgIssuers : 1;
     p.stages = stages;
     p.bw = pb.q < p.pb ? pb.q : p.pb;
     p.bh = (p.pb / p.bw) < pb.p ? (p.pb / p.bw) : pb.p;
@@ -466,6 +510,7 @@ b2c_status launch_conv_wgrad(b2c_ctx* ctx, const WgradProblem& pb, cudaStream_t 
     p.dw = pb.dw;
     p.status = ctx->d_status;
     p.spin_limit = ctx->spin_limit;
+    p.stall = ctx->stall_counters;
 
     if (!attr_set) {
         B2C_CUDA(cudaFuncSetAttribute(conv_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 212 * 1024));
