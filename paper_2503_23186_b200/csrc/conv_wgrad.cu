@@ -215,8 +215,8 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
             const int my = warp - 1;
             // SBO = eight pixel rows, LBO = next block of cw channels (the next box)
             const uint64_t proto_a = make_smem_desc(0u, (uint32_t)p.a_lbo, 16u * (uint32_t)p.cw_a, (uint32_t)p.swz_a);
-            // framed x: the 64-column blocks of an MMA are the three shifts, one pixel row (128 bytes) apart
-            const uint64_t proto_b = p.fx ? make_smem_desc(0u, 128u, p.fx_sbo, (uint32_t)p.swz_b)
+            // framed x: the column blocks of an MMA are the three shifts, one pixel row (cw_b channels) apart
+            const uint64_t proto_b = p.fx ? make_smem_desc(0u, 2u * (uint32_t)p.cw_b, p.fx_sbo, (uint32_t)p.swz_b)
                                           : make_smem_desc(0u, (uint32_t)p.box_b, 16u * (uint32_t)p.cw_b, (uint32_t)p.swz_b);
             const uint32_t a_hi = (uint32_t)(proto_a >> 32), a_lo_base = (uint32_t)proto_a;
             const uint32_t b_hi = (uint32_t)(proto_b >> 32), b_lo_base = (uint32_t)proto_b;
@@ -226,12 +226,11 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
             uint32_t idesc0 = 0, idesc1 = 0, idesc2 = 0, boff0 = 0, boff1 = 0, boff2 = 0, dcol0 = 0, dcol1 = 0, dcol2 = 0;
             int n_pieces = 0;
             for (int i = 0; i < p.n_pieces; ++i) {
-                if (!p.fx && p.piece_t0[i] >= grp.nb) break;
+                if (p.piece_t0[i] >= grp.nb) break;
                 const int nt = min(p.piece_nt[i], grp.nb - p.piece_t0[i]);
-                // framed x: piece i = channel block i, N = three shifts x 64 channels
-                const uint32_t id = p.fx ? make_idesc_bf16(128, 192, true, true) : make_idesc_bf16(128, nt * p.ct, true, true);
-                const uint32_t bo = p.fx ? (uint32_t)(p.a_bytes + i * p.fx_box) >> 4 : (uint32_t)(p.a_bytes + p.piece_t0[i] * p.b_boxes * p.box_b) >> 4;
-                const uint32_t dc = p.fx ? (uint32_t)(i * 192) : (uint32_t)(p.piece_t0[i] * p.ct);
+                const uint32_t id = make_idesc_bf16(128, nt * p.ct, true, true);
+                const uint32_t bo = (uint32_t)(p.a_bytes + p.piece_t0[i] * p.b_boxes * p.box_b) >> 4;
+                const uint32_t dc = (uint32_t)(p.piece_t0[i] * p.ct);
                 if (i == 0) { idesc0 = id; boff0 = bo; dcol0 = dc; }
                 else if (i == 1) { idesc1 = id; boff1 = bo; dcol1 = dc; }
                 else { idesc2 = id; boff2 = bo; dcol2 = dc; }
@@ -261,10 +260,12 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
                 const uint32_t st16 = smem_u32(smem + (size_t)s * p.stage_bytes) >> 4;
                 const uint32_t a_lo = a_lo_base + st16, b_lo = b_lo_base + st16;
                 const uint32_t acc0 = it != 0 ? 1u : 0u;
-                if (p.fx) {   // chunks of 64 pixels: four k-steps
-                    wg_issue_framed<4>(tmem_base + dcol0, a_lo, b_lo + boff0, a_hi, b_hi, idesc0, kstep_a, p.fx_koff[0], p.fx_koff[1], p.fx_koff[2], p.fx_koff[3], acc0);
-                    if (n_pieces > 1)
-                        wg_issue_framed<4>(tmem_base + dcol1, a_lo, b_lo + boff1, a_hi, b_hi, idesc1, kstep_a, p.fx_koff[0], p.fx_koff[1], p.fx_koff[2], p.fx_koff[3], acc0);
+                if (p.fx) {   // chunks of 64 pixels: four k-steps; one MMA per channel block, N = three shifts x cw_b channels
+                    const uint32_t id_fx = make_idesc_bf16(128, 3 * p.cw_b, true, true);
+                    const uint32_t b_first = b_lo + ((uint32_t)p.a_bytes >> 4), b_next = (uint32_t)p.fx_box >> 4, d_next = 3u * (uint32_t)p.cw_b;
+                    for (int i = 0; i < p.b_boxes; ++i)
+                        wg_issue_framed<4>(tmem_base + (uint32_t)i * d_next, a_lo, b_first + (uint32_t)i * b_next, a_hi, b_hi, id_fx, kstep_a, p.fx_koff[0],
+                                           p.fx_koff[1], p.fx_koff[2], p.fx_koff[3], acc0);
                 } else if (ksteps == 4) {
                     wg_issue<4>(tmem_base + dcol0, a_lo, b_lo + boff0, a_hi, b_hi, idesc0, kstep_a, kstep_b, acc0);
                     if (n_pieces > 1) wg_issue<4>(tmem_base + dcol1, a_lo, b_lo + boff1, a_hi, b_hi, idesc1, kstep_a, kstep_b, acc0);
@@ -312,7 +313,8 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
                 float* dst_row = p.dw + ((long long)(live ? k : 0) * p.rs_total + (live ? rs : 0)) * p.c_total + ctile * p.ct;
                 // accumulator column of 16-channel chunk ck of shift b (framed x: [channel block][shift][64 channels])
                 auto col = [&](int ck) -> uint32_t {
-                    return p.fx ? (uint32_t)((ck >> 2) * 192 + b * 64 + (ck & 3) * 16) : (uint32_t)(b * p.ct + ck * 16);
+                    const int per_block = p.cw_b >> 4;   // 16-channel chunks per x box
+                    return p.fx ? (uint32_t)((ck / per_block) * 3 * p.cw_b + b * p.cw_b + (ck % per_block) * 16) : (uint32_t)(b * p.ct + ck * 16);
                 };
                 auto send = [&](const uint32_t (&r)[16], int ck) {
                     if (live) {
@@ -390,20 +392,24 @@ b2c_status launch_conv_wgrad(b2c_ctx* ctx, const WgradProblem& pb, cudaStream_t 
     for (int cand = 160; cand >= p.cw_b; cand -= 16)
         if (pb.c % cand == 0 && cand % p.cw_b == 0) { p.ct = cand; break; }
     // framed x stages: 64 pixels of one image per chunk, 64-channel x boxes, at most two of them per CTA (2 x 192 TMEM columns)
-    p.fx = (R == 3 && pb.stride == 1 && pb.q >= 8 && pb.p * pb.q >= 64 && p.cw_b == 64 && ctx->use_wgrad_frame) ? 1 : 0;
-    if (p.fx) p.ct = (pb.c % 128 == 0) ? 128 : 64;
+    p.fx = (R == 3 && pb.stride == 1 && pb.q >= 8 && pb.p * pb.q >= 64 && p.cw_b >= 32 && ctx->use_wgrad_frame) ? 1 : 0;
+    if (p.fx) {   // as many boxes per CTA as TMEM holds (three shifts of cw_b columns each): 2 of 64 channels, up to 5 of 32
+        const int max_boxes = 512 / (3 * p.cw_b);
+        p.ct = p.cw_b;
+        for (int nb = max_boxes; nb >= 1; --nb)
+            if (pb.c % (nb * p.cw_b) == 0) { p.ct = nb * p.cw_b; break; }
+    }
     p.n_ctiles = pb.c / p.ct;
     p.n_ktiles = p.stack ? 1 : (pb.k + 127) / 128;
     p.a_boxes = p.stack ? 2 : 128 / p.cw_a;
     p.b_boxes = p.ct / p.cw_b;
     const int shifts = R == 3 ? 3 : 1;
     p.tmem_cols = 32;
-    while (p.tmem_cols < (p.fx ? p.b_boxes * 192 : shifts * p.ct)) p.tmem_cols *= 2;
+    while (p.tmem_cols < (p.fx ? p.b_boxes * 3 * p.cw_b : shifts * p.ct)) p.tmem_cols *= 2;
     if (p.tmem_cols > 512) return B2C_ERR_UNSUPPORTED_SHAPE;
     // MMAs per k-step: merge the column blocks of consecutive shifts while N stays within 256
     if (p.fx) {
-        p.n_pieces = p.b_boxes;   // one N = 192 MMA per 64-channel block
-        for (int i = 0; i < p.n_pieces; ++i) { p.piece_t0[i] = 0; p.piece_nt[i] = 3; }
+        p.n_pieces = 0;   // framed x: one MMA per x box, laid out by the kernel
     } else if (shifts * p.ct <= 256) {
         p.n_pieces = 1; p.piece_t0[0] = 0; p.piece_nt[0] = shifts;
     } else if (2 * p.ct <= 256) {
@@ -454,7 +460,7 @@ b2c_status launch_conv_wgrad(b2c_ctx* ctx, const WgradProblem& pb, cudaStream_t 
         p.stage_bytes = p.a_bytes + shifts * p.b_boxes * p.box_b;
         if (p.fx) {
             const int bw = pb.q < p.pb ? pb.q : p.pb, bh = p.pb / bw;
-            p.fx_tx = (bw + 2) * bh * 128;
+            p.fx_tx = (bw + 2) * bh * p.cw_b * 2;
             p.fx_box = (p.fx_tx + 1023) & ~1023;
             p.stage_bytes = p.a_bytes + p.b_boxes * p.fx_box;
         }
@@ -478,9 +484,9 @@ b2c_status launch_conv_wgrad(b2c_ctx* ctx, const WgradProblem& pb, cudaStream_t 
         if (p.bn != 1) return B2C_ERR_UNSUPPORTED_SHAPE;   // cannot happen: at least 64 pixels per image
         for (int kk = 0; kk < 4; ++kk) {
             const int pix = 16 * kk, h = pix / p.bw, w0 = pix % p.bw;   // bw == 8: a k-step covers image rows 2kk and 2kk + 1
-            p.fx_koff[kk] = (uint32_t)((h * (p.bw + 2) + w0) * 128) >> 4;
+            p.fx_koff[kk] = (uint32_t)((h * (p.bw + 2) + w0) * p.cw_b * 2) >> 4;
         }
-        p.fx_sbo = p.bw == 8 ? 10u * 128u : 1024u;
+        p.fx_sbo = (uint32_t)((p.bw == 8 ? 10 : 8) * p.cw_b * 2);   // eight pixel rows, or one framed image row of ten
     }
     p.tiles_w = pb.q / p.bw;
     p.tw_shift = 0;

@@ -38,6 +38,7 @@ CONV_SHAPES = [
     (5, 16, 16, 32, 64, 3, 2),
     (6, 4, 4, 128, 64, 3, 1),       # 8 images per tile, ragged
     (2, 16, 16, 160, 160, 3, 1),    # WRN width
+    (2, 32, 32, 160, 160, 3, 1),    # WRN width at full image size (framed weight-gradient stages with 32-channel boxes)
     (4, 8, 8, 512, 512, 3, 1),      # two channel tiles of 256, long reduction
     (2, 32, 32, 16, 160, 1, 1),
     (130, 1, 1, 512, 128, 1, 1),    # classifier-shaped
