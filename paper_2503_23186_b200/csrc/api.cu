@@ -44,6 +44,10 @@ b2c_status b2c_create(b2c_ctx** out, int device)
         ctx->use_wgrad_frame = env ? (env[0] != '0') : 1;
     }
     {
+        const char* env = std::getenv("B2C_ISSUE_SPLIT");
+        ctx->use_issue_split = env ? (env[0] != '0') : 1;
+    }
+    {
         const char* env = std::getenv("B2C_PDL");
         ctx->use_pdl = env ? (env[0] != '0') : 1;
     }

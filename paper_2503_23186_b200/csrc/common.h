@@ -25,6 +25,7 @@ struct b2c_ctx {
     int use_pairs;                       // forward / data-gradient convolutions may run on CTA pairs (cta_group::2)
     unsigned long long* stall_counters;  // optional device array the convolution kernels add their wait cycles to
     int use_wgrad_frame;                 // weight gradient of 3x3 stride-1 layers stages x once per chunk with a one-pixel frame (all three shifts from one box)
+    int use_issue_split;                 // forward / data-gradient tiles wider than 128 channels: two MMA-issuing threads share every unit
     int use_pdl;                         // kernels are launched with programmatic stream serialization (their set-up overlaps the previous kernel's tail)
 };
 

@@ -50,6 +50,7 @@ struct alignas(64) ConvKParams {
     int tx_a, tx_b;                  // bytes one A / B load delivers
     int a_step;                      // byte offset of one image row inside the A tile (vreuse)
     int issuers;                     // MMA-issuing threads at work (1 or 2)
+    int issue_split;                 // the two issuing threads share every unit: alternate stages into one accumulator (tiles wider than 128 channels)
     int pair;                        // CTA pairs (cta_group::2): M = 256 per MMA, each CTA holds half of every B tile
     int resident;                    // filter bank of this CTA's channel tile stays in shared memory
     int resident_bytes;
@@ -423,7 +424,7 @@ __device__ __forceinline__ void issue_stage_fh(uint32_t d_tmem, uint32_t a_lo, u
 template <int KS, int NB, bool PAIR>
 __device__ __forceinline__ void mma_issuer(const ConvKParams& p, const UnitWalk& walk, int my, uint32_t tmem_base, uint32_t smem_addr,
                                            uint32_t ring_addr, int stage_bytes, uint64_t* full_bar, uint64_t* empty_bar, uint64_t* acc_full,
-                                           uint64_t* acc_empty, uint64_t* w_bar, uint32_t* abort_flag, const int* slot_stage)
+                                           uint64_t* acc_empty, uint64_t* w_bar, uint64_t* init_bar, uint32_t* abort_flag, const int* slot_stage)
 {
     const uint32_t idesc = make_idesc_bf16(PAIR ? 256 : 128, p.n_tile, false, false);
     const uint32_t sbo = 8u * (uint32_t)p.kb * 2u;  // eight rows of kb bf16
@@ -454,7 +455,7 @@ __device__ __forceinline__ void mma_issuer(const ConvKParams& p, const UnitWalk&
         int n_it = n_it_fixed;
         if (p.n_par > 1) n_it = unit_iters(p, walk.unit(p, pu) / units_per_par);
         if (n_it == 0) continue;   // a parity without taps: the epilogue stores zeros without an accumulator
-        if ((j % p.issuers) != my) {   // another issuer's unit: step over its stages
+        if (!p.issue_split && (j % p.issuers) != my) {   // another issuer's unit: step over its stages
             i_stage += n_it;
             s += n_it;
             while (s >= S) { s -= S; ph ^= 1u; }
@@ -472,7 +473,27 @@ __device__ __forceinline__ void mma_issuer(const ConvKParams& p, const UnitWalk&
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * p.acc_cols);
         uint32_t b_res = bank_lo;   // resident bank: B tile of (tap or horizontal shift, channel block), consecutive per stage
+        // Shared units: stage i of the CTA belongs to thread i % 2 (the ring depth is even, so a slot keeps its thread).  The
+        // thread that does not own the unit's first stage, whose first MMA overwrites the accumulator, waits until that
+        // stage has completed before it adds to the same accumulator.
+        const int init_owner = i_stage & 1;
+        bool init_seen = !p.issue_split || init_owner == my;
         for (int it = 0; it < n_it; ++it) {
+            if (p.issue_split && (i_stage & 1) != my) {   // the other thread's stage
+                b_res += b_cb16;
+                ++i_stage;
+                if (++s == S) { s = 0; ph ^= 1u; }
+                continue;
+            }
+            if (!init_seen) {
+                if (!mbar_wait_bounded(&init_bar[buf], (uint32_t)(j >> p.acc_shift) & 1u, p.spin_limit, abort_flag)) {
+                    atomicOr(p.status, B2C_DEV_TIMEOUT);
+                    ok = false;
+                    break;
+                }
+                tc_fence_after();
+                init_seen = true;
+            }
             const long long w2 = timed ? clock64() : 0;
             // A parity wait tells a barrier's phases apart only modulo two, and with two issuers this thread may reach a
             // slot before the slot's previous stage (another issuer's) was even loaded.  A producer issues the load of
@@ -504,6 +525,7 @@ __device__ __forceinline__ void mma_issuer(const ConvKParams& p, const UnitWalk&
             // frees the stage (in both CTAs of a pair) once these MMAs have read it
             if constexpr (PAIR) umma_commit_pair(&empty_bar[s], (uint16_t)3);
             else umma_commit(&empty_bar[s]);
+            if (p.issue_split && it == 0) umma_commit(&init_bar[buf]);   // the overwriting stage of this unit
             ++i_stage;
             if (++s == S) { s = 0; ph ^= 1u; }
         }
@@ -523,7 +545,7 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
 {
     const int rank = PAIR ? (int)cluster_ctarank() : 0;   // 0 = leader of the pair: issues the MMAs, owns the barriers the pair shares
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], acc_full[kMaxAccBufs], acc_empty[kMaxAccBufs], w_bar, drain_bar;
+    __shared__ uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], acc_full[kMaxAccBufs], acc_empty[kMaxAccBufs], init_bar[kMaxAccBufs], w_bar, drain_bar;
     __shared__ uint32_t tmem_slot;
     __shared__ uint32_t abort_flag;
     __shared__ int slot_stage[kMaxStages];   // per ring slot: 1 + index of the stage whose loads were issued into it last
@@ -541,7 +563,8 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
             mbar_init(&empty_bar[s], 1);
         }
         for (int b = 0; b < kMaxAccBufs; ++b) {
-            mbar_init(&acc_full[b], 1);
+            mbar_init(&acc_full[b], p.issue_split ? 2 : 1);   // shared units: both issuing threads commit
+            mbar_init(&init_bar[b], 1);
             mbar_init(&acc_empty[b], PAIR ? 2 * kEpiWarps : kEpiWarps);   // one arrival per epilogue warp (of both CTAs of a pair)
         }
         mbar_init(&w_bar, 1);
@@ -677,7 +700,7 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
             if (my < p.issuers) {
             const uint32_t smem_addr = smem_u32(smem), ring_addr = smem_u32(ring);
             const int ksteps = p.kb >> 4;
-#define B2C_ISSUER(KS, NB) mma_issuer<KS, NB, PAIR>(p, walk, my, tmem_base, smem_addr, ring_addr, stage_bytes, full_bar, empty_bar, acc_full, acc_empty, &w_bar, &abort_flag, slot_stage)
+#define B2C_ISSUER(KS, NB) mma_issuer<KS, NB, PAIR>(p, walk, my, tmem_base, smem_addr, ring_addr, stage_bytes, full_bar, empty_bar, acc_full, acc_empty, &w_bar, init_bar, &abort_flag, slot_stage)
             if (p.nb == 3) {
                 if (ksteps == 4) B2C_ISSUER(4, 3);
                 else if (ksteps == 2) B2C_ISSUER(2, 3);
@@ -909,6 +932,12 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
     if (p.stages < 2) return B2C_ERR_UNSUPPORTED_SHAPE;
     // Two issuing threads where one cannot keep the tensor pipe busy: tiles of at most 128 channels.
     p.issuers = p.n_tile <= 128 ? kIssuers : 1;
+    // Wider tiles: both threads work on every unit, alternate stages (needs an even ring; single CTAs only).
+    if (p.n_tile > 128 && !p.pair && ctx->use_issue_split && p.stages >= 2) {
+        p.stages &= ~1;
+        p.issuers = kIssuers;
+        p.issue_split = 1;
+    }
     const int stage_bytes = p.a_bytes + (p.resident ? 0 : p.nb * p.b_bytes);
     const size_t smem_bytes = (size_t)p.resident_bytes + (size_t)p.stages * stage_bytes + 1024;
 

@@ -89,7 +89,11 @@ def _compare_step(ctx, spec, params, velocity, images, labels, micro_batch, n_mi
     w_again = net.unpack(net.w)
     for name in sorted(params):
         if np.any(params[name] != 0):
-            assert_close(w_again[name], w_new[name], f"w_new {name} (single call)")
+            # Two runs of the library differ in fp32 accumulation order (atomics; MMAs of two issuing threads interleave
+            # in one accumulator), which is unspecified; a deep net amplifies that like any other rounding difference,
+            # so its run-to-run gate is the free-running one used against the oracle above.
+            assert_close(w_again[name], w_new[name], f"w_new {name} (single call)", REL_FRO if gate_gradients else 1e-2,
+                         MAX_REL if gate_gradients else 5e-2)
     net.close()
     return rows
 
