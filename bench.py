@@ -140,23 +140,33 @@ class ClockSampler:
 # ------------------------------------------------------------------------------------------------
 # CPU oracle legs
 # ------------------------------------------------------------------------------------------------
-def oracle_sample_step(spec, params, images, labels):
+def oracle_sample_step(spec, params, images, labels, n_micro=1):
     from oracle import net as onet
     vel = {k: np.zeros_like(v) for k, v in params.items()}
     t = time.perf_counter()
-    onet.train_step(spec, params, vel, images, labels, 1, LR, MU, WD, rounding=True)
+    onet.train_step(spec, params, vel, images, labels, n_micro, LR, MU, WD, rounding=True)
     return time.perf_counter() - t
 
 
-def cpu_baseline(spec, sample_images: int):
-    """The oracle as it stands, timed on this host on a bounded sample of the workload."""
+def cpu_baseline(spec, micro_batch: int, n_micro: int, target_s: float = 12.0):
+    """The oracle as it stands, timed on this host on a bounded sample of the workload: a short probe of 8 images sizes
+    the sample so that the timed run is roughly `target_s` seconds of CPU work (part of a micro-batch, or a few whole
+    micro-batches of the step)."""
     import oracle
     oracle.lib()
     params = wl.init_params(spec, 0)
+    images, labels = wl.image_batch(0, 8, tag="cpu_probe")
+    probe = oracle_sample_step(spec, params, images.astype(np.float64), labels)
+    want = 8 * round(target_s / max(probe, 1e-3))
+    if want <= micro_batch:
+        groups, sample_images = 1, int(max(8, want))
+    else:
+        groups = int(min(n_micro, max(1, want // micro_batch)))
+        sample_images = groups * micro_batch
     images, labels = wl.image_batch(0, sample_images, tag="cpu")
-    dt = oracle_sample_step(spec, params, images.astype(np.float64), labels)
+    dt = oracle_sample_step(spec, params, images.astype(np.float64), labels, groups)
     return {"value": sample_images / dt, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
-            "sample": f"one optimiser step on one micro-batch of {sample_images} images (fp64, all layers, forward+backward+update), {dt:.1f} s"}
+            "sample": f"one optimiser step on {groups} micro-batch(es), {sample_images} images in all (fp64, all layers, forward+backward+update), {dt:.1f} s"}
 
 
 def run_reference(args, spec, name):
@@ -306,7 +316,6 @@ def run_b2c(args, spec, name, micro_batch, n_micro):
                 "algorithmic_bytes_per_launch": km_bytes / km_launches if km_launches else None,
                 "all_conv_tflops": conv_tf, "all_conv_frac_of_measured": conv_tf / peaks["bf16"] if conv_tf else None,
                 "all_conv_frac_of_nominal": conv_tf / NOMINAL_BF16_TFLOPS if conv_tf else None}
-    sample = 32
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
@@ -317,7 +326,7 @@ def run_b2c(args, spec, name, micro_batch, n_micro):
                    "profiled_ms_per_step": profiled_ms / args.steps},
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(sum(fam_launches.values())),
         "roofline": roofline, "kernels": kernels, "loss": loss,
-        "cpu_baseline": cpu_baseline(spec, sample) if world == 1 and not args.no_cpu_baseline else None,
+        "cpu_baseline": cpu_baseline(spec, micro_batch, n_micro) if world == 1 and not args.no_cpu_baseline else None,
     }
     print(json.dumps(out))
 
