@@ -398,6 +398,10 @@ b2c_status b2c_net_create_concurrent(b2c_ctx* ctx, const b2c_layer_desc* layers,
             const int pix = L.p * L.q;
             const int imgs_per_tile = pix >= 128 ? 1 : 128 / pix;
             o.fused_stats = net->fuse_stats && (micro_batch % imgs_per_tile == 0);
+            // 1x1 expansions (at least four times more outputs than inputs, short reduction): the per-column sums of the
+            // wide-tile epilogue take longer than the few MMAs of a unit and than one more pass over the output
+            // (measured at 1024 images: 64 -> 256 at 32x32 359 us fused, 167 us + a 110 us pass unfused).
+            if (L.d.r == 1 && L.d.k >= 4 * L.d.c && L.d.c <= 256 && L.d.k > 64) o.fused_stats = false;
         }
         if (L.d.kind == B2C_LAYER_BN) L.bwd_ws_off = alloc(b2c_bn_relu_bwd_workspace_bytes(L.d.c) * n_concurrent);
     }
