@@ -25,6 +25,8 @@
  *       B2C_FULL_HALO=0      one load per tap group instead of one framed tile per channel block (3x3 stride-1 layers)
  *       B2C_ISSUE_SPLIT=0    forward / data gradient, tiles wider than 128 channels: one MMA-issuing thread instead of two sharing every unit
  *       B2C_WGRAD_FRAME=0    weight gradient: one x box per horizontal shift instead of one framed box per channel block
+ *       B2C_FUSE_WIDE=0|1    BatchNorm statistics of tiles wider than 64 channels: never | always in the convolution epilogue
+ *                            (default: where the unit's MMAs take longer than the epilogue's column sums)
  *       B2C_FUSE_BN_STATS=0  BatchNorm statistics by a separate pass instead of the convolution epilogue (b2c_train_step)
  *       B2C_CHUNK_MB=<n>     b2c_train_step takes layers whose tensors exceed n MB a few micro-batches at a time (0 = off, default)
  */

@@ -398,10 +398,19 @@ b2c_status b2c_net_create_concurrent(b2c_ctx* ctx, const b2c_layer_desc* layers,
             const int pix = L.p * L.q;
             const int imgs_per_tile = pix >= 128 ? 1 : 128 / pix;
             o.fused_stats = net->fuse_stats && (micro_batch % imgs_per_tile == 0);
-            // 1x1 expansions (at least four times more outputs than inputs, short reduction): the per-column sums of the
-            // wide-tile epilogue take longer than the few MMAs of a unit and than one more pass over the output
-            // (measured at 1024 images: 64 -> 256 at 32x32 359 us fused, 167 us + a 110 us pass unfused).
-            if (L.d.r == 1 && L.d.k >= 4 * L.d.c && L.d.c <= 256 && L.d.k > 64) o.fused_stats = false;
+            // Tiles wider than 64 channels sum their columns with a shuffle butterfly (about 1400 cycles per 32 columns and
+            // unit, measured); where that exceeds the unit's MMA time the epilogue becomes the bottleneck and one more pass
+            // over the output (mostly still in L2) is cheaper.  Tiles of up to 64 channels keep their sums in registers.
+            {
+                int n_tile = 16;
+                for (int cand = 256; cand >= 16; cand -= 16)
+                    if (L.d.k % cand == 0) { n_tile = cand; break; }
+                const long long mma_cycles = (long long)(L.c_pad * L.gemm_r * L.gemm_r / 16) * (n_tile / 2 > 48 ? n_tile / 2 : 48);
+                const long long sum_cycles = 1400ll * n_tile / 32;
+                const char* e2 = std::getenv("B2C_FUSE_WIDE");   // 1: always fuse; 0: never on wide tiles; default: by the estimate
+                const bool wide_ok = e2 ? e2[0] != '0' : mma_cycles >= sum_cycles;
+                if (n_tile > 64 && !wide_ok) o.fused_stats = false;
+            }
         }
         if (L.d.kind == B2C_LAYER_BN) L.bwd_ws_off = alloc(b2c_bn_relu_bwd_workspace_bytes(L.d.c) * n_concurrent);
     }

@@ -35,9 +35,8 @@ __device__ __forceinline__ uint4 ld16(const void* base, long long vec_index) { r
 
 // Row/channel-group decomposition shared by the row-walking kernels.  blockIdx.y selects the
 // statistics group (a micro-batch): rows [g*m, (g+1)*m) of the tensor, its own accumulators and
-// its own saved mean / invstd.  Each thread keeps kRowsUnroll independent 16-byte loads per tensor
+// its own saved mean / invstd.  Each thread keeps several independent 16-byte loads per tensor
 // in flight (rows beyond the end read as zero and contribute nothing).
-static constexpr int kRowsUnroll = 4;
 struct RowWalk {
     int groups;         // c / 8
     int rows_per_iter;  // rows a block covers per step
@@ -49,6 +48,8 @@ __device__ __forceinline__ uint4 ld16_or_zero(const void* base, long long vec_in
 }
 
 // ------------------------------------------------------------------------------ BN forward
+// Rows in flight per thread in the statistics pass: it reads one tensor only (see bn_apply_kernel).
+static constexpr int kStatsUnroll = 8;
 __global__ void __launch_bounds__(kEwThreads, 2) bn_stats_kernel(const void* __restrict__ y, long long m, int c, double* __restrict__ stats)
 {
     pdl_wait();   // first global access comes after the previous kernel of the stream
@@ -64,12 +65,12 @@ __global__ void __launch_bounds__(kEwThreads, 2) bn_stats_kernel(const void* __r
 #pragma unroll
         for (int i = 0; i < 8; ++i) s[i] = ss[i] = 0.f;
         const long long step = (long long)gridDim.x * rw.rows_per_iter;
-        for (long long r = (long long)blockIdx.x * rw.rows_per_iter + rl; r < m; r += kRowsUnroll * step) {
-            uint4 v[kRowsUnroll];
+        for (long long r = (long long)blockIdx.x * rw.rows_per_iter + rl; r < m; r += kStatsUnroll * step) {
+            uint4 v[kStatsUnroll];
 #pragma unroll
-            for (int u = 0; u < kRowsUnroll; ++u) v[u] = ld16_or_zero(y, base + (r + u * step) * rw.groups + g, r + u * step < m);
+            for (int u = 0; u < kStatsUnroll; ++u) v[u] = ld16_or_zero(y, base + (r + u * step) * rw.groups + g, r + u * step < m);
 #pragma unroll
-            for (int u = 0; u < kRowsUnroll; ++u) {
+            for (int u = 0; u < kStatsUnroll; ++u) {
                 float f[8];
                 unpack8(v[u], f);
 #pragma unroll
