@@ -586,7 +586,9 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
                     const bool ready = in.fused_stats;
                     double* stats = reinterpret_cast<double*>(net->ws + (in.stats_off >= 0 ? in.stats_off : L.bwd_ws_off)) + (size_t)g0 * 2 * in.c;
                     ProfScope ps_(net, stream, B2C_PROF_BN_FWD, ready ? 1 : 2);
-                    B2C_TRY(launch_bn_fwd(ctx, Gc, (long long)mbs * in.h * in.w, in.c, act(d.src, img0), stats, ready, net->w + L.gamma_off,
+                    B2C_TRY(launch_bn_fwd(ctx, Gc, (long long)mbs * in.h * in.w, in.c, act(d.src, img0), stats,
+                                          ready ? 1 : (in.stats_off >= 0 ? 2 : 0),   // a convolution output's sums live in the region cleared once per pass
+                                          net->w + L.gamma_off,
                                           net->w + L.beta_off, d.res >= 0 ? act(d.res, img0) : nullptr, d.relu, 1e-5f, act(i + 1, img0),
                                           reinterpret_cast<float*>(net->ws + L.mean_off) + (size_t)g0 * in.c,
                                           reinterpret_cast<float*>(net->ws + L.invstd_off) + (size_t)g0 * in.c, nullptr, nullptr, 0.f,

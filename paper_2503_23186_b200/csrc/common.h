@@ -115,10 +115,11 @@ struct WgradProblem {
 b2c_status launch_conv_wgrad(b2c_ctx* ctx, const WgradProblem& pb, cudaStream_t stream);
 
 // BatchNorm over G statistics groups (micro-batches) of m rows each; stats / sums are fp64 [G][2c],
-// save_mean / save_invstd fp32 [G][c].  G > 1 requires acc != 0 in the backward pass.  relu_mask (optional): one bit per
+// save_mean / save_invstd fp32 [G][c].  G > 1 requires acc != 0 in the backward pass.  stats_ready: 1 = `stats` holds the
+// sums already (convolution epilogue), 0 = clear and compute them, 2 = compute them into `stats` the caller has cleared.  relu_mask (optional): one bit per
 // element, "stored output > 0" (a byte per 8 channels), written by the forward pass and read by the backward pass
 // in place of the output tensor.  sums_zeroed: the caller has already cleared `sums`.
-b2c_status launch_bn_fwd(b2c_ctx* ctx, int G, long long m, int c, const void* y, double* stats, bool stats_ready, const float* gamma,
+b2c_status launch_bn_fwd(b2c_ctx* ctx, int G, long long m, int c, const void* y, double* stats, int stats_ready, const float* gamma,
                          const float* beta, const void* residual, int relu, float eps, void* a, float* save_mean, float* save_invstd,
                          float* run_mean, float* run_var, float momentum, void* relu_mask, cudaStream_t stream);
 b2c_status launch_bn_bwd(b2c_ctx* ctx, int G, long long m, int c, const void* da1, const void* da2, const void* y, const void* a,

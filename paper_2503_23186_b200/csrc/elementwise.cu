@@ -852,14 +852,14 @@ static int ew_grid(b2c_ctx* ctx, int n_groups, long long m, int rows_per_iter)
     return (int)(blocks < cap ? (blocks < 1 ? 1 : blocks) : cap);
 }
 
-b2c_status launch_bn_fwd(b2c_ctx* ctx, int G, long long m, int c, const void* y, double* stats, bool stats_ready, const float* gamma,
+b2c_status launch_bn_fwd(b2c_ctx* ctx, int G, long long m, int c, const void* y, double* stats, int stats_ready, const float* gamma,
                          const float* beta, const void* residual, int relu, float eps, void* a, float* save_mean, float* save_invstd,
                          float* run_mean, float* run_var, float momentum, void* relu_mask, cudaStream_t stream)
 {
     const int rows_per_iter = kEwThreads / (c / 8);
     dim3 grid((unsigned)ew_grid(ctx, G, m, rows_per_iter), (unsigned)G);
-    if (!stats_ready) {
-        B2C_CUDA(cudaMemsetAsync(stats, 0, sizeof(double) * 2 * c * G, stream));
+    if (stats_ready != 1) {
+        if (stats_ready == 0) B2C_CUDA(cudaMemsetAsync(stats, 0, sizeof(double) * 2 * c * G, stream));
         B2C_CUDA(b2c_launch(ctx, bn_stats_kernel, dim3(grid), dim3(kEwThreads), sizeof(float) * 2 * c, stream, 1u, y, m, c, stats));
     }
     uint8_t* mask_out = relu ? reinterpret_cast<uint8_t*>(relu_mask) : nullptr;

@@ -295,7 +295,8 @@ def test_chunked_schedule_matches_oracle(ctx, monkeypatch):
     assert abs(loss_chunked - loss_whole) <= 1e-5 * abs(loss_whole)
     gw, gc = whole.unpack(whole.g), chunked.unpack(chunked.g)
     for name in sorted(params):
-        assert_close(gc[name], gw[name], f"grad {name} (chunked vs whole passes)", 1e-4, 1e-3)
+        # two runs differ in fp32 accumulation order (atomics, two MMA-issuing threads per accumulator): the per-tensor budget
+        assert_close(gc[name], gw[name], f"grad {name} (chunked vs whole passes)")
     whole.close(); chunked.close()
 
 
