@@ -284,6 +284,14 @@ b2c_status b2c_net_profile_enable(b2c_net* net, int enable);
  * last read (0 unless enabled), launches[kind] = kernels launched since the last read (always counted).
  * Both arrays are HOST memory of B2C_PROF_KINDS entries.  Resets the sums. */
 b2c_status b2c_net_profile_read(b2c_net* net, double* ms, long long* launches, void* stream);
+/* The same records per network component (the partition of the model into logical components that the paper's
+ * scheduling algorithm profiles is the layer list): ms[3*i + 0] = forward time of layer i, ms[3*i + 1] = its
+ * parameter-gradient time (weight gradient; bias gradient), ms[3*i + 2] = its data-gradient time (convolution data
+ * gradient, BatchNorm / pooling backward), summed since the last b2c_net_profile_read.  HOST memory of 3*n_layers
+ * doubles; n_layers must equal b2c_net_layer_count.  Synchronises `stream`; does not reset the records, so call it
+ * before b2c_net_profile_read.  All zero unless profiling is enabled. */
+b2c_status b2c_net_profile_read_layers(b2c_net* net, double* ms, int n_layers, void* stream);
+int b2c_net_layer_count(const b2c_net* net);
 
 #ifdef __cplusplus
 }

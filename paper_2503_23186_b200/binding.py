@@ -30,6 +30,7 @@ EXPORTS = [
     "b2c_net_create", "b2c_net_create_concurrent", "b2c_net_destroy", "b2c_net_param_count", "b2c_net_param_offset",
     "b2c_net_padded_image_channels", "b2c_net_first_conv_im2col", "b2c_im2col_3x3", "b2c_net_workspace_bytes", "b2c_net_tensor_offset", "b2c_net_bind",
     "b2c_net_sync_weights", "b2c_train_step", "b2c_net_apply_update", "b2c_net_profile_enable", "b2c_net_profile_read",
+    "b2c_net_profile_read_layers", "b2c_net_layer_count",
 ]
 PROF_KINDS = ["conv_fwd", "conv_dgrad", "conv_wgrad", "bn_fwd", "bn_bwd", "other", "update"]
 
@@ -307,6 +308,13 @@ class Net:
         n = (c_longlong * len(PROF_KINDS))()
         _check(lib().b2c_net_profile_read(self.handle, ms, n, _stream()), "b2c_net_profile_read")
         return dict(zip(PROF_KINDS, list(ms))), dict(zip(PROF_KINDS, list(n)))
+
+    def profile_read_layers(self):
+        """Per layer [forward ms, parameter-gradient ms, data-gradient ms] since the last profile_read (call before it)."""
+        n = len(self.spec)
+        ms = (c_double * (3 * n))()
+        _check(lib().b2c_net_profile_read_layers(self.handle, ms, c_int(n), _stream()), "b2c_net_profile_read_layers")
+        return np.array(list(ms)).reshape(n, 3)
 
     def tensor_view(self, tensor: int, shape, dtype=torch.bfloat16, grad=False, which=0):
         off = self.tensor_offset(tensor, grad, which)

@@ -222,7 +222,7 @@ struct b2c_net {
     bool fuse_stats = true;
     // optional per-launch timing (CUDA events on the step's stream), summed per kernel family
     bool profile = false;
-    struct Span { cudaEvent_t a, b; int kind; };
+    struct Span { cudaEvent_t a, b; int kind, layer, pass; };   // layer -1: not a layer's launch site; pass 0 forward, 1 parameter gradient, 2 data gradient
     std::vector<Span> spans;      // event pool, reused every step
     size_t spans_used = 0;
     long long launches[B2C_PROF_KINDS] = {0};   // kernels launched since the last profile read
@@ -236,7 +236,7 @@ namespace {
 // Brackets one launch site with events when profiling is on, and counts its kernels.
 struct ProfScope {
     b2c_net* net; cudaStream_t stream; b2c_net::Span* sp = nullptr;
-    ProfScope(b2c_net* n, cudaStream_t st, int kind, int kernels) : net(n), stream(st)
+    ProfScope(b2c_net* n, cudaStream_t st, int kind, int kernels, int layer = -1, int pass = 0) : net(n), stream(st)
     {
         net->launches[kind] += kernels;
         if (!net->profile) return;
@@ -247,6 +247,8 @@ struct ProfScope {
         }
         sp = &net->spans[net->spans_used++];
         sp->kind = kind;
+        sp->layer = layer;
+        sp->pass = pass;
         cudaEventRecord(sp->a, stream);
     }
     ~ProfScope() { if (sp) cudaEventRecord(sp->b, stream); }
@@ -577,7 +579,7 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
                     pb.in = act_in(d.src, img0); pb.wt = w_bf16 + L.w_off; pb.out = act(i + 1, img0);
                     pb.stats = o.fused_stats ? reinterpret_cast<double*>(net->ws + o.stats_off) + (size_t)g0 * 2 * d.k : nullptr;
                     pb.stats_group_images = mbs;
-                    ProfScope ps_(net, stream, B2C_PROF_CONV_FWD, 1);
+                    ProfScope ps_(net, stream, B2C_PROF_CONV_FWD, 1, i, 0);
                     B2C_TRY(launch_conv_kmajor(ctx, pb, stream));
                     break;
                 }
@@ -585,7 +587,7 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
                     const TensorPlan& in = net->tensors[d.src];
                     const bool ready = in.fused_stats;
                     double* stats = reinterpret_cast<double*>(net->ws + (in.stats_off >= 0 ? in.stats_off : L.bwd_ws_off)) + (size_t)g0 * 2 * in.c;
-                    ProfScope ps_(net, stream, B2C_PROF_BN_FWD, ready ? 1 : 2);
+                    ProfScope ps_(net, stream, B2C_PROF_BN_FWD, ready ? 1 : 2, i, 0);
                     B2C_TRY(launch_bn_fwd(ctx, Gc, (long long)mbs * in.h * in.w, in.c, act(d.src, img0), stats,
                                           ready ? 1 : (in.stats_off >= 0 ? 2 : 0),   // a convolution output's sums live in the region cleared once per pass
                                           net->w + L.gamma_off,
@@ -597,7 +599,7 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
                 }
                 case B2C_LAYER_AVGPOOL: {
                     const TensorPlan& in = net->tensors[d.src];
-                    ProfScope ps_(net, stream, B2C_PROF_OTHER, 1);
+                    ProfScope ps_(net, stream, B2C_PROF_OTHER, 1, i, 0);
                     B2C_TRY(b2c_avgpool_fwd(ctx, Nc, in.h * in.w, in.c, act(d.src, img0), act(i + 1, img0), stream));
                     break;
                 }
@@ -607,13 +609,13 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
                     pb.r = 1; pb.stride = 1; pb.pad = 0; pb.dgrad = false;
                     pb.in = act(d.src, img0); pb.wt = w_bf16 + L.w_off; pb.out = act(i + 1, img0);
                     pb.out_f32 = true; pb.bias = net->w + L.bias_off;
-                    ProfScope ps_(net, stream, B2C_PROF_OTHER, 1);
+                    ProfScope ps_(net, stream, B2C_PROF_OTHER, 1, i, 0);
                     B2C_TRY(launch_conv_kmajor(ctx, pb, stream));
                     break;
                 }
                 case B2C_LAYER_XENT: {
                     const TensorPlan& in = net->tensors[d.src];
-                    ProfScope ps_(net, stream, B2C_PROF_OTHER, 1);
+                    ProfScope ps_(net, stream, B2C_PROF_OTHER, 1, i, 0);
                     B2C_TRY(b2c_softmax_xent_fwd_bwd(ctx, Nc, d.k, reinterpret_cast<const float*>(act(d.src, img0)), in.c, lab + img0,
                                                      1.f / ((float)mbs * (float)n_micro), 1.f / (float)mbs, loss_dev,
                                                      grad(d.src, L.src_slot, img0), in.c, stream));
@@ -636,7 +638,7 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
                     WgradProblem wp{};
                     wp.n = Nc; wp.h = 1; wp.w = 1; wp.c = L.c_pad; wp.p = 1; wp.q = 1; wp.k = L.k_pad; wp.r = 1; wp.stride = 1; wp.pad = 0;
                     wp.dy = dz; wp.x = act(d.src, img0); wp.dw = net->g + L.w_off;
-                    ProfScope ps_(net, stream, B2C_PROF_OTHER, 3);
+                    ProfScope ps_(net, stream, B2C_PROF_OTHER, 3, i, 1);
                     B2C_TRY(launch_conv_wgrad(ctx, wp, stream));
                     B2C_TRY(b2c_bias_grad(ctx, Nc, L.k_pad, L.k_pad, dz, net->g + L.bias_off, 1, stream));
                     KMajorProblem pb{};
@@ -648,13 +650,13 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
                 }
                 case B2C_LAYER_AVGPOOL: {
                     const TensorPlan& in = net->tensors[d.src];
-                    ProfScope ps_(net, stream, B2C_PROF_OTHER, 1);
+                    ProfScope ps_(net, stream, B2C_PROF_OTHER, 1, i, 2);
                     B2C_TRY(b2c_avgpool_bwd(ctx, Nc, in.h * in.w, in.c, grad(i + 1, 0, img0), grad(d.src, L.src_slot, img0), stream));
                     break;
                 }
                 case B2C_LAYER_BN: {
                     const TensorPlan& in = net->tensors[d.src];
-                    ProfScope ps_(net, stream, B2C_PROF_BN_BWD, 2);
+                    ProfScope ps_(net, stream, B2C_PROF_BN_BWD, 2, i, 2);
                     B2C_TRY(launch_bn_bwd(ctx, Gc, (long long)mbs * in.h * in.w, in.c, grad(i + 1, 0, img0),
                                           o.n_contrib > 1 ? grad(i + 1, 1, img0) : nullptr, act(d.src, img0), act(i + 1, img0), net->w + L.gamma_off,
                                           reinterpret_cast<float*>(net->ws + L.mean_off) + (size_t)g0 * in.c,
@@ -671,7 +673,7 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
                     wp.r = L.gemm_r; wp.stride = d.stride; wp.pad = (L.gemm_r - 1) / 2;
                     wp.dy = dy; wp.x = act_in(d.src, img0); wp.dw = net->g + L.w_off;
                     {
-                        ProfScope ps_(net, stream, B2C_PROF_CONV_WGRAD, 1);
+                        ProfScope ps_(net, stream, B2C_PROF_CONV_WGRAD, 1, i, 1);
                         B2C_TRY(launch_conv_wgrad(ctx, wp, stream));
                     }
                     if (d.src != 0) {
@@ -679,7 +681,7 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
                         pb.n = Nc; pb.ih = L.p; pb.iw = L.q; pb.ic = d.k; pb.oh = d.h; pb.ow = d.w; pb.oc = L.c_pad;
                         pb.r = d.r; pb.stride = d.stride; pb.pad = (d.r - 1) / 2; pb.dgrad = true;
                         pb.in = dy; pb.wt = w_dg + L.w_off; pb.out = grad(d.src, L.src_slot, img0);
-                        ProfScope ps_(net, stream, B2C_PROF_CONV_DGRAD, 1);
+                        ProfScope ps_(net, stream, B2C_PROF_CONV_DGRAD, 1, i, 2);
                         B2C_TRY(launch_conv_kmajor(ctx, pb, stream));
                     }
                     break;
@@ -722,6 +724,21 @@ b2c_status b2c_net_profile_enable(b2c_net* net, int enable)
     for (int k = 0; k < B2C_PROF_KINDS; ++k) net->launches[k] = 0;
     return B2C_OK;
 }
+
+b2c_status b2c_net_profile_read_layers(b2c_net* net, double* ms, int n_layers, void* stream)
+{
+    if (!net || !ms || n_layers != (int)net->layers.size()) return B2C_ERR_INVALID_ARG;
+    B2C_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+    for (int i = 0; i < 3 * n_layers; ++i) ms[i] = 0.0;
+    for (size_t i = 0; i < net->spans_used; ++i) {
+        const b2c_net::Span& sp = net->spans[i];
+        float t = 0.f;
+        if (sp.layer >= 0 && sp.layer < n_layers && cudaEventElapsedTime(&t, sp.a, sp.b) == cudaSuccess) ms[3 * sp.layer + sp.pass] += t;
+    }
+    return B2C_OK;
+}
+
+int b2c_net_layer_count(const b2c_net* net) { return net ? (int)net->layers.size() : 0; }
 
 b2c_status b2c_net_profile_read(b2c_net* net, double* ms, long long* launches, void* stream)
 {

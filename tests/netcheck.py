@@ -123,10 +123,14 @@ def _wgrad_samples(rng, dy, x, R, stride, pad, count):
     return idx, out
 
 
-def check_step(net, spec, images, labels, n, n_micro_scale=1, sample=None, seed=0, groups=1):
+def check_step(net, spec, images, labels, n, n_micro_scale=1, sample=None, seed=0, groups=1, lowmem=False):
     """Checks the micro-batch whose state is in the workspace (run train_step with n_micro=1, update=False
     first).  `images` are the logical (unpadded) images of that pass: `groups` micro-batches side by side, each
-    with its own BatchNorm statistics (n = total images).  Returns a Report."""
+    with its own BatchNorm statistics (n = total images).  Returns a Report.
+
+    lowmem: for full-size workloads.  Host copies are fp32 (exact for bf16 data), fetched from the device each time a
+    layer needs them and dropped afterwards, so the host holds one layer's tensors at a time; every element is still
+    compared, against the same oracle functions."""
     rep = Report()
     rng = np.random.default_rng(seed)
     rb, rf = oracle.round_bf16, oracle.round_f32
@@ -135,19 +139,24 @@ def check_step(net, spec, images, labels, n, n_micro_scale=1, sample=None, seed=
     g = net.unpack(net.g)
     slots, n_contrib = grad_slots(spec)
 
+    def to_host(t):
+        return t.detach().float().cpu().numpy() if lowmem else host(t)
+
     def act(t):
         if t == 0:
-            return np.asarray(images, np.float64)
+            return np.asarray(images, np.float32 if lowmem else np.float64)
         shp = _shape(spec, t, n, net)
         dt = torch.float32 if spec[t - 1]["kind"] == "fc" else torch.bfloat16
-        return host(net.tensor_view(t, shp, dt))
+        return to_host(net.tensor_view(t, shp, dt))
 
     def grad(t, slot):
-        return host(net.tensor_view(t, _shape(spec, t, n, net), torch.bfloat16, True, slot))
+        return to_host(net.tensor_view(t, _shape(spec, t, n, net), torch.bfloat16, True, slot))
 
     cache = {}
 
     def A(t):
+        if lowmem:
+            return act(t)
         if t not in cache:
             cache[t] = act(t)
         return cache[t]
@@ -198,11 +207,13 @@ def check_step(net, spec, images, labels, n, n_micro_scale=1, sample=None, seed=
             two = n_contrib[i + 1] == 2
             per, parts = n // groups, []
             g1, g2 = grad(i + 1, 0), (grad(i + 1, 1) if two else None)
+            y_in, a_out = A(L["src"]), A(i + 1)
             for gi in range(groups):
                 sl = slice(gi * per, (gi + 1) * per)
                 mean, invstd = saved[i][gi]
-                parts.append(oracle.bn_relu_bwd(g1[sl], None if g2 is None else g2[sl], A(L["src"])[sl], A(i + 1)[sl], wm[f"gamma{i}"], mean, invstd,
+                parts.append(oracle.bn_relu_bwd(g1[sl], None if g2 is None else g2[sl], y_in[sl], a_out[sl], wm[f"gamma{i}"], mean, invstd,
                                                 L["relu"], L["res"] >= 0))
+            del g1, g2, y_in, a_out
             dy = np.concatenate([q[0] for q in parts])
             dres = np.concatenate([q[1] for q in parts]) if L["res"] >= 0 else None
             dg, db = sum(q[2] for q in parts), sum(q[3] for q in parts)

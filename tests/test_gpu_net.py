@@ -300,22 +300,29 @@ def test_chunked_schedule_matches_oracle(ctx, monkeypatch):
     whole.close(); chunked.close()
 
 
-def _full_size_sampled(ctx, spec, micro_batch, n_micro, seed):
-    """One pass of a full-size workload in the launch configuration bench.py times (all micro-batches side by side),
-    every layer checked on sampled outputs against the oracle; then the fused update against the oracle's update on
-    the device gradient sum, element by element."""
+def _full_size(ctx, spec, micro_batch, n_micro, seed, sampled=False):
+    """One pass of a full-size workload in the launch configuration bench.py times (all micro-batches side by side).
+    Every layer of the pass is checked teacher-forced against the oracle on the layer's own device inputs, every
+    element of every tensor at the per-tensor budget (sampled=True: on sampled outputs, for the workload the oracle
+    needs minutes for); then the fused update against the oracle's update on the device gradient sum, element by
+    element."""
     from paper_2503_23186_b200 import binding
-    from netcheck import check_step_sampled
+    from netcheck import check_step, check_step_sampled
     params = wl.init_params(spec, seed)
-    images, labels = wl.image_batch(seed, micro_batch * n_micro)
+    n = micro_batch * n_micro
+    images, labels = wl.image_batch(seed, n)
     net = binding.Net(ctx, spec, micro_batch, n_concurrent=n_micro)
     net.load_params(params)
     d_img, d_lab = dev_bf16(images), torch.from_numpy(labels).cuda()
     net.train_step(d_img, d_lab, n_micro, LR, MU, WD, update=False)
     assert ctx.device_status() == 0
-    rep = check_step_sampled(net, spec, images, labels, micro_batch * n_micro, groups=n_micro, samples=96, seed=seed)
+    if sampled:
+        rep = check_step_sampled(net, spec, images, labels, n, groups=n_micro, samples=96, seed=seed)
+    else:
+        rep = check_step(net, spec, images, labels, n, groups=n_micro, lowmem=True)
     worst = rep.worst()
-    print("full-size sampled check: %d comparisons, worst %s relF=%.3e max=%.3e" % (len(rep.rows), worst[0], worst[1], worst[2]))
+    print("full-size check (%s): %d comparisons, worst %s relF=%.3e max=%.3e" % ("sampled" if sampled else "every element", len(rep.rows), worst[0],
+                                                                                 worst[1], worst[2]))
     rep.assert_ok()
     # scale invariance of every convolution that feeds a BatchNorm: <w, dL/dw> ~ 0 (holds at any size)
     g, w = net.unpack(net.g), net.unpack(net.w)
@@ -335,11 +342,13 @@ def _full_size_sampled(ctx, spec, micro_batch, n_micro, seed):
 
 
 def test_resnet18_batch1024_config4_full_size(ctx):
-    _full_size_sampled(ctx, wl.resnet18_spec(), 128, 8, 0)
+    """Config 4: batch 1024 as eight micro-batches of 128 side by side, every element of every tensor against the oracle."""
+    _full_size(ctx, wl.resnet18_spec(), 128, 8, 0)
 
 
 def test_wrn28_10_batch256_config5_full_size(ctx):
-    _full_size_sampled(ctx, wl.wrn28_10_spec(), 256, 1, 0)
+    """Config 5: the WRN-28-10-shaped net at batch 256, every element of every tensor against the oracle."""
+    _full_size(ctx, wl.wrn28_10_spec(), 256, 1, 0)
 
 
 def test_tiny_bottleneck_net(ctx):
@@ -368,7 +377,7 @@ def test_resnet50_small_batch_layerwise(ctx):
 
 def test_resnet50_batch1024_full_size(ctx):
     """The ResNet-50-shaped net in the launch configuration bench.py times (eight micro-batches of 128 side by side)."""
-    _full_size_sampled(ctx, wl.resnet50_spec(), 128, 8, 0)
+    _full_size(ctx, wl.resnet50_spec(), 128, 8, 0, sampled=True)
 
 
 def test_wrn28_10_small_batch_layerwise(ctx):
