@@ -84,6 +84,11 @@ void b2c_set_stall_counters(b2c_ctx* ctx, unsigned long long* counters);
 
 /* ---- Forward pass (Algorithm 1, "Perform forward pass") -------------------------------- */
 
+/* Bytes of caller-owned scratch one convolution call needs (which: 0 forward, 1 data gradient, 2 weight gradient).
+ * Always 0: the three convolution entry points stage their operands in shared memory and accumulate in TMEM, and the
+ * weight gradient adds its partial sums straight into dw.  Kept so that callers can size buffers uniformly. */
+size_t b2c_conv2d_workspace_bytes(const b2c_conv_desc* d, int which);
+
 /* y[n,p,q,k] = sum_{r,s,c} x[n, p*stride+r-pad, q*stride+s-pad, c] * w[k,r,s,c]  (+ bias[k]),
  * x zero outside the image (cross-correlation, no kernel flip).  Implicit GEMM on tcgen05:
  * M = n*p*q, N = k, K = r*s*c.

@@ -24,7 +24,7 @@ LAYER_KINDS = {"conv": 0, "bn": 1, "avgpool": 2, "fc": 3, "xent": 4}
 # every symbol include/b2c.h declares
 EXPORTS = [
     "b2c_create", "b2c_destroy", "b2c_status_string", "b2c_get_device_status", "b2c_set_spin_limit", "b2c_set_stall_counters",
-    "b2c_conv2d_fwd", "b2c_bn_relu_fwd", "b2c_avgpool_fwd", "b2c_avgpool_bwd", "b2c_pad_channels",
+    "b2c_conv2d_workspace_bytes", "b2c_conv2d_fwd", "b2c_bn_relu_fwd", "b2c_avgpool_fwd", "b2c_avgpool_bwd", "b2c_pad_channels",
     "b2c_softmax_xent_fwd_bwd", "b2c_bn_relu_bwd_workspace_bytes", "b2c_bn_relu_bwd", "b2c_bn_relu_bwd_static", "b2c_conv2d_dgrad",
     "b2c_conv2d_wgrad", "b2c_bias_grad", "b2c_grad_accum_sgd_momentum", "b2c_weight_pack_dgrad",
     "b2c_net_create", "b2c_net_create_concurrent", "b2c_net_destroy", "b2c_net_param_count", "b2c_net_param_offset",
@@ -67,6 +67,7 @@ def lib() -> ctypes.CDLL:
         L.b2c_net_param_count.restype = c_size_t
         L.b2c_net_workspace_bytes.restype = c_size_t
         L.b2c_bn_relu_bwd_workspace_bytes.restype = c_size_t
+        L.b2c_conv2d_workspace_bytes.restype = c_size_t
         L.b2c_net_param_offset.restype = c_longlong
         L.b2c_net_tensor_offset.restype = c_longlong
         L.b2c_destroy.restype = None

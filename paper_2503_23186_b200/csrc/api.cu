@@ -31,6 +31,7 @@ b2c_status b2c_create(b2c_ctx** out, int device)
     ctx->sm_count = prop.multiProcessorCount;
     ctx->spin_limit = 1u << 22;
     ctx->stall_counters = nullptr;
+    ctx->smem_optin_done = 0u;
     {
         const char* env = std::getenv("B2C_CTA_PAIRS");
         ctx->use_pairs = env ? (env[0] == '2' ? 2 : env[0] == '1' ? 1 : 0) : 1;   // 0 never, 1 for 128-channel tiles (default), 2 wherever possible
@@ -122,6 +123,12 @@ static b2c_status check_desc(const b2c_conv_desc* d, int* p, int* q)
     return B2C_OK;
 }
 
+size_t b2c_conv2d_workspace_bytes(const b2c_conv_desc* d, int which)
+{
+    (void)d; (void)which;
+    return 0;   // forward, data gradient and weight gradient keep everything they need in shared memory and TMEM
+}
+
 b2c_status b2c_conv2d_fwd(b2c_ctx* ctx, const b2c_conv_desc* d, const void* x, const void* w_krsc, void* y, int y_is_f32, const float* bias,
                           double* ch_stats, void* stream)
 {
@@ -167,7 +174,10 @@ b2c_status b2c_conv2d_wgrad(b2c_ctx* ctx, const b2c_conv_desc* d, const void* dy
     pb.p = p; pb.q = q; pb.k = d->k;
     pb.r = d->r; pb.stride = d->stride; pb.pad = d->pad;
     pb.dy = dy; pb.x = x; pb.dw = dw_krsc;
-    if (d->c % 16 || d->k % 16) return B2C_ERR_UNSUPPORTED_SHAPE;
+    // everything the launcher would reject is rejected here, before anything is enqueued
+    if (d->c < 16 || d->c % 16 || d->k < 16 || d->k % 16) return B2C_ERR_UNSUPPORTED_SHAPE;
+    if (!b2c_is_pow2(p) || !b2c_is_pow2(q) || p > 128 || q > 128) return B2C_ERR_UNSUPPORTED_SHAPE;
+    if (!b2c_aligned16(dy) || !b2c_aligned16(x) || !b2c_aligned16(dw_krsc)) return B2C_ERR_MISALIGNED;
     if (!accumulate) B2C_CUDA(cudaMemsetAsync(dw_krsc, 0, sizeof(float) * (size_t)d->k * d->r * d->s * d->c, (cudaStream_t)stream));
     return launch_conv_wgrad(ctx, pb, (cudaStream_t)stream);
 }
@@ -542,9 +552,9 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
         return slot >= 0 && T.grad_off[slot] >= 0 ? net->ws + T.grad_off[slot] + (long long)img0 * T.h * T.w * T.c * 2 : nullptr;
     };
 
-    B2C_CUDA(cudaMemsetAsync(loss_dev, 0, sizeof(float), stream));
     const size_t image_bytes = (size_t)N * net->image_h * net->image_w * net->image_c * 2;
     if (image_bytes % 16) return B2C_ERR_MISALIGNED;
+    B2C_CUDA(cudaMemsetAsync(loss_dev, 0, sizeof(float), stream));
     const int mbs = net->micro_batch;
 
     for (int mb = 0; mb < n_passes; ++mb) {

@@ -27,7 +27,11 @@ struct b2c_ctx {
     int use_wgrad_frame;                 // weight gradient of 3x3 stride-1 layers stages x once per chunk with a one-pixel frame (all three shifts from one box)
     int use_issue_split;                 // forward / data-gradient tiles wider than 128 channels: two MMA-issuing threads share every unit
     int use_pdl;                         // kernels are launched with programmatic stream serialization (their set-up overlaps the previous kernel's tail)
+    unsigned smem_optin_done;            // kernels whose dynamic shared-memory opt-in was set on this context's device (B2C_OPTIN_* bits)
 };
+#define B2C_OPTIN_KMAJOR 1u
+#define B2C_OPTIN_WGRAD 2u
+#define B2C_OPTIN_BN_BWD 4u
 
 #define B2C_CUDA(call)                               \
     do {                                             \

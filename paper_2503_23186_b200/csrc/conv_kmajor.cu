@@ -810,7 +810,6 @@ void forward_taps(TapList& tl, int R, int stride, int pad)
 
 b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_t stream)
 {
-    static bool attr_set = false;
     ConvKParams p;
     memset(&p, 0, sizeof(p));
     const int R = pb.r;
@@ -1009,10 +1008,10 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
     p.spin_limit = ctx->spin_limit;
     p.stall = ctx->stall_counters;
 
-    if (!attr_set) {
+    if (!(ctx->smem_optin_done & B2C_OPTIN_KMAJOR)) {   // the attribute belongs to the device: kept per context, not per process
         B2C_CUDA(cudaFuncSetAttribute(conv_kmajor_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 212 * 1024));
         B2C_CUDA(cudaFuncSetAttribute(conv_kmajor_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 212 * 1024));
-        attr_set = true;
+        ctx->smem_optin_done |= B2C_OPTIN_KMAJOR;
     }
     if (p.pair) B2C_CUDA(b2c_launch(ctx, conv_kmajor_kernel<true>, dim3((unsigned)grid), dim3(kThreads), smem_bytes, stream, 2u, p));
     else B2C_CUDA(b2c_launch(ctx, conv_kmajor_kernel<false>, dim3((unsigned)grid), dim3(kThreads), smem_bytes, stream, 1u, p));

@@ -370,7 +370,6 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
 
 b2c_status launch_conv_wgrad(b2c_ctx* ctx, const WgradProblem& pb, cudaStream_t stream)
 {
-    static bool attr_set = false;
     WgradParams p;
     memset(&p, 0, sizeof(p));
     const int R = pb.r;
@@ -518,9 +517,9 @@ b2c_status launch_conv_wgrad(b2c_ctx* ctx, const WgradProblem& pb, cudaStream_t 
     p.spin_limit = ctx->spin_limit;
     p.stall = ctx->stall_counters;
 
-    if (!attr_set) {
+    if (!(ctx->smem_optin_done & B2C_OPTIN_WGRAD)) {
         B2C_CUDA(cudaFuncSetAttribute(conv_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 212 * 1024));
-        attr_set = true;
+        ctx->smem_optin_done |= B2C_OPTIN_WGRAD;
     }
     const size_t smem_bytes = (size_t)p.stages * p.stage_bytes + 1024;
     dim3 grid((unsigned)(base * n_splits));

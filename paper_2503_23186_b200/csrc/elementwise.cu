@@ -887,15 +887,14 @@ b2c_status launch_bn_bwd(b2c_ctx* ctx, int G, long long m, int c, const void* da
     const bool staged = (!relu || mask != nullptr) && chunk_vecs % 16 == 0 && (m * groups) % 16 == 0 && m >= 2ll * rows_per_iter * grid.x &&
                         reinterpret_cast<uintptr_t>(mask) % 16 == 0;
     if (staged) {
-        static bool attr_set = false;
         const int nt = da2 != nullptr ? 3 : 2;
         const size_t stage = (size_t)nt * chunk_vecs * 16 + (relu ? ((chunk_vecs + 127) & ~127) : 0);
         const size_t smem = kStStages * stage + sizeof(float) * 2 * c + 128;
         if (smem <= 110 * 1024) {
-            if (!attr_set) {
+            if (!(ctx->smem_optin_done & B2C_OPTIN_BN_BWD)) {
                 B2C_CUDA(cudaFuncSetAttribute(bn_bwd_reduce_staged_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024));
                 B2C_CUDA(cudaFuncSetAttribute(bn_bwd_apply_staged_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024));
-                attr_set = true;
+                ctx->smem_optin_done |= B2C_OPTIN_BN_BWD;
             }
             B2C_CUDA(b2c_launch(ctx, bn_bwd_reduce_staged_kernel, dim3(grid), dim3(kStThreads), smem, stream, 1u, da1, da2, y, m, c, relu, sums, mask, ctx->spin_limit, ctx->d_status));
             B2C_CUDA(b2c_launch(ctx, bn_bwd_apply_staged_kernel, dim3(grid), dim3(kStThreads), smem, stream, 1u, da1, da2, y, m, c, gamma, save_mean, save_invstd, relu, sums, dy, dres,
