@@ -160,6 +160,21 @@ b2c_status b2c_bn_relu_bwd(b2c_ctx* ctx, int n, int h, int w, int c, const void*
                            int relu, void* dy, void* dres, float* dgamma, float* dbeta, int acc,
                            const void* relu_mask, void* ws, size_t ws_bytes, void* stream);
 
+/* The same backward for several statistics groups side by side (replica-local BatchNorm of data parallelism: each
+ * replica, or micro-batch, normalises over its own images; Section III-A, data parallelism): the tensors hold `groups`
+ * runs of rows_per_group rows of c channels back to back, save_mean / save_invstd are fp32 [groups][c], and every
+ * group is differentiated with its own statistics.  dgamma / dbeta receive the sum over the groups (overwritten if
+ * acc == 0, accumulated into otherwise).  Both passes run in one cooperative launch, group by group: the reduction of
+ * a group, a grid-wide barrier, then the apply pass of that group while its tensors are still in L2 (about 6 bytes
+ * of DRAM traffic per element instead of 10).  Requires relu_mask when relu != 0.
+ *   ws: scratch of b2c_bn_relu_bwd_groups_workspace_bytes(c, groups) bytes, 8-byte aligned; the call zeroes it. */
+size_t b2c_bn_relu_bwd_groups_workspace_bytes(int c, int groups);
+b2c_status b2c_bn_relu_bwd_groups(b2c_ctx* ctx, int groups, long long rows_per_group, int c, const void* da1,
+                                  const void* da2, const void* y, const float* gamma, const float* save_mean,
+                                  const float* save_invstd, int relu, void* dy, void* dres, float* dgamma,
+                                  float* dbeta, int acc, const void* relu_mask, void* ws, size_t ws_bytes,
+                                  void* stream);
+
 /* (No counterpart in the paper: a packaging variant of b2c_bn_relu_bwd.)
  * The same computation, arguments and results as b2c_bn_relu_bwd, but without the `ws` argument: the per-channel
  * fp64 accumulators live in an array built into the library (B2C_BN_BWD_STATIC_MAX_C channels, 32 KB, resident on
@@ -274,6 +289,22 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
  * weight copies are refreshed and grad_sum is zeroed.  Data-parallel replicas call b2c_train_step with update == 0,
  * sum grad_sum across replicas (e.g. an NCCL all-reduce), then call this with n_avg = n_micro * replicas. */
 b2c_status b2c_net_apply_update(b2c_net* net, int n_avg, float lr, float momentum, float wd, void* stream);
+
+/* Pieces of the update for data-parallel replicas that shard the optimiser state (gradient synchronisation fused with
+ * the update: reduce-scatter of grad_sum, b2c_grad_accum_sgd_momentum on the replica's own slice of the flat arrays,
+ * all-gather of the bf16 copy): the filter banks of the weight layers occupy [begin, end) element ranges of the flat
+ * arrays in layer order (b2c_net_weight_range, index < b2c_net_weight_layer_count; the backward pass completes them
+ * last layer first), and b2c_net_refresh_dgrad_weights rewrites w_bf16_dgrad from the current w_bf16. */
+int b2c_net_weight_layer_count(const b2c_net* net);
+/* Gradient-ready events for buckets of the flat arrays: after b2c_net_set_buckets, every b2c_train_step records event k
+ * on its stream once weight layer first_layer[k] (an index < b2c_net_weight_layer_count) has finished its parameter
+ * gradient for the step; every later weight layer, and with first_layer[k] == 0 everything else, is final by then.
+ * b2c_net_bucket_wait makes `stream` (the stream of the collectives) wait for event k, so that a bucket's exchange
+ * starts while the backward pass of the earlier layers still runs.  n_buckets == 0 removes the events. */
+b2c_status b2c_net_set_buckets(b2c_net* net, int n_buckets, const int* first_layer);
+b2c_status b2c_net_bucket_wait(b2c_net* net, int bucket, void* stream);
+b2c_status b2c_net_weight_range(const b2c_net* net, int index, long long* begin, long long* end);
+b2c_status b2c_net_refresh_dgrad_weights(b2c_net* net, void* stream);
 
 /* ---- Per-component timing (the profiling phase of the paper's adaptive scheduling algorithm
  *      measures the execution time of each network component; this is the measurement hook) ---- */

@@ -25,12 +25,14 @@ LAYER_KINDS = {"conv": 0, "bn": 1, "avgpool": 2, "fc": 3, "xent": 4}
 EXPORTS = [
     "b2c_create", "b2c_destroy", "b2c_status_string", "b2c_get_device_status", "b2c_set_spin_limit", "b2c_set_stall_counters",
     "b2c_conv2d_workspace_bytes", "b2c_conv2d_fwd", "b2c_bn_relu_fwd", "b2c_avgpool_fwd", "b2c_avgpool_bwd", "b2c_pad_channels",
-    "b2c_softmax_xent_fwd_bwd", "b2c_bn_relu_bwd_workspace_bytes", "b2c_bn_relu_bwd", "b2c_bn_relu_bwd_static", "b2c_conv2d_dgrad",
+    "b2c_softmax_xent_fwd_bwd", "b2c_bn_relu_bwd_workspace_bytes", "b2c_bn_relu_bwd", "b2c_bn_relu_bwd_static",
+    "b2c_bn_relu_bwd_groups_workspace_bytes", "b2c_bn_relu_bwd_groups", "b2c_conv2d_dgrad",
     "b2c_conv2d_wgrad", "b2c_bias_grad", "b2c_grad_accum_sgd_momentum", "b2c_weight_pack_dgrad",
     "b2c_net_create", "b2c_net_create_concurrent", "b2c_net_destroy", "b2c_net_param_count", "b2c_net_param_offset",
     "b2c_net_padded_image_channels", "b2c_net_first_conv_im2col", "b2c_im2col_3x3", "b2c_net_workspace_bytes", "b2c_net_tensor_offset", "b2c_net_bind",
     "b2c_net_sync_weights", "b2c_train_step", "b2c_net_apply_update", "b2c_net_profile_enable", "b2c_net_profile_read",
     "b2c_net_profile_read_layers", "b2c_net_layer_count",
+    "b2c_net_weight_layer_count", "b2c_net_weight_range", "b2c_net_refresh_dgrad_weights", "b2c_net_set_buckets", "b2c_net_bucket_wait",
 ]
 PROF_KINDS = ["conv_fwd", "conv_dgrad", "conv_wgrad", "bn_fwd", "bn_bwd", "other", "update"]
 
@@ -68,6 +70,7 @@ def lib() -> ctypes.CDLL:
         L.b2c_net_workspace_bytes.restype = c_size_t
         L.b2c_bn_relu_bwd_workspace_bytes.restype = c_size_t
         L.b2c_conv2d_workspace_bytes.restype = c_size_t
+        L.b2c_bn_relu_bwd_groups_workspace_bytes.restype = c_size_t
         L.b2c_net_param_offset.restype = c_longlong
         L.b2c_net_tensor_offset.restype = c_longlong
         L.b2c_destroy.restype = None
@@ -170,6 +173,17 @@ class Context:
                                      _ptr(save_invstd), c_int(int(relu)), _ptr(dy), _ptr(dres), _ptr(dgamma), _ptr(dbeta), c_int(int(acc)),
                                      _ptr(relu_mask), _ptr(ws), c_size_t(ws.numel() * ws.element_size()), _stream()), "b2c_bn_relu_bwd")
 
+    @staticmethod
+    def bn_relu_bwd_groups_workspace_bytes(c, groups) -> int:
+        return lib().b2c_bn_relu_bwd_groups_workspace_bytes(c_int(c), c_int(groups))
+
+    def bn_relu_bwd_groups(self, groups, rows_per_group, c, da1, da2, y, gamma, save_mean, save_invstd, relu, dy, dres, dgamma, dbeta, acc, relu_mask, ws):
+        """BatchNorm backward of `groups` statistics groups stored back to back (both passes in one launch, group by group)."""
+        _check(lib().b2c_bn_relu_bwd_groups(self.handle, c_int(groups), c_longlong(rows_per_group), c_int(c), _ptr(da1), _ptr(da2), _ptr(y), _ptr(gamma),
+                                            _ptr(save_mean), _ptr(save_invstd), c_int(int(relu)), _ptr(dy), _ptr(dres), _ptr(dgamma), _ptr(dbeta),
+                                            c_int(int(acc)), _ptr(relu_mask), _ptr(ws), c_size_t(ws.numel() * ws.element_size()), _stream()),
+               "b2c_bn_relu_bwd_groups")
+
     def bn_relu_bwd_static(self, n, h, w, c, da1, da2, y, a, gamma, save_mean, save_invstd, relu, dy, dres, dgamma, dbeta, acc):
         """b2c_bn_relu_bwd without a caller-provided workspace: the accumulators live inside the library, so the
         call allocates nothing (for callers that cannot get device memory of their own; at most 2048 channels;
@@ -222,6 +236,7 @@ class Net:
         self.w_dgrad = torch.zeros_like(self.w_bf16)
         self.workspace = torch.zeros(self.workspace_bytes, dtype=torch.uint8, device=dev)
         self.loss = torch.zeros(1, dtype=torch.float32, device=dev)
+        self.bucket_events = None
         _check(lib().b2c_net_bind(self.handle, _ptr(self.w), _ptr(self.v), _ptr(self.g), _ptr(self.w_bf16), _ptr(self.w_dgrad),
                                   _ptr(self.workspace), c_size_t(self.workspace_bytes)), "b2c_net_bind")
 
@@ -299,6 +314,36 @@ class Net:
 
     def apply_update(self, n_avg, lr, momentum, wd):
         _check(lib().b2c_net_apply_update(self.handle, c_int(n_avg), c_float(lr), c_float(momentum), c_float(wd), _stream()), "b2c_net_apply_update")
+
+    # ---- pieces of the update for replicas that shard the optimiser state (data_parallel.dp_train_step_sharded)
+    def weight_layer_ranges(self):
+        """[(begin, end)] element ranges of the filter banks in the flat arrays, in layer order."""
+        out = []
+        for i in range(lib().b2c_net_weight_layer_count(self.handle)):
+            b, e = c_longlong(), c_longlong()
+            _check(lib().b2c_net_weight_range(self.handle, c_int(i), byref(b), byref(e)), "b2c_net_weight_range")
+            out.append((b.value, e.value))
+        return out
+
+    def set_buckets(self, buckets):
+        """buckets = data_parallel.bucket_plan(...): train_step then records a gradient-ready event per bucket."""
+        first = (c_int * len(buckets))(*[b[2] for b in buckets])
+        _check(lib().b2c_net_set_buckets(self.handle, c_int(len(buckets)), first), "b2c_net_set_buckets")
+        self.bucket_events = list(range(len(buckets))) if buckets else None
+
+    def bucket_wait(self, k, stream):
+        """Makes the torch stream `stream` wait until bucket k's gradients of the current step are final."""
+        _check(lib().b2c_net_bucket_wait(self.handle, c_int(k), c_void_p(stream.cuda_stream)), "b2c_net_bucket_wait")
+
+    def apply_update_range(self, begin, end, n_avg, lr, momentum, wd):
+        """The fused average + SGD-momentum update on elements [begin, end) of the flat arrays only (fp32 master, momentum,
+        gradient sum cleared, bf16 copy); begin a multiple of 8."""
+        self.ctx.grad_accum_sgd_momentum(end - begin, self.w[begin:end], self.v[begin:end], self.g[begin:end], 1.0 / n_avg, lr, momentum, wd,
+                                         self.w_bf16[begin:end], True)
+
+    def refresh_derived_weights(self):
+        """Rewrites the data-gradient layout of the bf16 weights from the current bf16 copy."""
+        _check(lib().b2c_net_refresh_dgrad_weights(self.handle, _stream()), "b2c_net_refresh_dgrad_weights")
 
     def profile_enable(self, enable: bool = True):
         _check(lib().b2c_net_profile_enable(self.handle, c_int(int(enable))), "b2c_net_profile_enable")

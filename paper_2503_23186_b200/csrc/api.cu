@@ -34,7 +34,7 @@ b2c_status b2c_create(b2c_ctx** out, int device)
     ctx->smem_optin_done = 0u;
     {
         const char* env = std::getenv("B2C_CTA_PAIRS");
-        ctx->use_pairs = env ? (env[0] == '2' ? 2 : env[0] == '1' ? 1 : 0) : 1;   // 0 never, 1 for 128-channel tiles (default), 2 wherever possible
+        ctx->use_pairs = env ? (env[0] == '3' ? 3 : env[0] == '2' ? 2 : env[0] == '1' ? 1 : 0) : 1;   // 0 never, 1 for 3x3 stride-1 layers with tiles of 128 channels or more (default), 2 wherever possible, 3 for 128-channel tiles only
     }
     {
         const char* env = std::getenv("B2C_FULL_HALO");
@@ -51,6 +51,10 @@ b2c_status b2c_create(b2c_ctx** out, int device)
     {
         const char* env = std::getenv("B2C_PDL");
         ctx->use_pdl = env ? (env[0] != '0') : 1;
+    }
+    {
+        const char* env = std::getenv("B2C_BN_GROUPED");
+        ctx->use_bn_grouped = env ? (env[0] != '0') : 1;
     }
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
@@ -206,9 +210,10 @@ struct LayerPlan {
     int gemm_r = 0;                // filter size the convolution kernels see (1 for the patch-matrix stem)
     int p = 0, q = 0;
     long long w_off = -1, gamma_off = -1, beta_off = -1, bias_off = -1;   // elements into the flat parameter arrays
-    long long mean_off = -1, invstd_off = -1, bwd_ws_off = -1, mask_off = -1;   // bytes into the workspace
+    long long mean_off = -1, invstd_off = -1, bwd_ws_off = -1, mask_off = -1, arrive_off = -1;   // bytes into the workspace
     int src_slot = -1, res_slot = -1;                                     // which gradient buffer of src / res this layer writes
     int chunk_groups = 1;          // micro-batches of a pass this layer takes per launch (divides n_conc)
+    int seg_index = -1;            // position of this layer's filter bank among the weight layers (conv, fc)
 };
 
 inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
@@ -236,9 +241,14 @@ struct b2c_net {
     std::vector<Span> spans;      // event pool, reused every step
     size_t spans_used = 0;
     long long launches[B2C_PROF_KINDS] = {0};   // kernels launched since the last profile read
+    // gradient-ready events of the update buckets: event k is recorded once the weight layer first_layer[k] has finished its
+    // parameter gradient in the last pass of a step (the backward pass completes weight layers last to first)
+    std::vector<int> bucket_first_layer;
+    std::vector<cudaEvent_t> bucket_events;
     ~b2c_net()
     {
         for (Span& sp : spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
+        for (cudaEvent_t e : bucket_events) cudaEventDestroy(e);
     }
 };
 
@@ -327,6 +337,7 @@ b2c_status b2c_net_create_concurrent(b2c_ctx* ctx, const b2c_layer_desc* layers,
                 o.act_off = alloc(o.elems() * 2);
                 L.gemm_r = patch ? 1 : d.r;
                 L.w_off = palloc((size_t)d.k * L.gemm_r * L.gemm_r * L.c_pad);
+                L.seg_index = (int)net->segs.size();
                 net->segs.push_back(b2c_weight_seg{L.w_off, d.k, L.gemm_r * L.gemm_r, L.c_pad});
                 break;
             }
@@ -355,6 +366,7 @@ b2c_status b2c_net_create_concurrent(b2c_ctx* ctx, const b2c_layer_desc* layers,
                 o.n = batch; o.h = 1; o.w = 1; o.c = L.k_pad; o.f32 = true; o.exists = true;
                 o.act_off = alloc(o.elems() * 4);
                 L.w_off = palloc((size_t)L.k_pad * L.c_pad);
+                L.seg_index = (int)net->segs.size();
                 net->segs.push_back(b2c_weight_seg{L.w_off, L.k_pad, 1, L.c_pad});
                 break;
             }
@@ -424,7 +436,10 @@ b2c_status b2c_net_create_concurrent(b2c_ctx* ctx, const b2c_layer_desc* layers,
                 if (n_tile > 64 && !wide_ok) o.fused_stats = false;
             }
         }
-        if (L.d.kind == B2C_LAYER_BN) L.bwd_ws_off = alloc(b2c_bn_relu_bwd_workspace_bytes(L.d.c) * n_concurrent);
+        if (L.d.kind == B2C_LAYER_BN) {
+            L.bwd_ws_off = alloc(b2c_bn_relu_bwd_workspace_bytes(L.d.c) * n_concurrent);
+            L.arrive_off = alloc(sizeof(unsigned) * (size_t)n_concurrent);   // one arrival counter per statistics group, cleared with the sums
+        }
     }
     net->stats_end = (long long)ws;
     net->ws_bytes = ws;
@@ -499,6 +514,46 @@ static b2c_status net_pack_dgrad(b2c_net* net, void* stream)
 {
     return b2c_weight_pack_dgrad(net->ctx, net->segs.data(), (int)net->segs.size(), net->w_bf16, net->w_dgrad, stream);
 }
+
+b2c_status b2c_net_set_buckets(b2c_net* net, int n_buckets, const int* first_layer)
+{
+    if (!net || n_buckets < 0 || (n_buckets > 0 && !first_layer)) return B2C_ERR_INVALID_ARG;
+    for (int b = 0; b < n_buckets; ++b)
+        if (first_layer[b] < 0 || first_layer[b] >= (int)net->segs.size()) return B2C_ERR_INVALID_ARG;
+    for (cudaEvent_t e : net->bucket_events) cudaEventDestroy(e);
+    net->bucket_events.clear();
+    net->bucket_first_layer.assign(first_layer, first_layer + n_buckets);
+    for (int b = 0; b < n_buckets; ++b) {
+        cudaEvent_t e;
+        if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return B2C_ERR_CUDA;
+        net->bucket_events.push_back(e);
+    }
+    return B2C_OK;
+}
+
+b2c_status b2c_net_bucket_wait(b2c_net* net, int bucket, void* stream)
+{
+    if (!net || bucket < 0 || bucket >= (int)net->bucket_events.size()) return B2C_ERR_INVALID_ARG;
+    B2C_CUDA(cudaStreamWaitEvent((cudaStream_t)stream, net->bucket_events[bucket], 0));
+    return B2C_OK;
+}
+
+b2c_status b2c_net_refresh_dgrad_weights(b2c_net* net, void* stream)
+{
+    if (!net || !net->ws) return B2C_ERR_INVALID_ARG;
+    return net_pack_dgrad(net, stream);
+}
+
+b2c_status b2c_net_weight_range(const b2c_net* net, int index, long long* begin, long long* end)
+{
+    if (!net || !begin || !end || index < 0 || index >= (int)net->segs.size()) return B2C_ERR_INVALID_ARG;
+    const b2c_weight_seg& sg = net->segs[index];
+    *begin = sg.offset;
+    *end = sg.offset + (long long)sg.k * sg.rs * sg.c;
+    return B2C_OK;
+}
+
+int b2c_net_weight_layer_count(const b2c_net* net) { return net ? (int)net->segs.size() : 0; }
 
 b2c_status b2c_net_sync_weights(b2c_net* net, void* stream)
 {
@@ -635,6 +690,12 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
             return B2C_OK;
         };
 
+        // the parameter gradient of weight layer `seg` is complete for this step: release the buckets that waited for it
+        auto weights_done = [&](int seg, int g0, int Gc) {
+            if (mb != n_passes - 1 || g0 + Gc != G) return;
+            for (size_t b = 0; b < net->bucket_events.size(); ++b)
+                if (net->bucket_first_layer[b] == seg) cudaEventRecord(net->bucket_events[b], stream);
+        };
         // backward pass of layer i over the same kind of run; parameter gradients are summed into the flat gradient array
         auto backward_layer = [&](int i, int g0, int Gc) -> b2c_status {
             const LayerPlan& L = net->layers[i];
@@ -651,6 +712,7 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
                     ProfScope ps_(net, stream, B2C_PROF_OTHER, 3, i, 1);
                     B2C_TRY(launch_conv_wgrad(ctx, wp, stream));
                     B2C_TRY(b2c_bias_grad(ctx, Nc, L.k_pad, L.k_pad, dz, net->g + L.bias_off, 1, stream));
+                    weights_done(L.seg_index, g0, Gc);
                     KMajorProblem pb{};
                     pb.n = Nc; pb.ih = 1; pb.iw = 1; pb.ic = L.k_pad; pb.oh = 1; pb.ow = 1; pb.oc = L.c_pad;
                     pb.r = 1; pb.stride = 1; pb.pad = 0; pb.dgrad = true;
@@ -673,7 +735,8 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
                                           reinterpret_cast<float*>(net->ws + L.invstd_off) + (size_t)g0 * in.c, d.relu, grad(d.src, L.src_slot, img0),
                                           d.res >= 0 ? grad(d.res, L.res_slot, img0) : nullptr, net->g + L.gamma_off, net->g + L.beta_off, 1,
                                           reinterpret_cast<double*>(net->ws + L.bwd_ws_off) + (size_t)g0 * 2 * in.c, /*sums_zeroed=*/in.stats_off >= 0,
-                                          L.mask_off >= 0 ? net->ws + L.mask_off + (long long)img0 * in.h * in.w * in.c / 8 : nullptr, stream));
+                                          L.mask_off >= 0 ? net->ws + L.mask_off + (long long)img0 * in.h * in.w * in.c / 8 : nullptr,
+                                          reinterpret_cast<unsigned*>(net->ws + L.arrive_off) + g0, stream));
                     break;
                 }
                 case B2C_LAYER_CONV: {
@@ -686,6 +749,7 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
                         ProfScope ps_(net, stream, B2C_PROF_CONV_WGRAD, 1, i, 1);
                         B2C_TRY(launch_conv_wgrad(ctx, wp, stream));
                     }
+                    weights_done(L.seg_index, g0, Gc);
                     if (d.src != 0) {
                         KMajorProblem pb{};
                         pb.n = Nc; pb.ih = L.p; pb.iw = L.q; pb.ic = d.k; pb.oh = d.h; pb.ow = d.w; pb.oc = L.c_pad;

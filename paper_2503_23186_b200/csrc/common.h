@@ -27,11 +27,13 @@ struct b2c_ctx {
     int use_wgrad_frame;                 // weight gradient of 3x3 stride-1 layers stages x once per chunk with a one-pixel frame (all three shifts from one box)
     int use_issue_split;                 // forward / data-gradient tiles wider than 128 channels: two MMA-issuing threads share every unit
     int use_pdl;                         // kernels are launched with programmatic stream serialization (their set-up overlaps the previous kernel's tail)
+    int use_bn_grouped;                  // BatchNorm backward of the training step: both passes in one cooperative launch, group by group
     unsigned smem_optin_done;            // kernels whose dynamic shared-memory opt-in was set on this context's device (B2C_OPTIN_* bits)
 };
 #define B2C_OPTIN_KMAJOR 1u
 #define B2C_OPTIN_WGRAD 2u
 #define B2C_OPTIN_BN_BWD 4u
+#define B2C_OPTIN_BN_GROUPED 8u
 
 #define B2C_CUDA(call)                               \
     do {                                             \
@@ -122,12 +124,13 @@ b2c_status launch_conv_wgrad(b2c_ctx* ctx, const WgradProblem& pb, cudaStream_t 
 // save_mean / save_invstd fp32 [G][c].  G > 1 requires acc != 0 in the backward pass.  stats_ready: 1 = `stats` holds the
 // sums already (convolution epilogue), 0 = clear and compute them, 2 = compute them into `stats` the caller has cleared.  relu_mask (optional): one bit per
 // element, "stored output > 0" (a byte per 8 channels), written by the forward pass and read by the backward pass
-// in place of the output tensor.  sums_zeroed: the caller has already cleared `sums`.
+// in place of the output tensor.  sums_zeroed: the caller has already cleared `sums` (and `arrivals`).  arrivals (optional): G
+// zeroed counters; with them the two passes run in one cooperative launch, group by group (bn_bwd_grouped_kernel).
 b2c_status launch_bn_fwd(b2c_ctx* ctx, int G, long long m, int c, const void* y, double* stats, int stats_ready, const float* gamma,
                          const float* beta, const void* residual, int relu, float eps, void* a, float* save_mean, float* save_invstd,
                          float* run_mean, float* run_var, float momentum, void* relu_mask, cudaStream_t stream);
 b2c_status launch_bn_bwd(b2c_ctx* ctx, int G, long long m, int c, const void* da1, const void* da2, const void* y, const void* a,
                          const float* gamma, const float* save_mean, const float* save_invstd, int relu, void* dy, void* dres, float* dgamma,
-                         float* dbeta, int acc, double* sums, bool sums_zeroed, const void* relu_mask, cudaStream_t stream);
+                         float* dbeta, int acc, double* sums, bool sums_zeroed, const void* relu_mask, unsigned* arrivals, cudaStream_t stream);
 
 }  // namespace b2c

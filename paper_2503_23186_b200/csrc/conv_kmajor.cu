@@ -525,7 +525,10 @@ __device__ __forceinline__ void mma_issuer(const ConvKParams& p, const UnitWalk&
             // frees the stage (in both CTAs of a pair) once these MMAs have read it
             if constexpr (PAIR) umma_commit_pair(&empty_bar[s], (uint16_t)3);
             else umma_commit(&empty_bar[s]);
-            if (p.issue_split && it == 0) umma_commit(&init_bar[buf]);   // the overwriting stage of this unit
+            if (p.issue_split && it == 0) {   // the overwriting stage of this unit (both issuing threads live in the leader CTA of a pair)
+                if constexpr (PAIR) umma_commit_pair(&init_bar[buf], (uint16_t)1);
+                else umma_commit(&init_bar[buf]);
+            }
             ++i_stage;
             if (++s == S) { s = 0; ph ^= 1u; }
         }
@@ -859,7 +862,8 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
     // default only 3x3 stride-1 layers with 128-channel tiles use them (use_pairs: 0 = never, 1 = those, 2 = every
     // eligible problem).
     const bool pair_ok = n_par == 1 && !pb.out_f32 && pb.bias == nullptr && n_tile % 32 == 0 && m_tiles % 2 == 0 && ctx->sm_count >= 2;
-    p.pair = (pair_ok && (ctx->use_pairs == 2 || (ctx->use_pairs == 1 && n_tile == 128 && R == 3 && pb.stride == 1))) ? 1 : 0;
+    p.pair = (pair_ok && (ctx->use_pairs == 2 || (ctx->use_pairs == 1 && n_tile >= 128 && R == 3 && pb.stride == 1) ||
+                          (ctx->use_pairs == 3 && n_tile == 128 && R == 3 && pb.stride == 1))) ? 1 : 0;
     const int b_rows = p.pair ? n_tile / 2 : n_tile;   // filter rows one CTA fetches per tile
 
     // launch shape: one persistent CTA per SM; the unit walk stride (CTAs, or pairs) is a multiple of n_ktiles so that a
@@ -931,8 +935,8 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
     if (p.stages < 2) return B2C_ERR_UNSUPPORTED_SHAPE;
     // Two issuing threads where one cannot keep the tensor pipe busy: tiles of at most 128 channels.
     p.issuers = p.n_tile <= 128 ? kIssuers : 1;
-    // Wider tiles: both threads work on every unit, alternate stages (needs an even ring; single CTAs only).
-    if (p.n_tile > 128 && !p.pair && ctx->use_issue_split && p.stages >= 2) {
+    // Wider tiles: both threads work on every unit, alternate stages (needs an even ring).
+    if (p.n_tile > 128 && ctx->use_issue_split && p.stages >= 2) {
         p.stages &= ~1;
         p.issuers = kIssuers;
         p.issue_split = 1;

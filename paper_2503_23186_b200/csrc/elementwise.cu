@@ -8,6 +8,7 @@
 // registers until the end of the walk.  Row sums are combined in shared memory, then added to
 // global fp64 accumulators (fp32 partials over few rows, fp64 across them: var = E[y^2] - E[y]^2
 // stays accurate for channels whose mean is large against their spread).
+#include <cstdlib>
 #include "common.h"
 #include "ptx.cuh"
 
@@ -620,6 +621,261 @@ __global__ void __launch_bounds__(kStThreads, 2) bn_bwd_apply_staged_kernel(cons
     __syncthreads();
 }
 
+// ------------------------------------------------------------------------------ BN backward, both passes in one launch
+// One cooperative launch walks the statistics groups (micro-batches) in order: the reduction pass R(g) of a group, a
+// grid-wide barrier, then the apply pass A(g) of the same group, which finds the group's tensors still in L2 (a group
+// of a 1024-image layer is an eighth of the tensor: da and y of 17 MB each against 134 MB for all groups, which do not
+// fit the L2).  HBM traffic per element drops from 10.25 bytes (two passes over da and y, one write) to about 6.1.
+// The barrier of group g is split: every block arrives after R(g), runs the reduction passes of the next `ahead`
+// groups, and only then waits, so the barrier latency hides behind useful work.  Small layers (whole tensor in L2
+// anyway) look further ahead; they gain the second launch.  The launch is cooperative (all blocks co-resident), every
+// wait is bounded, and a block that gives up raises the status word and winds down like the other staged kernels.
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kEwThreads) : "memory"); }
+__device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned* p)
+{
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+// Producer: the full chunks of one group, continuing the ring at stage index i.  False if a wait gave up.
+__device__ __forceinline__ bool staged_produce_group(const StagedWalk& sw, uint8_t* ring, uint64_t* full, uint64_t* empty, const void* t0,
+                                                     const void* t1, const void* t2, const uint8_t* mask, long long base_vec, int& i,
+                                                     unsigned spin_limit, uint32_t* abort_flag, unsigned* status)
+{
+    const uint32_t tbytes = (uint32_t)sw.chunk_vecs * 16u;
+    const uint32_t tx = (uint32_t)sw.nt * tbytes + (mask != nullptr ? (uint32_t)sw.chunk_vecs : 0u);
+    for (long long k = blockIdx.x; k < sw.n_full; k += gridDim.x, ++i) {
+        const int s = i % kStStages;
+        if (!mbar_wait_bounded(&empty[s], (((uint32_t)(i / kStStages)) & 1u) ^ 1u, spin_limit, abort_flag)) {
+            atomicOr(status, B2C_DEV_TIMEOUT);
+            return false;
+        }
+        uint8_t* dst = ring + (size_t)s * sw.stage_bytes;
+        const long long v0 = base_vec + k * sw.chunk_vecs;
+        mbar_expect_tx(&full[s], tx);
+        bulk_load(dst, reinterpret_cast<const uint4*>(t0) + v0, tbytes, &full[s]);
+        bulk_load(dst + tbytes, reinterpret_cast<const uint4*>(t1) + v0, tbytes, &full[s]);
+        if (sw.nt > 2) bulk_load(dst + 2 * tbytes, reinterpret_cast<const uint4*>(t2) + v0, tbytes, &full[s]);
+        if (mask != nullptr) bulk_load(dst + sw.nt * tbytes, mask + v0, (uint32_t)sw.chunk_vecs, &full[s]);
+    }
+    return true;
+}
+
+__global__ void __launch_bounds__(kStThreads, 2) bn_bwd_grouped_kernel(const void* __restrict__ da1, const void* __restrict__ da2,
+                                                                       const void* __restrict__ y, long long m, int c, int n_groups, int ahead,
+                                                                       const float* __restrict__ gamma, const float* __restrict__ mean_all,
+                                                                       const float* __restrict__ invstd_all, int relu, double* sums_all,
+                                                                       unsigned* arrivals, void* __restrict__ dy, void* __restrict__ dres,
+                                                                       float* dgamma, float* dbeta, int acc, const uint8_t* __restrict__ relu_mask,
+                                                                       unsigned spin_limit, unsigned* status)
+{
+    pdl_wait();   // first global access comes after the previous kernel of the stream
+    pdl_launch_dependents();
+    extern __shared__ uint8_t st_raw[];
+    __shared__ uint64_t full[kStStages], empty[kStStages];
+    __shared__ uint32_t abort_flag;
+    uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(st_raw) + 127u) & ~uintptr_t(127));
+    const StagedWalk sw(c, m, da2 != nullptr ? 3 : 2, relu != 0);
+    float* s_acc = reinterpret_cast<float*>(ring + (size_t)kStStages * sw.stage_bytes);
+    for (int i = threadIdx.x; i < 2 * c; i += kStThreads) s_acc[i] = 0.f;
+    staged_init(full, empty, &abort_flag);
+    __syncthreads();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint8_t* mask = relu ? relu_mask : nullptr;
+    const long long group_vecs = m * sw.groups;
+    const int n_steps = n_groups + ahead;   // step t: R(t) if t < n_groups, then A(t - ahead) if t >= ahead
+    int i = 0;                              // ring stage index, advanced identically by the producer and the consumers
+    if (warp == kEwThreads / 32) {
+        if (lane == 0) {
+            bool ok = true;
+            for (int t = 0; ok && t < n_steps; ++t) {
+                if (t < n_groups) ok = staged_produce_group(sw, ring, full, empty, da1, y, da2, mask, t * group_vecs, i, spin_limit, &abort_flag, status);
+                if (ok && t >= ahead)
+                    ok = staged_produce_group(sw, ring, full, empty, da1, y, da2, mask, (t - ahead) * group_vecs, i, spin_limit, &abort_flag, status);
+            }
+        }
+    } else {
+        const int g = threadIdx.x % sw.groups;
+        const bool act = threadIdx.x < sw.active;
+        const uint32_t tbytes = (uint32_t)sw.chunk_vecs * 16u;
+        const bool two = sw.nt > 2;
+        const bool ragged = (long long)sw.n_full * sw.chunk_rows < m && (sw.n_full % gridDim.x) == blockIdx.x;   // this block takes the group's tail
+        const double inv_m = 1.0 / (double)m;
+        // Every consumer warp runs the same sequence of consumer_sync() calls whether or not a wait has given up: after
+        // a failure (the abort flag is set before the failing thread reaches the next barrier) the warps only skip work.
+        bool ok = true;
+        for (int t = 0; t < n_steps; ++t) {
+            if (t < n_groups) {
+                // ---------------------------------------------------------------- R(t): S1 = sum dz, S2 = sum dz*y
+                if (ok) {
+                    const long long base = t * group_vecs;
+                    float sb[8], sg[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) sb[j] = sg[j] = 0.f;
+                    auto accumulate = [&](const uint4& v1, const uint4& vy, const uint4& v2, unsigned mk) {
+                        float d[8], d2[8], fy[8];
+                        unpack8(v1, d);
+                        if (two) unpack8(v2, d2);
+                        unpack8(vy, fy);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            float dz = d[j];
+                            if (two) dz += d2[j];
+                            if (!((mk >> j) & 1u)) dz = 0.f;
+                            sb[j] += dz;
+                            sg[j] = fmaf(dz, fy[j], sg[j]);
+                        }
+                    };
+                    for (long long k = blockIdx.x; k < sw.n_full; k += gridDim.x, ++i) {
+                        ok = staged_wait(full, i, lane, spin_limit, &abort_flag, status);
+                        if (!ok) break;
+                        if (act) {
+                            const uint8_t* st = ring + (size_t)(i % kStStages) * sw.stage_bytes;
+#pragma unroll
+                            for (int u = 0; u < 2; ++u) {
+                                const int v = u * sw.active + threadIdx.x;
+                                const uint4 v1 = reinterpret_cast<const uint4*>(st)[v];
+                                const uint4 vy = reinterpret_cast<const uint4*>(st + tbytes)[v];
+                                uint4 v2 = make_uint4(0u, 0u, 0u, 0u);
+                                if (two) v2 = reinterpret_cast<const uint4*>(st + 2 * tbytes)[v];
+                                const unsigned mk = mask != nullptr ? (unsigned)st[sw.nt * tbytes + v] : 0xffu;
+                                accumulate(v1, vy, v2, mk);
+                            }
+                        }
+                        staged_release(empty, i, lane);
+                    }
+                    if (ok && act && ragged) {
+                        for (long long r = sw.n_full * sw.chunk_rows + threadIdx.x / sw.groups; r < m; r += sw.rpi) {
+                            const long long vi = base + r * sw.groups + g;
+                            const uint4 v1 = ld16(da1, vi), vy = ld16(y, vi);
+                            const uint4 v2 = two ? ld16(da2, vi) : make_uint4(0u, 0u, 0u, 0u);
+                            const unsigned mk = mask != nullptr ? (unsigned)__ldg(mask + vi) : 0xffu;
+                            accumulate(v1, vy, v2, mk);
+                        }
+                    }
+                    if (ok && act) {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            atomicAdd(&s_acc[g * 8 + j], sb[j]);
+                            atomicAdd(&s_acc[c + g * 8 + j], sg[j]);
+                        }
+                    }
+                }
+                consumer_sync();
+                if (*(volatile uint32_t*)&abort_flag) ok = false;
+                if (ok) {
+                    double* out = sums_all + (size_t)t * 2 * c;
+                    for (int j = threadIdx.x; j < 2 * c; j += kEwThreads) {
+                        atomicAdd(out + j, (double)s_acc[j]);
+                        s_acc[j] = 0.f;
+                    }
+                    __threadfence();   // this block's sums are visible device-wide before its arrival is
+                }
+                consumer_sync();
+                if (ok && threadIdx.x == 0) {
+                    __threadfence();
+                    atomicAdd(arrivals + t, 1u);
+                }
+            }
+            if (t >= ahead) {
+                // ---------------------------------------------------------------- A(ga): dy (and dres), after every block has arrived at group ga
+                const int ga = t - ahead;
+                if (ok && threadIdx.x == 0) {
+                    bool seen = false;
+                    for (unsigned poll = 0; poll < spin_limit; ++poll) {
+                        if (ld_acquire_gpu(arrivals + ga) >= gridDim.x) { seen = true; break; }
+                        if (*(volatile uint32_t*)&abort_flag) break;
+                        __nanosleep(100);
+                    }
+                    if (!seen) {
+                        *(volatile uint32_t*)&abort_flag = 1u;
+                        atomicOr(status, B2C_DEV_TIMEOUT);
+                    }
+                }
+                consumer_sync();
+                if (*(volatile uint32_t*)&abort_flag) ok = false;
+                if (ok) {
+                    const long long base = ga * group_vecs;
+                    const double* sums = sums_all + (size_t)ga * 2 * c;
+                    const float* mean = mean_all + (size_t)ga * c;
+                    const float* invstd = invstd_all + (size_t)ga * c;
+                    if (blockIdx.x == 0) {
+                        for (int ch = threadIdx.x; ch < c; ch += kEwThreads) {
+                            const double s1 = __ldcg(sums + ch), s2 = __ldcg(sums + c + ch);
+                            const float db = (float)s1, dg = (float)((double)invstd[ch] * (s2 - (double)mean[ch] * s1));
+                            if (n_groups == 1) {
+                                dbeta[ch] = acc ? dbeta[ch] + db : db;
+                                dgamma[ch] = acc ? dgamma[ch] + dg : dg;
+                            } else {   // several groups add into the same gradient (always accumulating)
+                                atomicAdd(dbeta + ch, db);
+                                atomicAdd(dgamma + ch, dg);
+                            }
+                        }
+                    }
+                    float mu[8], k0[8], kb[8], kg[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const int ch = g * 8 + j;
+                        const double s1 = __ldcg(sums + ch), s2 = __ldcg(sums + c + ch);
+                        const double is = (double)invstd[ch], dgam = is * (s2 - (double)mean[ch] * s1);
+                        mu[j] = mean[ch];
+                        k0[j] = gamma[ch] * invstd[ch];                        // gamma*invstd
+                        kb[j] = (float)(s1 * inv_m);                           // dbeta/m
+                        kg[j] = (float)(dgam * inv_m * is);                    // (dgamma/m)*invstd, multiplies (y-mean)
+                    }
+                    auto emit = [&](const uint4& v1, const uint4& vy, const uint4& v2, unsigned mk, long long vi) {
+                        float d[8], d2[8], fy[8], o[8];
+                        unpack8(v1, d);
+                        if (two) unpack8(v2, d2);
+                        unpack8(vy, fy);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            float dz = d[j];
+                            if (two) dz += d2[j];
+                            if (!((mk >> j) & 1u)) dz = 0.f;
+                            d[j] = dz;
+                            o[j] = k0[j] * (dz - kb[j] - (fy[j] - mu[j]) * kg[j]);
+                        }
+                        reinterpret_cast<uint4*>(dy)[vi] = pack8(o);
+                        if (dres != nullptr) reinterpret_cast<uint4*>(dres)[vi] = pack8(d);
+                    };
+                    for (long long k = blockIdx.x; k < sw.n_full; k += gridDim.x, ++i) {
+                        ok = staged_wait(full, i, lane, spin_limit, &abort_flag, status);
+                        if (!ok) break;
+                        if (act) {
+                            const uint8_t* st = ring + (size_t)(i % kStStages) * sw.stage_bytes;
+#pragma unroll
+                            for (int u = 0; u < 2; ++u) {
+                                const int v = u * sw.active + threadIdx.x;
+                                const uint4 v1 = reinterpret_cast<const uint4*>(st)[v];
+                                const uint4 vy = reinterpret_cast<const uint4*>(st + tbytes)[v];
+                                uint4 v2 = make_uint4(0u, 0u, 0u, 0u);
+                                if (two) v2 = reinterpret_cast<const uint4*>(st + 2 * tbytes)[v];
+                                const unsigned mk = mask != nullptr ? (unsigned)st[sw.nt * tbytes + v] : 0xffu;
+                                emit(v1, vy, v2, mk, base + k * sw.chunk_vecs + v);
+                            }
+                        }
+                        staged_release(empty, i, lane);
+                    }
+                    if (ok && act && ragged) {
+                        for (long long r = sw.n_full * sw.chunk_rows + threadIdx.x / sw.groups; r < m; r += sw.rpi) {
+                            const long long vi = base + r * sw.groups + g;
+                            const uint4 v1 = ld16(da1, vi), vy = ld16(y, vi);
+                            const uint4 v2 = two ? ld16(da2, vi) : make_uint4(0u, 0u, 0u, 0u);
+                            const unsigned mk = mask != nullptr ? (unsigned)__ldg(mask + vi) : 0xffu;
+                            emit(v1, vy, v2, mk, vi);
+                        }
+                    }
+                }
+            }
+        }
+    }
+    __syncthreads();
+    // After an aborted wait the copies already issued must land before the block may exit.
+    if (abort_flag && warp == kEwThreads / 32 && lane == 0) staged_drain(i, full);   // the producer lane's i = stages it issued
+    __syncthreads();
+}
+
 // ------------------------------------------------------------------------------ pooling, padding
 __global__ void avgpool_fwd_kernel(const void* __restrict__ a, int n, int hw, int c, void* __restrict__ pooled)
 {
@@ -875,12 +1131,60 @@ b2c_status launch_bn_fwd(b2c_ctx* ctx, int G, long long m, int c, const void* y,
 
 b2c_status launch_bn_bwd(b2c_ctx* ctx, int G, long long m, int c, const void* da1, const void* da2, const void* y, const void* a,
                          const float* gamma, const float* save_mean, const float* save_invstd, int relu, void* dy, void* dres, float* dgamma,
-                         float* dbeta, int acc, double* sums, bool sums_zeroed, const void* relu_mask, cudaStream_t stream)
+                         float* dbeta, int acc, double* sums, bool sums_zeroed, const void* relu_mask, unsigned* arrivals, cudaStream_t stream)
 {
     const int rows_per_iter = kEwThreads / (c / 8);
     dim3 grid((unsigned)ew_grid(ctx, G, m, rows_per_iter), (unsigned)G);
     const uint8_t* mask = relu ? reinterpret_cast<const uint8_t*>(relu_mask) : nullptr;
-    if (!sums_zeroed) B2C_CUDA(cudaMemsetAsync(sums, 0, sizeof(double) * 2 * c * G, stream));
+    if (!sums_zeroed) {
+        B2C_CUDA(cudaMemsetAsync(sums, 0, sizeof(double) * 2 * c * G, stream));
+        if (arrivals != nullptr) B2C_CUDA(cudaMemsetAsync(arrivals, 0, sizeof(unsigned) * G, stream));
+    }
+    // Both passes in one cooperative launch, group by group (the apply pass of a group re-reads its tensors from L2).
+    if (arrivals != nullptr && ctx->use_bn_grouped) {
+        const int groups = c / 8, active = rows_per_iter * groups, chunk_vecs = 2 * active;
+        const int nt = da2 != nullptr ? 3 : 2;
+        const size_t stage = (size_t)nt * chunk_vecs * 16 + (relu ? ((chunk_vecs + 127) & ~127) : 0);
+        const size_t smem = kStStages * stage + sizeof(float) * 2 * c + 128;
+        const long long n_full = m / (2 * rows_per_iter);
+        const bool eligible = (!relu || mask != nullptr) && chunk_vecs % 16 == 0 && (m * groups) % 16 == 0 && n_full >= 1 &&
+                              reinterpret_cast<uintptr_t>(mask) % 16 == 0 && smem <= 110 * 1024;
+        if (eligible) {
+            if (!(ctx->smem_optin_done & B2C_OPTIN_BN_GROUPED)) {
+                B2C_CUDA(cudaFuncSetAttribute(bn_bwd_grouped_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024));
+                ctx->smem_optin_done |= B2C_OPTIN_BN_GROUPED;
+            }
+            int per_sm = 0;
+            B2C_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, bn_bwd_grouped_kernel, kStThreads, smem));
+            if (per_sm > 2) per_sm = 2;
+            if (per_sm >= 1) {
+                long long blocks = (long long)per_sm * ctx->sm_count;   // all blocks co-resident: the groups' barriers need every block running
+                if (blocks > n_full) blocks = n_full;
+                // Groups whose reduction pass runs ahead of a group's apply pass: as many as keep the inputs of the waiting
+                // groups (da, y, second gradient, mask) within a part of the L2, at least one.
+                const double group_bytes = (double)m * c * (2.0 * nt + 0.125);
+                int ahead = (int)(40e6 / group_bytes);
+                if (ahead < 1) ahead = 1;
+                if (const char* e = getenv("B2C_BN_AHEAD")) ahead = atoi(e);
+                if (ahead < 1) ahead = 1;
+                if (ahead > G) ahead = G;
+                cudaLaunchConfig_t cfg = {};
+                cfg.gridDim = dim3((unsigned)blocks);
+                cfg.blockDim = dim3(kStThreads);
+                cfg.dynamicSmemBytes = smem;
+                cfg.stream = stream;
+                cudaLaunchAttribute attr[1];
+                attr[0].id = cudaLaunchAttributeCooperative;
+                attr[0].val.cooperative = 1;
+                cfg.attrs = attr;
+                cfg.numAttrs = 1;
+                B2C_CUDA(cudaLaunchKernelEx(&cfg, bn_bwd_grouped_kernel, da1, da2, y, m, c, G, ahead, gamma, save_mean, save_invstd, relu, sums, arrivals, dy,
+                                            dres, dgamma, dbeta, acc, mask, ctx->spin_limit, ctx->d_status));
+                B2C_CUDA(cudaGetLastError());
+                return B2C_OK;
+            }
+        }
+    }
     // The staged kernels need the ReLU mask (not the activation), chunk offsets that keep the mask copies 16-byte
     // aligned, and at least one full chunk per block to be worth their set-up.
     const int groups = c / 8, active = rows_per_iter * groups, chunk_vecs = 2 * active;
@@ -945,7 +1249,37 @@ b2c_status b2c_bn_relu_bwd(b2c_ctx* ctx, int n, int h, int w, int c, const void*
         (dres && !b2c_aligned16(dres)) || (reinterpret_cast<uintptr_t>(ws) & 7u))
         return B2C_ERR_MISALIGNED;
     return launch_bn_bwd(ctx, 1, (long long)n * h * w, c, da1, da2, y, a, gamma, save_mean, save_invstd, relu, dy, dres, dgamma, dbeta, acc,
-                         reinterpret_cast<double*>(ws), false, relu_mask, stream);
+                         reinterpret_cast<double*>(ws), false, relu_mask, nullptr, stream);
+}
+
+size_t b2c_bn_relu_bwd_groups_workspace_bytes(int c, int groups)
+{
+    if (c <= 0 || groups <= 0) return 0;
+    return sizeof(double) * 2 * (size_t)c * groups + ((sizeof(unsigned) * (size_t)groups + 7) & ~size_t(7));   // sums, then arrival counters
+}
+
+b2c_status b2c_bn_relu_bwd_groups(b2c_ctx* ctx, int groups, long long rows_per_group, int c, const void* da1, const void* da2, const void* y,
+                                  const float* gamma, const float* save_mean, const float* save_invstd, int relu, void* dy, void* dres,
+                                  float* dgamma, float* dbeta, int acc, const void* relu_mask, void* ws, size_t ws_bytes, void* stream_)
+{
+    cudaStream_t stream = (cudaStream_t)stream_;
+    if (!ctx || !da1 || !y || !gamma || !save_mean || !save_invstd || !dy || !dgamma || !dbeta || !ws) return B2C_ERR_INVALID_ARG;
+    if (relu && !relu_mask) return B2C_ERR_INVALID_ARG;
+    if (groups < 1 || groups > 4096 || rows_per_group < 1 || c < 8 || c % 8 || c > 2048) return B2C_ERR_UNSUPPORTED_SHAPE;
+    if (ws_bytes < b2c_bn_relu_bwd_groups_workspace_bytes(c, groups)) return B2C_ERR_WORKSPACE_TOO_SMALL;
+    if (!b2c_aligned16(da1) || (da2 && !b2c_aligned16(da2)) || !b2c_aligned16(y) || !b2c_aligned16(dy) || (dres && !b2c_aligned16(dres)) ||
+        (relu_mask && !b2c_aligned16(relu_mask)) || (reinterpret_cast<uintptr_t>(ws) & 7u))
+        return B2C_ERR_MISALIGNED;
+    if ((rows_per_group * (c / 8)) % 16) return B2C_ERR_UNSUPPORTED_SHAPE;   // a group's slice of the bit mask must start on a 16-byte boundary
+    double* sums = reinterpret_cast<double*>(ws);
+    unsigned* arrivals = reinterpret_cast<unsigned*>(sums + (size_t)2 * c * groups);
+    B2C_CUDA(cudaMemsetAsync(ws, 0, b2c_bn_relu_bwd_groups_workspace_bytes(c, groups), stream));
+    if (!acc && groups > 1) {   // several groups always add into the gradients: start them at zero
+        B2C_CUDA(cudaMemsetAsync(dgamma, 0, sizeof(float) * c, stream));
+        B2C_CUDA(cudaMemsetAsync(dbeta, 0, sizeof(float) * c, stream));
+    }
+    return launch_bn_bwd(ctx, groups, rows_per_group, c, da1, da2, y, nullptr, gamma, save_mean, save_invstd, relu, dy, dres, dgamma, dbeta,
+                         groups > 1 ? 1 : acc, sums, true, relu_mask, arrivals, stream);
 }
 
 b2c_status b2c_avgpool_fwd(b2c_ctx* ctx, int n, int hw, int c, const void* a, void* pooled, void* stream_)
@@ -1097,7 +1431,7 @@ b2c_status b2c_bn_relu_bwd_static(b2c_ctx* ctx, int n, int h, int w, int c, cons
     }
     // the array keeps the previous call's sums: the launcher clears the part this call uses
     return launch_bn_bwd(ctx, 1, (long long)n * h * w, c, da1, da2, y, a, gamma, save_mean, save_invstd, relu, dy, dres, dgamma, dbeta, acc,
-                         g_bn_bwd_static_ptr[current], false, nullptr, stream);
+                         g_bn_bwd_static_ptr[current], false, nullptr, nullptr, stream);
 }
 
 }  // extern "C"

@@ -214,6 +214,54 @@ def test_bn_relu_fwd_bwd(ctx, shape, relu, use_res):
     assert ctx.device_status() == 0
 
 
+# (groups, rows per group, channels): ragged tails, more groups than fit the look-ahead, one chunk per block at most,
+# idle threads at 160 channels, and a 64-channel case whose groups are large enough to be taken one at a time
+BN_GROUP_SHAPES = [(4, 2048, 64), (3, 1000, 160), (8, 96, 512), (1, 4096, 128), (5, 16 * 1024, 64), (2, 640, 8)]
+
+
+@pytest.mark.parametrize("shape", BN_GROUP_SHAPES, ids=lambda s: "x".join(map(str, s)))
+@pytest.mark.parametrize("relu,use_res", [(True, False), (True, True), (False, False)])
+def test_bn_relu_bwd_groups(ctx, shape, relu, use_res):
+    """Several statistics groups (micro-batches) back to back, each differentiated with its own statistics, both passes
+    in one cooperative launch: every group against the oracle, the parameter gradients against the sum over groups."""
+    G, M, C = shape
+    r = wl.rng_for(14, f"bng{shape}{relu}{use_res}")
+    y = wl.to_bf16_grid(r.standard_normal((G, M, C)) * (0.5 + r.random(C)) + 1.5 * r.standard_normal((G, 1, C)))
+    da1 = wl.to_bf16_grid(r.standard_normal((G, M, C)))
+    da2 = wl.to_bf16_grid(r.standard_normal((G, M, C))) if use_res else None
+    gamma = (1.0 + 0.3 * r.standard_normal(C)).astype(np.float32)
+    beta = (0.2 * r.standard_normal(C)).astype(np.float32)
+    means, invstds, a_ref, dy_ref, dres_ref = [], [], [], [], []
+    dg_ref, db_ref = np.zeros(C), np.zeros(C)
+    for g in range(G):
+        mean, _, invstd = oracle.bn_stats(y[g], 1e-5)
+        mean, invstd = oracle.round_f32(mean), oracle.round_f32(invstd)
+        a = oracle.round_bf16(oracle.bn_relu_apply(y[g], mean, invstd, gamma, beta, None, relu))
+        q = oracle.bn_relu_bwd(da1[g], None if da2 is None else da2[g], y[g], a, gamma, mean, invstd, relu, use_res)
+        means.append(mean); invstds.append(invstd); a_ref.append(a); dy_ref.append(q[0]); dres_ref.append(q[1])
+        dg_ref += q[2]; db_ref += q[3]
+    mask = torch.from_numpy(np.packbits(np.stack(a_ref).reshape(-1) > 0, bitorder="little")).cuda() if relu else None
+    dyo = torch.full((G, M, C), float("nan"), dtype=torch.bfloat16, device="cuda")
+    dres = torch.full((G, M, C), float("nan"), dtype=torch.bfloat16, device="cuda") if use_res else None
+    dg, db = torch.full((C,), 1.0, device="cuda"), torch.full((C,), -2.0, device="cuda")
+    ws = torch.full((ctx.bn_relu_bwd_groups_workspace_bytes(C, G),), 0x5A, dtype=torch.uint8, device="cuda")   # stale contents must not matter
+    args = (G, M, C, dev_bf16(da1), None if da2 is None else dev_bf16(da2), dev_bf16(y), dev_f32(gamma), dev_f32(np.stack(means)),
+            dev_f32(np.stack(invstds)), relu, dyo, dres, dg, db)
+    ctx.bn_relu_bwd_groups(*args, True, mask, ws)
+    assert ctx.device_status() == 0
+    assert_close(dyo, np.stack(dy_ref), "dy")
+    if use_res:
+        assert_close(dres, oracle.round_bf16(np.stack(dres_ref)), "dres", 1e-6, 1e-6)
+    assert_close(dg, dg_ref + 1.0, "dgamma (accumulated)", 2e-3, 2e-3)
+    assert_close(db, db_ref - 2.0, "dbeta (accumulated)", 2e-3, 2e-3)
+    # overwrite mode, and a second call on the same workspace
+    ctx.bn_relu_bwd_groups(*args, False, mask, ws)
+    assert ctx.device_status() == 0
+    assert_close(dg, dg_ref, "dgamma", 2e-3, 2e-3)
+    assert_close(db, db_ref, "dbeta", 2e-3, 2e-3)
+    assert_close(dyo, np.stack(dy_ref), "dy (second call)")
+
+
 def test_bn_large_mean_small_spread(ctx):
     # |mean| ~ 50x the spread: E[y^2] - E[y]^2 must not lose the variance
     N, H, W, C = 8, 16, 16, 16

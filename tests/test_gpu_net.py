@@ -392,3 +392,41 @@ def test_wrn28_10_small_batch_layerwise(ctx):
     assert ctx.device_status() == 0
     check_step(net, spec, images, labels, 8).assert_ok()
     net.close()
+
+
+def test_sharded_update_pieces_match_fused_update(ctx):
+    """The device side of the sharded data-parallel update: gradient-ready events per bucket (waited for on a second
+    stream while the backward pass runs), the update applied slice by slice as three replicas would own them, and the
+    refresh of the data-gradient weight layout, against the fused whole-array update: bit-identical arrays."""
+    from paper_2503_23186_b200 import binding, data_parallel as dp
+    spec = wl.tiny_net_spec(classes=10, hw=16, c=3, width=64, width2=128)
+    params = wl.perturb_bn_params(wl.init_params(spec, 21), 21)
+    images, labels = wl.image_batch(21, 16, hw=16, c=3, classes=10)
+    d_img, d_lab = dev_bf16(images), torch.from_numpy(labels).cuda()
+    fused, pieces = binding.Net(ctx, spec, 8), binding.Net(ctx, spec, 8)
+    for n in (fused, pieces):
+        n.load_params(params)
+    buckets = dp.bucket_plan(pieces.param_count, pieces.weight_layer_ranges(), 3)
+    assert sorted((b, e) for b, e, _ in buckets)[0][0] == 0 and max(e for _, e, _ in buckets) == pieces.param_count
+    pieces.set_buckets(buckets)
+    side = torch.cuda.Stream()
+    for step in range(2):
+        fused.train_step(d_img, d_lab, 2, LR, MU, WD, update=False)
+        # same inputs, same kernels: the gradient sums are compared within the run-to-run budget, then made identical
+        pieces.train_step(d_img, d_lab, 2, LR, MU, WD, update=False)
+        for k, (begin, end, _) in enumerate(buckets):
+            with torch.cuda.stream(side):
+                pieces.bucket_wait(k, side)
+                assert_close(pieces.g[begin:end], host(fused.g[begin:end]), f"gradient sums of bucket {k}", 1e-2, 3e-2)
+                pieces.g[begin:end].copy_(fused.g[begin:end])
+                for rank in range(3):
+                    b, e = dp.slice_of(begin, end, rank, 3)
+                    if e > b:
+                        pieces.apply_update_range(b, e, 2, LR, MU, WD)
+        torch.cuda.current_stream().wait_stream(side)
+        pieces.refresh_derived_weights()
+        fused.apply_update(2, LR, MU, WD)
+        assert ctx.device_status() == 0
+        for name in ("w", "v", "g", "w_bf16", "w_dgrad"):
+            assert torch.equal(getattr(pieces, name), getattr(fused, name)), (step, name)
+    fused.close(); pieces.close()
