@@ -54,7 +54,7 @@ b2c_status b2c_create(b2c_ctx** out, int device)
     }
     {
         const char* env = std::getenv("B2C_BN_GROUPED");
-        ctx->use_bn_grouped = env ? (env[0] != '0') : 1;
+        ctx->use_bn_grouped = env ? (env[0] != '0') : 0;
     }
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
@@ -736,7 +736,7 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
                                           d.res >= 0 ? grad(d.res, L.res_slot, img0) : nullptr, net->g + L.gamma_off, net->g + L.beta_off, 1,
                                           reinterpret_cast<double*>(net->ws + L.bwd_ws_off) + (size_t)g0 * 2 * in.c, /*sums_zeroed=*/in.stats_off >= 0,
                                           L.mask_off >= 0 ? net->ws + L.mask_off + (long long)img0 * in.h * in.w * in.c / 8 : nullptr,
-                                          reinterpret_cast<unsigned*>(net->ws + L.arrive_off) + g0, stream));
+                                          ctx->use_bn_grouped ? reinterpret_cast<unsigned*>(net->ws + L.arrive_off) + g0 : nullptr, stream));
                     break;
                 }
                 case B2C_LAYER_CONV: {

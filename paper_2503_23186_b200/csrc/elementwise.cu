@@ -1141,7 +1141,7 @@ b2c_status launch_bn_bwd(b2c_ctx* ctx, int G, long long m, int c, const void* da
         if (arrivals != nullptr) B2C_CUDA(cudaMemsetAsync(arrivals, 0, sizeof(unsigned) * G, stream));
     }
     // Both passes in one cooperative launch, group by group (the apply pass of a group re-reads its tensors from L2).
-    if (arrivals != nullptr && ctx->use_bn_grouped) {
+    if (arrivals != nullptr) {
         const int groups = c / 8, active = rows_per_iter * groups, chunk_vecs = 2 * active;
         const int nt = da2 != nullptr ? 3 : 2;
         const size_t stage = (size_t)nt * chunk_vecs * 16 + (relu ? ((chunk_vecs + 127) & ~127) : 0);
