@@ -255,11 +255,15 @@ def run_b2c(args, spec, name, micro_batch, n_micro):
             dist.barrier()
         torch.cuda.synchronize()
         ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        host_s = 0.0
         for a, b in ev:
             flush.zero_()            # untimed: evicts the previous step's lines from L2
             a.record()
+            t_h = time.perf_counter()
             step(d_img, d_lab)
+            host_s += time.perf_counter() - t_h
             b.record()
+        timed_region.host_ms = 1e3 * host_s / args.steps   # host time to enqueue one step (no synchronisation inside)
         torch.cuda.synchronize()
         if world > 1:
             dist.barrier()
@@ -273,6 +277,7 @@ def run_b2c(args, spec, name, micro_batch, n_micro):
     # the headline: K steps as a user runs them
     sampler.mark()
     total_ms = timed_region()
+    host_enqueue_ms = timed_region.host_ms
     clocks = sampler.stop() if rank == 0 else None
     # the same K steps again with CUDA events around every launch site (two event records per launch cost about 7 % of
     # the step, so they stay out of the headline): per-kernel-family times for the roofline figures
@@ -358,7 +363,7 @@ def run_b2c(args, spec, name, micro_batch, n_micro):
         "config": {"workload": name, "global_batch": world * batch, "micro_batch": micro_batch, "n_micro": n_micro, "micro_batches_per_pass": net.n_concurrent, "params": n_params,
                    "l2": "per-step working set (~0.5 GB of activations) exceeds the 126 MB L2; a 256 MB buffer is rewritten between timed steps (untimed)",
                    "timing": "CUDA events per step on the launching stream, summed, max over ranks; kernel-family times from a second region of the same steps with events around every launch site (b2c_net_profile_enable)",
-                   "profiled_ms_per_step": profiled_ms / args.steps},
+                   "profiled_ms_per_step": profiled_ms / args.steps, "host_enqueue_ms_per_step": host_enqueue_ms},
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(sum(fam_launches.values())),
         "roofline": roofline, "kernels": kernels, "loss": loss,
         "cpu_baseline": cpu_baseline(spec, micro_batch, n_micro) if world == 1 and not args.no_cpu_baseline else None,

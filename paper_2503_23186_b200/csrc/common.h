@@ -5,6 +5,10 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <string>
+#include <unordered_map>
+#include <vector>
+
 #include "../../include/b2c.h"
 
 // Bits of the sticky device status word.
@@ -28,6 +32,10 @@ struct b2c_ctx {
     int use_issue_split;                 // forward / data-gradient tiles wider than 128 channels: two MMA-issuing threads share every unit
     int use_pdl;                         // kernels are launched with programmatic stream serialization (their set-up overlaps the previous kernel's tail)
     int use_bn_grouped;                  // BatchNorm backward of the training step: both passes in one cooperative launch, group by group
+    // Launch plans (kernel parameter blocks with their tensor maps, grid and shared-memory size) of the convolution
+    // kernels, keyed by the bytes of the problem description: pointers and shapes of a bound network repeat every
+    // step, so a plan is built once and its launches cost one parameter copy.
+    std::unordered_map<std::string, std::vector<unsigned char>> plan_cache;
     unsigned smem_optin_done;            // kernels whose dynamic shared-memory opt-in was set on this context's device (B2C_OPTIN_* bits)
 };
 #define B2C_OPTIN_KMAJOR 1u

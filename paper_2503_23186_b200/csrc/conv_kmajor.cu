@@ -811,10 +811,17 @@ void forward_taps(TapList& tl, int R, int stride, int pad)
         }
 }
 
-b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_t stream)
-{
+// A launch plan: the kernel's parameter block (tensor maps included), launch shape and shared-memory size.
+struct KMajorPlan {
     ConvKParams p;
-    memset(&p, 0, sizeof(p));
+    int grid;
+    size_t smem_bytes;
+};
+
+static b2c_status build_kmajor_plan(b2c_ctx* ctx, const KMajorProblem& pb, KMajorPlan& plan)
+{
+    ConvKParams& p = plan.p;
+    memset(&plan, 0, sizeof(plan));
     const int R = pb.r;
     if (!(R == 1 || R == 3) || !(pb.stride == 1 || pb.stride == 2) || pb.pad != (R - 1) / 2) return B2C_ERR_UNSUPPORTED_SHAPE;
     if (pb.n < 1 || pb.ic < 16 || pb.ic % 16 || pb.oc < 16 || pb.oc % 16) return B2C_ERR_UNSUPPORTED_SHAPE;
@@ -1008,6 +1015,41 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
     p.grp_shift = log2_exact(p.stats_group_images);
     p.cb_shift = log2_exact(p.c_blocks);
     if (p.stats && p.stats_group_images > 0 && (p.stats_group_images % p.bn) != 0) return B2C_ERR_UNSUPPORTED_SHAPE;  // a tile must not straddle groups
+    plan.grid = grid;
+    plan.smem_bytes = smem_bytes;
+    return B2C_OK;
+}
+
+// Appends the bytes of a value to a cache key.
+template <typename T>
+static inline void key_add(std::string& key, const T& v)
+{
+    key.append(reinterpret_cast<const char*>(&v), sizeof(T));
+}
+
+b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_t stream)
+{
+    // plans are keyed by everything the planner reads: the problem and the context's switches
+    std::string key("K");
+    key_add(key, pb.n); key_add(key, pb.ih); key_add(key, pb.iw); key_add(key, pb.ic); key_add(key, pb.oh); key_add(key, pb.ow); key_add(key, pb.oc);
+    key_add(key, pb.r); key_add(key, pb.stride); key_add(key, pb.pad); key_add(key, pb.dgrad); key_add(key, pb.in); key_add(key, pb.wt);
+    key_add(key, pb.out); key_add(key, pb.out_f32); key_add(key, pb.bias); key_add(key, pb.stats); key_add(key, pb.stats_group_images);
+    key_add(key, ctx->use_pairs); key_add(key, ctx->use_full_halo); key_add(key, ctx->use_issue_split);
+    auto it = ctx->plan_cache.find(key);
+    if (it == ctx->plan_cache.end()) {
+        KMajorPlan fresh;
+        b2c_status st = build_kmajor_plan(ctx, pb, fresh);
+        if (st != B2C_OK) return st;
+        if (ctx->plan_cache.size() >= 8192) ctx->plan_cache.clear();   // callers that pass new buffers every call: keep the table bounded
+        std::vector<unsigned char> bytes(sizeof(KMajorPlan));
+        memcpy(bytes.data(), &fresh, sizeof(KMajorPlan));
+        it = ctx->plan_cache.emplace(std::move(key), std::move(bytes)).first;
+    }
+    KMajorPlan plan;   // a copy: the 64-byte alignment of the tensor maps is the parameter block's, not the table's
+    memcpy(&plan, it->second.data(), sizeof(KMajorPlan));
+    ConvKParams& p = plan.p;
+    const int grid = plan.grid;
+    const size_t smem_bytes = plan.smem_bytes;
     p.status = ctx->d_status;
     p.spin_limit = ctx->spin_limit;
     p.stall = ctx->stall_counters;

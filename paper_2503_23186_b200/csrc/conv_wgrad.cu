@@ -368,10 +368,16 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
     }
 }
 
-b2c_status launch_conv_wgrad(b2c_ctx* ctx, const WgradProblem& pb, cudaStream_t stream)
-{
+struct WgradPlan {
     WgradParams p;
-    memset(&p, 0, sizeof(p));
+    int grid;
+    size_t smem_bytes;
+};
+
+static b2c_status build_wgrad_plan(b2c_ctx* ctx, const WgradProblem& pb, WgradPlan& plan)
+{
+    WgradParams& p = plan.p;
+    memset(&plan, 0, sizeof(plan));
     const int R = pb.r;
     if (!(R == 1 || R == 3) || !(pb.stride == 1 || pb.stride == 2) || pb.pad != (R - 1) / 2) return B2C_ERR_UNSUPPORTED_SHAPE;
     if (pb.n < 1 || pb.c < 16 || pb.c % 16 || pb.k < 16 || pb.k % 16) return B2C_ERR_UNSUPPORTED_SHAPE;
@@ -513,6 +519,36 @@ b2c_status launch_conv_wgrad(b2c_ctx* ctx, const WgradProblem& pb, cudaStream_t 
     p.c_total = pb.c;
     p.rs_total = R * R;
     p.dw = pb.dw;
+    plan.smem_bytes = (size_t)p.stages * p.stage_bytes + 1024;
+    plan.grid = base * n_splits;
+    return B2C_OK;
+}
+
+template <typename T>
+static inline void key_add(std::string& key, const T& v)
+{
+    key.append(reinterpret_cast<const char*>(&v), sizeof(T));
+}
+
+b2c_status launch_conv_wgrad(b2c_ctx* ctx, const WgradProblem& pb, cudaStream_t stream)
+{
+    std::string key("W");
+    key_add(key, pb.n); key_add(key, pb.h); key_add(key, pb.w); key_add(key, pb.c); key_add(key, pb.p); key_add(key, pb.q); key_add(key, pb.k);
+    key_add(key, pb.r); key_add(key, pb.stride); key_add(key, pb.pad); key_add(key, pb.dy); key_add(key, pb.x); key_add(key, pb.dw);
+    key_add(key, ctx->use_wgrad_frame);
+    auto it = ctx->plan_cache.find(key);
+    if (it == ctx->plan_cache.end()) {
+        WgradPlan fresh;
+        b2c_status st = build_wgrad_plan(ctx, pb, fresh);
+        if (st != B2C_OK) return st;
+        if (ctx->plan_cache.size() >= 8192) ctx->plan_cache.clear();
+        std::vector<unsigned char> bytes(sizeof(WgradPlan));
+        memcpy(bytes.data(), &fresh, sizeof(WgradPlan));
+        it = ctx->plan_cache.emplace(std::move(key), std::move(bytes)).first;
+    }
+    WgradPlan plan;
+    memcpy(&plan, it->second.data(), sizeof(WgradPlan));
+    WgradParams& p = plan.p;
     p.status = ctx->d_status;
     p.spin_limit = ctx->spin_limit;
     p.stall = ctx->stall_counters;
@@ -521,8 +557,8 @@ b2c_status launch_conv_wgrad(b2c_ctx* ctx, const WgradProblem& pb, cudaStream_t 
         B2C_CUDA(cudaFuncSetAttribute(conv_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 212 * 1024));
         ctx->smem_optin_done |= B2C_OPTIN_WGRAD;
     }
-    const size_t smem_bytes = (size_t)p.stages * p.stage_bytes + 1024;
-    dim3 grid((unsigned)(base * n_splits));
+    const size_t smem_bytes = plan.smem_bytes;
+    dim3 grid((unsigned)plan.grid);
     B2C_CUDA(b2c_launch(ctx, conv_wgrad_kernel, grid, dim3(kWgThreads), smem_bytes, stream, 1u, p));
     B2C_CUDA(cudaGetLastError());
     return B2C_OK;
