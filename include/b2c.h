@@ -9,7 +9,7 @@
  *   - All tensor pointers are DEVICE pointers owned by the caller, 16-byte aligned, and must
  *     stay valid until the stream has passed the call.  Descriptor structs are HOST memory and
  *     are read before the call returns.  The library allocates no device memory in any call
- *     except b2c_create (one status word) and b2c_net_create (a few KB of tables).
+ *     except b2c_create (one status word); b2c_net_create builds host-side tables only.
  *   - `stream` is a cudaStream_t passed as void*.  Calls only enqueue work and return.
  *   - Layouts: activations NHWC bf16; convolution weights KRSC bf16 (K output channels, R x S
  *     taps, C input channels); accumulation is always fp32; fp32 -> bf16 is round-to-nearest-even.
@@ -21,10 +21,14 @@
  *   - Environment switches, read by b2c_create (kernel variants) and b2c_net_create (step plan); all default to the
  *     fastest measured setting and exist for A/B measurements:
  *       B2C_PDL=0            launch kernels without programmatic stream serialization
- *       B2C_CTA_PAIRS=0|1|2  CTA pairs in the forward / data-gradient kernel: never | 128-channel 3x3 layers (default) | wherever possible
+ *       B2C_CTA_PAIRS=0|1|2|3  CTA pairs in the forward / data-gradient kernel: never | 3x3 stride-1 layers with tiles of 128 or
+ *                            256 channels (default) | wherever possible | 128-channel tiles only
  *       B2C_FULL_HALO=0      one load per tap group instead of one framed tile per channel block (3x3 stride-1 layers)
  *       B2C_ISSUE_SPLIT=0    forward / data gradient, tiles wider than 128 channels: one MMA-issuing thread instead of two sharing every unit
  *       B2C_WGRAD_FRAME=0    weight gradient: one x box per horizontal shift instead of one framed box per channel block
+ *       B2C_WGRAD_ISSUERS=1  weight gradient: one MMA-issuing thread instead of two on alternate chunks of one accumulator
+ *       B2C_BN_GROUPED=1     b2c_train_step runs the BatchNorm backward as one cooperative launch per layer, group by group
+ *                            (b2c_bn_relu_bwd_groups); off by default: measured slower inside the step
  *       B2C_FUSE_WIDE=0|1    BatchNorm statistics of tiles wider than 64 channels: never | always in the convolution epilogue
  *                            (default: where the unit's MMAs take longer than the epilogue's column sums)
  *       B2C_FUSE_BN_STATS=0  BatchNorm statistics by a separate pass instead of the convolution epilogue (b2c_train_step)

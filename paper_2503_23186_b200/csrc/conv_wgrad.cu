@@ -479,7 +479,7 @@ static b2c_status build_wgrad_plan(b2c_ctx* ctx, const WgradProblem& pb, WgradPl
     // Two issuing threads need an even ring.  Measured: four stages with two threads beat five with one (128 -> 128:
     // 67 us against 79 us), three stages with one thread beat two with two (512 -> 512 at 4x4: 79 us against 106 us).
     if (stages >= 4) stages &= ~1;
-    p.issuers = (stages % 2 == 0) ? kWgIssuers : 1;
+    p.issuers = (stages % 2 == 0 && ctx->use_wgrad_two_issuers) ? kWgIssuers : 1;
     p.stages = stages;
     p.bw = pb.q < p.pb ? pb.q : p.pb;
     p.bh = (p.pb / p.bw) < pb.p ? (p.pb / p.bw) : pb.p;
@@ -535,7 +535,7 @@ b2c_status launch_conv_wgrad(b2c_ctx* ctx, const WgradProblem& pb, cudaStream_t 
     std::string key("W");
     key_add(key, pb.n); key_add(key, pb.h); key_add(key, pb.w); key_add(key, pb.c); key_add(key, pb.p); key_add(key, pb.q); key_add(key, pb.k);
     key_add(key, pb.r); key_add(key, pb.stride); key_add(key, pb.pad); key_add(key, pb.dy); key_add(key, pb.x); key_add(key, pb.dw);
-    key_add(key, ctx->use_wgrad_frame);
+    key_add(key, ctx->use_wgrad_frame); key_add(key, ctx->use_wgrad_two_issuers);
     auto it = ctx->plan_cache.find(key);
     if (it == ctx->plan_cache.end()) {
         WgradPlan fresh;

@@ -1,4 +1,4 @@
-"""The allocation-free BatchNorm backward entry point (b2c_bn_relu_bwd_static) against the regular one.
+"""The allocation-free BatchNorm backward entry point (b2c_bn_relu_bwd_static) against the regular one and the oracle.
 
 Some callers of this library cannot allocate device memory where they call it: they run under an allocator they do
 not own, inside a fixed memory budget, or must not trigger the device synchronisation that CUDA's allocation calls
@@ -8,6 +8,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2503_23186_b200 import workloads as wl
 from parity import assert_close, dev_bf16, dev_f32, host
 
@@ -27,14 +28,14 @@ def _problem(seed, shape, use_res):
     return y, a, da1, da2, gamma, mean, invstd
 
 
-def _run(ctx, shape, prob, static):
+def _run(ctx, shape, prob, static, relu=True):
     N, H, W, C = shape
     y, a, da1, da2, gamma, mean, invstd = prob
     dy = torch.empty(shape, dtype=torch.bfloat16, device="cuda")
     dres = torch.empty(shape, dtype=torch.bfloat16, device="cuda") if da2 is not None else None
     dg, db = torch.zeros(C, device="cuda"), torch.zeros(C, device="cuda")
     args = (N, H, W, C, dev_bf16(da1), None if da2 is None else dev_bf16(da2), dev_bf16(y), dev_bf16(a), dev_f32(gamma), dev_f32(mean),
-            dev_f32(invstd), True, dy, dres, dg, db, False)
+            dev_f32(invstd), relu, dy, dres, dg, db, False)
     if static:
         ctx.bn_relu_bwd_static(*args)
     else:
@@ -49,15 +50,20 @@ def test_static_scratch_variant_matches_regular_entry_point():
     ctx = binding.Context(0)
     try:
         # two calls in a row with different channel counts: the second must not see the first one's sums
-        for seed, shape, use_res in [(0, (8, 16, 16, 256), True), (1, (5, 8, 8, 64), False)]:
+        # (the third problem has no ReLU and is large enough for the bulk-copy ring of the backward kernels)
+        for seed, shape, use_res, relu in [(0, (8, 16, 16, 256), True, True), (1, (5, 8, 8, 64), False, True), (2, (33, 31, 32, 64), False, False)]:
             prob = _problem(seed, shape, use_res)
-            ref = _run(ctx, shape, prob, static=False)
-            got = _run(ctx, shape, prob, static=True)
-            for name, g, r in zip(("dy", "dres", "dgamma", "dbeta"), got, ref):
+            ref = _run(ctx, shape, prob, static=False, relu=relu)
+            got = _run(ctx, shape, prob, static=True, relu=relu)
+            y, a, da1, da2, gamma, mean, invstd = prob
+            want = oracle.bn_relu_bwd(da1, da2, y, a, gamma, mean, invstd, relu, use_res)
+            want = (oracle.round_bf16(want[0]), None if want[1] is None else oracle.round_bf16(want[1]), want[2], want[3])
+            for name, g, r, o in zip(("dy", "dres", "dgamma", "dbeta"), got, ref, want):
                 if r is None:
                     assert g is None
                     continue
-                assert_close(g, host(r), name)
+                assert_close(g, host(r), name + " (against the regular entry point)")
+                assert_close(g, o, name + " (against the oracle)")
         # sizes beyond the built-in scratch are refused with a clear status and nothing is enqueued
         big = (1, 1, 1, 2048 + 8)
         t = torch.zeros(big, dtype=torch.bfloat16, device="cuda")
