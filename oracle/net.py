@@ -20,7 +20,11 @@ from . import (avgpool_bwd, avgpool_fwd, bn_relu_apply, bn_relu_bwd, bn_stats, c
 BN_EPS = 1e-5
 
 
-def _rb(x, rounding):
+def _rb(x, rounding, site=None):
+    """bf16 storage point.  ``rounding`` may also be a callable ``f(x, site)`` standing in for the bf16 rounding at the
+    named storage point (the tests use it to study how sensitive the step is to which way single roundings fall)."""
+    if callable(rounding):
+        return rounding(x, site)
     return round_bf16(x) if rounding else x
 
 
@@ -39,8 +43,8 @@ def forward(spec, params, images, labels, rounding=True, grad_scale=None):
     for i, L in enumerate(spec):
         k = L["kind"]
         if k == "conv":
-            w = _rb(params[f"w{i}"], rounding)
-            T.append(_rb(conv2d_fwd(T[L["src"]], w, L["stride"], L["pad"]), rounding))
+            w = _rb(params[f"w{i}"], rounding, "weights")
+            T.append(_rb(conv2d_fwd(T[L["src"]], w, L["stride"], L["pad"]), rounding, "conv"))
         elif k == "bn":
             y = T[L["src"]]
             mean, var, invstd = bn_stats(y, BN_EPS)
@@ -48,11 +52,11 @@ def forward(spec, params, images, labels, rounding=True, grad_scale=None):
             res = T[L["res"]] if L["res"] >= 0 else None
             a = bn_relu_apply(y, mean, invstd, params[f"gamma{i}"], params[f"beta{i}"], res, L["relu"])
             saved[i] = (mean, invstd, var)
-            T.append(_rb(a, rounding))
+            T.append(_rb(a, rounding, "bn"))
         elif k == "avgpool":
-            T.append(_rb(avgpool_fwd(T[L["src"]]), rounding))
+            T.append(_rb(avgpool_fwd(T[L["src"]]), rounding, "pool"))
         elif k == "fc":
-            w = _rb(params[f"w{i}"], rounding)
+            w = _rb(params[f"w{i}"], rounding, "weights")
             z = T[L["src"]] @ np.asarray(w, np.float64).T + np.asarray(params[f"b{i}"], np.float64)
             T.append(_rf(z, rounding))
         elif k == "xent":
@@ -79,18 +83,18 @@ def backward(spec, params, fw, rounding=True, dout=None):
         k = L["kind"]
         out_t = i + 1
         if k == "xent":
-            contrib[L["src"]].append(_rb(fw["dlogits"], rounding))
+            contrib[L["src"]].append(_rb(fw["dlogits"], rounding, "dlogits"))
             continue
         if not contrib[out_t]:
             raise RuntimeError(f"layer {i} output has no gradient")
         if k == "fc":
             dz = contrib[out_t][0]
-            w = np.asarray(_rb(params[f"w{i}"], rounding), np.float64)
+            w = np.asarray(_rb(params[f"w{i}"], rounding, "weights"), np.float64)
             grads[f"w{i}"] = dz.T @ T[L["src"]]
             grads[f"b{i}"] = dz.sum(axis=0)
-            contrib[L["src"]].append(_rb(dz @ w, rounding))
+            contrib[L["src"]].append(_rb(dz @ w, rounding, "fc_dgrad"))
         elif k == "avgpool":
-            contrib[L["src"]].append(_rb(avgpool_bwd(contrib[out_t][0], L["H"], L["W"]), rounding))
+            contrib[L["src"]].append(_rb(avgpool_bwd(contrib[out_t][0], L["H"], L["W"]), rounding, "pool_bwd"))
         elif k == "bn":
             c = contrib[out_t]
             assert len(c) <= 2
@@ -98,17 +102,17 @@ def backward(spec, params, fw, rounding=True, dout=None):
             dy, dres, dgamma, dbeta = bn_relu_bwd(c[0], c[1] if len(c) == 2 else None, T[L["src"]], T[out_t],
                                                   params[f"gamma{i}"], mean, invstd, L["relu"], L["res"] >= 0)
             grads[f"gamma{i}"], grads[f"beta{i}"] = dgamma, dbeta
-            contrib[L["src"]].append(_rb(dy, rounding))
+            contrib[L["src"]].append(_rb(dy, rounding, "bn_bwd"))
             if L["res"] >= 0:
-                contrib[L["res"]].append(_rb(dres, rounding))
+                contrib[L["res"]].append(_rb(dres, rounding, "bn_bwd_res"))
         elif k == "conv":
             dy = contrib[out_t][0]
             assert len(contrib[out_t]) == 1
             x = T[L["src"]]
             grads[f"w{i}"] = conv2d_wgrad(dy, x, L["R"], L["R"], L["stride"], L["pad"])
             if L["src"] != 0:  # the image batch needs no gradient
-                w = _rb(params[f"w{i}"], rounding)
-                contrib[L["src"]].append(_rb(conv2d_dgrad(dy, w, x.shape, L["stride"], L["pad"]), rounding))
+                w = _rb(params[f"w{i}"], rounding, "weights")
+                contrib[L["src"]].append(_rb(conv2d_dgrad(dy, w, x.shape, L["stride"], L["pad"]), rounding, "conv_dgrad"))
     return grads, contrib
 
 

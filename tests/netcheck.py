@@ -51,10 +51,13 @@ def grad_slots(spec):
 class Report:
     def __init__(self):
         self.rows = []
+        self.differ = {}
 
     def add(self, name, got, ref, rel_fro=REL_FRO, max_rel=MAX_REL):
         rel, mx = errors(got, ref)
         self.rows.append((name, rel, mx, rel <= rel_fro and mx <= max_rel and bool(np.all(np.isfinite(got)))))
+        # share of elements that differ at all: for tensors stored in bf16 these are the roundings that fell the other way
+        self.differ[name] = float(np.mean(np.asarray(got, np.float64).reshape(-1) != np.asarray(ref, np.float64).reshape(-1)))
 
     def failures(self):
         return [r for r in self.rows if not r[3]]

@@ -23,16 +23,21 @@ def ctx():
     c.close()
 
 
-def _compare_step(ctx, spec, params, velocity, images, labels, micro_batch, n_micro, table=None, gate_gradients=True):
+def _compare_step(ctx, spec, params, velocity, images, labels, micro_batch, n_micro, table=None, seeds=(1, 2)):
     """Three checks of one optimiser step.
-    (1) Teacher-forced: every layer's device outputs against the oracle applied to that layer's device inputs
-        (per-kernel tolerances; first micro-batch).
-    (2) Free-running: loss, logits, updated parameters and momentum of the library's whole chain against the
-        oracle's whole chain.
-    (3) Free-running parameter gradients: reported per tensor; gated with the conditioning of each sum taken into
-        account (see _gradient_gate)."""
+    (1) Teacher-forced: every layer's device outputs against the oracle applied to that layer's device inputs, at the
+        per-tensor budget (first micro-batch).  This is where the stated tolerances are enforced.
+    (2) The update alone, on the device's own gradient sum: fp32 arithmetic on identical inputs, 1e-6.
+    (3) Free-running: loss, every parameter gradient and the updated parameters of the library's whole chain against
+        the oracle's whole chain, and two runs of the library against each other.  The library and the oracle store a
+        small share of the bf16 elements one step apart (fp32 sums in an unspecified order against fp64 sums), and
+        the gradient of a randomly initialised BatchNorm residual net amplifies that strongly, so the gate is measured,
+        not assumed: the share of differing elements per kind of tensor is read off check (1), the oracle is rerun with
+        that share of its roundings flipped (tests/sensitivity.py), and every free-running deviation must stay within
+        FREE_RUNNING_FACTOR times the spread of those reruns (never tighter than the per-tensor budget itself)."""
     from paper_2503_23186_b200 import binding
     from netcheck import check_step
+    from sensitivity import DEFAULT_RATES, rates_from_report, step_spread
     net = binding.Net(ctx, spec, micro_batch)
     net.load_params(params, velocity)
     d_img, d_lab = dev_bf16(images), torch.from_numpy(labels).cuda()
@@ -47,24 +52,31 @@ def _compare_step(ctx, spec, params, velocity, images, labels, micro_batch, n_mi
     rep.assert_ok()
     net.g.zero_()
 
-    # (2), (3)
-    ref = onet.train_step(spec, params, vel, images.astype(np.float64), labels, n_micro, LR, MU, WD, rounding=True)
+    # the yardstick of (3): flip shares as measured above (not below the shares seen on the ResNet-18-shaped net, so that
+    # tensors too small to show a flip in one run are still perturbed), spread over the seeded reruns of the oracle
+    rates = rates_from_report(rep, floor=DEFAULT_RATES)
+    ref, spread = step_spread(spec, params, vel, images.astype(np.float64), labels, n_micro, LR, MU, WD, rates, seeds)
+
+    def gate(name, kind):
+        return max(FREE_RUNNING_FACTOR * spread[kind][name], REL_FRO)
+
     loss = net.train_step(d_img, d_lab, n_micro, LR, MU, WD, update=False).item()
     assert ctx.device_status() == 0
-    assert abs(loss - ref["loss"]) <= 2e-3 * abs(ref["loss"]), (loss, ref["loss"])
+    assert abs(loss - ref["loss"]) <= max(FREE_RUNNING_FACTOR * spread["loss"], 1e-5) * abs(ref["loss"]), (loss, ref["loss"], spread["loss"])
     grads = net.unpack(net.g)
     rows = []
     for name in sorted(params):
         rel, mx = errors(grads[name], ref["grads"][name])
-        rows.append((name, rel, mx))
+        rows.append((name, rel, spread["grads"][name]))
     if table is not None:
         table["free_running_gradients"] = rows
     # zero padding of the flat arrays receives no gradient
     packed_mask = net.pack({k: np.ones_like(v) for k, v in params.items()})
     assert torch.count_nonzero(net.g[torch.from_numpy(packed_mask == 0).cuda()]).item() == 0
-    _gradient_gate(rows, grads, ref["grads"], gate_gradients)
+    bad = [(n, r, sp) for (n, r, sp) in rows if r > gate(n, "grads")]
+    assert not bad, bad
 
-    # the update alone, teacher-forced on the device's own gradient sum: fp32 arithmetic on identical inputs
+    # (2) the update alone, teacher-forced on the device's own gradient sum
     g_dev = net.unpack(net.g)
     net.apply_update(n_micro, LR, MU, WD)
     assert ctx.device_status() == 0
@@ -75,45 +87,25 @@ def _compare_step(ctx, spec, params, velocity, images, labels, micro_batch, n_mi
         assert_close(v_new[name], rv, f"v_new {name} (given the device gradient)", SGD_REL, 1e-5)
     assert torch.count_nonzero(net.g).item() == 0
     assert torch.equal(net.w_bf16, net.w.to(torch.bfloat16))
-    # free-running: updated parameters against the oracle's whole chain (tensors that start at zero are pure
-    # gradient and fall under the gradient discussion above)
+    # (3) updated parameters of the whole chain
     for name in sorted(params):
-        if np.any(params[name] != 0):
-            # deep nets: the 20 % free-running gradient error times lr*|g|/|w| ~ 1e-2 shows up here
-            assert_close(w_new[name], ref["params"][name], f"w_new {name}", REL_FRO if gate_gradients else 1e-2, MAX_REL if gate_gradients else 5e-2)
-    # the same step in one call (forward, backward and update fused in b2c_train_step)
+        rel, _ = errors(w_new[name], ref["params"][name])
+        assert rel <= gate(name, "params"), (name, rel, spread["params"][name])
+    # the same step in one call (forward, backward and update fused in b2c_train_step): a second realisation of the
+    # unspecified accumulation order, held to the same yardstick
     net.load_params(params, velocity)
     loss2 = net.train_step(d_img, d_lab, n_micro, LR, MU, WD, update=True).item()
     assert ctx.device_status() == 0
-    assert abs(loss2 - loss) <= 1e-3 * abs(loss)   # run-to-run: BatchNorm statistics are combined with atomics
+    assert abs(loss2 - loss) <= max(FREE_RUNNING_FACTOR * spread["loss"], 1e-5) * abs(loss)
     w_again = net.unpack(net.w)
     for name in sorted(params):
-        if np.any(params[name] != 0):
-            # Two runs of the library differ in fp32 accumulation order (atomics; MMAs of two issuing threads interleave
-            # in one accumulator), which is unspecified; a deep net amplifies that like any other rounding difference,
-            # so its run-to-run gate is the free-running one used against the oracle above.
-            assert_close(w_again[name], w_new[name], f"w_new {name} (single call)", REL_FRO if gate_gradients else 1e-2,
-                         MAX_REL if gate_gradients else 5e-2)
+        rel, _ = errors(w_again[name], w_new[name])
+        assert rel <= gate(name, "params"), (name, rel, spread["params"][name])
     net.close()
     return rows
 
 
-def _gradient_gate(rows, got, ref, tight):
-    """Free-running gradients differ from the oracle's by the legitimate bf16 rounding flips of every upstream tensor
-    (an fp32 tensor-core sum and an fp64 sum land on opposite sides of a rounding boundary for ~1e-3 of the elements,
-    a relative perturbation of ~1e-4 per stored tensor).  The gradient of a randomly initialised BatchNorm residual
-    network amplifies such perturbations by two to three orders of magnitude (pinned on the oracle alone in
-    tests/test_oracle_pins.py), so the per-tensor budget cannot hold for the free-running chain of a deep net: there
-    the gate is the direction of every gradient (cosine >= 0.9 rules out sign, index and scaling mistakes) and the
-    errors are reported; the per-tensor budget is enforced teacher-forced, layer by layer.  Shallow nets keep a
-    relative gate with slack for the chain length."""
-    for name in got:
-        a, b = np.asarray(got[name], np.float64).reshape(-1), np.asarray(ref[name], np.float64).reshape(-1)
-        cos = float(np.dot(a, b) / max(np.linalg.norm(a) * np.linalg.norm(b), 1e-300))
-        assert cos >= 0.9, (name, cos)
-    if tight:
-        bad = [(n, r, m) for (n, r, m) in rows if r > 2e-2 or m > 5e-2]
-        assert not bad, bad
+FREE_RUNNING_FACTOR = 3.0   # free-running deviations may reach this multiple of the oracle's own spread under rounding flips
 
 
 def test_tiny_net_two_micro_batches(ctx):
@@ -123,11 +115,11 @@ def test_tiny_net_two_micro_batches(ctx):
     images, labels = wl.image_batch(1, 2 * 12, hw=8, c=16, classes=10)
     table = {}
     try:
-        _compare_step(ctx, spec, params, vel, images, labels, 12, 2, table)
+        _compare_step(ctx, spec, params, vel, images, labels, 12, 2, table, seeds=tuple(range(1, 7)))
     finally:
         print("teacher-forced worst:", table.get("teacher_forced_worst"))
         for row in table.get("free_running_gradients", []):
-            print("free-running grad %-10s relF=%.3e max=%.3e" % row)
+            print("free-running grad %-10s relF=%.3e (oracle spread under rounding flips %.3e)" % row)
 
 
 def test_tiny_net_three_channel_images(ctx):
@@ -135,7 +127,7 @@ def test_tiny_net_three_channel_images(ctx):
     spec = wl.tiny_net_spec(classes=10, hw=16, c=3, width=16, width2=32)
     params = wl.perturb_bn_params(wl.init_params(spec, 2), 2)
     images, labels = wl.image_batch(2, 8, hw=16, c=3, classes=10)
-    _compare_step(ctx, spec, params, None, images, labels, 8, 1)
+    _compare_step(ctx, spec, params, None, images, labels, 8, 1, seeds=tuple(range(1, 7)))
 
 
 def test_basic_block_config2(ctx):
@@ -149,23 +141,37 @@ def test_basic_block_config2(ctx):
     w2 = wl.normal_bf16(0, "w2", (C, 3, 3, C), std=float(np.sqrt(2.0 / (9 * C))))
     g = wl.normal_bf16(0, "g", (N, H, H, C))
     gamma, beta = np.ones(C, np.float32), np.zeros(C, np.float32)
-    rb, rf = oracle.round_bf16, oracle.round_f32
+    rf = oracle.round_f32
 
-    # oracle, with rounding at the storage points
-    y1 = rb(oracle.conv2d_fwd(x, w1, 1, 1))
-    m1, _, i1 = oracle.bn_stats(y1, 1e-5); m1, i1 = rf(m1), rf(i1)
-    a1 = rb(oracle.bn_relu_apply(y1, m1, i1, gamma, beta, None, True))
-    y2 = rb(oracle.conv2d_fwd(a1, w2, 1, 1))
-    m2, _, i2 = oracle.bn_stats(y2, 1e-5); m2, i2 = rf(m2), rf(i2)
-    out = rb(oracle.bn_relu_apply(y2, m2, i2, gamma, beta, x, True))
-    dy2, dres, dg2, db2 = oracle.bn_relu_bwd(g, None, y2, out, gamma, m2, i2, True, True)
-    dy2, dres = rb(dy2), rb(dres)
-    dw2 = oracle.conv2d_wgrad(dy2, a1, 3, 3, 1, 1)
-    da1 = rb(oracle.conv2d_dgrad(dy2, w2, a1.shape, 1, 1))
-    dy1, _, dg1, db1 = oracle.bn_relu_bwd(da1, None, y1, a1, gamma, m1, i1, True, False)
-    dy1 = rb(dy1)
-    dw1 = oracle.conv2d_wgrad(dy1, x, 3, 3, 1, 1)
-    dx = rb(oracle.conv2d_dgrad(dy1, w1, x.shape, 1, 1)) + dres   # two contributions reach the block input
+    def chain(rb):
+        """The block's forward and backward pass in the oracle, rb(x, site) = rounding at the storage points."""
+        y1 = rb(oracle.conv2d_fwd(x, w1, 1, 1), "conv")
+        m1, _, i1 = oracle.bn_stats(y1, 1e-5); m1, i1 = rf(m1), rf(i1)
+        a1 = rb(oracle.bn_relu_apply(y1, m1, i1, gamma, beta, None, True), "bn")
+        y2 = rb(oracle.conv2d_fwd(a1, w2, 1, 1), "conv")
+        m2, _, i2 = oracle.bn_stats(y2, 1e-5); m2, i2 = rf(m2), rf(i2)
+        out = rb(oracle.bn_relu_apply(y2, m2, i2, gamma, beta, x, True), "bn")
+        dy2, dres, dg2, db2 = oracle.bn_relu_bwd(g, None, y2, out, gamma, m2, i2, True, True)
+        dy2, dres = rb(dy2, "bn_bwd"), rb(dres, "bn_bwd_res")
+        dw2 = oracle.conv2d_wgrad(dy2, a1, 3, 3, 1, 1)
+        da1 = rb(oracle.conv2d_dgrad(dy2, w2, a1.shape, 1, 1), "conv_dgrad")
+        dy1, _, dg1, db1 = oracle.bn_relu_bwd(da1, None, y1, a1, gamma, m1, i1, True, False)
+        dy1 = rb(dy1, "bn_bwd")
+        dw1 = oracle.conv2d_wgrad(dy1, x, 3, 3, 1, 1)
+        dx = rb(oracle.conv2d_dgrad(dy1, w1, x.shape, 1, 1), "conv_dgrad") + dres   # two contributions reach the block input
+        return dict(y1=y1, a1=a1, y2=y2, out=out, dw2=dw2, dw1=dw1, dg2=dg2, db2=db2, dg1=dg1, db1=db1, dx=dx)
+
+    from sensitivity import DEFAULT_RATES, flipping_round, rel_fro
+    rb = lambda v, site=None: oracle.round_bf16(v)
+    ref = chain(rb)
+    y1, a1, y2, out = ref["y1"], ref["a1"], ref["y2"], ref["out"]
+    # free-running yardstick: the oracle's own spread when the measured share of its roundings falls the other way
+    spread = {k: 0.0 for k in ref}
+    for seed in (1, 2, 3):
+        run = chain(flipping_round(DEFAULT_RATES, seed))
+        for k in ref:
+            spread[k] = max(spread[k], rel_fro(run[k], ref[k]))
+    gate = lambda k: max(FREE_RUNNING_FACTOR * spread[k], REL_FRO)
 
     # library
     bf = lambda: torch.empty((N, H, H, C), dtype=torch.bfloat16, device="cuda")
@@ -194,15 +200,16 @@ def test_basic_block_config2(ctx):
     ctx.conv2d_dgrad(d, DY1, W1d, DX1)
     assert ctx.device_status() == 0
 
-    assert_close(Y1, y1, "y1"); assert_close(A1, a1, "a1"); assert_close(Y2, y2, "y2"); assert_close(OUT, out, "out")
-    # backward quantities of the free-running chain: per-tensor budget with slack for the chain of rounding flips
-    loose = dict(rel_fro=1e-2, max_rel=3e-2)
-    assert_close(DW2.reshape(C, 3, 3, C), dw2, "dw2", **loose); assert_close(DW1.reshape(C, 3, 3, C), dw1, "dw1", **loose)
-    assert_close(DG2, dg2, "dgamma2", **loose); assert_close(DB2, db2, "dbeta2", **loose)
-    assert_close(DG1, dg1, "dgamma1", **loose); assert_close(DB1, db1, "dbeta1", **loose)
-    # a ReLU mask may legitimately flip where |z| is below fp32 resolution: one element then differs by a whole dz,
-    # so the free-running input gradient is held to the Frobenius budget only
-    assert_close(host(DX1) + host(DRES), dx, "dx", rel_fro=1e-2, max_rel=float("inf"))
+    assert_close(Y1, y1, "y1")   # identical inputs: the per-tensor budget
+    # everything further down the free-running chain: within FREE_RUNNING_FACTOR times the oracle's spread under rounding
+    # flips, never tighter than the per-tensor budget.  No max-error bound: where a ReLU mask flips (|z| below the
+    # resolution of the sums), single elements legitimately differ by a whole dz.
+    for name, got in (("a1", A1), ("y2", Y2), ("out", OUT), ("dw2", DW2.reshape(C, 3, 3, C)), ("dw1", DW1.reshape(C, 3, 3, C)), ("dg2", DG2), ("db2", DB2),
+                      ("dg1", DG1), ("db1", DB1), ("dx", host(DX1) + host(DRES))):
+        rel = rel_fro(host(got) if isinstance(got, torch.Tensor) else got, ref[name])
+        print("config 2 free-running %-4s relF=%.3e (oracle spread %.3e)" % (name, rel, spread[name]))
+        assert rel <= gate(name), (name, rel, spread[name])
+    rb = oracle.round_bf16
     # the same backward kernels teacher-forced on the device's own tensors: the per-tensor budget proper
     hy2, hout, ha1, hy1 = host(Y2), host(OUT), host(A1), host(Y1)
     t_dy2, t_dres, t_dg2, t_db2 = oracle.bn_relu_bwd(g, None, hy2, hout, gamma, host(M2), host(I2), True, True)
@@ -221,11 +228,11 @@ def test_resnet18_batch128_config3(ctx):
     images, labels = wl.image_batch(0, 128)
     table = {}
     try:
-        _compare_step(ctx, spec, params, None, images, labels, 128, 1, table, gate_gradients=False)
+        _compare_step(ctx, spec, params, None, images, labels, 128, 1, table)
     finally:
         print("teacher-forced worst:", table.get("teacher_forced_worst"))
         for row in table.get("free_running_gradients", []):
-            print("free-running grad %-10s relF=%.3e max=%.3e" % row)
+            print("free-running grad %-10s relF=%.3e (oracle spread under rounding flips %.3e)" % row)
 
 
 def test_teacher_forced_report_resnet18(ctx, capsys):
@@ -241,7 +248,7 @@ def test_teacher_forced_report_resnet18(ctx, capsys):
     rep = check_step(net, spec, images, labels, 32)
     with capsys.disabled():
         for name, rel, mx, ok in rep.rows:
-            print("teacher-forced %-22s relF=%.3e max=%.3e %s" % (name, rel, mx, "" if ok else "FAIL"))
+            print("teacher-forced %-22s relF=%.3e max=%.3e differing=%.2e %s" % (name, rel, mx, rep.differ[name], "" if ok else "FAIL"))
     rep.assert_ok()
     net.close()
 
@@ -264,9 +271,14 @@ def test_concurrent_micro_batches_match_sequential(ctx):
     assert ctx.device_status() == 0
     check_step(par, spec, images, labels, 32, groups=4).assert_ok()
     assert abs(loss_par - loss_seq) <= 1e-4 * abs(loss_seq)
+    # two realisations of the unspecified accumulation order: within the oracle's spread under rounding flips
+    from sensitivity import DEFAULT_RATES, step_spread
+    _, spread = step_spread(spec, params, {k: np.zeros_like(v) for k, v in params.items()}, images.astype(np.float64), labels, 4, LR, MU, WD,
+                            DEFAULT_RATES, seeds=tuple(range(1, 7)))
     gs, gp = seq.unpack(seq.g), par.unpack(par.g)
     for name in sorted(params):
-        assert_close(gp[name], gs[name], f"grad {name} (concurrent vs sequential)", 1e-2, 3e-2)
+        rel, _ = errors(gp[name], gs[name])
+        assert rel <= max(FREE_RUNNING_FACTOR * spread["grads"][name], REL_FRO), (name, rel, spread["grads"][name])
     seq.close(); par.close()
 
 
@@ -354,11 +366,11 @@ def test_wrn28_10_batch256_config5_full_size(ctx):
 def test_tiny_bottleneck_net(ctx):
     """Bottleneck blocks (1x1 -> 3x3 -> 1x1 with expansion, projection and identity shortcuts, a stride-2 block): the
     whole step against the oracle, two micro-batches.  Ten convolutions and BatchNorms deep: the free-running gradients
-    are held to direction (see _gradient_gate), every layer to the per-kernel budget on identical inputs."""
+    are held to the oracle's own spread under rounding flips (see _compare_step), every layer to the per-kernel budget on identical inputs."""
     spec = wl.tiny_bottleneck_spec(classes=10, hw=8, c=16, width=16)
     params = wl.perturb_bn_params(wl.init_params(spec, 7), 7)
     images, labels = wl.image_batch(7, 2 * 12, hw=8, c=16, classes=10)
-    _compare_step(ctx, spec, params, None, images, labels, 12, 2, gate_gradients=False)
+    _compare_step(ctx, spec, params, None, images, labels, 12, 2, seeds=tuple(range(1, 7)))
 
 
 def test_resnet50_small_batch_layerwise(ctx):
