@@ -442,3 +442,28 @@ def test_sharded_update_pieces_match_fused_update(ctx):
         for name in ("w", "v", "g", "w_bf16", "w_dgrad"):
             assert torch.equal(getattr(pieces, name), getattr(fused, name)), (step, name)
     fused.close(); pieces.close()
+
+
+def test_profile_components_and_strategy_selection(ctx):
+    """The profiling phase of the adaptive scheduling algorithm on the device (per-layer times from the step's own
+    launch sites) feeding the host-side cost model and solver."""
+    from paper_2503_23186_b200 import asa, binding
+    spec = wl.tiny_net_spec(classes=10, hw=16, c=3, width=64, width2=128)
+    net = binding.Net(ctx, spec, 8, n_concurrent=4)
+    net.load_params(wl.init_params(spec, 22))
+    images, labels = wl.image_batch(22, 32, hw=16, c=3, classes=10)
+    ms = asa.profile_components(net, dev_bf16(images), torch.from_numpy(labels).cuda(), 4, LR, MU, WD, steps=3)
+    assert ctx.device_status() == 0
+    assert ms.shape == (len(spec), 3) and np.all(ms >= 0)
+    for i, L in enumerate(spec):
+        if L["kind"] == "conv":
+            assert ms[i, 0] > 0 and ms[i, 1] > 0                    # forward and weight gradient of every convolution were timed
+            assert (ms[i, 2] > 0) == (L["src"] != 0)                # the image batch needs no data gradient
+        if L["kind"] == "bn":
+            assert ms[i, 0] > 0 and ms[i, 2] > 0 and ms[i, 1] == 0
+    fam, _ = net.profile_read()
+    assert all(v == 0 for v in fam.values())                        # profile_components left the records cleared and switched off
+    comps = asa.components_from_spec(spec, 32, ms)
+    plan = asa.select_strategies(comps, asa.Links(devices=8, bandwidth_gbs=770.0), 180e9)
+    assert len(plan["strategy"]) == len(spec) and plan["time_ms"] <= min(plan["uniform_time_ms"].values()) + 1e-9
+    net.close()
