@@ -279,6 +279,17 @@ long long b2c_net_tensor_offset(const b2c_net* net, int tensor, int grad, int wh
  * (w_master, velocity, grad_sum fp32; w_bf16, w_bf16_dgrad bf16) and the workspace. */
 b2c_status b2c_net_bind(b2c_net* net, float* w_master, float* velocity, float* grad_sum, void* w_bf16,
                         void* w_bf16_dgrad, void* workspace, size_t workspace_bytes);
+/* Running statistics of the BatchNorm layers (optional; they do not enter the step's results).  After
+ * b2c_net_bind_running_stats(net, running, momentum) every pass of b2c_train_step updates, after its forward pass,
+ *   running_mean = (1 - momentum) * running_mean + momentum * mean,
+ *   running_var  = (1 - momentum) * running_var  + momentum * var * m / (m - 1)      (unbiased, m rows per micro-batch)
+ * for every BatchNorm layer, the micro-batches of a pass applied in order.  `running` is a caller-owned fp32 DEVICE
+ * array of b2c_net_running_stats_count elements; layer i's block [mean c][var c] starts at
+ * b2c_net_running_stats_offset(net, i) (-1 for layers without statistics).  The caller initialises it (mean 0,
+ * variance 1).  running == NULL switches the update off (the default). */
+size_t b2c_net_running_stats_count(const b2c_net* net);
+long long b2c_net_running_stats_offset(const b2c_net* net, int layer);
+b2c_status b2c_net_bind_running_stats(b2c_net* net, float* running, float momentum);
 /* Refreshes w_bf16 and w_bf16_dgrad from w_master (call once after initialising the masters). */
 b2c_status b2c_net_sync_weights(b2c_net* net, void* stream);
 /* One optimiser step: for each of n_micro micro-batches (images bf16 [n_micro*micro_batch, h, w, c],

@@ -33,6 +33,7 @@ EXPORTS = [
     "b2c_net_sync_weights", "b2c_train_step", "b2c_net_apply_update", "b2c_net_profile_enable", "b2c_net_profile_read",
     "b2c_net_profile_read_layers", "b2c_net_layer_count",
     "b2c_net_weight_layer_count", "b2c_net_weight_range", "b2c_net_refresh_dgrad_weights", "b2c_net_set_buckets", "b2c_net_bucket_wait",
+    "b2c_net_running_stats_count", "b2c_net_running_stats_offset", "b2c_net_bind_running_stats",
 ]
 PROF_KINDS = ["conv_fwd", "conv_dgrad", "conv_wgrad", "bn_fwd", "bn_bwd", "other", "update"]
 
@@ -73,6 +74,8 @@ def lib() -> ctypes.CDLL:
         L.b2c_bn_relu_bwd_groups_workspace_bytes.restype = c_size_t
         L.b2c_net_param_offset.restype = c_longlong
         L.b2c_net_tensor_offset.restype = c_longlong
+        L.b2c_net_running_stats_count.restype = c_size_t
+        L.b2c_net_running_stats_offset.restype = c_longlong
         L.b2c_destroy.restype = None
         L.b2c_net_destroy.restype = None
         L.b2c_set_spin_limit.restype = None
@@ -324,6 +327,23 @@ class Net:
             _check(lib().b2c_net_weight_range(self.handle, c_int(i), byref(b), byref(e)), "b2c_net_weight_range")
             out.append((b.value, e.value))
         return out
+
+    def enable_running_stats(self, momentum: float = 0.1):
+        """Allocates and binds the running statistics (mean 0, variance 1); returns {layer: (mean view, var view)}."""
+        n = lib().b2c_net_running_stats_count(self.handle)
+        self.running = torch.zeros(max(n, 1), dtype=torch.float32, device="cuda")
+        views = {}
+        for i, L in enumerate(self.spec):
+            if L["kind"] != "bn":
+                continue
+            off = lib().b2c_net_running_stats_offset(self.handle, c_int(i))
+            if off < 0:
+                continue
+            c = L["C"]
+            self.running[off + c:off + 2 * c] = 1.0
+            views[i] = (self.running[off:off + c], self.running[off + c:off + 2 * c])
+        _check(lib().b2c_net_bind_running_stats(self.handle, _ptr(self.running), c_float(momentum)), "b2c_net_bind_running_stats")
+        return views
 
     def set_buckets(self, buckets):
         """buckets = data_parallel.bucket_plan(...): train_step then records a gradient-ready event per bucket."""

@@ -215,6 +215,7 @@ struct LayerPlan {
     int p = 0, q = 0;
     long long w_off = -1, gamma_off = -1, beta_off = -1, bias_off = -1;   // elements into the flat parameter arrays
     long long mean_off = -1, invstd_off = -1, bwd_ws_off = -1, mask_off = -1, arrive_off = -1;   // bytes into the workspace
+    long long run_off = -1;                                                // elements into the running-statistics array
     int src_slot = -1, res_slot = -1;                                     // which gradient buffer of src / res this layer writes
     int chunk_groups = 1;          // micro-batches of a pass this layer takes per launch (divides n_conc)
     int seg_index = -1;            // position of this layer's filter bank among the weight layers (conv, fc)
@@ -247,6 +248,11 @@ struct b2c_net {
     long long launches[B2C_PROF_KINDS] = {0};   // kernels launched since the last profile read
     // gradient-ready events of the update buckets: event k is recorded once the weight layer first_layer[k] has finished its
     // parameter gradient in the last pass of a step (the backward pass completes weight layers last to first)
+    // running statistics of the BatchNorm layers (optional): caller-owned array, one [mean c][var c] block per layer
+    std::vector<BnRunEntry> run_entries;
+    size_t run_count = 0;
+    float* run_stats = nullptr;
+    float run_momentum = 0.1f;
     std::vector<int> bucket_first_layer;
     std::vector<cudaEvent_t> bucket_events;
     ~b2c_net()
@@ -447,6 +453,16 @@ b2c_status b2c_net_create_concurrent(b2c_ctx* ctx, const b2c_layer_desc* layers,
     }
     net->stats_end = (long long)ws;
     net->ws_bytes = ws;
+    // running statistics: every BatchNorm whose input is a convolution output (its sums stay in the workspace for the pass)
+    for (int i = 0; i < n_layers; ++i) {
+        LayerPlan& L = net->layers[i];
+        if (L.d.kind != B2C_LAYER_BN) continue;
+        const TensorPlan& in = net->tensors[L.d.src];
+        if (in.stats_off < 0) continue;
+        L.run_off = (long long)net->run_count;
+        net->run_entries.push_back(BnRunEntry{in.stats_off, in.c, (int)net->run_count, (float)((long long)micro_batch * in.h * in.w)});
+        net->run_count += 2 * (size_t)in.c;
+    }
     // Chunking for L2: a layer takes as many micro-batches per launch as keep its largest tensor under the budget (a
     // power-of-two divisor of the pass; B2C_CHUNK_MB sets the budget in MB, 0 = whole passes).
     {
@@ -517,6 +533,23 @@ b2c_status b2c_net_bind(b2c_net* net, float* w_master, float* velocity, float* g
 static b2c_status net_pack_dgrad(b2c_net* net, void* stream)
 {
     return b2c_weight_pack_dgrad(net->ctx, net->segs.data(), (int)net->segs.size(), net->w_bf16, net->w_dgrad, stream);
+}
+
+size_t b2c_net_running_stats_count(const b2c_net* net) { return net ? net->run_count : 0; }
+
+long long b2c_net_running_stats_offset(const b2c_net* net, int layer)
+{
+    if (!net || layer < 0 || layer >= (int)net->layers.size()) return -1;
+    return net->layers[layer].run_off;
+}
+
+b2c_status b2c_net_bind_running_stats(b2c_net* net, float* running, float momentum)
+{
+    if (!net || momentum < 0.f || momentum > 1.f) return B2C_ERR_INVALID_ARG;
+    if (running && (reinterpret_cast<uintptr_t>(running) & 3u)) return B2C_ERR_MISALIGNED;
+    net->run_stats = running;
+    net->run_momentum = momentum;
+    return B2C_OK;
 }
 
 b2c_status b2c_net_set_buckets(b2c_net* net, int n_buckets, const int* first_layer)
@@ -779,6 +812,11 @@ b2c_status b2c_train_step(b2c_net* net, const void* images, const int32_t* label
             for (int g0 = 0; g0 < G; g0 += Gc)
                 for (int i = seg; i < seg_end; ++i) B2C_TRY(forward_layer(i, g0, Gc));
             seg = seg_end;
+        }
+        if (net->run_stats != nullptr && !net->run_entries.empty()) {   // the forward pass of all micro-batches of the pass is enqueued
+            ProfScope ps_(net, stream, B2C_PROF_BN_FWD, (int)((net->run_entries.size() + 63) / 64));
+            B2C_TRY(launch_bn_running_update(ctx, net->run_entries.data(), (int)net->run_entries.size(), net->ws, net->run_stats, G, net->run_momentum,
+                                             stream));
         }
         for (int seg_end = n_layers; seg_end > 0;) {
             const int Gc = net->layers[seg_end - 1].chunk_groups;

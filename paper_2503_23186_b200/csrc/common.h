@@ -142,4 +142,16 @@ b2c_status launch_bn_bwd(b2c_ctx* ctx, int G, long long m, int c, const void* da
                          const float* gamma, const float* save_mean, const float* save_invstd, int relu, void* dy, void* dres, float* dgamma,
                          float* dbeta, int acc, double* sums, bool sums_zeroed, const void* relu_mask, unsigned* arrivals, cudaStream_t stream);
 
+// Running statistics of the BatchNorm layers of a step (momentum update with the unbiased variance), taken from the fp64
+// sums the forward pass left in the workspace.  One entry per layer; the G statistics groups of a pass are applied in
+// order, as if the micro-batches had run one after the other.
+struct BnRunEntry {
+    long long stats_off;   // bytes into the workspace: fp64 [G][2c] sum / sum of squares
+    int c;                 // channels
+    int run_off;           // elements into the running-statistics array: [mean c][var c]
+    float m;               // rows per group
+};
+b2c_status launch_bn_running_update(b2c_ctx* ctx, const BnRunEntry* entries, int n_entries, const char* ws, float* run, int G, float momentum,
+                                    cudaStream_t stream);
+
 }  // namespace b2c

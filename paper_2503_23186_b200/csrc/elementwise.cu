@@ -1098,6 +1098,32 @@ __global__ void weight_pack_dgrad_kernel(const __grid_constant__ PackSegs segs, 
     }
 }
 
+// ------------------------------------------------------------------------------ running statistics
+static constexpr int kRunEntries = 64;
+struct BnRunTable {
+    BnRunEntry e[kRunEntries];
+};
+__global__ void bn_running_update_kernel(const __grid_constant__ BnRunTable tab, const char* __restrict__ ws, float* __restrict__ run, int G, float momentum)
+{
+    pdl_wait();   // first global access comes after the previous kernel of the stream
+    pdl_launch_dependents();
+    const BnRunEntry& en = tab.e[blockIdx.x];
+    const double* stats = reinterpret_cast<const double*>(ws + en.stats_off);
+    const double inv_m = 1.0 / (double)en.m;
+    const float unbias = en.m > 1.f ? (float)((double)en.m / ((double)en.m - 1.0)) : 1.f;
+    for (int ch = threadIdx.x; ch < en.c; ch += blockDim.x) {
+        float rm = run[en.run_off + ch], rv = run[en.run_off + en.c + ch];
+        for (int g = 0; g < G; ++g) {
+            float mean, invstd, var;
+            bn_moments(stats + (size_t)g * 2 * en.c, en.c, ch, inv_m, 0.f, mean, invstd, var);
+            rm = (1.f - momentum) * rm + momentum * mean;
+            rv = (1.f - momentum) * rv + momentum * var * unbias;
+        }
+        run[en.run_off + ch] = rm;
+        run[en.run_off + en.c + ch] = rv;
+    }
+}
+
 // ------------------------------------------------------------------------------ launchers
 // Blocks per statistics group: one wave of two resident blocks per SM across all groups.
 static int ew_grid(b2c_ctx* ctx, int n_groups, long long m, int rows_per_iter)
@@ -1125,6 +1151,19 @@ b2c_status launch_bn_fwd(b2c_ctx* ctx, int G, long long m, int c, const void* y,
     else
         B2C_CUDA(b2c_launch(ctx, bn_apply_kernel<8, false>, dim3(grid), dim3(kEwThreads), 0, stream, 1u, y, m, c, stats, gamma, beta, residual, relu, eps, a,
                             save_mean, save_invstd, run_mean, run_var, momentum, mask_out));
+    B2C_CUDA(cudaGetLastError());
+    return B2C_OK;
+}
+
+b2c_status launch_bn_running_update(b2c_ctx* ctx, const BnRunEntry* entries, int n_entries, const char* ws, float* run, int G, float momentum,
+                                    cudaStream_t stream)
+{
+    for (int first = 0; first < n_entries; first += kRunEntries) {
+        BnRunTable tab;
+        const int n = n_entries - first < kRunEntries ? n_entries - first : kRunEntries;
+        for (int i = 0; i < n; ++i) tab.e[i] = entries[first + i];
+        B2C_CUDA(b2c_launch(ctx, bn_running_update_kernel, dim3((unsigned)n), dim3(128), 0, stream, 1u, tab, ws, run, G, momentum));
+    }
     B2C_CUDA(cudaGetLastError());
     return B2C_OK;
 }

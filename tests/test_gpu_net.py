@@ -467,3 +467,35 @@ def test_profile_components_and_strategy_selection(ctx):
     plan = asa.select_strategies(comps, asa.Links(devices=8, bandwidth_gbs=770.0), 180e9)
     assert len(plan["strategy"]) == len(spec) and plan["time_ms"] <= min(plan["uniform_time_ms"].values()) + 1e-9
     net.close()
+
+
+def test_running_statistics_inside_the_step(ctx):
+    """b2c_train_step keeps the BatchNorm running statistics when an array is bound: two steps of four micro-batches
+    side by side, each layer's running mean / unbiased variance against the oracle's statistics of the layer's own
+    device input, the micro-batches applied in order with momentum 0.1."""
+    from paper_2503_23186_b200 import binding
+    from netcheck import _shape
+    spec = wl.tiny_net_spec(classes=10, hw=16, c=3, width=64, width2=128)
+    net = binding.Net(ctx, spec, 8, n_concurrent=4)
+    net.load_params(wl.perturb_bn_params(wl.init_params(spec, 23), 23))
+    views = net.enable_running_stats(0.1)
+    assert set(views) == {i for i, L in enumerate(spec) if L["kind"] == "bn"}
+    images, labels = wl.image_batch(23, 32, hw=16, c=3, classes=10)
+    d_img, d_lab = dev_bf16(images), torch.from_numpy(labels).cuda()
+    want = {i: (np.zeros(spec[i]["C"]), np.ones(spec[i]["C"])) for i in views}
+    for step in range(2):
+        net.train_step(d_img, d_lab, 4, LR, MU, WD, update=True)
+        assert ctx.device_status() == 0
+        for i in views:
+            y = host(net.tensor_view(spec[i]["src"], _shape(spec, spec[i]["src"], 32, net), torch.bfloat16))
+            rm, rv = want[i]
+            for g in range(4):
+                yg = y[g * 8:(g + 1) * 8]
+                mean, var, _ = oracle.bn_stats(yg, 1e-5)
+                m = yg.size // yg.shape[-1]
+                rm = 0.9 * rm + 0.1 * mean
+                rv = 0.9 * rv + 0.1 * var * m / (m - 1)
+            want[i] = (rm, rv)
+            assert_close(views[i][0], rm, f"running mean of layer {i}, step {step}", 1e-5, 1e-5)
+            assert_close(views[i][1], rv, f"running variance of layer {i}, step {step}", 1e-4, 1e-4)
+    net.close()
