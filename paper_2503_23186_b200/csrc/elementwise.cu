@@ -353,13 +353,13 @@ static constexpr int kStThreads = kEwThreads + 32;   // consumer warps + the pro
 struct StagedWalk {
     int groups, rpi, active, chunk_rows, chunk_vecs, nt, mask_stride, stage_bytes;
     long long n_full;
-    __device__ StagedWalk(int c, long long m, int n_tensors, bool has_mask)
+    __device__ StagedWalk(int c, long long m, int n_tensors, bool has_mask, int vecs = 2)   // vecs: vectors per thread, tensor and stage
     {
         groups = c >> 3;
         rpi = kEwThreads / groups;
         active = rpi * groups;
-        chunk_rows = 2 * rpi;
-        chunk_vecs = 2 * active;
+        chunk_rows = vecs * rpi;
+        chunk_vecs = vecs * active;
         nt = n_tensors;
         mask_stride = has_mask ? ((chunk_vecs + 127) & ~127) : 0;
         stage_bytes = nt * chunk_vecs * 16 + mask_stride;
@@ -392,27 +392,28 @@ __device__ __forceinline__ int staged_produce(const StagedWalk& sw, uint8_t* rin
     return i;
 }
 // After an aborted wait: the copies already issued must land before the block may exit.
-__device__ __forceinline__ void staged_drain(int issued, uint64_t* full)
+__device__ __forceinline__ void staged_drain(int issued, uint64_t* full, int S = kStStages)
 {
-    for (int back = 0; back < kStStages && back < issued; ++back) {
+    for (int back = 0; back < S && back < issued; ++back) {
         const int it = issued - 1 - back;
-        for (uint32_t i = 0; i < (1u << 22) && !mbar_try_wait(&full[it % kStStages], (uint32_t)(it / kStStages) & 1u); ++i) {}
+        for (uint32_t i = 0; i < (1u << 22) && !mbar_try_wait(&full[it % S], (uint32_t)(it / S) & 1u); ++i) {}
     }
 }
 // Consumer side of one chunk: wait (one poller per warp), then the caller reads its two vectors per tensor.
-__device__ __forceinline__ bool staged_wait(uint64_t* full, int i, int lane, unsigned spin_limit, uint32_t* abort_flag, unsigned* status)
+__device__ __forceinline__ bool staged_wait(uint64_t* full, int i, int lane, unsigned spin_limit, uint32_t* abort_flag, unsigned* status,
+                                            int S = kStStages)
 {
     bool ok = true;
     if (lane == 0) {
-        ok = mbar_wait_bounded(&full[i % kStStages], (uint32_t)(i / kStStages) & 1u, spin_limit, abort_flag);
+        ok = mbar_wait_bounded(&full[i % S], (uint32_t)(i / S) & 1u, spin_limit, abort_flag);
         if (!ok) atomicOr(status, B2C_DEV_TIMEOUT);
     }
     return __all_sync(0xffffffffu, ok);
 }
-__device__ __forceinline__ void staged_release(uint64_t* empty, int i, int lane)
+__device__ __forceinline__ void staged_release(uint64_t* empty, int i, int lane, int S = kStStages)
 {
     __syncwarp();
-    if (lane == 0) mbar_arrive(&empty[i % kStStages]);
+    if (lane == 0) mbar_arrive(&empty[i % S]);
 }
 __device__ __forceinline__ void staged_init(uint64_t* full, uint64_t* empty, uint32_t* abort_flag)
 {
@@ -626,8 +627,9 @@ __global__ void __launch_bounds__(kStThreads, 2) bn_bwd_apply_staged_kernel(cons
 // grid-wide barrier, then the apply pass A(g) of the same group, which finds the group's tensors still in L2 (a group
 // of a 1024-image layer is an eighth of the tensor: da and y of 17 MB each against 134 MB for all groups, which do not
 // fit the L2).  HBM traffic per element drops from 10.25 bytes (two passes over da and y, one write) to about 6.1.
-// The barrier of group g is split: every block arrives after R(g), runs the reduction passes of the next `ahead`
-// groups, and only then waits, so the barrier latency hides behind useful work.  Small layers (whole tensor in L2
+// The barrier of group g is split: a block arrives after R(g), runs the reduction passes of the next `ahead` groups, and
+// only then needs the group's sums, so the barrier latency hides behind useful work; a helper warp does the arriving,
+// the waiting and the coefficient arithmetic beside the streaming warps.  Small layers (whole tensor in L2
 // anyway) look further ahead; they gain the second launch.  The launch is cooperative (all blocks co-resident), every
 // wait is bounded, and a block that gives up raises the status word and winds down like the other staged kernels.
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kEwThreads) : "memory"); }
@@ -640,34 +642,48 @@ __device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned* p)
 // Producer: the full chunks of one group, continuing the ring at stage index i.  False if a wait gave up.
 __device__ __forceinline__ bool staged_produce_group(const StagedWalk& sw, uint8_t* ring, uint64_t* full, uint64_t* empty, const void* t0,
                                                      const void* t1, const void* t2, const uint8_t* mask, long long base_vec, int& i,
-                                                     unsigned spin_limit, uint32_t* abort_flag, unsigned* status)
+                                                     unsigned spin_limit, uint32_t* abort_flag, unsigned* status, uint64_t policy, int S)
 {
     const uint32_t tbytes = (uint32_t)sw.chunk_vecs * 16u;
     const uint32_t tx = (uint32_t)sw.nt * tbytes + (mask != nullptr ? (uint32_t)sw.chunk_vecs : 0u);
     for (long long k = blockIdx.x; k < sw.n_full; k += gridDim.x, ++i) {
-        const int s = i % kStStages;
-        if (!mbar_wait_bounded(&empty[s], (((uint32_t)(i / kStStages)) & 1u) ^ 1u, spin_limit, abort_flag)) {
+        const int s = i % S;
+        if (!mbar_wait_bounded(&empty[s], (((uint32_t)(i / S)) & 1u) ^ 1u, spin_limit, abort_flag)) {
             atomicOr(status, B2C_DEV_TIMEOUT);
             return false;
         }
         uint8_t* dst = ring + (size_t)s * sw.stage_bytes;
         const long long v0 = base_vec + k * sw.chunk_vecs;
         mbar_expect_tx(&full[s], tx);
-        bulk_load(dst, reinterpret_cast<const uint4*>(t0) + v0, tbytes, &full[s]);
-        bulk_load(dst + tbytes, reinterpret_cast<const uint4*>(t1) + v0, tbytes, &full[s]);
-        if (sw.nt > 2) bulk_load(dst + 2 * tbytes, reinterpret_cast<const uint4*>(t2) + v0, tbytes, &full[s]);
-        if (mask != nullptr) bulk_load(dst + sw.nt * tbytes, mask + v0, (uint32_t)sw.chunk_vecs, &full[s]);
+        bulk_load_hint(dst, reinterpret_cast<const uint4*>(t0) + v0, tbytes, &full[s], policy);
+        bulk_load_hint(dst + tbytes, reinterpret_cast<const uint4*>(t1) + v0, tbytes, &full[s], policy);
+        if (sw.nt > 2) bulk_load_hint(dst + 2 * tbytes, reinterpret_cast<const uint4*>(t2) + v0, tbytes, &full[s], policy);
+        if (mask != nullptr) bulk_load_hint(dst + sw.nt * tbytes, mask + v0, (uint32_t)sw.chunk_vecs, &full[s], policy);
     }
     return true;
 }
 
-__global__ void __launch_bounds__(kStThreads, 2) bn_bwd_grouped_kernel(const void* __restrict__ da1, const void* __restrict__ da2,
+// Block of the grouped kernel: eight consumer warps, the producer warp, and a helper warp that takes the work between
+// two passes off the consumers' path (adding the block's partial sums to the group's global sums, the arrival at the
+// group's barrier, the wait for the other blocks and the group's coefficients), so that the consumers only stream.
+static constexpr int kGrThreads = kEwThreads + 64;
+// Named barriers between the consumers (c) and the helper (h); a barrier completes once kEwThreads + 32 threads have
+// arrived or synchronised on it.  Every role runs the same sequence of barrier operations whether or not a wait has
+// given up (after a failure only the work in between is skipped), so none of them can be left waiting.
+//   2: partial sums of R(t) are in shared memory        (c arrive, h sync)
+//   3: the partial-sum slots may be overwritten          (h arrive, c sync)
+//   4: coefficients of A(ga) are in shared memory        (h arrive, c sync)
+//   5: the coefficient table may be overwritten          (c arrive, h sync)
+__device__ __forceinline__ void named_sync(int id) { asm volatile("bar.sync %0, %1;" ::"r"(id), "n"(kEwThreads + 32) : "memory"); }
+__device__ __forceinline__ void named_arrive(int id) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "n"(kEwThreads + 32) : "memory"); }
+
+__global__ void __launch_bounds__(kGrThreads, 2) bn_bwd_grouped_kernel(const void* __restrict__ da1, const void* __restrict__ da2,
                                                                        const void* __restrict__ y, long long m, int c, int n_groups, int ahead,
                                                                        const float* __restrict__ gamma, const float* __restrict__ mean_all,
                                                                        const float* __restrict__ invstd_all, int relu, double* sums_all,
                                                                        unsigned* arrivals, void* __restrict__ dy, void* __restrict__ dres,
                                                                        float* dgamma, float* dbeta, int acc, const uint8_t* __restrict__ relu_mask,
-                                                                       unsigned spin_limit, unsigned* status)
+                                                                       unsigned spin_limit, unsigned* status, int vecs, int S)
 {
     pdl_wait();   // first global access comes after the previous kernel of the stream
     pdl_launch_dependents();
@@ -675,43 +691,122 @@ __global__ void __launch_bounds__(kStThreads, 2) bn_bwd_grouped_kernel(const voi
     __shared__ uint64_t full[kStStages], empty[kStStages];
     __shared__ uint32_t abort_flag;
     uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(st_raw) + 127u) & ~uintptr_t(127));
-    const StagedWalk sw(c, m, da2 != nullptr ? 3 : 2, relu != 0);
-    float* s_acc = reinterpret_cast<float*>(ring + (size_t)kStStages * sw.stage_bytes);
-    for (int i = threadIdx.x; i < 2 * c; i += kStThreads) s_acc[i] = 0.f;
+    const StagedWalk sw(c, m, da2 != nullptr ? 3 : 2, relu != 0, vecs);   // S ring stages of `vecs` vectors per thread and tensor
+    // Per-block partial sums without atomics: every consumer thread owns one (row, channel group) pair, so it stores
+    // its 16 sums into its own slot [slot][2c]; channel groups narrower than a warp first add up the rows a warp holds
+    // with shuffles (slot = warp), otherwise slot = the thread's row.  The helper warp adds the slots up.
+    const bool warp_reduce = sw.groups < 32 && (sw.groups & (sw.groups - 1)) == 0;
+    const int n_slots = warp_reduce ? kEwThreads / 32 : sw.rpi;
+    float* s_part = reinterpret_cast<float*>(ring + (size_t)S * sw.stage_bytes);   // [n_slots][2c]
+    float* s_coef = s_part + (size_t)n_slots * 2 * c;                                     // [4][c]: mean, gamma*invstd, dbeta/m, (dgamma/m)*invstd
     staged_init(full, empty, &abort_flag);
     __syncthreads();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint8_t* mask = relu ? relu_mask : nullptr;
     const long long group_vecs = m * sw.groups;
     const int n_steps = n_groups + ahead;   // step t: R(t) if t < n_groups, then A(t - ahead) if t >= ahead
+    const double inv_m = 1.0 / (double)m;
     int i = 0;                              // ring stage index, advanced identically by the producer and the consumers
     if (warp == kEwThreads / 32) {
+        // ------------------------------------------------------------------------------------ producer
         if (lane == 0) {
+            // the reduction pass asks L2 to keep the group's lines (the apply pass reads them again), the apply pass releases them
+            const uint64_t keep = l2_policy_evict_last(), release = l2_policy_evict_first();
             bool ok = true;
             for (int t = 0; ok && t < n_steps; ++t) {
-                if (t < n_groups) ok = staged_produce_group(sw, ring, full, empty, da1, y, da2, mask, t * group_vecs, i, spin_limit, &abort_flag, status);
+                if (t < n_groups)
+                    ok = staged_produce_group(sw, ring, full, empty, da1, y, da2, mask, t * group_vecs, i, spin_limit, &abort_flag, status, keep, S);
                 if (ok && t >= ahead)
-                    ok = staged_produce_group(sw, ring, full, empty, da1, y, da2, mask, (t - ahead) * group_vecs, i, spin_limit, &abort_flag, status);
+                    ok = staged_produce_group(sw, ring, full, empty, da1, y, da2, mask, (t - ahead) * group_vecs, i, spin_limit, &abort_flag, status,
+                                              release, S);
+            }
+        }
+    } else if (warp == kEwThreads / 32 + 1) {
+        // ------------------------------------------------------------------------------------ helper
+        named_arrive(3);   // the partial-sum slots start out free
+        for (int t = 0; t < n_steps; ++t) {
+            // first the coefficients of the apply pass of this step (its group's arrivals were posted a whole reduction pass
+            // ago), then this step's own sums: the consumers find the table ready when they get there
+            if (t >= ahead) {
+                const int ga = t - ahead;
+                bool ok = *(volatile uint32_t*)&abort_flag == 0u;
+                if (ok && lane == 0) {   // every block has added its sums of group ga
+                    bool seen = false;
+                    for (unsigned poll = 0; poll < spin_limit; ++poll) {
+                        if (ld_acquire_gpu(arrivals + ga) >= gridDim.x) { seen = true; break; }
+                        if (*(volatile uint32_t*)&abort_flag) break;
+                        __nanosleep(100);
+                    }
+                    if (!seen) {
+                        *(volatile uint32_t*)&abort_flag = 1u;
+                        atomicOr(status, B2C_DEV_TIMEOUT);
+                    }
+                }
+                __syncwarp();
+                ok = *(volatile uint32_t*)&abort_flag == 0u;
+                named_sync(5);   // the consumers have taken the previous group's coefficients
+                if (ok) {
+                    const double* sums = sums_all + (size_t)ga * 2 * c;
+                    const float* mean = mean_all + (size_t)ga * c;
+                    const float* invstd = invstd_all + (size_t)ga * c;
+                    for (int ch = lane; ch < c; ch += 32) {
+                        const double s1 = __ldcg(sums + ch), s2 = __ldcg(sums + c + ch);
+                        const float mn = mean[ch], istd = invstd[ch];
+                        const double dgam = (double)istd * (s2 - (double)mn * s1);
+                        s_coef[ch] = mn;
+                        s_coef[c + ch] = gamma[ch] * istd;                          // gamma*invstd
+                        s_coef[2 * c + ch] = (float)(s1 * inv_m);                   // dbeta/m
+                        s_coef[3 * c + ch] = (float)(dgam * inv_m * (double)istd);  // (dgamma/m)*invstd, multiplies (y-mean)
+                        if (blockIdx.x == 0) {   // block 0 also emits the parameter gradients
+                            const float db = (float)s1, dg = (float)dgam;
+                            if (n_groups == 1) {
+                                dbeta[ch] = acc ? dbeta[ch] + db : db;
+                                dgamma[ch] = acc ? dgamma[ch] + dg : dg;
+                            } else {   // several groups add into the same gradient (always accumulating)
+                                atomicAdd(dbeta + ch, db);
+                                atomicAdd(dgamma + ch, dg);
+                            }
+                        }
+                    }
+                }
+                named_arrive(4);
+            }
+            if (t < n_groups) {
+                named_sync(2);
+                const bool ok = *(volatile uint32_t*)&abort_flag == 0u;
+                if (ok) {
+                    double* out = sums_all + (size_t)t * 2 * c;
+                    for (int j = lane; j < 2 * c; j += 32) {
+                        float tot = 0.f;
+                        for (int sl = 0; sl < n_slots; ++sl) tot += s_part[(size_t)sl * 2 * c + j];
+                        atomicAdd(out + j, (double)tot);
+                    }
+                }
+                if (t + 1 < n_groups) named_arrive(3);   // the slots have been read (nobody waits for it after the last group)
+                if (ok) {
+                    __threadfence();   // this block's sums are visible device-wide before its arrival is
+                    __syncwarp();
+                    if (lane == 0) atomicAdd(arrivals + t, 1u);
+                }
             }
         }
     } else {
+        // ------------------------------------------------------------------------------------ consumers
         const int g = threadIdx.x % sw.groups;
         const bool act = threadIdx.x < sw.active;
         const uint32_t tbytes = (uint32_t)sw.chunk_vecs * 16u;
         const bool two = sw.nt > 2;
         const bool ragged = (long long)sw.n_full * sw.chunk_rows < m && (sw.n_full % gridDim.x) == blockIdx.x;   // this block takes the group's tail
-        const double inv_m = 1.0 / (double)m;
-        // Every consumer warp runs the same sequence of consumer_sync() calls whether or not a wait has given up: after
-        // a failure (the abort flag is set before the failing thread reaches the next barrier) the warps only skip work.
+        named_arrive(5);   // the coefficient table starts out free
         bool ok = true;
         for (int t = 0; t < n_steps; ++t) {
             if (t < n_groups) {
                 // ---------------------------------------------------------------- R(t): S1 = sum dz, S2 = sum dz*y
+                float sb[8], sg[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) sb[j] = sg[j] = 0.f;
                 if (ok) {
                     const long long base = t * group_vecs;
-                    float sb[8], sg[8];
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) sb[j] = sg[j] = 0.f;
                     auto accumulate = [&](const uint4& v1, const uint4& vy, const uint4& v2, unsigned mk) {
                         float d[8], d2[8], fy[8];
                         unpack8(v1, d);
@@ -727,12 +822,12 @@ __global__ void __launch_bounds__(kStThreads, 2) bn_bwd_grouped_kernel(const voi
                         }
                     };
                     for (long long k = blockIdx.x; k < sw.n_full; k += gridDim.x, ++i) {
-                        ok = staged_wait(full, i, lane, spin_limit, &abort_flag, status);
+                        ok = staged_wait(full, i, lane, spin_limit, &abort_flag, status, S);
                         if (!ok) break;
                         if (act) {
-                            const uint8_t* st = ring + (size_t)(i % kStStages) * sw.stage_bytes;
-#pragma unroll
-                            for (int u = 0; u < 2; ++u) {
+                            const uint8_t* st = ring + (size_t)(i % S) * sw.stage_bytes;
+#pragma unroll 2
+                            for (int u = 0; u < vecs; ++u) {
                                 const int v = u * sw.active + threadIdx.x;
                                 const uint4 v1 = reinterpret_cast<const uint4*>(st)[v];
                                 const uint4 vy = reinterpret_cast<const uint4*>(st + tbytes)[v];
@@ -742,7 +837,7 @@ __global__ void __launch_bounds__(kStThreads, 2) bn_bwd_grouped_kernel(const voi
                                 accumulate(v1, vy, v2, mk);
                             }
                         }
-                        staged_release(empty, i, lane);
+                        staged_release(empty, i, lane, S);
                     }
                     if (ok && act && ragged) {
                         for (long long r = sw.n_full * sw.chunk_rows + threadIdx.x / sw.groups; r < m; r += sw.rpi) {
@@ -753,76 +848,47 @@ __global__ void __launch_bounds__(kStThreads, 2) bn_bwd_grouped_kernel(const voi
                             accumulate(v1, vy, v2, mk);
                         }
                     }
-                    if (ok && act) {
+                }
+                if (warp_reduce) {   // every lane of the warp is active here (the group count divides the block); uniform branch
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            atomicAdd(&s_acc[g * 8 + j], sb[j]);
-                            atomicAdd(&s_acc[c + g * 8 + j], sg[j]);
-                        }
-                    }
-                }
-                consumer_sync();
-                if (*(volatile uint32_t*)&abort_flag) ok = false;
-                if (ok) {
-                    double* out = sums_all + (size_t)t * 2 * c;
-                    for (int j = threadIdx.x; j < 2 * c; j += kEwThreads) {
-                        atomicAdd(out + j, (double)s_acc[j]);
-                        s_acc[j] = 0.f;
-                    }
-                    __threadfence();   // this block's sums are visible device-wide before its arrival is
-                }
-                consumer_sync();
-                if (ok && threadIdx.x == 0) {
-                    __threadfence();
-                    atomicAdd(arrivals + t, 1u);
-                }
-            }
-            if (t >= ahead) {
-                // ---------------------------------------------------------------- A(ga): dy (and dres), after every block has arrived at group ga
-                const int ga = t - ahead;
-                if (ok && threadIdx.x == 0) {
-                    bool seen = false;
-                    for (unsigned poll = 0; poll < spin_limit; ++poll) {
-                        if (ld_acquire_gpu(arrivals + ga) >= gridDim.x) { seen = true; break; }
-                        if (*(volatile uint32_t*)&abort_flag) break;
-                        __nanosleep(100);
-                    }
-                    if (!seen) {
-                        *(volatile uint32_t*)&abort_flag = 1u;
-                        atomicOr(status, B2C_DEV_TIMEOUT);
-                    }
-                }
-                consumer_sync();
-                if (*(volatile uint32_t*)&abort_flag) ok = false;
-                if (ok) {
-                    const long long base = ga * group_vecs;
-                    const double* sums = sums_all + (size_t)ga * 2 * c;
-                    const float* mean = mean_all + (size_t)ga * c;
-                    const float* invstd = invstd_all + (size_t)ga * c;
-                    if (blockIdx.x == 0) {
-                        for (int ch = threadIdx.x; ch < c; ch += kEwThreads) {
-                            const double s1 = __ldcg(sums + ch), s2 = __ldcg(sums + c + ch);
-                            const float db = (float)s1, dg = (float)((double)invstd[ch] * (s2 - (double)mean[ch] * s1));
-                            if (n_groups == 1) {
-                                dbeta[ch] = acc ? dbeta[ch] + db : db;
-                                dgamma[ch] = acc ? dgamma[ch] + dg : dg;
-                            } else {   // several groups add into the same gradient (always accumulating)
-                                atomicAdd(dbeta + ch, db);
-                                atomicAdd(dgamma + ch, dg);
+                    for (int off = 16; off >= 1; off >>= 1) {
+                        if (off >= sw.groups) {
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                sb[j] += __shfl_xor_sync(0xffffffffu, sb[j], off);
+                                sg[j] += __shfl_xor_sync(0xffffffffu, sg[j], off);
                             }
                         }
                     }
-                    float mu[8], k0[8], kb[8], kg[8];
+                }
+                named_sync(3);   // the helper has read the previous group's partial sums
+                if (act && (!warp_reduce || lane < sw.groups)) {
+                    float* mine = s_part + (size_t)(warp_reduce ? warp : threadIdx.x / sw.groups) * 2 * c + g * 8;
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
-                        const int ch = g * 8 + j;
-                        const double s1 = __ldcg(sums + ch), s2 = __ldcg(sums + c + ch);
-                        const double is = (double)invstd[ch], dgam = is * (s2 - (double)mean[ch] * s1);
-                        mu[j] = mean[ch];
-                        k0[j] = gamma[ch] * invstd[ch];                        // gamma*invstd
-                        kb[j] = (float)(s1 * inv_m);                           // dbeta/m
-                        kg[j] = (float)(dgam * inv_m * is);                    // (dgamma/m)*invstd, multiplies (y-mean)
+                        mine[j] = sb[j];
+                        mine[c + j] = sg[j];
                     }
+                }
+                named_arrive(2);   // hand the partial sums to the helper and go on streaming
+            }
+            if (t >= ahead) {
+                // ---------------------------------------------------------------- A(ga): dy (and dres) from the coefficients the helper has prepared
+                const int ga = t - ahead;
+                named_sync(4);
+                if (*(volatile uint32_t*)&abort_flag) ok = false;
+                float mu[8], k0[8], kb[8], kg[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int ch = act ? g * 8 + j : 0;
+                    mu[j] = s_coef[ch];
+                    k0[j] = s_coef[c + ch];
+                    kb[j] = s_coef[2 * c + ch];
+                    kg[j] = s_coef[3 * c + ch];
+                }
+                if (t + 1 < n_steps) named_arrive(5);   // the table may be rewritten (nobody waits for it after the last group)
+                if (ok) {
+                    const long long base = ga * group_vecs;
                     auto emit = [&](const uint4& v1, const uint4& vy, const uint4& v2, unsigned mk, long long vi) {
                         float d[8], d2[8], fy[8], o[8];
                         unpack8(v1, d);
@@ -836,16 +902,16 @@ __global__ void __launch_bounds__(kStThreads, 2) bn_bwd_grouped_kernel(const voi
                             d[j] = dz;
                             o[j] = k0[j] * (dz - kb[j] - (fy[j] - mu[j]) * kg[j]);
                         }
-                        reinterpret_cast<uint4*>(dy)[vi] = pack8(o);
-                        if (dres != nullptr) reinterpret_cast<uint4*>(dres)[vi] = pack8(d);
+                        __stcs(reinterpret_cast<uint4*>(dy) + vi, pack8(o));   // streaming stores: the outputs should not push the waiting group out of L2
+                        if (dres != nullptr) __stcs(reinterpret_cast<uint4*>(dres) + vi, pack8(d));
                     };
                     for (long long k = blockIdx.x; k < sw.n_full; k += gridDim.x, ++i) {
-                        ok = staged_wait(full, i, lane, spin_limit, &abort_flag, status);
+                        ok = staged_wait(full, i, lane, spin_limit, &abort_flag, status, S);
                         if (!ok) break;
                         if (act) {
-                            const uint8_t* st = ring + (size_t)(i % kStStages) * sw.stage_bytes;
-#pragma unroll
-                            for (int u = 0; u < 2; ++u) {
+                            const uint8_t* st = ring + (size_t)(i % S) * sw.stage_bytes;
+#pragma unroll 2
+                            for (int u = 0; u < vecs; ++u) {
                                 const int v = u * sw.active + threadIdx.x;
                                 const uint4 v1 = reinterpret_cast<const uint4*>(st)[v];
                                 const uint4 vy = reinterpret_cast<const uint4*>(st + tbytes)[v];
@@ -855,7 +921,7 @@ __global__ void __launch_bounds__(kStThreads, 2) bn_bwd_grouped_kernel(const voi
                                 emit(v1, vy, v2, mk, base + k * sw.chunk_vecs + v);
                             }
                         }
-                        staged_release(empty, i, lane);
+                        staged_release(empty, i, lane, S);
                     }
                     if (ok && act && ragged) {
                         for (long long r = sw.n_full * sw.chunk_rows + threadIdx.x / sw.groups; r < m; r += sw.rpi) {
@@ -872,7 +938,7 @@ __global__ void __launch_bounds__(kStThreads, 2) bn_bwd_grouped_kernel(const voi
     }
     __syncthreads();
     // After an aborted wait the copies already issued must land before the block may exit.
-    if (abort_flag && warp == kEwThreads / 32 && lane == 0) staged_drain(i, full);   // the producer lane's i = stages it issued
+    if (abort_flag && warp == kEwThreads / 32 && lane == 0) staged_drain(i, full, S);   // the producer lane's i = stages it issued
     __syncthreads();
 }
 
@@ -1181,12 +1247,26 @@ b2c_status launch_bn_bwd(b2c_ctx* ctx, int G, long long m, int c, const void* da
     }
     // Both passes in one cooperative launch, group by group (the apply pass of a group re-reads its tensors from L2).
     if (arrivals != nullptr) {
-        const int groups = c / 8, active = rows_per_iter * groups, chunk_vecs = 2 * active;
+        // Stage size (vectors per thread and tensor) and ring depth: as many stages as fit, four at most.
+        const int groups = c / 8, active = rows_per_iter * groups;
         const int nt = da2 != nullptr ? 3 : 2;
-        const size_t stage = (size_t)nt * chunk_vecs * 16 + (relu ? ((chunk_vecs + 127) & ~127) : 0);
-        const size_t smem = kStStages * stage + sizeof(float) * 2 * c + 128;
-        const long long n_full = m / (2 * rows_per_iter);
-        const bool eligible = (!relu || mask != nullptr) && chunk_vecs % 16 == 0 && (m * groups) % 16 == 0 && n_full >= 1 &&
+        const bool warp_reduce = groups < 32 && (groups & (groups - 1)) == 0;
+        const int n_slots = warp_reduce ? kEwThreads / 32 : rows_per_iter;
+        const size_t extra = sizeof(float) * ((size_t)n_slots * 2 * c + 4 * (size_t)c) + 128;
+        int vecs = 2, ring_stages = 0;   // (stages of four vectors leave a ring of two or three and measured slower: 159 against 136 us on the 64-channel layers)
+        size_t stage = 0;
+        for (;;) {
+            const int cv = vecs * active;
+            stage = (size_t)nt * cv * 16 + (relu ? ((cv + 127) & ~127) : 0);
+            ring_stages = (int)((110 * 1024 - extra) / stage);
+            if (ring_stages > kStStages) ring_stages = kStStages;
+            if ((ring_stages >= 2 && m / (vecs * rows_per_iter) >= 4ll * ctx->sm_count) || vecs == 2) break;
+            vecs = 2;
+        }
+        const int chunk_vecs = vecs * active;
+        const size_t smem = (size_t)(ring_stages > 0 ? ring_stages : 1) * stage + extra;
+        const long long n_full = m / (vecs * rows_per_iter);
+        const bool eligible = ring_stages >= 2 && (!relu || mask != nullptr) && chunk_vecs % 16 == 0 && (m * groups) % 16 == 0 && n_full >= 1 &&
                               reinterpret_cast<uintptr_t>(mask) % 16 == 0 && smem <= 110 * 1024;
         if (eligible) {
             if (!(ctx->smem_optin_done & B2C_OPTIN_BN_GROUPED)) {
@@ -1194,7 +1274,7 @@ b2c_status launch_bn_bwd(b2c_ctx* ctx, int G, long long m, int c, const void* da
                 ctx->smem_optin_done |= B2C_OPTIN_BN_GROUPED;
             }
             int per_sm = 0;
-            B2C_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, bn_bwd_grouped_kernel, kStThreads, smem));
+            B2C_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, bn_bwd_grouped_kernel, kGrThreads, smem));
             if (per_sm > 2) per_sm = 2;
             if (per_sm >= 1) {
                 long long blocks = (long long)per_sm * ctx->sm_count;   // all blocks co-resident: the groups' barriers need every block running
@@ -1209,7 +1289,7 @@ b2c_status launch_bn_bwd(b2c_ctx* ctx, int G, long long m, int c, const void* da
                 if (ahead > G) ahead = G;
                 cudaLaunchConfig_t cfg = {};
                 cfg.gridDim = dim3((unsigned)blocks);
-                cfg.blockDim = dim3(kStThreads);
+                cfg.blockDim = dim3(kGrThreads);
                 cfg.dynamicSmemBytes = smem;
                 cfg.stream = stream;
                 cudaLaunchAttribute attr[1];
@@ -1218,7 +1298,7 @@ b2c_status launch_bn_bwd(b2c_ctx* ctx, int G, long long m, int c, const void* da
                 cfg.attrs = attr;
                 cfg.numAttrs = 1;
                 B2C_CUDA(cudaLaunchKernelEx(&cfg, bn_bwd_grouped_kernel, da1, da2, y, m, c, G, ahead, gamma, save_mean, save_invstd, relu, sums, arrivals, dy,
-                                            dres, dgamma, dbeta, acc, mask, ctx->spin_limit, ctx->d_status));
+                                            dres, dgamma, dbeta, acc, mask, ctx->spin_limit, ctx->d_status, vecs, ring_stages));
                 B2C_CUDA(cudaGetLastError());
                 return B2C_OK;
             }
