@@ -48,6 +48,35 @@ __device__ __forceinline__ uint4 ld16_or_zero(const void* base, long long vec_in
     return ok ? __ldg(reinterpret_cast<const uint4*>(base) + vec_index) : make_uint4(0u, 0u, 0u, 0u);
 }
 
+// A thread's 8 + 8 per-channel sums into the block's shared accumulators.  Threads of a warp whose lanes differ by a
+// multiple of the group count hold the same channels: where the group count is a power of two below 32 those lanes add
+// up with shuffles first and one lane per channel group issues the shared-memory atomics, which leaves one contender
+// per warp and address instead of one per row (32 rows on the same address took several microseconds per block).
+// `whole_warps`: every lane of every calling warp is active (the group count divides the block).
+__device__ __forceinline__ void block_accumulate(float* s_acc, int c, int groups, int g, float (&a)[8], float (&b)[8], bool active)
+{
+    const bool warp_reduce = groups < 32 && (groups & (groups - 1)) == 0;   // uniform over the block; all threads are active then
+    if (warp_reduce) {
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) {
+            if (off >= groups) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    a[i] += __shfl_xor_sync(0xffffffffu, a[i], off);
+                    b[i] += __shfl_xor_sync(0xffffffffu, b[i], off);
+                }
+            }
+        }
+        if ((int)(threadIdx.x & 31) >= groups) return;
+    }
+    if (!active) return;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        atomicAdd(&s_acc[g * 8 + i], a[i]);
+        atomicAdd(&s_acc[c + g * 8 + i], b[i]);
+    }
+}
+
 // ------------------------------------------------------------------------------ BN forward
 // Rows in flight per thread in the statistics pass: it reads one tensor only (see bn_apply_kernel).
 static constexpr int kStatsUnroll = 8;
@@ -81,11 +110,7 @@ __global__ void __launch_bounds__(kEwThreads, 2) bn_stats_kernel(const void* __r
                 }
             }
         }
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            atomicAdd(&s_acc[g * 8 + i], s[i]);
-            atomicAdd(&s_acc[c + g * 8 + i], ss[i]);
-        }
+        block_accumulate(s_acc, c, rw.groups, g, s, ss, true);
     }
     __syncthreads();
     double* out = stats + (size_t)blockIdx.y * 2 * c;
@@ -239,11 +264,7 @@ __global__ void __launch_bounds__(kEwThreads, 2) bn_bwd_reduce_kernel(const void
                 }
             }
         }
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            atomicAdd(&s_acc[g * 8 + i], sb[i]);
-            atomicAdd(&s_acc[c + g * 8 + i], sg[i]);
-        }
+        block_accumulate(s_acc, c, rw.groups, g, sb, sg, true);
     }
     __syncthreads();
     double* out = sums_all + (size_t)blockIdx.y * 2 * c;
@@ -500,13 +521,7 @@ __global__ void __launch_bounds__(kStThreads, 2) bn_bwd_reduce_staged_kernel(con
                 accumulate(v1, vy, v2, da2 != nullptr, mk);
             }
         }
-        if (act) {
-#pragma unroll
-            for (int i2 = 0; i2 < 8; ++i2) {
-                atomicAdd(&s_acc[g * 8 + i2], sb[i2]);
-                atomicAdd(&s_acc[c + g * 8 + i2], sg[i2]);
-            }
-        }
+        block_accumulate(s_acc, c, sw.groups, g, sb, sg, act);
     }
     __syncthreads();
     if (abort_flag && warp == kEwThreads / 32 && lane == 0) staged_drain(issued, full);
