@@ -43,6 +43,9 @@ struct alignas(64) ConvKParams {
     int acc_bufs, acc_shift;         // accumulators in TMEM (2 or 4) and log2 of that: unit j uses accumulator j % acc_bufs
     int vreuse;                      // a stage serves the three vertical taps of one horizontal shift
     int fh;                          // full halo: a stage holds the tile with a one-pixel frame and serves all nine taps
+    int hm;                          // merged horizontal taps: one N = 3 x n_tile MMA per vertical tap and k-step, the three column blocks are
+                                     // shifted by one pixel and added in the epilogue (tiles of whole image rows, 64 output channels)
+    int mma_n;                       // UMMA N (n_tile, or 3 x n_tile with merged horizontal taps)
     int nb;                          // B tiles per stage (1, or 3 with vreuse)
     int b_merged;                    // the three B tiles of a stage come with one load (box of three filter rows)
     int r_filter;                    // filter height = width
@@ -122,7 +125,7 @@ struct UnitWalk {
 __device__ __forceinline__ int unit_iters(const ConvKParams& p, int par)
 {
     const int taps = p.taps[par].count;
-    if (p.fh) return p.c_blocks;
+    if (p.fh || p.hm) return p.c_blocks;
     return (p.vreuse ? taps / 3 : taps) * p.c_blocks;
 }
 
@@ -150,7 +153,7 @@ __device__ __forceinline__ void butterfly16(float (&a)[16], float (&b)[16], int 
 // of every accumulator.  NCH > 0: the warp owns exactly NCH 16-column chunks per unit and keeps the BatchNorm sums of
 // its rows in registers across units, reducing them over rows once per statistics group.  NCH == 0: any width; sums
 // are reduced over rows per unit into a per-warp shared-memory array.
-template <int NCH>
+template <int NCH, bool HM = false>
 __device__ __forceinline__ void epilogue_loop(const ConvKParams& p, uint32_t tmem_base, uint64_t* acc_full, uint64_t* acc_empty,
                                               uint32_t* abort_flag, float* my_stats, int e, int lane, int rank)
 {
@@ -231,13 +234,21 @@ __device__ __forceinline__ void epilogue_loop(const ConvKParams& p, uint32_t tme
             tc_fence_after();
             ++jacc;
         }
+        // A new statistics group: the finished group's sums go out.  Narrow tiles (sums in registers) do that after this unit's
+        // accumulator has been read and handed back, so that the MMA threads do not wait for the reduction over rows.
+        bool flush_pending = false;
+        int next_group = cur_group;
         if (do_stats) {
             const int grp = p.stats_group_images > 0 ? (p.grp_shift >= 0 ? c.n0 >> p.grp_shift : c.n0 / p.stats_group_images) : 0;
             if (grp != cur_group) {
-                if (cur_group >= 0) flush_stats();
-                cur_group = grp;
+                if (cur_group >= 0) {
+                    if constexpr (NCH > 0) flush_pending = true;
+                    else flush_stats();
+                }
+                next_group = grp;
+                if constexpr (NCH == 0) cur_group = grp;
             }
-            cur_ktile = c.ktile;
+            if constexpr (NCH == 0) cur_ktile = c.ktile;
         }
         const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * p.acc_cols + col_begin);
         // the accumulator is handed back to the MMA thread as soon as this warp has read its last column
@@ -286,6 +297,28 @@ __device__ __forceinline__ void epilogue_loop(const ConvKParams& p, uint32_t tme
         if constexpr (NCH > 0) {
             // narrow tiles: read all of this warp's columns at once, free the accumulator, then work from registers
             uint32_t r[NCH][16];
+            if constexpr (HM) {
+                // Merged horizontal taps: the accumulator holds three blocks of n_tile columns, block s = the contribution of
+                // filter column s evaluated at this row's own pixel.  Output pixel w takes block 0 of pixel w - 1, block 1 of its
+                // own pixel and block 2 of pixel w + 1; a warp's 32 rows are whole image rows, so the neighbours are the
+                // adjacent lanes, and the first / last pixel of an image row has no left / right neighbour (zero padding).
+                const float m_left = lw != 0 ? 1.f : 0.f, m_right = lw != p.bw - 1 ? 1.f : 0.f;
+#pragma unroll
+                for (int ck = 0; ck < NCH; ++ck) {
+                    uint32_t d0[16], d1[16], d2[16];
+                    tmem_ld16(t_row + (uint32_t)(ck * 16), d0);
+                    tmem_ld16(t_row + (uint32_t)(p.n_tile + ck * 16), d1);
+                    tmem_ld16(t_row + (uint32_t)(2 * p.n_tile + ck * 16), d2);
+                    tmem_ld_wait();
+                    if (ck == NCH - 1) release();
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const float left = __shfl_up_sync(0xffffffffu, __uint_as_float(d0[i]), 1);
+                        const float right = __shfl_down_sync(0xffffffffu, __uint_as_float(d2[i]), 1);
+                        r[ck][i] = __float_as_uint(fmaf(left, m_left, fmaf(right, m_right, __uint_as_float(d1[i]))));
+                    }
+                }
+            } else {
 #pragma unroll
             for (int ck = 0; ck < NCH; ++ck) {
                 if (n_it > 0 && ck < n_chunks) {
@@ -297,6 +330,10 @@ __device__ __forceinline__ void epilogue_loop(const ConvKParams& p, uint32_t tme
             }
             if (n_it > 0) tmem_ld_wait();
             release();
+            }
+            if (flush_pending) flush_stats();   // still the previous group's sums and channel tile
+            cur_group = next_group;
+            cur_ktile = c.ktile;
 #pragma unroll
             for (int ck = 0; ck < NCH; ++ck) {
                 if (ck < n_chunks) {
@@ -426,7 +463,7 @@ __device__ __forceinline__ void mma_issuer(const ConvKParams& p, const UnitWalk&
                                            uint32_t ring_addr, int stage_bytes, uint64_t* full_bar, uint64_t* empty_bar, uint64_t* acc_full,
                                            uint64_t* acc_empty, uint64_t* w_bar, uint64_t* init_bar, uint32_t* abort_flag, const int* slot_stage)
 {
-    const uint32_t idesc = make_idesc_bf16(PAIR ? 256 : 128, p.n_tile, false, false);
+    const uint32_t idesc = make_idesc_bf16(PAIR ? 256 : 128, p.mma_n, false, false);
     const uint32_t sbo = 8u * (uint32_t)p.kb * 2u;  // eight rows of kb bf16
     const uint64_t desc_proto = make_smem_desc(0u, 16u, sbo, (uint32_t)p.swz);
     const uint32_t desc_hi = (uint32_t)(desc_proto >> 32), desc_lo_base = (uint32_t)desc_proto;
@@ -610,7 +647,14 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
             const int b_rows = PAIR ? p.n_tile >> 1 : p.n_tile;
             const int R = p.r_filter;
             const uint32_t w_bar_cl = PAIR ? map_to_cta(smem_u32(&w_bar), 0) : 0u;
-            if (p.resident && w == 0) {
+            if (p.hm && w == 0) {
+                // merged horizontal taps: per channel block one box of all nine taps, landing as [r][s][out][64 in]:
+                // three tiles (one per filter row) of 3 x n_tile rows
+                const int oc0 = (walk.first % p.n_ktiles) * p.n_tile;
+                mbar_expect_tx(&w_bar, (uint32_t)(p.c_blocks * 3 * p.tx_b));
+                for (int cb = 0; cb < p.c_blocks; ++cb)
+                    tma_load_4d(smem + (size_t)cb * 3 * p.b_bytes, &p.tmB, &w_bar, cb * p.kb, oc0, 0, 0);
+            } else if (p.resident && w == 0) {
                 // bank order: [tap or horizontal shift][channel block][vertical tap]
                 const int ktile = walk.first % p.n_ktiles;   // the walk stride is a multiple of n_ktiles: fixed per CTA
                 const TapList& tl = p.taps[0];
@@ -660,7 +704,7 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
                     if (p.issuers > 1) st_volatile_shared(&slot_stage[s], i + 1);
                     int t0 = p.cb_shift >= 0 ? it >> p.cb_shift : it / p.c_blocks;   // tap (or horizontal shift)
                     const int cb = it - t0 * p.c_blocks;                               // channel block
-                    if (p.fh) t0 = 0;   // one framed box per channel block: the entry of tap (0, 0) carries its origin
+                    if (p.fh || p.hm) t0 = 0;   // one box per channel block: the entry of tap (0, 0) carries its origin
                     uint8_t* a_dst = ring + (size_t)s * stage_bytes;
                     // with vreuse the table entry of vertical tap 0 carries the shift of the whole haloed tile
                     if constexpr (PAIR) {
@@ -673,7 +717,7 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
                         }
                     } else {
                         mbar_expect_tx(&full_bar[s], stage_tx);
-                        tma_load_4d(a_dst, &p.tmA[tl.map[t0]], &full_bar[s], cb * p.kb, c.ow0 + tl.dw[t0], c.oh0 + tl.dh[t0], c.n0);
+                        tma_load_4d(a_dst, &p.tmA[tl.map[t0]], &full_bar[s], cb * p.kb, c.ow0 + (p.hm ? 0 : tl.dw[t0]), c.oh0 + tl.dh[t0], c.n0);   // merged taps: no horizontal shift
                         for (int v = 0; v < n_b_loads; ++v) {
                             const int rs = tl.rs[t0 + 3 * v], fr = (rs * 11) >> 5;   // rs / 3 for rs < 9 (R is 1 or 3)
                             tma_load_4d(a_dst + p.a_bytes + (size_t)v * p.b_bytes, &p.tmB, &full_bar[s], cb * p.kb, rs - fr * R, oc0, fr);
@@ -721,6 +765,8 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
         const int e = warp - 2;
         if (p.n_tile <= 32 && !p.out_is_f32)
             epilogue_loop<1>(p, tmem_base, acc_full, acc_empty, &abort_flag, s_stats[e], e, lane, rank);
+        else if (p.hm)
+            epilogue_loop<2, true>(p, tmem_base, acc_full, acc_empty, &abort_flag, s_stats[e], e, lane, rank);
         else if (p.n_tile <= 64 && !p.out_is_f32)
             epilogue_loop<2>(p, tmem_base, acc_full, acc_empty, &abort_flag, s_stats[e], e, lane, rank);
         else
@@ -896,7 +942,35 @@ static b2c_status build_kmajor_plan(b2c_ctx* ctx, const KMajorProblem& pb, KMajo
     const int taps_total = R * R;
     const int attempts[3][2] = {{kb_natural, 1}, {32, 1}, {kb_natural, 0}};   // (kb, vreuse)
     bool planned = false;
-    if (fh_ok && units_per_cta >= 2) {
+    // Merged horizontal taps (3x3, stride 1, one channel tile of 64, 64-channel k-blocks, image rows of 8 / 16 / 32 pixels that
+    // fill a tile with whole rows): per vertical tap and k-step ONE MMA with N = 192 against the three filter columns, so
+    // the A operand crosses the shared-memory port once per 192 columns instead of once per 64 (an N = 64 MMA is bound by
+    // its operand fetch: 48 cycles for 32 cycles of tensor work).  The stage is the tile with a halo row above and below
+    // (vertical taps are row offsets, as with vertical tap reuse); the horizontal shifts are applied to the three column
+    // blocks of the accumulator by the epilogue.
+    const bool hm_ok = ctx->use_hmerge && !p.pair && R == 3 && pb.stride == 1 && n_par == 1 && n_tile == 64 && pb.oc == 64 && pb.ic % 64 == 0 && !pb.out_f32 &&
+                       pb.bias == nullptr && (gw == 8 || gw == 16 || gw == 32) && gh >= 128 / gw && 9 * pb.ic * 64 * 2 <= 148 * 1024;
+    if (hm_ok && units_per_cta >= 2) {
+        const int bank = 9 * pb.ic * 64 * 2;
+        p.bw = gw; p.bh = 128 / gw; p.bn = 1;
+        p.tiles_w = 1; p.tiles_h = gh / p.bh; p.tiles_n = pb.n;
+        p.total_units = p.tiles_n * p.tiles_h * p.n_ktiles;
+        const int a_bytes = (p.bh + 2) * p.bw * 128;   // multiples of 1 KB for every row length used here
+        int stages = (ring_budget - bank) / a_bytes;
+        if (stages > kMaxStages) stages = kMaxStages;
+        if (stages >= 3) {
+            p.hm = 1; p.fh = 0; p.vreuse = 0; p.pair = 0;
+            p.kb = 64; p.c_blocks = pb.ic / 64; p.swz = SWZ_128B;
+            p.nb = 3; p.b_merged = 1;
+            p.tx_b = 3 * 64 * 64 * 2; p.b_bytes = p.tx_b;          // one tile = the three filter columns of one filter row: 192 rows of 128 bytes
+            p.tx_a = a_bytes; p.a_bytes = a_bytes; p.a_step = p.bw * 128;   // one image row per vertical tap
+            p.resident = 1; p.resident_bytes = bank;
+            p.stages = stages;
+            p.acc_cols = 192; p.acc_bufs = 2; p.acc_shift = 1; p.tmem_cols = 512;
+            planned = true;
+        }
+    }
+    if (!planned && fh_ok && units_per_cta >= 2) {
         const int tx_b = b_rows * 64 * 2, bank = taps_total * (pb.ic / 64) * tx_b, a_bytes = ((10 * 18 * 128) + 1023) & ~1023;
         int stages = (ring_budget - bank) / a_bytes;
         if (stages > kMaxStages) stages = kMaxStages;
@@ -941,6 +1015,7 @@ static b2c_status build_kmajor_plan(b2c_ctx* ctx, const KMajorProblem& pb, KMajo
     }
     if (p.stages < 2) return B2C_ERR_UNSUPPORTED_SHAPE;
     // Two issuing threads where one cannot keep the tensor pipe busy: tiles of at most 128 channels.
+    p.mma_n = p.hm ? 3 * p.n_tile : p.n_tile;
     p.issuers = p.n_tile <= 128 ? kIssuers : 1;
     // Wider tiles: both threads work on every unit, alternate stages (needs an even ring).
     if (p.n_tile > 128 && ctx->use_issue_split && p.stages >= 2) {
@@ -952,7 +1027,7 @@ static b2c_status build_kmajor_plan(b2c_ctx* ctx, const KMajorProblem& pb, KMajo
     const size_t smem_bytes = (size_t)p.resident_bytes + (size_t)p.stages * stage_bytes + 1024;
 
     // tensor maps
-    const int box_h = (p.vreuse || p.fh) ? p.bh + 2 : p.bh;
+    const int box_h = (p.vreuse || p.fh || p.hm) ? p.bh + 2 : p.bh;
     const int box_w = p.fh ? p.bw + 2 : p.bw;
     if (!pb.dgrad && pb.stride == 2) {
         for (int ph = 0; ph < 2; ++ph)
@@ -962,7 +1037,14 @@ static b2c_status build_kmajor_plan(b2c_ctx* ctx, const KMajorProblem& pb, KMajo
     } else {
         if (!encode_activation_map(ctx, &p.tmA[0], pb.in, pb.n, pb.ih, pb.iw, pb.ic, 1, 0, 0, p.kb, box_w, box_h, p.bn)) return B2C_ERR_CUDA;
     }
-    {
+    if (p.hm) {
+        // weights [out][r][s][in] viewed as (in, out, s, r): a box of all nine taps lands as [r][s][out][in], i.e. per filter row
+        // one K-major tile whose 192 rows are the three filter columns of the 64 output channels
+        cuuint64_t dims[4] = {(cuuint64_t)pb.ic, (cuuint64_t)pb.oc, (cuuint64_t)R, (cuuint64_t)R};
+        cuuint64_t str[3] = {(cuuint64_t)R * R * pb.ic * 2, (cuuint64_t)pb.ic * 2, (cuuint64_t)R * pb.ic * 2};
+        cuuint32_t box[4] = {64u, 64u, 3u, 3u};
+        if (!encode_map(ctx, &p.tmB, pb.wt, 4, dims, str, box, 128)) return B2C_ERR_CUDA;
+    } else {
         // weights [out][r][s][in] viewed as (in, s, out, r): a box of three filter rows lands as three tiles [r][out][in]
         cuuint64_t dims[4] = {(cuuint64_t)pb.ic, (cuuint64_t)R, (cuuint64_t)pb.oc, (cuuint64_t)R};
         cuuint64_t str[3] = {(cuuint64_t)pb.ic * 2, (cuuint64_t)R * R * pb.ic * 2, (cuuint64_t)R * pb.ic * 2};
@@ -1034,7 +1116,7 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
     key_add(key, pb.n); key_add(key, pb.ih); key_add(key, pb.iw); key_add(key, pb.ic); key_add(key, pb.oh); key_add(key, pb.ow); key_add(key, pb.oc);
     key_add(key, pb.r); key_add(key, pb.stride); key_add(key, pb.pad); key_add(key, pb.dgrad); key_add(key, pb.in); key_add(key, pb.wt);
     key_add(key, pb.out); key_add(key, pb.out_f32); key_add(key, pb.bias); key_add(key, pb.stats); key_add(key, pb.stats_group_images);
-    key_add(key, ctx->use_pairs); key_add(key, ctx->use_full_halo); key_add(key, ctx->use_issue_split);
+    key_add(key, ctx->use_pairs); key_add(key, ctx->use_full_halo); key_add(key, ctx->use_issue_split); key_add(key, ctx->use_hmerge);
     auto it = ctx->plan_cache.find(key);
     if (it == ctx->plan_cache.end()) {
         KMajorPlan fresh;
