@@ -1299,8 +1299,6 @@ b2c_status launch_bn_bwd(b2c_ctx* ctx, int G, long long m, int c, const void* da
                 const double group_bytes = (double)m * c * (2.0 * nt + 0.125);
                 int ahead = (int)(40e6 / group_bytes);
                 if (ahead < 1) ahead = 1;
-                if (const char* e = getenv("B2C_BN_AHEAD")) ahead = atoi(e);
-                if (ahead < 1) ahead = 1;
                 if (ahead > G) ahead = G;
                 cudaLaunchConfig_t cfg = {};
                 cfg.gridDim = dim3((unsigned)blocks);
