@@ -57,6 +57,10 @@ b2c_status b2c_create(b2c_ctx** out, int device)
         ctx->use_hmerge = env ? (env[0] != '0') : 1;
     }
     {
+        const char* env = std::getenv("B2C_GROUP_KBLOCKS");
+        ctx->use_group_kblocks = env ? (env[0] != '0') : 1;
+    }
+    {
         const char* env = std::getenv("B2C_WGRAD_ISSUERS");
         ctx->use_wgrad_two_issuers = env ? (env[0] != '1') : 1;   // B2C_WGRAD_ISSUERS=1: one issuing thread
     }

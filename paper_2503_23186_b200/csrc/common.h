@@ -32,6 +32,7 @@ struct b2c_ctx {
     int use_issue_split;                 // forward / data-gradient tiles wider than 128 channels: two MMA-issuing threads share every unit
     int use_pdl;                         // kernels are launched with programmatic stream serialization (their set-up overlaps the previous kernel's tail)
     int use_hmerge;                      // forward / data gradient of 3x3 stride-1 layers with 64 output channels: horizontal taps merged into N = 192 MMAs
+    int use_group_kblocks;               // short k-blocks of stride-2 and 1x1 layers share ring slots (fewer barrier waits per MMA)
     int use_wgrad_two_issuers;           // weight gradient: two MMA-issuing threads on alternate chunks of one accumulator where the ring depth is even
     int use_bn_grouped;                  // BatchNorm backward of the training step: both passes in one cooperative launch, group by group
     // Launch plans (kernel parameter blocks with their tensor maps, grid and shared-memory size) of the convolution

@@ -53,6 +53,7 @@ struct alignas(64) ConvKParams {
     int tx_a, tx_b;                  // bytes one A / B load delivers
     int a_step;                      // byte offset of one image row inside the A tile (vreuse)
     int issuers;                     // MMA-issuing threads at work (1 or 2)
+    int gsub;                        // k-blocks that share a ring slot, one barrier wait and one commit (short k-blocks: the waits would bound the issuing threads)
     int issue_split;                 // the two issuing threads share every unit: alternate stages into one accumulator (tiles wider than 128 channels)
     int pair;                        // CTA pairs (cta_group::2): M = 256 per MMA, each CTA holds half of every B tile
     int resident;                    // filter bank of this CTA's channel tile stays in shared memory
@@ -127,6 +128,13 @@ __device__ __forceinline__ int unit_iters(const ConvKParams& p, int par)
     const int taps = p.taps[par].count;
     if (p.fh || p.hm) return p.c_blocks;
     return (p.vreuse ? taps / 3 : taps) * p.c_blocks;
+}
+
+// ring slots a unit takes: gsub k-blocks per slot, the last slot of a unit possibly with fewer
+__device__ __forceinline__ int unit_stages(const ConvKParams& p, int par)
+{
+    const int n = unit_iters(p, par);
+    return p.gsub > 1 ? (n + p.gsub - 1) / p.gsub : n;
 }
 
 // Column sums over the 32 rows a warp holds (one row per lane, 16 columns each): a butterfly that halves the
@@ -458,7 +466,7 @@ __device__ __forceinline__ void issue_stage_fh(uint32_t d_tmem, uint32_t a_lo, u
 // thread cannot keep the tensor pipe busy on narrow tiles: it pays roughly 45 cycles per tcgen05.mma, 180 per barrier
 // wait and 55 per commit, all serial, against 48-64 cycles the pipe needs per MMA at N <= 128; two threads working on
 // different accumulators can.
-template <int KS, int NB, bool PAIR>
+template <int KS, int NB, bool PAIR, bool GROUP>
 __device__ __forceinline__ void mma_issuer(const ConvKParams& p, const UnitWalk& walk, int my, uint32_t tmem_base, uint32_t smem_addr,
                                            uint32_t ring_addr, int stage_bytes, uint64_t* full_bar, uint64_t* empty_bar, uint64_t* acc_full,
                                            uint64_t* acc_empty, uint64_t* w_bar, uint64_t* init_bar, uint32_t* abort_flag, const int* slot_stage)
@@ -475,6 +483,8 @@ __device__ __forceinline__ void mma_issuer(const ConvKParams& p, const UnitWalk&
     // B tiles of consecutive vertical taps are adjacent, in a stage and in the resident bank alike
     const uint32_t b_step16 = (uint32_t)p.b_bytes >> 4;
     const uint32_t b_cb16 = (uint32_t)(p.nb * p.b_bytes) >> 4, stage16 = (uint32_t)stage_bytes >> 4;
+    const int G = GROUP ? p.gsub : 1;
+    const uint32_t sub16 = GROUP ? stage16 / (uint32_t)G : stage16;   // one k-block inside a slot
     const uint32_t ring_lo = desc_lo_base + (ring_addr >> 4), bank_lo = desc_lo_base + (smem_addr >> 4);
     const int S = p.stages;
     const bool timed = p.stall != nullptr;
@@ -489,9 +499,10 @@ __device__ __forceinline__ void mma_issuer(const ConvKParams& p, const UnitWalk&
     uint32_t ph = 0;
     long long wait_ring = 0, wait_acc = 0;
     for (int pu = walk.first; ok && pu < walk.count; pu += walk.stride) {
-        int n_it = n_it_fixed;
-        if (p.n_par > 1) n_it = unit_iters(p, walk.unit(p, pu) / units_per_par);
-        if (n_it == 0) continue;   // a parity without taps: the epilogue stores zeros without an accumulator
+        int n_sub = n_it_fixed;   // k-blocks of the unit
+        if (p.n_par > 1) n_sub = unit_iters(p, walk.unit(p, pu) / units_per_par);
+        if (n_sub == 0) continue;   // a parity without taps: the epilogue stores zeros without an accumulator
+        const int n_it = GROUP ? (n_sub + G - 1) / G : n_sub;   // ring slots of the unit
         if (!p.issue_split && (j % p.issuers) != my) {   // another issuer's unit: step over its stages
             i_stage += n_it;
             s += n_it;
@@ -516,8 +527,10 @@ __device__ __forceinline__ void mma_issuer(const ConvKParams& p, const UnitWalk&
         const int init_owner = i_stage & 1;
         bool init_seen = !p.issue_split || init_owner == my;
         for (int it = 0; it < n_it; ++it) {
+            int n_k = 1;   // k-blocks in this slot
+            if constexpr (GROUP) n_k = n_sub - it * G < G ? n_sub - it * G : G;
             if (p.issue_split && (i_stage & 1) != my) {   // the other thread's stage
-                b_res += b_cb16;
+                b_res += GROUP ? (uint32_t)n_k * b_cb16 : b_cb16;
                 ++i_stage;
                 if (++s == S) { s = 0; ph ^= 1u; }
                 continue;
@@ -536,7 +549,9 @@ __device__ __forceinline__ void mma_issuer(const ConvKParams& p, const UnitWalk&
             // slot before the slot's previous stage (another issuer's) was even loaded.  A producer issues the load of
             // stage i only after the previous stage in that slot was consumed, and then stamps the slot with i + 1:
             // seeing the stamp pass i makes the parity wait unambiguous.
-            if (p.issuers > 1) {
+            // (Threads that share every unit take alternate slots of an even ring: a slot has one consumer, which has waited for
+            // the slot's previous stage itself, and needs no stamp.)
+            if (p.issuers > 1 && !p.issue_split) {
                 uint32_t polls = 0;
                 while (ld_volatile_shared(&slot_stage[s]) <= i_stage) {
                     if (++polls > p.spin_limit || *(volatile uint32_t*)abort_flag != 0u) {
@@ -554,11 +569,21 @@ __device__ __forceinline__ void mma_issuer(const ConvKParams& p, const UnitWalk&
             if (timed) wait_ring += clock64() - w2;
             tc_fence_after();
             // descriptors differ from stage to stage only in the 14-bit address field: add offsets to the low word
-            const uint32_t a_lo = ring_lo + (uint32_t)s * stage16;
-            const uint32_t b_lo = p.resident ? b_res : a_lo + a_to_b16;
-            if (p.fh) issue_stage_fh<KS, PAIR>(d_tmem, a_lo, b_lo, a_hi_fh, desc_hi, idesc, a_row16, a_rowpitch16, b_step16, b_s16, it != 0 ? 1u : 0u);
-            else issue_stage<KS, NB, PAIR>(d_tmem, a_lo, b_lo, desc_hi, idesc, a_step16, b_step16, it != 0 ? 1u : 0u);
-            b_res += b_cb16;
+            if constexpr (GROUP) {   // (never with full-halo or merged-tap stages)
+                uint32_t a_lo = ring_lo + (uint32_t)s * stage16;
+                for (int g = 0; g < n_k; ++g) {
+                    const uint32_t b_lo = p.resident ? b_res : a_lo + a_to_b16;
+                    issue_stage<KS, NB, PAIR>(d_tmem, a_lo, b_lo, desc_hi, idesc, a_step16, b_step16, (it | g) != 0 ? 1u : 0u);
+                    b_res += b_cb16;
+                    a_lo += sub16;
+                }
+            } else {
+                const uint32_t a_lo = ring_lo + (uint32_t)s * stage16;
+                const uint32_t b_lo = p.resident ? b_res : a_lo + a_to_b16;
+                if (p.fh) issue_stage_fh<KS, PAIR>(d_tmem, a_lo, b_lo, a_hi_fh, desc_hi, idesc, a_row16, a_rowpitch16, b_step16, b_s16, it != 0 ? 1u : 0u);
+                else issue_stage<KS, NB, PAIR>(d_tmem, a_lo, b_lo, desc_hi, idesc, a_step16, b_step16, it != 0 ? 1u : 0u);
+                b_res += b_cb16;
+            }
             // frees the stage (in both CTAs of a pair) once these MMAs have read it
             if constexpr (PAIR) umma_commit_pair(&empty_bar[s], (uint16_t)3);
             else umma_commit(&empty_bar[s]);
@@ -572,6 +597,104 @@ __device__ __forceinline__ void mma_issuer(const ConvKParams& p, const UnitWalk&
         if (!ok) break;
         if constexpr (PAIR) umma_commit_pair(&acc_full[buf], (uint16_t)3);
         else umma_commit(&acc_full[buf]);
+        ++j;
+    }
+    if (timed) {
+        atomicAdd(p.stall + 1, (unsigned long long)wait_ring);
+        atomicAdd(p.stall + 2, (unsigned long long)wait_acc);
+    }
+}
+
+// The two MMA-issuing threads of a CTA sharing every unit (tiles wider than 128 channels, where TMEM holds two accumulators
+// and the threads cannot take alternate units).  Stage i of the CTA belongs to thread i % 2; the ring depth is even, so
+// thread `my` owns the slots my, my + 2, ... and walks them in order with its own phase bit: a slot has one consumer and
+// needs no stamp.  Both threads accumulate into the unit's accumulator (accumulation commutes; the tensor pipe runs MMAs
+// one after the other).  The thread that does not own a unit's first stage, whose first MMA overwrites the accumulator,
+// waits for that stage's completion barrier instead of the accumulator-free barrier (the first stage was issued after
+// the accumulator had been freed); both threads commit to the accumulator-full barrier (count 2).  This thread's chain
+// of dependent instructions per slot is what bounds these layers, so the loop carries nothing it does not need.
+template <int KS, int NB, bool PAIR, bool GROUP>
+__device__ __forceinline__ void mma_issuer_split(const ConvKParams& p, const UnitWalk& walk, int my, uint32_t tmem_base, uint32_t smem_addr,
+                                                 uint32_t ring_addr, int stage_bytes, uint64_t* full_bar, uint64_t* empty_bar, uint64_t* acc_full,
+                                                 uint64_t* acc_empty, uint64_t* w_bar, uint64_t* init_bar, uint32_t* abort_flag)
+{
+    const uint32_t idesc = make_idesc_bf16(PAIR ? 256 : 128, p.mma_n, false, false);
+    const uint64_t desc_proto = make_smem_desc(0u, 16u, 8u * (uint32_t)p.kb * 2u, (uint32_t)p.swz);
+    const uint32_t desc_hi = (uint32_t)(desc_proto >> 32), desc_lo_base = (uint32_t)desc_proto;
+    const uint32_t a_to_b16 = (uint32_t)p.a_bytes >> 4, a_step16 = (uint32_t)p.a_step >> 4, b_step16 = (uint32_t)p.b_bytes >> 4;
+    const uint32_t b_cb16 = (uint32_t)(p.nb * p.b_bytes) >> 4, stage16 = (uint32_t)stage_bytes >> 4;
+    const int G = GROUP ? p.gsub : 1;
+    const uint32_t sub16 = GROUP ? stage16 / (uint32_t)G : stage16;
+    const uint32_t ring_lo = desc_lo_base + (ring_addr >> 4), bank_lo = desc_lo_base + (smem_addr >> 4);
+    const int S = p.stages;
+    const bool timed = p.stall != nullptr, resident = p.resident != 0;
+    const int n_sub_fixed = unit_iters(p, 0);
+    const int units_per_par = p.n_par > 1 ? p.total_units / p.n_par : 1;
+    long long wait_ring = 0, wait_acc = 0;
+    bool ok = true;
+    if (resident && !mbar_wait_bounded(w_bar, 0u, p.spin_limit, abort_flag)) {
+        atomicOr(p.status, B2C_DEV_TIMEOUT);
+        ok = false;
+    }
+    int s = my, k = my;   // this thread's next slot, and the index (in CTA order) of the stage that goes there
+    uint32_t ph = 0;
+    int i0 = 0, j = 0;    // index of the unit's first stage, count of units with stages
+    for (int pu = walk.first; ok && pu < walk.count; pu += walk.stride) {
+        int n_sub = n_sub_fixed;
+        if (p.n_par > 1) n_sub = unit_iters(p, walk.unit(p, pu) / units_per_par);
+        if (n_sub == 0) continue;
+        const int i_end = i0 + (GROUP ? (n_sub + G - 1) / G : n_sub);
+        const int buf = j & (p.acc_bufs - 1);
+        const uint32_t acc_par = (uint32_t)(j >> p.acc_shift) & 1u;
+        if (k < i_end) {
+            const long long w1 = timed ? clock64() : 0;
+            const bool mine_first = k == i0;
+            if (!mbar_wait_bounded(mine_first ? &acc_empty[buf] : &init_bar[buf], mine_first ? acc_par ^ 1u : acc_par, p.spin_limit, abort_flag)) {
+                atomicOr(p.status, B2C_DEV_TIMEOUT);
+                ok = false;
+                break;
+            }
+            if (timed) wait_acc += clock64() - w1;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + (uint32_t)(buf * p.acc_cols);
+            do {
+                const int it = k - i0;
+                const long long w2 = timed ? clock64() : 0;
+                if (!mbar_wait_bounded(&full_bar[s], ph, p.spin_limit, abort_flag)) {
+                    atomicOr(p.status, B2C_DEV_TIMEOUT);
+                    ok = false;
+                    break;
+                }
+                if (timed) wait_ring += clock64() - w2;
+                tc_fence_after();
+                uint32_t a_lo = ring_lo + (uint32_t)s * stage16;
+                if constexpr (GROUP) {
+                    const int n_k = n_sub - it * G < G ? n_sub - it * G : G;
+                    uint32_t b_res = bank_lo + (uint32_t)(it * G) * b_cb16;
+                    for (int g = 0; g < n_k; ++g) {
+                        issue_stage<KS, NB, PAIR>(d_tmem, a_lo, resident ? b_res : a_lo + a_to_b16, desc_hi, idesc, a_step16, b_step16, (it | g) != 0 ? 1u : 0u);
+                        b_res += b_cb16;
+                        a_lo += sub16;
+                    }
+                } else {
+                    issue_stage<KS, NB, PAIR>(d_tmem, a_lo, resident ? bank_lo + (uint32_t)it * b_cb16 : a_lo + a_to_b16, desc_hi, idesc, a_step16, b_step16,
+                                              it != 0 ? 1u : 0u);
+                }
+                if constexpr (PAIR) umma_commit_pair(&empty_bar[s], (uint16_t)3);   // frees the stage in both CTAs of a pair
+                else umma_commit(&empty_bar[s]);
+                if (it == 0) {   // the overwriting stage (both issuing threads live in the leader CTA of a pair)
+                    if constexpr (PAIR) umma_commit_pair(&init_bar[buf], (uint16_t)1);
+                    else umma_commit(&init_bar[buf]);
+                }
+                k += 2;
+                s += 2;
+                if (s >= S) { s = my; ph ^= 1u; }
+            } while (k < i_end);
+            if (!ok) break;
+        }
+        if constexpr (PAIR) umma_commit_pair(&acc_full[buf], (uint16_t)3);
+        else umma_commit(&acc_full[buf]);
+        i0 = i_end;
         ++j;
     }
     if (timed) {
@@ -595,7 +718,8 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
     uint8_t* ring = smem + p.resident_bytes;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int S = p.stages;
-    const int stage_bytes = p.a_bytes + (p.resident ? 0 : p.nb * p.b_bytes);
+    const int sub_bytes = p.a_bytes + (p.resident ? 0 : p.nb * p.b_bytes);   // one k-block: the A tile and, unless the bank is resident, its filter tiles
+    const int stage_bytes = p.gsub * sub_bytes;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
@@ -682,7 +806,9 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
             const int n_b_loads = p.resident ? 0 : (p.b_merged ? 1 : p.nb);
             for (int pu = walk.first; ok && pu < walk.count; pu += walk.stride) {
                 const int u = walk.unit(p, pu);
-                const int n_it = unit_iters(p, p.n_par > 1 ? u / (p.total_units / p.n_par) : 0);
+                const int n_sub = unit_iters(p, p.n_par > 1 ? u / (p.total_units / p.n_par) : 0);
+                const int G = p.gsub;
+                const int n_it = G > 1 ? (n_sub + G - 1) / G : n_sub;   // ring slots of the unit
                 if (i >= i_base + n_it) {   // no stage of this unit is mine
                     i_base += n_it;
                     continue;
@@ -701,26 +827,56 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
                     if (timed) waited += clock64() - w0;
                     // The previous stage in this slot has been consumed, so its barrier phase is over: the stamp lets the
                     // issuers tell this slot's phases apart (a relaxed store: the wait above orders it).
-                    if (p.issuers > 1) st_volatile_shared(&slot_stage[s], i + 1);
-                    int t0 = p.cb_shift >= 0 ? it >> p.cb_shift : it / p.c_blocks;   // tap (or horizontal shift)
-                    const int cb = it - t0 * p.c_blocks;                               // channel block
-                    if (p.fh || p.hm) t0 = 0;   // one box per channel block: the entry of tap (0, 0) carries its origin
-                    uint8_t* a_dst = ring + (size_t)s * stage_bytes;
-                    // with vreuse the table entry of vertical tap 0 carries the shift of the whole haloed tile
-                    if constexpr (PAIR) {
-                        const uint32_t full_cl = map_to_cta(smem_u32(&full_bar[s]), 0);
-                        if (rank == 0) mbar_expect_tx(&full_bar[s], 2u * stage_tx);
-                        tma_load_4d_pair(a_dst, &p.tmA[tl.map[t0]], full_cl, cb * p.kb, c.ow0 + tl.dw[t0], c.oh0 + tl.dh[t0], c.n0);
-                        for (int v = 0; v < n_b_loads; ++v) {
-                            const int rs = tl.rs[t0 + 3 * v], fr = (rs * 11) >> 5;   // rs / 3 for rs < 9 (R is 1 or 3)
-                            tma_load_4d_pair(a_dst + p.a_bytes + (size_t)v * p.b_bytes, &p.tmB, full_cl, cb * p.kb, rs - fr * R, oc0, fr);
+                    if (p.issuers > 1 && !p.issue_split) st_volatile_shared(&slot_stage[s], i + 1);
+                    if (G > 1) {
+                        // the k-blocks that share this slot (one, except where short k-blocks are grouped)
+                        const int k_first = it * G, n_k = n_sub - k_first < G ? n_sub - k_first : G;
+                        if constexpr (PAIR) {
+                            if (rank == 0) mbar_expect_tx(&full_bar[s], 2u * (uint32_t)n_k * stage_tx);
+                        } else {
+                            mbar_expect_tx(&full_bar[s], (uint32_t)n_k * stage_tx);
+                        }
+                        for (int g = 0; g < n_k; ++g) {
+                            const int kblk = k_first + g;
+                            const int t0 = p.cb_shift >= 0 ? kblk >> p.cb_shift : kblk / p.c_blocks;   // tap
+                            const int cb = kblk - t0 * p.c_blocks;                                       // channel block
+                            uint8_t* a_dst = ring + (size_t)s * stage_bytes + (size_t)g * sub_bytes;
+                            if constexpr (PAIR) {
+                                const uint32_t full_cl = map_to_cta(smem_u32(&full_bar[s]), 0);
+                                tma_load_4d_pair(a_dst, &p.tmA[tl.map[t0]], full_cl, cb * p.kb, c.ow0 + tl.dw[t0], c.oh0 + tl.dh[t0], c.n0);
+                                for (int v = 0; v < n_b_loads; ++v) {
+                                    const int rs = tl.rs[t0 + 3 * v], fr = (rs * 11) >> 5;   // rs / 3 for rs < 9 (R is 1 or 3)
+                                    tma_load_4d_pair(a_dst + p.a_bytes + (size_t)v * p.b_bytes, &p.tmB, full_cl, cb * p.kb, rs - fr * R, oc0, fr);
+                                }
+                            } else {
+                                tma_load_4d(a_dst, &p.tmA[tl.map[t0]], &full_bar[s], cb * p.kb, c.ow0 + tl.dw[t0], c.oh0 + tl.dh[t0], c.n0);
+                                for (int v = 0; v < n_b_loads; ++v) {
+                                    const int rs = tl.rs[t0 + 3 * v], fr = (rs * 11) >> 5;   // rs / 3 for rs < 9 (R is 1 or 3)
+                                    tma_load_4d(a_dst + p.a_bytes + (size_t)v * p.b_bytes, &p.tmB, &full_bar[s], cb * p.kb, rs - fr * R, oc0, fr);
+                                }
+                            }
                         }
                     } else {
-                        mbar_expect_tx(&full_bar[s], stage_tx);
-                        tma_load_4d(a_dst, &p.tmA[tl.map[t0]], &full_bar[s], cb * p.kb, c.ow0 + (p.hm ? 0 : tl.dw[t0]), c.oh0 + tl.dh[t0], c.n0);   // merged taps: no horizontal shift
-                        for (int v = 0; v < n_b_loads; ++v) {
-                            const int rs = tl.rs[t0 + 3 * v], fr = (rs * 11) >> 5;   // rs / 3 for rs < 9 (R is 1 or 3)
-                            tma_load_4d(a_dst + p.a_bytes + (size_t)v * p.b_bytes, &p.tmB, &full_bar[s], cb * p.kb, rs - fr * R, oc0, fr);
+                        int t0 = p.cb_shift >= 0 ? it >> p.cb_shift : it / p.c_blocks;   // tap (or horizontal shift)
+                        const int cb = it - t0 * p.c_blocks;                               // channel block
+                        if (p.fh || p.hm) t0 = 0;   // one box per channel block: the entry of tap (0, 0) carries its origin
+                        uint8_t* a_dst = ring + (size_t)s * stage_bytes;
+                        // with vreuse the table entry of vertical tap 0 carries the shift of the whole haloed tile
+                        if constexpr (PAIR) {
+                            const uint32_t full_cl = map_to_cta(smem_u32(&full_bar[s]), 0);
+                            if (rank == 0) mbar_expect_tx(&full_bar[s], 2u * stage_tx);
+                            tma_load_4d_pair(a_dst, &p.tmA[tl.map[t0]], full_cl, cb * p.kb, c.ow0 + tl.dw[t0], c.oh0 + tl.dh[t0], c.n0);
+                            for (int v = 0; v < n_b_loads; ++v) {
+                                const int rs = tl.rs[t0 + 3 * v], fr = (rs * 11) >> 5;   // rs / 3 for rs < 9 (R is 1 or 3)
+                                tma_load_4d_pair(a_dst + p.a_bytes + (size_t)v * p.b_bytes, &p.tmB, full_cl, cb * p.kb, rs - fr * R, oc0, fr);
+                            }
+                        } else {
+                            mbar_expect_tx(&full_bar[s], stage_tx);
+                            tma_load_4d(a_dst, &p.tmA[tl.map[t0]], &full_bar[s], cb * p.kb, c.ow0 + (p.hm ? 0 : tl.dw[t0]), c.oh0 + tl.dh[t0], c.n0);   // merged taps: no horizontal shift
+                            for (int v = 0; v < n_b_loads; ++v) {
+                                const int rs = tl.rs[t0 + 3 * v], fr = (rs * 11) >> 5;   // rs / 3 for rs < 9 (R is 1 or 3)
+                                tma_load_4d(a_dst + p.a_bytes + (size_t)v * p.b_bytes, &p.tmB, &full_bar[s], cb * p.kb, rs - fr * R, oc0, fr);
+                            }
                         }
                     }
                     last_issued = i;
@@ -747,15 +903,39 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
             if (my < p.issuers) {
             const uint32_t smem_addr = smem_u32(smem), ring_addr = smem_u32(ring);
             const int ksteps = p.kb >> 4;
-#define B2C_ISSUER(KS, NB) mma_issuer<KS, NB, PAIR>(p, walk, my, tmem_base, smem_addr, ring_addr, stage_bytes, full_bar, empty_bar, acc_full, acc_empty, &w_bar, init_bar, &abort_flag, slot_stage)
+            if (p.issue_split && !p.fh && !p.hm) {
+#define B2C_ISSUER_S(KS, NB, GR) mma_issuer_split<KS, NB, PAIR, GR>(p, walk, my, tmem_base, smem_addr, ring_addr, stage_bytes, full_bar, empty_bar, acc_full, acc_empty, &w_bar, init_bar, &abort_flag)
+                if (p.nb == 3) {
+                    if (ksteps == 4) B2C_ISSUER_S(4, 3, false);
+                    else if (ksteps == 2) B2C_ISSUER_S(2, 3, false);
+                    else B2C_ISSUER_S(1, 3, false);
+                } else if (p.gsub > 1) {
+                    if (ksteps == 4) B2C_ISSUER_S(4, 1, true);
+                    else if (ksteps == 2) B2C_ISSUER_S(2, 1, true);
+                    else B2C_ISSUER_S(1, 1, true);
+                } else {
+                    if (ksteps == 4) B2C_ISSUER_S(4, 1, false);
+                    else if (ksteps == 2) B2C_ISSUER_S(2, 1, false);
+                    else B2C_ISSUER_S(1, 1, false);
+                }
+#undef B2C_ISSUER_S
+            } else {
+#define B2C_ISSUER(KS, NB) mma_issuer<KS, NB, PAIR, false>(p, walk, my, tmem_base, smem_addr, ring_addr, stage_bytes, full_bar, empty_bar, acc_full, acc_empty, &w_bar, init_bar, &abort_flag, slot_stage)
             if (p.nb == 3) {
                 if (ksteps == 4) B2C_ISSUER(4, 3);
                 else if (ksteps == 2) B2C_ISSUER(2, 3);
                 else B2C_ISSUER(1, 3);
+            } else if (p.gsub > 1) {
+#define B2C_ISSUER_G(KS) mma_issuer<KS, 1, PAIR, true>(p, walk, my, tmem_base, smem_addr, ring_addr, stage_bytes, full_bar, empty_bar, acc_full, acc_empty, &w_bar, init_bar, &abort_flag, slot_stage)
+                if (ksteps == 4) B2C_ISSUER_G(4);
+                else if (ksteps == 2) B2C_ISSUER_G(2);
+                else B2C_ISSUER_G(1);
+#undef B2C_ISSUER_G
             } else {
                 if (ksteps == 4) B2C_ISSUER(4, 1);
                 else if (ksteps == 2) B2C_ISSUER(2, 1);
                 else B2C_ISSUER(1, 1);
+            }
             }
 #undef B2C_ISSUER
             }
@@ -1014,8 +1194,28 @@ static b2c_status build_kmajor_plan(b2c_ctx* ctx, const KMajorProblem& pb, KMajo
         if (stages >= 4 || !vr) break;
     }
     if (p.stages < 2) return B2C_ERR_UNSUPPORTED_SHAPE;
-    // Two issuing threads where one cannot keep the tensor pipe busy: tiles of at most 128 channels.
     p.mma_n = p.hm ? 3 * p.n_tile : p.n_tile;
+    // Short k-blocks share a ring slot.  An issuing thread pays 700-900 cycles per slot on top of its MMAs (the slot's stamp,
+    // the barrier wait, two commits; measured inside the running kernel), which bounds the stride-2 and 1x1 layers
+    // (one k-block = 2-4 MMAs of 48-128 cycles): group k-blocks while a slot holds less than about 1000 tensor-pipe
+    // cycles, three slots remain (four where two threads take alternate slots) and the unit has that many k-blocks.
+    p.gsub = 1;
+    if (ctx->use_group_kblocks && !p.fh && !p.hm && !p.vreuse) {
+        // k-blocks of the longest unit (stride-2 data gradient: the parity that takes every other tap in both directions)
+        const int max_sub = (n_par > 1 ? ((R + 1) / 2) * ((R + 1) / 2) : taps_total) * p.c_blocks;
+        const int per_sub = (p.kb / 16) * (p.mma_n / 2 > 48 ? p.mma_n / 2 : 48);
+        const bool split = p.n_tile > 128 && ctx->use_issue_split;   // two threads on alternate slots: an even ring, and four slots so that each keeps two
+        int g = 1;
+        while (g < 4 && g * per_sub < 1000 && 2 * g <= max_sub) {
+            int slots = p.stages / (2 * g);
+            if (split) slots &= ~1;
+            if (slots < (split ? 4 : 3)) break;
+            g *= 2;
+        }
+        p.gsub = g;
+        p.stages /= g;
+    }
+    // Two issuing threads where one cannot keep the tensor pipe busy: tiles of at most 128 channels.
     p.issuers = p.n_tile <= 128 ? kIssuers : 1;
     // Wider tiles: both threads work on every unit, alternate stages (needs an even ring).
     if (p.n_tile > 128 && ctx->use_issue_split && p.stages >= 2) {
@@ -1023,7 +1223,7 @@ static b2c_status build_kmajor_plan(b2c_ctx* ctx, const KMajorProblem& pb, KMajo
         p.issuers = kIssuers;
         p.issue_split = 1;
     }
-    const int stage_bytes = p.a_bytes + (p.resident ? 0 : p.nb * p.b_bytes);
+    const int stage_bytes = p.gsub * (p.a_bytes + (p.resident ? 0 : p.nb * p.b_bytes));
     const size_t smem_bytes = (size_t)p.resident_bytes + (size_t)p.stages * stage_bytes + 1024;
 
     // tensor maps
@@ -1116,7 +1316,7 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
     key_add(key, pb.n); key_add(key, pb.ih); key_add(key, pb.iw); key_add(key, pb.ic); key_add(key, pb.oh); key_add(key, pb.ow); key_add(key, pb.oc);
     key_add(key, pb.r); key_add(key, pb.stride); key_add(key, pb.pad); key_add(key, pb.dgrad); key_add(key, pb.in); key_add(key, pb.wt);
     key_add(key, pb.out); key_add(key, pb.out_f32); key_add(key, pb.bias); key_add(key, pb.stats); key_add(key, pb.stats_group_images);
-    key_add(key, ctx->use_pairs); key_add(key, ctx->use_full_halo); key_add(key, ctx->use_issue_split); key_add(key, ctx->use_hmerge);
+    key_add(key, ctx->use_pairs); key_add(key, ctx->use_full_halo); key_add(key, ctx->use_issue_split); key_add(key, ctx->use_hmerge); key_add(key, ctx->use_group_kblocks);
     auto it = ctx->plan_cache.find(key);
     if (it == ctx->plan_cache.end()) {
         KMajorPlan fresh;
