@@ -466,7 +466,7 @@ __device__ __forceinline__ void issue_stage_fh(uint32_t d_tmem, uint32_t a_lo, u
 // thread cannot keep the tensor pipe busy on narrow tiles: it pays roughly 45 cycles per tcgen05.mma, 180 per barrier
 // wait and 55 per commit, all serial, against 48-64 cycles the pipe needs per MMA at N <= 128; two threads working on
 // different accumulators can.
-template <int KS, int NB, bool PAIR, bool GROUP>
+template <int KS, int NB, bool PAIR, bool GROUP, bool FH>
 __device__ __forceinline__ void mma_issuer(const ConvKParams& p, const UnitWalk& walk, int my, uint32_t tmem_base, uint32_t smem_addr,
                                            uint32_t ring_addr, int stage_bytes, uint64_t* full_bar, uint64_t* empty_bar, uint64_t* acc_full,
                                            uint64_t* acc_empty, uint64_t* w_bar, uint64_t* init_bar, uint32_t* abort_flag, const int* slot_stage)
@@ -580,7 +580,7 @@ __device__ __forceinline__ void mma_issuer(const ConvKParams& p, const UnitWalk&
             } else {
                 const uint32_t a_lo = ring_lo + (uint32_t)s * stage16;
                 const uint32_t b_lo = p.resident ? b_res : a_lo + a_to_b16;
-                if (p.fh) issue_stage_fh<KS, PAIR>(d_tmem, a_lo, b_lo, a_hi_fh, desc_hi, idesc, a_row16, a_rowpitch16, b_step16, b_s16, it != 0 ? 1u : 0u);
+                if constexpr (FH) issue_stage_fh<KS, PAIR>(d_tmem, a_lo, b_lo, a_hi_fh, desc_hi, idesc, a_row16, a_rowpitch16, b_step16, b_s16, it != 0 ? 1u : 0u);
                 else issue_stage<KS, NB, PAIR>(d_tmem, a_lo, b_lo, desc_hi, idesc, a_step16, b_step16, it != 0 ? 1u : 0u);
                 b_res += b_cb16;
             }
@@ -703,7 +703,13 @@ __device__ __forceinline__ void mma_issuer_split(const ConvKParams& p, const Uni
     }
 }
 
-template <bool PAIR>
+// The kernel comes in four kinds, one per family of launch plans, so that each carries only the issuing and epilogue code its
+// plans use (with all of them in one kernel the code of a launch was spread over several hundred KB and the 64- and
+// 128-channel layers ran 7-12 % slower inside a training step, where every launch starts on a cold instruction cache):
+// general (one MMA per tap or vertical tap reuse, any tile width up to 128 channels), split (tiles wider than 128 channels:
+// two issuing threads share every unit), merged horizontal taps, full-halo stages.
+enum : int { KIND_GENERAL = 0, KIND_SPLIT = 1, KIND_HMERGE = 2, KIND_FULL_HALO = 3 };
+template <bool PAIR, int KIND>
 __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_constant__ ConvKParams p)
 {
     const int rank = PAIR ? (int)cluster_ctarank() : 0;   // 0 = leader of the pair: issues the MMAs, owns the barriers the pair shares
@@ -818,17 +824,21 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
                 const int oc0 = c.ktile * p.n_tile + rank * b_rows;
                 while (i < i_base + n_it) {
                     const int it = i - i_base;
-                    const long long w0 = timed ? clock64() : 0;
-                    if (!mbar_wait_bounded(&empty_bar[s], ph ^ 1u, p.spin_limit, &abort_flag)) {
-                        atomicOr(p.status, B2C_DEV_TIMEOUT);
-                        ok = false;
-                        break;
-                    }
-                    if (timed) waited += clock64() - w0;
-                    // The previous stage in this slot has been consumed, so its barrier phase is over: the stamp lets the
-                    // issuers tell this slot's phases apart (a relaxed store: the wait above orders it).
-                    if (p.issuers > 1 && !p.issue_split) st_volatile_shared(&slot_stage[s], i + 1);
+                    // waits until the slot's previous stage has been consumed; that stage's barrier phase is then over, and the
+                    // stamp lets issuers that take alternate units tell the slot's phases apart (a relaxed store: the wait orders it)
+                    auto wait_empty = [&]() -> bool {
+                        const long long w0 = timed ? clock64() : 0;
+                        if (!mbar_wait_bounded(&empty_bar[s], ph ^ 1u, p.spin_limit, &abort_flag)) {
+                            atomicOr(p.status, B2C_DEV_TIMEOUT);
+                            ok = false;
+                            return false;
+                        }
+                        if (timed) waited += clock64() - w0;
+                        if (p.issuers > 1 && !p.issue_split) st_volatile_shared(&slot_stage[s], i + 1);
+                        return true;
+                    };
                     if (G > 1) {
+                        if (!wait_empty()) break;
                         // the k-blocks that share this slot (one, except where short k-blocks are grouped)
                         const int k_first = it * G, n_k = n_sub - k_first < G ? n_sub - k_first : G;
                         if constexpr (PAIR) {
@@ -857,26 +867,35 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
                             }
                         }
                     } else {
+                        // (operands first, the wait second: the address arithmetic is off the chain wait -> expect -> issue)
                         int t0 = p.cb_shift >= 0 ? it >> p.cb_shift : it / p.c_blocks;   // tap (or horizontal shift)
                         const int cb = it - t0 * p.c_blocks;                               // channel block
                         if (p.fh || p.hm) t0 = 0;   // one box per channel block: the entry of tap (0, 0) carries its origin
                         uint8_t* a_dst = ring + (size_t)s * stage_bytes;
                         // with vreuse the table entry of vertical tap 0 carries the shift of the whole haloed tile
+                        const CUtensorMap* map_a = &p.tmA[tl.map[t0]];
+                        const int ca = cb * p.kb, wa = c.ow0 + (p.hm ? 0 : tl.dw[t0]), ha = c.oh0 + tl.dh[t0];   // merged taps: no horizontal shift
+                        int b_s[3], b_r[3];
+#pragma unroll
+                        for (int v = 0; v < 3; ++v) {
+                            const int rs = v < n_b_loads ? tl.rs[t0 + 3 * v] : 0, fr = (rs * 11) >> 5;   // rs / 3 for rs < 9 (R is 1 or 3)
+                            b_s[v] = rs - fr * R;
+                            b_r[v] = fr;
+                        }
+                        if (!wait_empty()) break;
                         if constexpr (PAIR) {
                             const uint32_t full_cl = map_to_cta(smem_u32(&full_bar[s]), 0);
                             if (rank == 0) mbar_expect_tx(&full_bar[s], 2u * stage_tx);
-                            tma_load_4d_pair(a_dst, &p.tmA[tl.map[t0]], full_cl, cb * p.kb, c.ow0 + tl.dw[t0], c.oh0 + tl.dh[t0], c.n0);
-                            for (int v = 0; v < n_b_loads; ++v) {
-                                const int rs = tl.rs[t0 + 3 * v], fr = (rs * 11) >> 5;   // rs / 3 for rs < 9 (R is 1 or 3)
-                                tma_load_4d_pair(a_dst + p.a_bytes + (size_t)v * p.b_bytes, &p.tmB, full_cl, cb * p.kb, rs - fr * R, oc0, fr);
-                            }
+                            tma_load_4d_pair(a_dst, map_a, full_cl, ca, wa, ha, c.n0);
+#pragma unroll
+                            for (int v = 0; v < 3; ++v)
+                                if (v < n_b_loads) tma_load_4d_pair(a_dst + p.a_bytes + (size_t)v * p.b_bytes, &p.tmB, full_cl, ca, b_s[v], oc0, b_r[v]);
                         } else {
                             mbar_expect_tx(&full_bar[s], stage_tx);
-                            tma_load_4d(a_dst, &p.tmA[tl.map[t0]], &full_bar[s], cb * p.kb, c.ow0 + (p.hm ? 0 : tl.dw[t0]), c.oh0 + tl.dh[t0], c.n0);   // merged taps: no horizontal shift
-                            for (int v = 0; v < n_b_loads; ++v) {
-                                const int rs = tl.rs[t0 + 3 * v], fr = (rs * 11) >> 5;   // rs / 3 for rs < 9 (R is 1 or 3)
-                                tma_load_4d(a_dst + p.a_bytes + (size_t)v * p.b_bytes, &p.tmB, &full_bar[s], cb * p.kb, rs - fr * R, oc0, fr);
-                            }
+                            tma_load_4d(a_dst, map_a, &full_bar[s], ca, wa, ha, c.n0);
+#pragma unroll
+                            for (int v = 0; v < 3; ++v)
+                                if (v < n_b_loads) tma_load_4d(a_dst + p.a_bytes + (size_t)v * p.b_bytes, &p.tmB, &full_bar[s], ca, b_s[v], oc0, b_r[v]);
                         }
                     }
                     last_issued = i;
@@ -903,7 +922,7 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
             if (my < p.issuers) {
             const uint32_t smem_addr = smem_u32(smem), ring_addr = smem_u32(ring);
             const int ksteps = p.kb >> 4;
-            if (p.issue_split && !p.fh && !p.hm) {
+            if constexpr (KIND == KIND_SPLIT) {
 #define B2C_ISSUER_S(KS, NB, GR) mma_issuer_split<KS, NB, PAIR, GR>(p, walk, my, tmem_base, smem_addr, ring_addr, stage_bytes, full_bar, empty_bar, acc_full, acc_empty, &w_bar, init_bar, &abort_flag)
                 if (p.nb == 3) {
                     if (ksteps == 4) B2C_ISSUER_S(4, 3, false);
@@ -920,37 +939,43 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
                 }
 #undef B2C_ISSUER_S
             } else {
-#define B2C_ISSUER(KS, NB) mma_issuer<KS, NB, PAIR, false>(p, walk, my, tmem_base, smem_addr, ring_addr, stage_bytes, full_bar, empty_bar, acc_full, acc_empty, &w_bar, init_bar, &abort_flag, slot_stage)
-            if (p.nb == 3) {
-                if (ksteps == 4) B2C_ISSUER(4, 3);
-                else if (ksteps == 2) B2C_ISSUER(2, 3);
-                else B2C_ISSUER(1, 3);
-            } else if (p.gsub > 1) {
-#define B2C_ISSUER_G(KS) mma_issuer<KS, 1, PAIR, true>(p, walk, my, tmem_base, smem_addr, ring_addr, stage_bytes, full_bar, empty_bar, acc_full, acc_empty, &w_bar, init_bar, &abort_flag, slot_stage)
-                if (ksteps == 4) B2C_ISSUER_G(4);
-                else if (ksteps == 2) B2C_ISSUER_G(2);
-                else B2C_ISSUER_G(1);
-#undef B2C_ISSUER_G
-            } else {
-                if (ksteps == 4) B2C_ISSUER(4, 1);
-                else if (ksteps == 2) B2C_ISSUER(2, 1);
-                else B2C_ISSUER(1, 1);
-            }
-            }
+#define B2C_ISSUER(KS, NB, GR, FH) mma_issuer<KS, NB, PAIR, GR, FH>(p, walk, my, tmem_base, smem_addr, ring_addr, stage_bytes, full_bar, empty_bar, acc_full, acc_empty, &w_bar, init_bar, &abort_flag, slot_stage)
+                if constexpr (KIND == KIND_HMERGE) {
+                    B2C_ISSUER(4, 3, false, false);   // 64-channel k-blocks, the three filter rows of a channel block per stage
+                } else if constexpr (KIND == KIND_FULL_HALO) {
+                    B2C_ISSUER(4, 3, false, true);
+                } else if (p.nb == 3) {
+                    if (ksteps == 4) B2C_ISSUER(4, 3, false, false);
+                    else if (ksteps == 2) B2C_ISSUER(2, 3, false, false);
+                    else B2C_ISSUER(1, 3, false, false);
+                } else if (p.gsub > 1) {
+                    if (ksteps == 4) B2C_ISSUER(4, 1, true, false);
+                    else if (ksteps == 2) B2C_ISSUER(2, 1, true, false);
+                    else B2C_ISSUER(1, 1, true, false);
+                } else {
+                    if (ksteps == 4) B2C_ISSUER(4, 1, false, false);
+                    else if (ksteps == 2) B2C_ISSUER(2, 1, false, false);
+                    else B2C_ISSUER(1, 1, false, false);
+                }
 #undef B2C_ISSUER
+            }
             }
         }
     } else {
         // ---------------------------------------------------------------- epilogue (8 warps)
         const int e = warp - 2;
-        if (p.n_tile <= 32 && !p.out_is_f32)
-            epilogue_loop<1>(p, tmem_base, acc_full, acc_empty, &abort_flag, s_stats[e], e, lane, rank);
-        else if (p.hm)
-            epilogue_loop<2, true>(p, tmem_base, acc_full, acc_empty, &abort_flag, s_stats[e], e, lane, rank);
-        else if (p.n_tile <= 64 && !p.out_is_f32)
-            epilogue_loop<2>(p, tmem_base, acc_full, acc_empty, &abort_flag, s_stats[e], e, lane, rank);
-        else
+        if constexpr (KIND == KIND_SPLIT) {   // tiles wider than 128 channels
             epilogue_loop<0>(p, tmem_base, acc_full, acc_empty, &abort_flag, s_stats[e], e, lane, rank);
+        } else if constexpr (KIND == KIND_HMERGE) {
+            epilogue_loop<2, true>(p, tmem_base, acc_full, acc_empty, &abort_flag, s_stats[e], e, lane, rank);
+        } else {
+            if (KIND == KIND_GENERAL && p.n_tile <= 32 && !p.out_is_f32)
+                epilogue_loop<1>(p, tmem_base, acc_full, acc_empty, &abort_flag, s_stats[e], e, lane, rank);
+            else if (p.n_tile <= 64 && !p.out_is_f32)
+                epilogue_loop<2>(p, tmem_base, acc_full, acc_empty, &abort_flag, s_stats[e], e, lane, rank);
+            else
+                epilogue_loop<0>(p, tmem_base, acc_full, acc_empty, &abort_flag, s_stats[e], e, lane, rank);
+        }
     }
     tc_fence_before();
     __syncthreads();
@@ -1336,13 +1361,21 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
     p.spin_limit = ctx->spin_limit;
     p.stall = ctx->stall_counters;
 
+    // the kernel kind of the plan (merged taps run on single CTAs only)
+    typedef void (*kernel_t)(const ConvKParams);
+    static const kernel_t kernels[2][4] = {
+        {conv_kmajor_kernel<false, KIND_GENERAL>, conv_kmajor_kernel<false, KIND_SPLIT>, conv_kmajor_kernel<false, KIND_HMERGE>, conv_kmajor_kernel<false, KIND_FULL_HALO>},
+        {conv_kmajor_kernel<true, KIND_GENERAL>, conv_kmajor_kernel<true, KIND_SPLIT>, nullptr, conv_kmajor_kernel<true, KIND_FULL_HALO>}};
+    const int kind = p.hm ? KIND_HMERGE : p.fh ? KIND_FULL_HALO : p.issue_split ? KIND_SPLIT : KIND_GENERAL;
+    const kernel_t kernel = kernels[p.pair ? 1 : 0][kind];
+    if (kernel == nullptr) return B2C_ERR_UNSUPPORTED_SHAPE;
     if (!(ctx->smem_optin_done & B2C_OPTIN_KMAJOR)) {   // the attribute belongs to the device: kept per context, not per process
-        B2C_CUDA(cudaFuncSetAttribute(conv_kmajor_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 212 * 1024));
-        B2C_CUDA(cudaFuncSetAttribute(conv_kmajor_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 212 * 1024));
+        for (int a = 0; a < 2; ++a)
+            for (int b = 0; b < 4; ++b)
+                if (kernels[a][b] != nullptr) B2C_CUDA(cudaFuncSetAttribute(kernels[a][b], cudaFuncAttributeMaxDynamicSharedMemorySize, 212 * 1024));
         ctx->smem_optin_done |= B2C_OPTIN_KMAJOR;
     }
-    if (p.pair) B2C_CUDA(b2c_launch(ctx, conv_kmajor_kernel<true>, dim3((unsigned)grid), dim3(kThreads), smem_bytes, stream, 2u, p));
-    else B2C_CUDA(b2c_launch(ctx, conv_kmajor_kernel<false>, dim3((unsigned)grid), dim3(kThreads), smem_bytes, stream, 1u, p));
+    B2C_CUDA(b2c_launch(ctx, kernel, dim3((unsigned)grid), dim3(kThreads), smem_bytes, stream, p.pair ? 2u : 1u, p));
     B2C_CUDA(cudaGetLastError());
     return B2C_OK;
 }

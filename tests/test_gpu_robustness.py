@@ -159,15 +159,16 @@ def test_kernel_switches_off_and_on(name, value, monkeypatch):
             N, H, W, C, K, R, st = shape
             x, w, g = wl.conv_problem(33, *shape)
             P = H // st
+            pad = (R - 1) // 2
             y = torch.full((N, P, P, K), float("nan"), dtype=torch.bfloat16, device="cuda")
             c.conv2d_fwd(_desc(*shape), dev_bf16(x), dev_bf16(w), y)
-            assert_close(y, oracle.conv2d_fwd(x, w, st, 1), f"y {shape} {name}={value}")
+            assert_close(y, oracle.conv2d_fwd(x, w, st, pad), f"y {shape} {name}={value}")
             dx = torch.full(x.shape, float("nan"), dtype=torch.bfloat16, device="cuda")
             c.conv2d_dgrad(_desc(*shape), dev_bf16(g), _dgrad_weights(c, w), dx)
-            assert_close(dx, oracle.conv2d_dgrad(g, w, x.shape, st, 1), f"dx {shape} {name}={value}")
+            assert_close(dx, oracle.conv2d_dgrad(g, w, x.shape, st, pad), f"dx {shape} {name}={value}")
             dw = torch.full(w.shape, float("nan"), dtype=torch.float32, device="cuda")
             c.conv2d_wgrad(_desc(*shape), dev_bf16(g), dev_bf16(x), dw, accumulate=False)
-            assert_close(dw, oracle.conv2d_wgrad(g, x, R, R, st, 1), f"dw {shape} {name}={value}")
+            assert_close(dw, oracle.conv2d_wgrad(g, x, R, R, st, pad), f"dw {shape} {name}={value}")
             assert c.device_status() == 0
     finally:
         c.close()
