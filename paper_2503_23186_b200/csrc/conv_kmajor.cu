@@ -276,11 +276,11 @@ __device__ __forceinline__ void epilogue_loop(const ConvKParams& p, uint32_t tme
             float v[16];
 #pragma unroll
             for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
-            if (p.bias != nullptr) {
+            if (!HM && p.bias != nullptr) {   // (merged-tap plans have neither a bias nor fp32 output)
 #pragma unroll
                 for (int i = 0; i < 16; ++i) v[i] += (ch0 + i < p.oc_valid) ? __ldg(p.bias + ch0 + i) : 0.f;
             }
-            if (p.out_is_f32) {
+            if (!HM && p.out_is_f32) {
                 if (row_valid) {
                     float* dst = reinterpret_cast<float*>(p.out) + row_off + ch0;
 #pragma unroll
@@ -777,14 +777,14 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
             const int b_rows = PAIR ? p.n_tile >> 1 : p.n_tile;
             const int R = p.r_filter;
             const uint32_t w_bar_cl = PAIR ? map_to_cta(smem_u32(&w_bar), 0) : 0u;
-            if (p.hm && w == 0) {
+            if (KIND == KIND_HMERGE && w == 0) {
                 // merged horizontal taps: per channel block one box of all nine taps, landing as [r][s][out][64 in]:
                 // three tiles (one per filter row) of 3 x n_tile rows
                 const int oc0 = (walk.first % p.n_ktiles) * p.n_tile;
                 mbar_expect_tx(&w_bar, (uint32_t)(p.c_blocks * 3 * p.tx_b));
                 for (int cb = 0; cb < p.c_blocks; ++cb)
                     tma_load_4d(smem + (size_t)cb * 3 * p.b_bytes, &p.tmB, &w_bar, cb * p.kb, oc0, 0, 0);
-            } else if (p.resident && w == 0) {
+            } else if (KIND != KIND_HMERGE && p.resident && w == 0) {
                 // bank order: [tap or horizontal shift][channel block][vertical tap]
                 const int ktile = walk.first % p.n_ktiles;   // the walk stride is a multiple of n_ktiles: fixed per CTA
                 const TapList& tl = p.taps[0];
@@ -813,7 +813,7 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
             for (int pu = walk.first; ok && pu < walk.count; pu += walk.stride) {
                 const int u = walk.unit(p, pu);
                 const int n_sub = unit_iters(p, p.n_par > 1 ? u / (p.total_units / p.n_par) : 0);
-                const int G = p.gsub;
+                const int G = (KIND == KIND_GENERAL || KIND == KIND_SPLIT) ? p.gsub : 1;   // (full-halo and merged-tap stages are never grouped)
                 const int n_it = G > 1 ? (n_sub + G - 1) / G : n_sub;   // ring slots of the unit
                 if (i >= i_base + n_it) {   // no stage of this unit is mine
                     i_base += n_it;
@@ -870,11 +870,11 @@ __global__ void __launch_bounds__(kThreads, 1) conv_kmajor_kernel(const __grid_c
                         // (operands first, the wait second: the address arithmetic is off the chain wait -> expect -> issue)
                         int t0 = p.cb_shift >= 0 ? it >> p.cb_shift : it / p.c_blocks;   // tap (or horizontal shift)
                         const int cb = it - t0 * p.c_blocks;                               // channel block
-                        if (p.fh || p.hm) t0 = 0;   // one box per channel block: the entry of tap (0, 0) carries its origin
+                        if (KIND == KIND_HMERGE || KIND == KIND_FULL_HALO) t0 = 0;   // one box per channel block: the entry of tap (0, 0) carries its origin
                         uint8_t* a_dst = ring + (size_t)s * stage_bytes;
                         // with vreuse the table entry of vertical tap 0 carries the shift of the whole haloed tile
                         const CUtensorMap* map_a = &p.tmA[tl.map[t0]];
-                        const int ca = cb * p.kb, wa = c.ow0 + (p.hm ? 0 : tl.dw[t0]), ha = c.oh0 + tl.dh[t0];   // merged taps: no horizontal shift
+                        const int ca = cb * p.kb, wa = c.ow0 + (KIND == KIND_HMERGE ? 0 : tl.dw[t0]), ha = c.oh0 + tl.dh[t0];   // merged taps: no horizontal shift
                         int b_s[3], b_r[3];
 #pragma unroll
                         for (int v = 0; v < 3; ++v) {
