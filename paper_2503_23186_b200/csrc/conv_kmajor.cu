@@ -1141,7 +1141,7 @@ static b2c_status build_kmajor_plan(b2c_ctx* ctx, const KMajorProblem& pb, KMajo
                        9 * (pb.ic / 64) * b_rows * 64 * 2 <= (p.pair ? 148 : 96) * 1024;
     // shared-memory plan.  Preference: haloed stages (vertical tap reuse) with 64-channel k-blocks, then with
     // 32-channel k-blocks (smaller stages, so that a ring of at least four still fits), else one tap per stage.
-    const int ring_budget = 210 * 1024;
+    const int ring_budget = 217 * 1024;   // 227 KB per CTA less the static arrays (8.3 KB) and the alignment slack
     const int kb_natural = (pb.ic % 64 == 0) ? 64 : (pb.ic % 32 == 0) ? 32 : 16;
     const bool can_vreuse = (R == 3 && pb.stride == 1 && p.bn == 1);
     const int taps_total = R * R;
@@ -1372,7 +1372,7 @@ b2c_status launch_conv_kmajor(b2c_ctx* ctx, const KMajorProblem& pb, cudaStream_
     if (!(ctx->smem_optin_done & B2C_OPTIN_KMAJOR)) {   // the attribute belongs to the device: kept per context, not per process
         for (int a = 0; a < 2; ++a)
             for (int b = 0; b < 4; ++b)
-                if (kernels[a][b] != nullptr) B2C_CUDA(cudaFuncSetAttribute(kernels[a][b], cudaFuncAttributeMaxDynamicSharedMemorySize, 212 * 1024));
+                if (kernels[a][b] != nullptr) B2C_CUDA(cudaFuncSetAttribute(kernels[a][b], cudaFuncAttributeMaxDynamicSharedMemorySize, 218 * 1024));
         ctx->smem_optin_done |= B2C_OPTIN_KMAJOR;
     }
     B2C_CUDA(b2c_launch(ctx, kernel, dim3((unsigned)grid), dim3(kThreads), smem_bytes, stream, p.pair ? 2u : 1u, p));
