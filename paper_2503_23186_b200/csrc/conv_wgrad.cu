@@ -49,7 +49,8 @@ struct alignas(64) WgradParams {
     int box_a, box_b, a_boxes, b_boxes;   // bytes per dy / x box; dy boxes per stage; x boxes per shift
     int a_bytes, a_lbo;                   // dy bytes per stage; byte distance between the two 64-row halves of the A operand
     int tw_shift;                         // log2(tiles_w)
-    int stage_bytes;
+    int stage_bytes;                      // bytes of a ring slot = gsub chunks
+    int gsub, sub_bytes;                  // pixel chunks that share a ring slot, one barrier wait and one commit; bytes of one chunk's operands
     int n_pieces, piece_t0[3], piece_nt[3];   // MMAs per k-step: first shift and number of shifts each covers
     int fx;                               // framed x stages: one box of (bw + 2) x bh pixels per 64-channel block serves the three shifts
     int fx_box, fx_tx;                    // shared-memory footprint (1 KB multiple) and bytes delivered per framed box
@@ -161,25 +162,28 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
             prefetch_tensormap(&p.tmDy);
             prefetch_tensormap(&p.tmX[0]);
             const uint32_t tx = p.fx ? (uint32_t)(p.a_bytes + p.b_boxes * p.fx_tx) : (uint32_t)(p.a_bytes + grp.nb * p.b_boxes * p.box_b);
-            int it = w, s = w;
+            int it = w, s = w;   // it counts ring slots; a slot holds G consecutive chunks (the last one of the CTA possibly fewer)
             uint32_t ph = 0u;
             const bool timed = p.stall != nullptr && w == 0;
             long long waited = 0;
-            while (it < n_chunks) {
+            const int G = p.gsub, n_slots = (n_chunks + G - 1) / G;
+            while (it < n_slots) {
                 const long long w0 = timed ? clock64() : 0;
                 if (!mbar_wait_bounded(&empty_bar[s], ph ^ 1u, p.spin_limit, &abort_flag)) {
                     atomicOr(p.status, B2C_DEV_TIMEOUT);
                     break;
                 }
                 if (timed) waited += clock64() - w0;
-                int ch = chunk_begin + it;
+                const int n_g = n_chunks - it * G < G ? n_chunks - it * G : G;
+                mbar_expect_tx(&full_bar[s], (uint32_t)n_g * tx);
+                for (int g = 0; g < n_g; ++g) {
+                int ch = chunk_begin + it * G + g;
                 const int ow0 = (ch & (p.tiles_w - 1)) * p.bw;
                 ch >>= p.tw_shift;
                 const int th = ch / p.tiles_h;
                 const int oh0 = (ch - th * p.tiles_h) * p.bh;
                 const int n0 = th * p.bn;
-                uint8_t* dst = smem + (size_t)s * p.stage_bytes;
-                mbar_expect_tx(&full_bar[s], tx);
+                uint8_t* dst = smem + (size_t)s * p.stage_bytes + (size_t)g * p.sub_bytes;
                 if (p.stack) {
                     // one box with a halo row on top: copy 1 of dy (gathered one row higher) is its first pb pixels,
                     // copy 0 starts one image row further down
@@ -198,6 +202,7 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
                     for (int j = 0; j < p.b_boxes; ++j)
                         tma_load_4d(dst + (size_t)(b * p.b_boxes + j) * p.box_b, &p.tmX[grp.map[b]], &full_bar[s], ctile * p.ct + j * p.cw_b,
                                     ow0 + grp.dw[b], oh0 + grp.dh[b], n0);
+                }
                 last_issued = it;
                 if (s + kWgProducers < S) {
                     it += kWgProducers;
@@ -240,14 +245,23 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
             const bool timed = p.stall != nullptr;
             const long long t_begin = timed ? clock64() : 0;
             long long waited = 0, issuing = 0;
-            if (my != 0 && n_chunks > 1 && !mbar_wait_bounded(&init_bar, 0u, p.spin_limit, &abort_flag)) {   // chunk 0 has initialised the accumulator
+            const int G = p.gsub, n_slots = (n_chunks + G - 1) / G;
+            const uint32_t sub16 = (uint32_t)p.sub_bytes >> 4;
+            if (my != 0 && n_slots > 1 && !mbar_wait_bounded(&init_bar, 0u, p.spin_limit, &abort_flag)) {   // slot 0 has initialised the accumulator
                 atomicOr(p.status, B2C_DEV_TIMEOUT);
                 ok = false;
             }
             if (my != 0) tc_fence_after();
-            for (int it = my; ok && it < n_chunks; it += p.issuers) {
-                const int s = it % S;
-                const uint32_t ph = (uint32_t)(it / S) & 1u;
+            // (this thread's chain of dependent instructions per slot bounds chunks with few MMAs: nothing is recomputed in the loop)
+            const bool fx = p.fx != 0;
+            const int n_issuers = p.issuers, b_boxes = p.b_boxes;
+            const uint32_t id_fx = make_idesc_bf16(128, 3 * p.cw_b, true, true);
+            const uint32_t fx_b_first = (uint32_t)p.a_bytes >> 4, fx_b_next = (uint32_t)p.fx_box >> 4, fx_d_next = 3u * (uint32_t)p.cw_b;
+            const uint32_t fk0 = p.fx_koff[0], fk1 = p.fx_koff[1], fk2 = p.fx_koff[2], fk3 = p.fx_koff[3];
+            const uint32_t stage16 = (uint32_t)p.stage_bytes >> 4, smem16 = smem_u32(smem) >> 4;
+            int s = my;            // S is even with two threads: a thread's slots are my, my + 2, ...
+            uint32_t ph = 0u;
+            for (int it = my; ok && it < n_slots; it += n_issuers) {
                 const long long w0 = timed ? clock64() : 0;
                 if (!mbar_wait_bounded(&full_bar[s], ph, p.spin_limit, &abort_flag)) {
                     atomicOr(p.status, B2C_DEV_TIMEOUT);
@@ -257,15 +271,16 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
                 const long long w1 = timed ? clock64() : 0;
                 waited += w1 - w0;
                 tc_fence_after();
-                const uint32_t st16 = smem_u32(smem + (size_t)s * p.stage_bytes) >> 4;
-                const uint32_t a_lo = a_lo_base + st16, b_lo = b_lo_base + st16;
-                const uint32_t acc0 = it != 0 ? 1u : 0u;
-                if (p.fx) {   // chunks of 64 pixels: four k-steps; one MMA per channel block, N = three shifts x cw_b channels
-                    const uint32_t id_fx = make_idesc_bf16(128, 3 * p.cw_b, true, true);
-                    const uint32_t b_first = b_lo + ((uint32_t)p.a_bytes >> 4), b_next = (uint32_t)p.fx_box >> 4, d_next = 3u * (uint32_t)p.cw_b;
-                    for (int i = 0; i < p.b_boxes; ++i)
-                        wg_issue_framed<4>(tmem_base + (uint32_t)i * d_next, a_lo, b_first + (uint32_t)i * b_next, a_hi, b_hi, id_fx, kstep_a, p.fx_koff[0],
-                                           p.fx_koff[1], p.fx_koff[2], p.fx_koff[3], acc0);
+                const uint32_t st16 = smem16 + (uint32_t)s * stage16;
+                const int n_g = n_chunks - it * G < G ? n_chunks - it * G : G;
+                for (int g = 0; g < n_g; ++g) {
+                const uint32_t a_lo = a_lo_base + st16 + (uint32_t)g * sub16, b_lo = b_lo_base + st16 + (uint32_t)g * sub16;
+                const uint32_t acc0 = (it | g) != 0 ? 1u : 0u;
+                if (fx) {   // chunks of 64 pixels: four k-steps; one MMA per channel block, N = three shifts x cw_b channels
+                    const uint32_t b_first = b_lo + fx_b_first;
+                    for (int i = 0; i < b_boxes; ++i)
+                        wg_issue_framed<4>(tmem_base + (uint32_t)i * fx_d_next, a_lo, b_first + (uint32_t)i * fx_b_next, a_hi, b_hi, id_fx, kstep_a, fk0, fk1, fk2,
+                                           fk3, acc0);
                 } else if (ksteps == 4) {
                     wg_issue<4>(tmem_base + dcol0, a_lo, b_lo + boff0, a_hi, b_hi, idesc0, kstep_a, kstep_b, acc0);
                     if (n_pieces > 1) wg_issue<4>(tmem_base + dcol1, a_lo, b_lo + boff1, a_hi, b_hi, idesc1, kstep_a, kstep_b, acc0);
@@ -275,9 +290,12 @@ __global__ void __launch_bounds__(kWgThreads, 1) conv_wgrad_kernel(const __grid_
                     if (n_pieces > 1) wg_issue<2>(tmem_base + dcol1, a_lo, b_lo + boff1, a_hi, b_hi, idesc1, kstep_a, kstep_b, acc0);
                     if (n_pieces > 2) wg_issue<2>(tmem_base + dcol2, a_lo, b_lo + boff2, a_hi, b_hi, idesc2, kstep_a, kstep_b, acc0);
                 }
+                }
                 umma_commit(&empty_bar[s]);
                 if (it == 0) umma_commit(&init_bar);
                 if (timed) issuing += clock64() - w1;
+                s += n_issuers;
+                if (s >= S) { s -= S; ph ^= 1u; }
             }
             if (ok && n_chunks > 0) umma_commit(&accum_bar);
             if (timed && my == 0) {
@@ -473,7 +491,18 @@ static b2c_status build_wgrad_plan(b2c_ctx* ctx, const WgradProblem& pb, WgradPl
         p.pb = 32;
     }
     if (p.fx && p.pb != 64) return B2C_ERR_UNSUPPORTED_SHAPE;   // cannot happen: a framed stage is under 40 KB
-    int stages = (200 * 1024) / p.stage_bytes;
+    // Chunks with few MMAs share a ring slot (an issuing thread pays 700-900 cycles per slot for the barrier wait and the
+    // commits on top of its MMAs): two chunks per slot where one holds under half of that in tensor-pipe cycles and four
+    // slots remain.
+    p.sub_bytes = p.stage_bytes;
+    p.gsub = 1;
+    {
+        const int total_cols = p.fx ? p.b_boxes * 3 * p.cw_b : shifts * p.ct;
+        const int per_chunk = (p.pb / 16) * (total_cols / 2);
+        if (ctx->use_group_kblocks && per_chunk < 500 && ((216 * 1024) / p.sub_bytes) / 2 >= 4) p.gsub = 2;
+    }
+    p.stage_bytes = p.gsub * p.sub_bytes;
+    int stages = ((p.gsub > 1 ? 216 : 200) * 1024) / p.stage_bytes;
     if (stages > kWgStages) stages = kWgStages;
     if (stages < 2) return B2C_ERR_UNSUPPORTED_SHAPE;
     // Two issuing threads need an even ring.  Measured: four stages with two threads beat five with one (128 -> 128:
@@ -535,7 +564,7 @@ b2c_status launch_conv_wgrad(b2c_ctx* ctx, const WgradProblem& pb, cudaStream_t 
     std::string key("W");
     key_add(key, pb.n); key_add(key, pb.h); key_add(key, pb.w); key_add(key, pb.c); key_add(key, pb.p); key_add(key, pb.q); key_add(key, pb.k);
     key_add(key, pb.r); key_add(key, pb.stride); key_add(key, pb.pad); key_add(key, pb.dy); key_add(key, pb.x); key_add(key, pb.dw);
-    key_add(key, ctx->use_wgrad_frame); key_add(key, ctx->use_wgrad_two_issuers);
+    key_add(key, ctx->use_wgrad_frame); key_add(key, ctx->use_wgrad_two_issuers); key_add(key, ctx->use_group_kblocks);
     auto it = ctx->plan_cache.find(key);
     if (it == ctx->plan_cache.end()) {
         WgradPlan fresh;
@@ -554,7 +583,7 @@ b2c_status launch_conv_wgrad(b2c_ctx* ctx, const WgradProblem& pb, cudaStream_t 
     p.stall = ctx->stall_counters;
 
     if (!(ctx->smem_optin_done & B2C_OPTIN_WGRAD)) {
-        B2C_CUDA(cudaFuncSetAttribute(conv_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 212 * 1024));
+        B2C_CUDA(cudaFuncSetAttribute(conv_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 218 * 1024));
         ctx->smem_optin_done |= B2C_OPTIN_WGRAD;
     }
     const size_t smem_bytes = plan.smem_bytes;
