@@ -514,7 +514,7 @@ __device__ __forceinline__ void mma_issuer(const ConvKParams& p, const UnitWalk&
         if (p.n_par > 1) n_sub = unit_iters(p, walk.unit(p, pu) / units_per_par);
         if (n_sub == 0) continue;   // a parity without taps: the epilogue stores zeros without an accumulator
         const int n_it = GROUP ? (n_sub + G - 1) / G : n_sub;   // ring slots of the unit
-        if (!p.issue_split && (j % p.issuers) != my) {   // another issuer's unit: step over its stages
+        if ((j % p.issuers) != my) {   // another issuer's unit: step over its stages
             i_stage += n_it;
             s += n_it;
             while (s >= S) { s -= S; ph ^= 1u; }
@@ -522,47 +522,17 @@ __device__ __forceinline__ void mma_issuer(const ConvKParams& p, const UnitWalk&
             continue;
         }
         const int buf = j & (p.acc_bufs - 1);
-        const long long w1 = timed ? clock64() : 0;
-        if (!mbar_wait_bounded(&acc_empty[buf], ((uint32_t)(j >> p.acc_shift) & 1u) ^ 1u, p.spin_limit, abort_flag)) {
-            atomicOr(p.status, B2C_DEV_TIMEOUT);
-            ok = false;
-            break;
-        }
-        if (timed) wait_acc += clock64() - w1;
-        tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * p.acc_cols);
         uint32_t b_res = bank_lo;   // resident bank: B tile of (tap or horizontal shift, channel block), consecutive per stage
-        // Shared units: stage i of the CTA belongs to thread i % 2 (the ring depth is even, so a slot keeps its thread).  The
-        // thread that does not own the unit's first stage, whose first MMA overwrites the accumulator, waits until that
-        // stage has completed before it adds to the same accumulator.
-        const int init_owner = i_stage & 1;
-        bool init_seen = !p.issue_split || init_owner == my;
         for (int it = 0; it < n_it; ++it) {
             int n_k = 1;   // k-blocks in this slot
             if constexpr (GROUP) n_k = n_sub - it * G < G ? n_sub - it * G : G;
-            if (p.issue_split && (i_stage & 1) != my) {   // the other thread's stage
-                b_res += GROUP ? (uint32_t)n_k * b_cb16 : b_cb16;
-                ++i_stage;
-                if (++s == S) { s = 0; ph ^= 1u; }
-                continue;
-            }
-            if (!init_seen) {
-                if (!mbar_wait_bounded(&init_bar[buf], (uint32_t)(j >> p.acc_shift) & 1u, p.spin_limit, abort_flag)) {
-                    atomicOr(p.status, B2C_DEV_TIMEOUT);
-                    ok = false;
-                    break;
-                }
-                tc_fence_after();
-                init_seen = true;
-            }
             const long long w2 = timed ? clock64() : 0;
             // A parity wait tells a barrier's phases apart only modulo two, and with two issuers this thread may reach a
             // slot before the slot's previous stage (another issuer's) was even loaded.  A producer issues the load of
             // stage i only after the previous stage in that slot was consumed, and then stamps the slot with i + 1:
             // seeing the stamp pass i makes the parity wait unambiguous.
-            // (Threads that share every unit take alternate slots of an even ring: a slot has one consumer, which has waited for
-            // the slot's previous stage itself, and needs no stamp.)
-            if (p.issuers > 1 && !p.issue_split) {
+            if (p.issuers > 1) {
                 uint32_t polls = 0;
                 while (ld_volatile_shared(&slot_stage[s]) <= i_stage) {
                     if (++polls > p.spin_limit || *(volatile uint32_t*)abort_flag != 0u) {
@@ -578,6 +548,18 @@ __device__ __forceinline__ void mma_issuer(const ConvKParams& p, const UnitWalk&
                 break;
             }
             if (timed) wait_ring += clock64() - w2;
+            // The accumulator comes second: the unit's first slot is usually full long before the epilogue hands the accumulator
+            // back, so the slot's stamp and barrier (600-700 cycles of this thread) are off the path from "accumulator free" to
+            // the first MMA, the loop that bounds narrow tiles with two accumulators.
+            if (it == 0) {
+                const long long w1 = timed ? clock64() : 0;
+                if (!mbar_wait_bounded(&acc_empty[buf], ((uint32_t)(j >> p.acc_shift) & 1u) ^ 1u, p.spin_limit, abort_flag)) {
+                    atomicOr(p.status, B2C_DEV_TIMEOUT);
+                    ok = false;
+                    break;
+                }
+                if (timed) wait_acc += clock64() - w1;
+            }
             tc_fence_after();
             // descriptors differ from stage to stage only in the 14-bit address field: add offsets to the low word
             if constexpr (GROUP) {   // (never with full-halo or merged-tap stages)
@@ -598,10 +580,6 @@ __device__ __forceinline__ void mma_issuer(const ConvKParams& p, const UnitWalk&
             // frees the stage (in both CTAs of a pair) once these MMAs have read it
             if constexpr (PAIR) umma_commit_pair(&empty_bar[s], (uint16_t)3);
             else umma_commit(&empty_bar[s]);
-            if (p.issue_split && it == 0) {   // the overwriting stage of this unit (both issuing threads live in the leader CTA of a pair)
-                if constexpr (PAIR) umma_commit_pair(&init_bar[buf], (uint16_t)1);
-                else umma_commit(&init_bar[buf]);
-            }
             ++i_stage;
             if (++s == S) { s = 0; ph ^= 1u; }
         }
