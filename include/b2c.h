@@ -26,8 +26,9 @@
  *       B2C_FULL_HALO=0      one load per tap group instead of one framed tile per channel block (3x3 stride-1 layers)
  *       B2C_HMERGE=0         3x3 stride-1 layers with 64 output channels: one MMA per tap (N = 64) instead of the three horizontal taps
  *                            merged into N = 192 MMAs whose column blocks the epilogue shifts and adds
- *       B2C_GROUP_KBLOCKS=0  forward / data gradient of stride-2 and 1x1 layers: one 64-channel k-block per ring slot instead of two to four
- *                            sharing a slot, a barrier wait and a commit
+ *       B2C_GROUP_KBLOCKS=0  forward / data gradient of stride-2 and 1x1 layers: one k-block per ring slot instead of two sharing a slot,
+ *                            a barrier wait and a commit; weight gradient of layers with few MMAs per 64-pixel chunk: one chunk per slot
+ *                            instead of two
  *       B2C_ISSUE_SPLIT=0    forward / data gradient, tiles wider than 128 channels: one MMA-issuing thread instead of two sharing every unit
  *       B2C_WGRAD_FRAME=0    weight gradient: one x box per horizontal shift instead of one framed box per channel block
  *       B2C_WGRAD_ISSUERS=1  weight gradient: one MMA-issuing thread instead of two on alternate chunks of one accumulator
