@@ -148,14 +148,15 @@ SWITCHES = [("B2C_ISSUE_SPLIT", "0"), ("B2C_ISSUE_SPLIT", "1"), ("B2C_WGRAD_FRAM
 def test_kernel_switches_off_and_on(name, value, monkeypatch):
     """Each switch of b2c_create in both positions: forward, data gradient and weight gradient of layers that reach the
     switched path (256-channel tiles, 3x3 stride-1 layers with 8- and 32-pixel rows, 64 output channels, stride-2 and 1x1 layers
-    whose short k-blocks share ring slots, with one and with two issuing threads per unit) against the oracle."""
+    whose short k-blocks share ring slots, with an even and an odd number of k-blocks, with one and with two issuing threads per unit)
+    against the oracle."""
     from paper_2503_23186_b200 import binding
     monkeypatch.setenv(name, value)
     c = binding.Context(0)
     try:
         # (the 64-output-channel layers are large enough for merged horizontal taps: at least two tiles per SM, rows of 32 / 16 / 8 pixels)
         for shape in [(4, 16, 16, 128, 256, 3, 1), (4, 8, 8, 512, 512, 3, 1), (40, 32, 32, 64, 64, 3, 1), (160, 16, 16, 64, 64, 3, 1), (600, 8, 8, 128, 64, 3, 1),
-                      (16, 8, 8, 128, 128, 3, 1), (8, 32, 32, 64, 128, 3, 2), (8, 16, 16, 256, 64, 1, 1), (4, 16, 16, 160, 320, 3, 2)]:
+                      (16, 8, 8, 128, 128, 3, 1), (8, 32, 32, 64, 128, 3, 2), (8, 16, 16, 256, 64, 1, 1), (8, 16, 16, 192, 64, 1, 1), (4, 16, 16, 160, 320, 3, 2)]:
             N, H, W, C, K, R, st = shape
             x, w, g = wl.conv_problem(33, *shape)
             P = H // st
